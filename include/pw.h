@@ -1,0 +1,210 @@
+/*
+ * pw.h -- C ABI of the paged-weight MoE hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library executes one Mixture-of-Experts layer whose expert weight matrices
+ * ("linear-blocks", one row of the paper's weight page table each, Sec. 3.1) are
+ * resident in GPU memory as weight pages of differing, runtime-changing bitwidths,
+ * and lowers the bitwidth of a page at runtime (the "offload" direction of
+ * Sec. 3.1 / 3.3).  The paper's pages are Any-Precision bit-planes plus a centroid
+ * table; here a page is a group-wise uniform code (group of 128 weights along the
+ * input dimension, fp16 scale, fp16 zero-point = the value code 0 decodes to):
+ *
+ *      weight = fp16( code * scale + zero_point ),   code in [0, 2^bits - 1]
+ *
+ * General rules
+ *   - Plain C.  Every call returns a pw_status; nothing throws, traps or hangs.
+ *   - "device" pointers are CUDA global memory of the current device, "host"
+ *     pointers are ordinary host memory.  All device buffers are owned and
+ *     allocated by the caller; the library never allocates device memory.
+ *     pw_create allocates only a small host object and a pinned host staging area.
+ *   - Work is enqueued on the caller's stream and returns immediately.  Argument
+ *     errors are detected on the host before anything is enqueued.  Problems met
+ *     on the device (a bounded wait that ran out, a failed self check) are written
+ *     to a status word that pw_last_device_status reads back.
+ *   - Every device pointer must be 16-byte aligned.  rows and cols of a block
+ *     must be multiples of 128.  Inputs must be finite.
+ */
+#ifndef PW_H_
+#define PW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PW_OK = 0,
+  PW_ERR_INVALID_ARG = 1, /* null pointer, value out of range                         */
+  PW_ERR_SHAPE = 2,       /* rows/cols not multiples of 128, shape differs from ctx   */
+  PW_ERR_BITS = 3,        /* bitwidth not in {16,8,4,3,2}, or a demote that does not lower */
+  PW_ERR_ALIGN = 4,       /* device pointer not 16-byte aligned                        */
+  PW_ERR_STATE = 5,       /* page-table row missing, wrong page layout, not resident   */
+  PW_ERR_NOMEM = 6,       /* caller's workspace too small                              */
+  PW_ERR_CUDA = 7,        /* a CUDA runtime call failed                                */
+  PW_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out (see pw_last_device_status) */
+} pw_status;
+
+typedef enum { PW_GATE = 0, PW_UP = 1, PW_DOWN = 2 } pw_kind;
+
+/* Which expert-FFN kernel family pw_moe_forward uses.
+ * AUTO picks TENSOR unless every expert holds at most a few tokens. */
+typedef enum {
+  PW_MODE_AUTO = 0,
+  PW_MODE_SIMT = 1,  /* CUDA-core kernel, thread per weight row; right for a handful of tokens */
+  PW_MODE_TENSOR = 2 /* tcgen05 tensor-core kernel, pages dequantized into tensor memory      */
+} pw_mode;
+
+/* Page layouts.  CANONICAL: codes are a little-endian bit stream in row-major element
+ * order (code of element n at stream bits [n*bits, (n+1)*bits)), scales / zero-points
+ * fp16 [rows, cols/group] row-major; a 16-bit page is the fp16 matrix itself.
+ * TILED: the same bytes regrouped per (128-row, one-group) tile so that a kernel reads a
+ * tile with contiguous 16-byte loads; produced by pw_quantize_block / pw_demote_block /
+ * pw_import_page and required by pw_moe_forward.  Both layouts have identical sizes. */
+enum { PW_LAYOUT_CANONICAL = 0, PW_LAYOUT_TILED = 1 };
+
+/* Residency state of a page-table row (Sec. 3.1).  Only GPU_RESIDENT rows can be used. */
+enum { PW_STATE_GPU_RESIDENT = 0, PW_STATE_CPU_RESIDENT = 1, PW_STATE_IN_TRANSFER = 2 };
+
+typedef struct CUstream_st* pw_stream; /* a cudaStream_t */
+typedef struct pw_ctx pw_ctx;
+typedef struct pw_page_table pw_page_table; /* the committed table of a context */
+
+typedef struct {
+  int32_t n_layers;   /* MoE layers the page table covers                        */
+  int32_t n_experts;  /* routed experts E per layer                              */
+  int32_t n_shared;   /* always-on shared experts per layer (gate 1, 16-bit pages) */
+  int32_t hidden;     /* H, multiple of 128                                      */
+  int32_t ffn;        /* F, expert FFN size, multiple of 128                     */
+  int32_t group;      /* quantization group size; must be 128                    */
+  int32_t max_tokens; /* largest T of a forward call                             */
+  int32_t max_top_k;  /* largest top_k of a forward call                         */
+  void* workspace;    /* device, >= pw_workspace_bytes(cfg), 256-byte aligned, owned by the caller,
+                         must outlive the context; holds the committed table and all scratch   */
+  size_t workspace_bytes;
+} pw_config;
+
+/* One weight page = one linear-block at one bitwidth (Sec. 3.1).  All pointers device. */
+typedef struct {
+  void* codes;    /* bits < 16: packed codes, rows*cols*bits/8 bytes; bits == 16: fp16 weights   */
+  void* scales;   /* fp16, rows*cols/group values; ignored (may be NULL) when bits == 16         */
+  void* zps;      /* fp16, rows*cols/group values; ignored (may be NULL) when bits == 16         */
+  uint32_t rows;  /* output features                                                            */
+  uint32_t cols;  /* input features (the grouped, contracted dimension)                         */
+  uint16_t group; /* 128                                                                        */
+  uint8_t bits;   /* 16, 8, 4, 3 or 2 -- the committed bitwidth q_i once the row is published    */
+  uint8_t layout; /* PW_LAYOUT_*                                                                */
+} pw_page;
+
+/* One page-table row, index i = (layer, expert, kind) (Sec. 3.1).  Experts
+ * n_experts .. n_experts+n_shared-1 are the shared experts. */
+typedef struct {
+  int32_t layer, expert;
+  int32_t kind;         /* pw_kind                                            */
+  pw_page page;         /* page at the committed bitwidth q_i                 */
+  uint8_t desired_bits; /* d_i chosen by a planner; recorded, not acted on    */
+  uint8_t state;        /* PW_STATE_*; must be GPU_RESIDENT                   */
+} pw_table_entry;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Bytes of device workspace a context with this configuration needs (0 if cfg is invalid). */
+size_t pw_workspace_bytes(const pw_config* cfg);
+
+/* Creates a context on the current device.  cfg->workspace is zero-initialised on `the
+ * legacy default stream` and the call returns after that has completed.
+ * Errors: INVALID_ARG, SHAPE, ALIGN, NOMEM (workspace too small), CUDA. */
+pw_status pw_create(pw_ctx** ctx, const pw_config* cfg);
+
+/* Waits for the device, then frees the host object.  Device buffers stay with the caller. */
+pw_status pw_destroy(pw_ctx* ctx);
+
+/* Size table M_i^b of Eq. 3: total bytes of a rows x cols block at `bits`, metadata included;
+ * the three parts are returned through the optional out pointers.  0 on invalid arguments.
+ * Released bytes of a demotion b -> b' are pw_page_bytes(b) - pw_page_bytes(b'). */
+size_t pw_page_bytes(uint32_t rows, uint32_t cols, int bits, int group, size_t* codes_bytes, size_t* scales_bytes,
+                     size_t* zps_bytes);
+
+/* ---- pages -------------------------------------------------------------------------- */
+
+/* Group-quantizes an fp16 block into a new page.  w_fp16: device, [rows, cols] row-major.
+ * dst: host struct whose codes / scales / zps point to caller-allocated device buffers of the
+ * sizes pw_page_bytes reports; the call fills rows, cols, group, bits, layout (TILED).
+ * bits == 16 stores the weights unchanged (a re-tiled copy).  Per group of 128 along cols, in
+ * fp32 with one rounding per operation: lo = min, hi = max, scale = fp16((hi-lo)/(2^bits-1))
+ * (1.0 if hi == lo, 2^-24 if it rounds to zero), zero-point = fp16(lo),
+ * code = clamp(rint((w-lo) * (1/scale)), 0, 2^bits-1) with round-half-to-even.
+ * The paper has no runtime quantizer (its lower precisions pre-exist as bit-plane subsets,
+ * Sec. 2.2); this is the page constructor of this build's format.
+ * Errors: INVALID_ARG, SHAPE, BITS, ALIGN. */
+pw_status pw_quantize_block(pw_ctx* ctx, const void* w_fp16, uint32_t rows, uint32_t cols, int bits, pw_page* dst,
+                            pw_stream stream);
+
+/* Lowers a page: dst = quantize(dequantize(src), dst_bits), dst_bits < src->bits.  The offload
+ * direction of Sec. 3.1 / 3.3: the new page is written to separate caller-allocated buffers, the
+ * source is never modified, and the lower bitwidth takes effect only when the caller publishes
+ * dst with pw_set_page_table.  src must be TILED.  Meant to run on a side stream while
+ * pw_moe_forward runs on another.  Errors: INVALID_ARG, BITS, ALIGN, STATE (src not TILED). */
+pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bits, pw_page* dst, pw_stream stream);
+
+/* Layout conversion, same bitwidth: TILED -> CANONICAL (export) and CANONICAL -> TILED (import).
+ * dst buffers are caller-allocated, same sizes as src; the call fills dst's header fields.
+ * Export is how pages are compared bit for bit and saved; import restores them. */
+pw_status pw_export_page(pw_ctx* ctx, const pw_page* src_tiled, pw_page* dst_canonical, pw_stream stream);
+pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst_tiled, pw_stream stream);
+
+/* ---- page table --------------------------------------------------------------------- */
+
+/* Publishes n rows of the weight page table (Sec. 3.1): for each entry the row
+ * (layer, expert, kind) now maps to entry.page with committed bitwidth page.bits.  Rows not
+ * named keep their value.  The update is ordered on `stream`: forward calls enqueued on the same
+ * stream before this call read the old rows, calls enqueued after it read the new rows -- the
+ * "safe boundary" of Sec. 3.3 is the gap between two forward calls.  The previous page of a row
+ * may be released once work enqueued before this call has finished.  entries: host.  epoch_out
+ * (optional, host) receives the table epoch after the update; each call increments it by one.
+ * Errors: INVALID_ARG, SHAPE (page shape does not match kind and ctx), BITS, ALIGN,
+ * STATE (layout not TILED, state not GPU_RESIDENT, shared expert below 16 bits), CUDA. */
+pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entries, size_t n, pw_stream stream,
+                            uint64_t* epoch_out);
+
+/* Handle of the committed table, for pw_moe_forward. */
+const pw_page_table* pw_get_page_table(pw_ctx* ctx);
+
+/* Host-side query of a committed row (what the last pw_set_page_table published). */
+pw_status pw_query_row(pw_ctx* ctx, int layer, int expert, int kind, pw_table_entry* out);
+
+/* ---- forward ------------------------------------------------------------------------ */
+
+/* One MoE layer (Sec. 2.1, Sec. 3.3): top_k routing of T tokens over the E routed experts
+ * (ties: lower expert index; gates = softmax over the k selected logits), stable grouping of
+ * the (token, slot) pairs into per-expert segments, per expert y = W_down(silu(W_gate x) * W_up x)
+ * with every block read at its committed bitwidth from `table`, and
+ * out[t] = sum_j gate[t,j] * y_{e_j}[t] + sum over shared experts y_s[t].
+ * hidden_fp16: device [T, H] fp16.  router_logits: device [T, E] fp32.  out: device [T, H] fp32.
+ * table: pw_get_page_table(ctx) or NULL (same thing).  All rows of `layer` must have been
+ * published.  Operands of the contractions are fp16, accumulation is fp32.
+ * Errors: INVALID_ARG (T < 1, T > max_tokens, top_k < 1, top_k > min(E, max_top_k), bad layer),
+ * ALIGN, STATE (a row of the layer is unpublished). */
+pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden_fp16, const float* router_logits, int T,
+                         int top_k, const pw_page_table* table, float* out, pw_mode mode, pw_stream stream);
+
+/* Copies the routing of the last forward call out of the workspace (device pointers, any may
+ * be NULL): topk_ids int32 [T, k], gates fp32 [T, k], counts int32 [E], offsets int32 [E+1],
+ * perm int32 [T*k] (pair ids p = t*k + j sorted by expert, then by p). */
+pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
+                         int32_t* perm, pw_stream stream);
+
+/* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
+ * then clears it. */
+pw_status pw_last_device_status(pw_ctx* ctx);
+
+/* Number of kernels the library has launched through this context since creation. */
+uint64_t pw_launch_count(pw_ctx* ctx);
+
+const char* pw_status_str(pw_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PW_H_ */

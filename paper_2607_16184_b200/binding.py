@@ -1,0 +1,257 @@
+"""Thin ctypes binding of the C ABI declared in ``include/pw.h``.
+
+Argument marshalling only: every step of the hot path runs inside ``libpw.so``.
+PyTorch supplies device memory (``tensor.data_ptr()``) and streams.  There is no
+CPU fallback: if the library cannot be loaded, importing names from here raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpw.so")
+
+PW_OK = 0
+STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_SHAPE", 3: "PW_ERR_BITS", 4: "PW_ERR_ALIGN",
+                5: "PW_ERR_STATE", 6: "PW_ERR_NOMEM", 7: "PW_ERR_CUDA", 8: "PW_ERR_TIMEOUT"}
+PW_GATE, PW_UP, PW_DOWN = 0, 1, 2
+PW_MODE_AUTO, PW_MODE_SIMT, PW_MODE_TENSOR = 0, 1, 2
+PW_LAYOUT_CANONICAL, PW_LAYOUT_TILED = 0, 1
+PW_STATE_GPU_RESIDENT, PW_STATE_CPU_RESIDENT, PW_STATE_IN_TRANSFER = 0, 1, 2
+GROUP = 128
+
+# every symbol include/pw.h declares
+EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
+           "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
+           "pw_moe_forward", "pw_get_routing", "pw_last_device_status", "pw_launch_count", "pw_status_str")
+
+
+class PwError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, STATUS_NAMES.get(status, str(status))))
+
+
+class pw_config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_experts", C.c_int32), ("n_shared", C.c_int32), ("hidden", C.c_int32),
+                ("ffn", C.c_int32), ("group", C.c_int32), ("max_tokens", C.c_int32), ("max_top_k", C.c_int32),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class pw_page(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p), ("zps", C.c_void_p), ("rows", C.c_uint32),
+                ("cols", C.c_uint32), ("group", C.c_uint16), ("bits", C.c_uint8), ("layout", C.c_uint8)]
+
+
+class pw_table_entry(C.Structure):
+    _fields_ = [("layer", C.c_int32), ("expert", C.c_int32), ("kind", C.c_int32), ("page", pw_page),
+                ("desired_bits", C.c_uint8), ("state", C.c_uint8)]
+
+
+_lib = None
+
+
+def load():
+    """Loads libpw.so (built by ``paper_2607_16184_b200.build``).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libpw.so is missing: run `python -m paper_2607_16184_b200.build` (there is no fallback path)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, u32, sz = C.c_void_p, C.c_int, C.c_uint32, C.c_size_t
+    L.pw_workspace_bytes.restype = sz
+    L.pw_workspace_bytes.argtypes = [C.POINTER(pw_config)]
+    L.pw_create.restype = i32
+    L.pw_create.argtypes = [C.POINTER(vp), C.POINTER(pw_config)]
+    L.pw_destroy.restype = i32
+    L.pw_destroy.argtypes = [vp]
+    L.pw_page_bytes.restype = sz
+    L.pw_page_bytes.argtypes = [u32, u32, i32, i32, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+    L.pw_quantize_block.restype = i32
+    L.pw_quantize_block.argtypes = [vp, vp, u32, u32, i32, C.POINTER(pw_page), vp]
+    L.pw_demote_block.restype = i32
+    L.pw_demote_block.argtypes = [vp, C.POINTER(pw_page), i32, C.POINTER(pw_page), vp]
+    L.pw_export_page.restype = i32
+    L.pw_export_page.argtypes = [vp, C.POINTER(pw_page), C.POINTER(pw_page), vp]
+    L.pw_import_page.restype = i32
+    L.pw_import_page.argtypes = [vp, C.POINTER(pw_page), C.POINTER(pw_page), vp]
+    L.pw_set_page_table.restype = i32
+    L.pw_set_page_table.argtypes = [vp, C.POINTER(pw_table_entry), sz, vp, C.POINTER(C.c_uint64)]
+    L.pw_get_page_table.restype = vp
+    L.pw_get_page_table.argtypes = [vp]
+    L.pw_query_row.restype = i32
+    L.pw_query_row.argtypes = [vp, i32, i32, i32, C.POINTER(pw_table_entry)]
+    L.pw_moe_forward.restype = i32
+    L.pw_moe_forward.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp]
+    L.pw_get_routing.restype = i32
+    L.pw_get_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.pw_last_device_status.restype = i32
+    L.pw_last_device_status.argtypes = [vp]
+    L.pw_launch_count.restype = C.c_uint64
+    L.pw_launch_count.argtypes = [vp]
+    L.pw_status_str.restype = C.c_char_p
+    L.pw_status_str.argtypes = [i32]
+    _lib = L
+    return L
+
+
+def _check(st: int, where: str):
+    if st != PW_OK:
+        raise PwError(st, where)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def pw_page_bytes(rows: int, cols: int, bits: int, group: int = GROUP) -> Tuple[int, int, int, int]:
+    """(total, codes, scales, zps) bytes -- the size table M_i^b of Eq. 3.  total == 0 means invalid arguments."""
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    tot = load().pw_page_bytes(rows, cols, bits, group, C.byref(a), C.byref(b), C.byref(c))
+    return int(tot), int(a.value), int(b.value), int(c.value)
+
+
+class Page:
+    """Device buffers of one weight page plus its ``pw_page`` header."""
+
+    def __init__(self, rows: int, cols: int, bits: int, device="cuda", layout: int = PW_LAYOUT_TILED):
+        tot, cb, sb, zb = pw_page_bytes(rows, cols, bits)
+        if tot == 0:
+            # unallocatable request: keep a header with null buffers so the C call reports the precise error
+            self.codes = self.scales = self.zps = None
+            self.c = pw_page(None, None, None, rows, cols, GROUP, bits & 0xff, layout)
+            self.nbytes = 0
+            return
+        self.codes = torch.empty(cb, dtype=torch.uint8, device=device)
+        self.scales = torch.empty(sb // 2, dtype=torch.float16, device=device) if sb else None
+        self.zps = torch.empty(zb // 2, dtype=torch.float16, device=device) if zb else None
+        self.c = pw_page(self.codes.data_ptr(), self.scales.data_ptr() if sb else None,
+                         self.zps.data_ptr() if zb else None, rows, cols, GROUP, bits, layout)
+        self.nbytes = tot
+
+    rows = property(lambda self: self.c.rows)
+    cols = property(lambda self: self.c.cols)
+    bits = property(lambda self: self.c.bits)
+    layout = property(lambda self: self.c.layout)
+
+
+class Context:
+    """Owns the workspace tensor and the ``pw_ctx``; methods carry the names of the C calls."""
+
+    def __init__(self, n_layers: int, n_experts: int, n_shared: int, hidden: int, ffn: int, max_tokens: int,
+                 max_top_k: int, device="cuda"):
+        self.L = load()
+        self.device = torch.device(device)
+        cfg = pw_config(n_layers, n_experts, n_shared, hidden, ffn, GROUP, max_tokens, max_top_k, None, 0)
+        nbytes = self.L.pw_workspace_bytes(C.byref(cfg))
+        if nbytes == 0:
+            raise PwError(1, "pw_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        cfg.workspace, cfg.workspace_bytes = base, nbytes
+        self.cfg = cfg
+        self.handle = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(self.L.pw_create(C.byref(self.handle), C.byref(cfg)), "pw_create")
+        self.n_segments = n_experts + n_shared
+
+    def close(self):
+        if self.handle:
+            self.L.pw_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- pages ----
+    def pw_quantize_block(self, w_fp16: torch.Tensor, bits: int, dst: Optional[Page] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> Page:
+        assert w_fp16.dtype == torch.float16 and w_fp16.is_contiguous() and w_fp16.is_cuda
+        rows, cols = w_fp16.shape
+        dst = dst or Page(rows, cols, bits, self.device)
+        _check(self.L.pw_quantize_block(self.handle, w_fp16.data_ptr(), rows, cols, bits, C.byref(dst.c),
+                                        _stream_ptr(stream)), "pw_quantize_block")
+        return dst
+
+    def pw_demote_block(self, src: Page, dst_bits: int, dst: Optional[Page] = None,
+                        stream: Optional[torch.cuda.Stream] = None) -> Page:
+        dst = dst or Page(src.rows, src.cols, dst_bits, self.device)
+        _check(self.L.pw_demote_block(self.handle, C.byref(src.c), dst_bits, C.byref(dst.c), _stream_ptr(stream)),
+               "pw_demote_block")
+        return dst
+
+    def pw_export_page(self, src: Page, stream: Optional[torch.cuda.Stream] = None) -> Page:
+        dst = Page(src.rows, src.cols, src.bits, self.device, PW_LAYOUT_CANONICAL)
+        _check(self.L.pw_export_page(self.handle, C.byref(src.c), C.byref(dst.c), _stream_ptr(stream)),
+               "pw_export_page")
+        return dst
+
+    def pw_import_page(self, src: Page, stream: Optional[torch.cuda.Stream] = None) -> Page:
+        dst = Page(src.rows, src.cols, src.bits, self.device, PW_LAYOUT_TILED)
+        _check(self.L.pw_import_page(self.handle, C.byref(src.c), C.byref(dst.c), _stream_ptr(stream)),
+               "pw_import_page")
+        return dst
+
+    # ---- page table ----
+    def pw_set_page_table(self, entries: Sequence[Tuple[int, int, int, Page]],
+                          stream: Optional[torch.cuda.Stream] = None, desired_bits: int = 0,
+                          state: int = PW_STATE_GPU_RESIDENT) -> int:
+        """entries: (layer, expert, kind, page).  Returns the table epoch after the commit."""
+        arr = (pw_table_entry * len(entries))()
+        for i, (layer, expert, kind, page) in enumerate(entries):
+            arr[i].layer, arr[i].expert, arr[i].kind = layer, expert, kind
+            arr[i].page = page.c
+            arr[i].desired_bits = desired_bits
+            arr[i].state = state
+        epoch = C.c_uint64()
+        _check(self.L.pw_set_page_table(self.handle, arr, len(entries), _stream_ptr(stream), C.byref(epoch)),
+               "pw_set_page_table")
+        return int(epoch.value)
+
+    def pw_query_row(self, layer: int, expert: int, kind: int) -> pw_table_entry:
+        out = pw_table_entry()
+        _check(self.L.pw_query_row(self.handle, layer, expert, kind, C.byref(out)), "pw_query_row")
+        return out
+
+    # ---- forward ----
+    def pw_moe_forward(self, layer: int, hidden: torch.Tensor, router_logits: torch.Tensor, top_k: int,
+                       out: Optional[torch.Tensor] = None, mode: int = PW_MODE_AUTO,
+                       stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        assert hidden.dtype == torch.float16 and hidden.is_contiguous()
+        assert router_logits.dtype == torch.float32 and router_logits.is_contiguous()
+        T, H = hidden.shape
+        if out is None:
+            out = torch.empty(T, H, dtype=torch.float32, device=hidden.device)
+        table = self.L.pw_get_page_table(self.handle)
+        _check(self.L.pw_moe_forward(self.handle, layer, hidden.data_ptr(), router_logits.data_ptr(), T, top_k,
+                                     table, out.data_ptr(), mode, _stream_ptr(stream)), "pw_moe_forward")
+        return out
+
+    def pw_get_routing(self, T: int, top_k: int, stream: Optional[torch.cuda.Stream] = None) -> Dict[str, torch.Tensor]:
+        E = self.cfg.n_experts
+        d = self.device
+        r = {"topk_ids": torch.empty(T, top_k, dtype=torch.int32, device=d),
+             "gates": torch.empty(T, top_k, dtype=torch.float32, device=d),
+             "counts": torch.empty(E, dtype=torch.int32, device=d),
+             "offsets": torch.empty(E + 1, dtype=torch.int32, device=d),
+             "perm": torch.empty(T * top_k, dtype=torch.int32, device=d)}
+        _check(self.L.pw_get_routing(self.handle, r["topk_ids"].data_ptr(), r["gates"].data_ptr(),
+                                     r["counts"].data_ptr(), r["offsets"].data_ptr(), r["perm"].data_ptr(),
+                                     _stream_ptr(stream)), "pw_get_routing")
+        return r
+
+    def pw_last_device_status(self) -> int:
+        return int(self.L.pw_last_device_status(self.handle))
+
+    def pw_launch_count(self) -> int:
+        return int(self.L.pw_launch_count(self.handle))

@@ -1,0 +1,289 @@
+// Context, workspace map, page-table commits and the forward-call orchestration.
+#include <new>
+#include <string.h>
+
+#include "pw_common.cuh"
+
+namespace pw {
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+static bool bits_ok(int b) { return b == 16 || b == 8 || b == 4 || b == 3 || b == 2; }
+
+static bool config_ok(const pw_config& c) {
+  if (c.n_layers < 1 || c.n_experts < 1 || c.n_experts > 256 || c.n_shared < 0 || c.n_shared > 16) return false;
+  if (c.hidden < kGroup || c.ffn < kGroup || c.hidden % kGroup || c.ffn % kGroup) return false;
+  if (c.group != kGroup) return false;
+  if (c.max_tokens < 1 || c.max_top_k < 1 || c.max_top_k > 32 || c.max_top_k > c.n_experts) return false;
+  if ((long long)c.max_tokens * (c.max_top_k + c.n_shared) > (1ll << 24)) return false;
+  return true;
+}
+
+WsMap make_wsmap(const pw_config& c) {
+  WsMap m{};
+  m.S = c.n_experts + c.n_shared;
+  const int P = c.max_tokens * c.max_top_k;
+  m.Rmax = P + c.n_shared * c.max_tokens;
+  m.Rpad = m.Rmax + kPadRows;
+  const int maxdim = c.hidden > c.ffn ? c.hidden : c.ffn;
+  m.max_units = (m.Rmax / 16 + m.S + 1) * (maxdim / kTileRows) * 8;
+  const size_t eight = (size_t)8 * m.Rmax;
+  m.y_slots = eight < 8192 ? eight : ((size_t)m.Rmax > 8192 ? (size_t)m.Rmax : 8192);
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o = align_up(o + bytes, 256);
+    return at;
+  };
+  m.status = take(64 * 4);
+  m.counter = take(64 * 4);
+  m.table = take(sizeof(DevRow) * (size_t)c.n_layers * m.S * 3);
+  m.topk_ids = take(4 * (size_t)P);
+  m.gates = take(4 * (size_t)P);
+  m.counts = take(4 * (size_t)m.S);
+  m.offsets = take(4 * (size_t)(m.S + 1));
+  m.perm = take(4 * (size_t)P);
+  m.inv_perm = take(4 * (size_t)P);
+  m.row_token = take(4 * (size_t)m.Rpad);
+  m.seg_order = take(4 * (size_t)m.S);
+  m.units_gu = take(sizeof(Unit) * (size_t)m.max_units);
+  m.units_dn = take(sizeof(Unit) * (size_t)m.max_units);
+  m.n_units = take(16);
+  m.xt = take((size_t)c.hidden * 2 * m.Rpad);
+  m.ht = take((size_t)c.ffn * 2 * m.Rpad);
+  m.y = take(m.y_slots * c.hidden * 4);
+  m.total = o;
+  return m;
+}
+
+static size_t row_index(const pw_ctx* ctx, int layer, int expert, int kind) {
+  return ((size_t)layer * ctx->ws.S + expert) * 3 + kind;
+}
+
+}  // namespace pw
+
+using namespace pw;
+
+extern "C" size_t pw_workspace_bytes(const pw_config* cfg) {
+  if (!cfg || !config_ok(*cfg)) return 0;
+  return make_wsmap(*cfg).total;
+}
+
+extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
+  if (!out || !cfg) return PW_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->group != kGroup || cfg->hidden % kGroup || cfg->ffn % kGroup) return PW_ERR_SHAPE;
+  if (!config_ok(*cfg) || !cfg->workspace) return PW_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cfg->workspace) & 255) return PW_ERR_ALIGN;
+  WsMap m = make_wsmap(*cfg);
+  if (cfg->workspace_bytes < m.total) return PW_ERR_NOMEM;
+  pw_ctx* ctx = new (std::nothrow) pw_ctx();
+  if (!ctx) return PW_ERR_NOMEM;
+  ctx->cfg = *cfg;
+  ctx->ws = m;
+  ctx->base = reinterpret_cast<char*>(cfg->workspace);
+  ctx->table_handle.owner = ctx;
+  ctx->epoch = 0;
+  ctx->launches = 0;
+  ctx->last_T = ctx->last_k = 0;
+  ctx->tc_state = nullptr;
+  ctx->stage_next = 0;
+  const size_t nrows = (size_t)cfg->n_layers * m.S * 3;
+  ctx->stage_rows = nrows;
+  ctx->host_rows = new (std::nothrow) pw_table_entry[nrows]();
+  ctx->host_valid = new (std::nothrow) uint8_t[nrows]();
+  for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
+    ctx->stage[i] = nullptr;
+    ctx->stage_ev[i] = nullptr;
+    ctx->stage_used[i] = false;
+  }
+  bool ok = ctx->host_rows && ctx->host_valid;
+  int dev = 0;
+  ok = ok && cudaGetDevice(&dev) == cudaSuccess;
+  ok = ok && cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
+  for (int i = 0; ok && i < pw_ctx::kStageSlots; ++i) {
+    ok = cudaMallocHost(reinterpret_cast<void**>(&ctx->stage[i]), sizeof(DevRow) * nrows) == cudaSuccess &&
+         cudaEventCreateWithFlags(&ctx->stage_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  }
+  // the table (valid = 0), status word, counters and operand padding start out as zeros
+  ok = ok && cudaMemset(ctx->base, 0, m.total) == cudaSuccess;
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    pw_destroy(ctx);
+    return PW_ERR_CUDA;
+  }
+  *out = ctx;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_destroy(pw_ctx* ctx) {
+  if (!ctx) return PW_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
+    if (ctx->stage[i]) cudaFreeHost(ctx->stage[i]);
+    if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+  }
+  delete[] ctx->host_rows;
+  delete[] ctx->host_valid;
+  delete ctx;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entries, size_t n, pw_stream stream,
+                                       uint64_t* epoch_out) {
+  if (!ctx || (!entries && n)) return PW_ERR_INVALID_ARG;
+  const pw_config& c = ctx->cfg;
+  if (n > ctx->stage_rows) return PW_ERR_INVALID_ARG;
+  // validate everything before anything is enqueued
+  for (size_t i = 0; i < n; ++i) {
+    const pw_table_entry& e = entries[i];
+    const pw_page& p = e.page;
+    if (e.layer < 0 || e.layer >= c.n_layers || e.expert < 0 || e.expert >= ctx->ws.S || e.kind < 0 || e.kind > 2)
+      return PW_ERR_INVALID_ARG;
+    if (!bits_ok(p.bits)) return PW_ERR_BITS;
+    const uint32_t er = e.kind == PW_DOWN ? c.hidden : c.ffn, ec = e.kind == PW_DOWN ? c.ffn : c.hidden;
+    if (p.rows != er || p.cols != ec || p.group != kGroup) return PW_ERR_SHAPE;
+    if (!p.codes || (p.bits < 16 && (!p.scales || !p.zps))) return PW_ERR_INVALID_ARG;
+    if (!aligned16(p.codes) || (p.bits < 16 && (!aligned16(p.scales) || !aligned16(p.zps)))) return PW_ERR_ALIGN;
+    if (p.layout != PW_LAYOUT_TILED || e.state != PW_STATE_GPU_RESIDENT) return PW_ERR_STATE;
+    if (e.expert >= c.n_experts && p.bits != 16) return PW_ERR_STATE;
+    if (e.desired_bits != 0 && !bits_ok(e.desired_bits)) return PW_ERR_BITS;
+  }
+  if (n) {
+    const int slot = ctx->stage_next;
+    ctx->stage_next = (slot + 1) % pw_ctx::kStageSlots;
+    if (ctx->stage_used[slot]) PW_CUDA_OK(cudaEventSynchronize(ctx->stage_ev[slot]));
+    DevRow* st = ctx->stage[slot];
+    DevRow* dtab = reinterpret_cast<DevRow*>(ctx->base + ctx->ws.table);
+    size_t run_begin = 0;  // entries [run_begin, i) map to consecutive device rows
+    for (size_t i = 0; i < n; ++i) {
+      const pw_table_entry& e = entries[i];
+      DevRow r{};
+      r.codes = e.page.codes;
+      r.scales = reinterpret_cast<const __half*>(e.page.scales);
+      r.zps = reinterpret_cast<const __half*>(e.page.zps);
+      r.rows = e.page.rows;
+      r.cols = e.page.cols;
+      r.bits = e.page.bits;
+      r.valid = 1;
+      st[i] = r;
+      const size_t idx = row_index(ctx, e.layer, e.expert, e.kind);
+      ctx->host_rows[idx] = e;
+      ctx->host_valid[idx] = 1;
+      const bool last = i + 1 == n;
+      const bool contiguous =
+          !last && row_index(ctx, entries[i + 1].layer, entries[i + 1].expert, entries[i + 1].kind) == idx + 1;
+      if (!contiguous) {
+        const size_t first = idx - (i - run_begin);
+        PW_CUDA_OK(cudaMemcpyAsync(dtab + first, st + run_begin, sizeof(DevRow) * (i + 1 - run_begin),
+                                   cudaMemcpyHostToDevice, stream));
+        run_begin = i + 1;
+      }
+    }
+    PW_CUDA_OK(cudaEventRecord(ctx->stage_ev[slot], stream));
+    ctx->stage_used[slot] = true;
+  }
+  ctx->epoch++;
+  if (epoch_out) *epoch_out = ctx->epoch;
+  return PW_OK;
+}
+
+extern "C" const pw_page_table* pw_get_page_table(pw_ctx* ctx) { return ctx ? &ctx->table_handle : nullptr; }
+
+extern "C" pw_status pw_query_row(pw_ctx* ctx, int layer, int expert, int kind, pw_table_entry* out) {
+  if (!ctx || !out) return PW_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.n_layers || expert < 0 || expert >= ctx->ws.S || kind < 0 || kind > 2)
+    return PW_ERR_INVALID_ARG;
+  const size_t idx = row_index(ctx, layer, expert, kind);
+  if (!ctx->host_valid[idx]) return PW_ERR_STATE;
+  *out = ctx->host_rows[idx];
+  return PW_OK;
+}
+
+extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int top_k,
+                                    const pw_page_table* table, float* out, pw_mode mode, pw_stream stream) {
+  if (!ctx || !hidden || !logits || !out) return PW_ERR_INVALID_ARG;
+  const pw_config& c = ctx->cfg;
+  if (table && table->owner != ctx) return PW_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c.n_layers || T < 1 || T > c.max_tokens || top_k < 1 || top_k > c.max_top_k ||
+      top_k > c.n_experts)
+    return PW_ERR_INVALID_ARG;
+  if (mode != PW_MODE_AUTO && mode != PW_MODE_SIMT && mode != PW_MODE_TENSOR) return PW_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(logits) || !aligned16(out)) return PW_ERR_ALIGN;
+  for (int e = 0; e < ctx->ws.S; ++e)
+    for (int u = 0; u < 3; ++u)
+      if (!ctx->host_valid[row_index(ctx, layer, e, u)]) return PW_ERR_STATE;
+
+  if (mode == PW_MODE_AUTO) {
+    // a handful of tokens per expert at most: the CUDA-core kernel streams the pages once and is done
+    const long long pairs = (long long)T * top_k;
+    mode = (pairs <= 8 && c.n_shared == 0) ? PW_MODE_SIMT : PW_MODE_TENSOR;
+  }
+  int nt_tile = 0, ksplit = 1;
+  if (mode == PW_MODE_TENSOR) {
+    nt_tile = tensor_token_tile(ctx, T, top_k);
+    // split the down projection's contraction until there are a few units per SM
+    const int R = T * top_k + c.n_shared * T;
+    const int active = ctx->ws.S < R ? ctx->ws.S : R;
+    const long long tiles = (long long)active * ((R / active + nt_tile - 1) / nt_tile) * (c.hidden / kTileRows);
+    long long want = (4ll * ctx->num_sms + tiles - 1) / tiles;
+    const int ng = c.ffn / kGroup;
+    if (want > 8) want = 8;
+    if (want > ng) want = ng;
+    if (want < 1) want = 1;
+    while (want > 1 && (size_t)want * R > ctx->ws.y_slots) --want;
+    ksplit = (int)want;
+  }
+  pw_status st = launch_route(ctx, layer, hidden, logits, T, top_k, nt_tile, ksplit, stream);
+  if (st != PW_OK) return st;
+  st = mode == PW_MODE_SIMT ? launch_ffn_simt(ctx, layer, T, top_k, stream)
+                            : launch_ffn_tensor(ctx, layer, T, top_k, nt_tile, ksplit, stream);
+  if (st != PW_OK) return st;
+  st = launch_combine(ctx, T, top_k, ksplit, out, stream);
+  ctx->last_T = T;
+  ctx->last_k = top_k;
+  return st;
+}
+
+extern "C" pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
+                                    int32_t* perm, pw_stream stream) {
+  if (!ctx) return PW_ERR_INVALID_ARG;
+  if (ctx->last_T == 0) return PW_ERR_STATE;
+  const size_t P = (size_t)ctx->last_T * ctx->last_k;
+  const int E = ctx->cfg.n_experts;
+  char* b = ctx->base;
+  const WsMap& w = ctx->ws;
+  if (topk_ids) PW_CUDA_OK(cudaMemcpyAsync(topk_ids, b + w.topk_ids, 4 * P, cudaMemcpyDeviceToDevice, stream));
+  if (gates) PW_CUDA_OK(cudaMemcpyAsync(gates, b + w.gates, 4 * P, cudaMemcpyDeviceToDevice, stream));
+  if (counts) PW_CUDA_OK(cudaMemcpyAsync(counts, b + w.counts, 4 * (size_t)E, cudaMemcpyDeviceToDevice, stream));
+  if (offsets) PW_CUDA_OK(cudaMemcpyAsync(offsets, b + w.offsets, 4 * (size_t)(E + 1), cudaMemcpyDeviceToDevice, stream));
+  if (perm) PW_CUDA_OK(cudaMemcpyAsync(perm, b + w.perm, 4 * P, cudaMemcpyDeviceToDevice, stream));
+  return PW_OK;
+}
+
+extern "C" pw_status pw_last_device_status(pw_ctx* ctx) {
+  if (!ctx) return PW_ERR_INVALID_ARG;
+  int32_t v = 0;
+  PW_CUDA_OK(cudaDeviceSynchronize());
+  PW_CUDA_OK(cudaMemcpy(&v, ctx->base + ctx->ws.status, 4, cudaMemcpyDeviceToHost));
+  if (v != 0) {
+    PW_CUDA_OK(cudaMemset(ctx->base + ctx->ws.status, 0, 4));
+  }
+  return (pw_status)v;
+}
+
+extern "C" uint64_t pw_launch_count(pw_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" const char* pw_status_str(pw_status s) {
+  switch (s) {
+    case PW_OK: return "ok";
+    case PW_ERR_INVALID_ARG: return "invalid argument";
+    case PW_ERR_SHAPE: return "bad shape";
+    case PW_ERR_BITS: return "bad bitwidth";
+    case PW_ERR_ALIGN: return "misaligned pointer";
+    case PW_ERR_STATE: return "bad state";
+    case PW_ERR_NOMEM: return "workspace too small";
+    case PW_ERR_CUDA: return "CUDA error";
+    case PW_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown";
+}

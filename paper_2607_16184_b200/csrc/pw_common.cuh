@@ -1,0 +1,115 @@
+// Shared declarations of the library's translation units (host object, device table row,
+// workspace map, launch helpers).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/pw.h"
+
+namespace pw {
+
+constexpr int kGroup = 128;      // weights per quantization group
+constexpr int kTileRows = 128;   // rows of one page tile
+constexpr int kPadRows = 256;    // zero rows appended to the token-major operand buffers
+
+// One row of the device-resident page table (48 bytes).
+struct DevRow {
+  const void* codes;
+  const __half* scales;
+  const __half* zps;
+  uint32_t rows, cols;
+  uint32_t bits;
+  uint32_t valid;
+  uint64_t pad_;
+};
+static_assert(sizeof(DevRow) == 48, "DevRow layout");
+
+// One unit of work of the tensor-core FFN kernels.
+struct Unit {
+  int32_t seg;       // segment index: routed expert e, or E + s for shared expert s
+  int32_t row_tile;  // 128-row tile of the weight block
+  int32_t tok0;      // first operand row of the token tile (absolute row in Xt / Ht)
+  int32_t ntok;      // valid tokens in the tile
+  int32_t g0, g1;    // group range [g0, g1) of the contraction
+  int32_t split;     // split-K slot the partial result goes to
+  int32_t pad_;
+};
+
+// Offsets (bytes) of everything that lives in the caller's workspace.
+struct WsMap {
+  size_t status;      // int32[64]
+  size_t counter;     // int32[64]  dynamic work counters
+  size_t table;       // DevRow[n_layers * S * 3]
+  size_t topk_ids;    // int32[Tmax * kmax]
+  size_t gates;       // float[Tmax * kmax]
+  size_t counts;      // int32[S]
+  size_t offsets;     // int32[S + 1]   (absolute operand rows; shared segments follow the routed pairs)
+  size_t perm;        // int32[Pmax]
+  size_t inv_perm;    // int32[Pmax]
+  size_t row_token;   // int32[Rpad]    operand row -> token (-1 for padding)
+  size_t seg_order;   // int32[S]
+  size_t units_gu;    // Unit[max_units]
+  size_t units_dn;    // Unit[max_units]
+  size_t n_units;     // int32[4]
+  size_t xt;          // fp16 operand rows, k-chunk major: [H/8][Rpad][8]
+  size_t ht;          // fp16 SwiGLU output,  k-chunk major: [F/8][Rpad][8]
+  size_t y;           // float [y_slots][H]  split-K partial outputs of the down projection
+  size_t total;
+  // derived sizes
+  int S;              // segments = E + n_shared
+  int Rmax;           // max operand rows = Tmax*kmax + n_shared*Tmax
+  int Rpad;           // Rmax + kPadRows
+  int max_units;
+  size_t y_slots;     // rows of the y buffer (split * R must fit)
+};
+
+WsMap make_wsmap(const pw_config& c);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace pw
+
+struct pw_page_table {
+  pw_ctx* owner;
+};
+
+struct pw_ctx {
+  pw_config cfg;
+  pw::WsMap ws;
+  char* base;                     // cfg.workspace
+  pw_page_table table_handle;
+  pw_table_entry* host_rows;      // mirror of the committed table
+  uint8_t* host_valid;
+  uint64_t epoch;
+  // pinned staging ring for table updates
+  static constexpr int kStageSlots = 8;
+  pw::DevRow* stage[kStageSlots];
+  size_t stage_rows;
+  cudaEvent_t stage_ev[kStageSlots];
+  bool stage_used[kStageSlots];
+  int stage_next;
+  uint64_t launches;
+  int last_T, last_k;
+  int num_sms;
+  void* tc_state;                 // tensor-core path state (set up lazily)
+};
+
+#define PW_CUDA_OK(expr)                                   \
+  do {                                                     \
+    cudaError_t e__ = (expr);                              \
+    if (e__ != cudaSuccess) return PW_ERR_CUDA;            \
+  } while (0)
+
+namespace pw {
+
+// entry points of the other translation units
+pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
+                       int ksplit, cudaStream_t s);
+pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cudaStream_t s);
+pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
+pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
+int tensor_token_tile(const pw_ctx* ctx, int T, int k);
+
+}  // namespace pw

@@ -1,0 +1,202 @@
+// The TILED page layout and the bit-level packing of codes inside it.
+//
+// A page of `rows x cols` at `bits` is cut into tiles of 128 rows x one group (128 columns).
+// Tile (rt, g) is stored contiguously at byte offset (rt * n_groups + g) * bits * 2048 of the
+// codes buffer.  A row of a tile owns bits * 16 bytes = `bits` units of 16 bytes; unit j of row r
+// sits at ((j * 128) + r) * 16 inside the tile, so that the 128 threads of a row-per-thread kernel
+// read unit j with one contiguous 2 KB access.  Scales and zero-points are stored
+// [(rt * n_groups + g) * 128 + r].
+//
+// Inside a row's units the 128 codes are ordered for cheap unpacking to half2 pairs
+// (k, k+1), k even:
+//   16 bits: unit j = fp16 weights k = 8j .. 8j+7.
+//    8 bits: unit j = codes k = 16j .. 16j+15, one per byte, natural order.
+//    4 bits: unit j = codes k = 32j .. 32j+31; word w of it = k0 = 32j + 8w; nibble m (m < 4) holds
+//            k0 + 2m, nibble 4+m holds k0 + 2m + 1.
+//    2 bits: unit j = codes k = 64j .. 64j+63; word w = k0 = 64j + 16w; field m (m < 8) holds
+//            k0 + 2m, field 8+m holds k0 + 2m + 1.
+//    3 bits: units 0, 1 = the low two bits of every code in the 2-bit arrangement; unit 2 = the high
+//            bits: word w = k0 = 32w; bit m (m < 16) holds k0 + 2m, bit 16+m holds k0 + 2m + 1.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+namespace pw {
+
+__host__ __device__ inline size_t tile_code_bytes(int bits) { return (size_t)bits * 2048; }
+
+// ---- integer codes of a 32-weight slice (quarter of a row-group) -----------------------------
+// Slice q (0..3) of a row covers k = 32q .. 32q+31.  Word addresses inside a tile image:
+//   8 bits: units 2q, 2q+1 (8 words)   4 bits: unit q (4 words)
+//   2 bits: unit q/2, words 2(q%2), 2(q%2)+1          3 bits: that, plus unit 2 word q.
+template <int BITS>
+struct SliceWords {
+  static constexpr int kWords = BITS == 16 ? 16 : BITS == 8 ? 8 : BITS == 4 ? 4 : BITS == 3 ? 3 : 2;
+};
+
+// byte offset, inside a tile, of word `i` of slice q of row r
+template <int BITS>
+__host__ __device__ inline int slice_word_offset(int r, int q, int i) {
+  if constexpr (BITS == 16) return ((4 * q + (i >> 2)) * 128 + r) * 16 + (i & 3) * 4;
+  if constexpr (BITS == 8) return ((2 * q + (i >> 2)) * 128 + r) * 16 + (i & 3) * 4;
+  if constexpr (BITS == 4) return (q * 128 + r) * 16 + i * 4;
+  if constexpr (BITS == 2) return ((q >> 1) * 128 + r) * 16 + (2 * (q & 1) + i) * 4;
+  // BITS == 3: i = 0, 1 low-plane words, i = 2 high-plane word
+  if (i < 2) return ((q >> 1) * 128 + r) * 16 + (2 * (q & 1) + i) * 4;
+  return (2 * 128 + r) * 16 + q * 4;
+}
+
+template <int BITS>
+__device__ inline void unpack_slice(const uint32_t* w, int (&code)[32]) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) code[4 * i + j] = (w[i] >> (8 * j)) & 0xff;
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        code[8 * i + 2 * m] = (w[i] >> (4 * m)) & 0xf;
+        code[8 * i + 2 * m + 1] = (w[i] >> (16 + 4 * m)) & 0xf;
+      }
+  } else {  // 2 or 3
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int m = 0; m < 8; ++m) {
+        code[16 * i + 2 * m] = (w[i] >> (2 * m)) & 3;
+        code[16 * i + 2 * m + 1] = (w[i] >> (16 + 2 * m)) & 3;
+      }
+    if constexpr (BITS == 3) {
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        code[2 * m] |= ((w[2] >> m) & 1) << 2;
+        code[2 * m + 1] |= ((w[2] >> (16 + m)) & 1) << 2;
+      }
+    }
+  }
+}
+
+template <int BITS>
+__device__ inline void pack_slice(const int (&code)[32], uint32_t* w) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v |= (uint32_t)code[4 * i + j] << (8 * j);
+      w[i] = v;
+    }
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        v |= (uint32_t)code[8 * i + 2 * m] << (4 * m);
+        v |= (uint32_t)code[8 * i + 2 * m + 1] << (16 + 4 * m);
+      }
+      w[i] = v;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int m = 0; m < 8; ++m) {
+        v |= (uint32_t)(code[16 * i + 2 * m] & 3) << (2 * m);
+        v |= (uint32_t)(code[16 * i + 2 * m + 1] & 3) << (16 + 2 * m);
+      }
+      w[i] = v;
+    }
+    if constexpr (BITS == 3) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        v |= (uint32_t)((code[2 * m] >> 2) & 1) << m;
+        v |= (uint32_t)((code[2 * m + 1] >> 2) & 1) << (16 + m);
+      }
+      w[2] = v;
+    }
+  }
+}
+
+// ---- fast unpack of a whole row-group to half2 pairs (forward kernels) -------------------------
+// out[p] = (weight k = 2p, weight k = 2p + 1), p = 0 .. 63.  `u` are the row's units in order.
+// code -> fp16 via the 0x6400 (= 1024.0) mantissa trick, then one HFMA2 with (scale, zero-point).
+__device__ inline __half2 u32_as_h2(uint32_t x) { return *reinterpret_cast<__half2*>(&x); }
+
+__device__ inline __half2 dq_pair(uint32_t magic_or_code, __half2 s2, __half2 z2) {
+  const __half2 k1024 = u32_as_h2(0x64006400u);
+  return __hfma2(__hsub2(u32_as_h2(magic_or_code), k1024), s2, z2);
+}
+
+// Half h (0 or 1) of a row-group: out[p] = weights (64h + 2p, 64h + 2p + 1), p = 0 .. 31.
+// `row_units` points at unit 0 of the row inside a tile image (shared or global memory); unit j
+// of the same row is kTileRowsStride uint4 further on.
+constexpr int kUnitStride = 128;  // uint4 elements between consecutive units of one row
+
+template <int BITS>
+__device__ __forceinline__ void decode_half(const uint4* row_units, int h, __half2 s2, __half2 z2, __half2* out) {
+  if constexpr (BITS == 16) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint4 u = row_units[(8 * h + j) * kUnitStride];
+      out[4 * j + 0] = u32_as_h2(u.x);
+      out[4 * j + 1] = u32_as_h2(u.y);
+      out[4 * j + 2] = u32_as_h2(u.z);
+      out[4 * j + 3] = u32_as_h2(u.w);
+    }
+  } else if constexpr (BITS == 8) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint4 u = row_units[(4 * h + j) * kUnitStride];
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        out[8 * j + 2 * i] = dq_pair(__byte_perm(w[i], 0x64646464u, 0x4140), s2, z2);
+        out[8 * j + 2 * i + 1] = dq_pair(__byte_perm(w[i], 0x64646464u, 0x4342), s2, z2);
+      }
+    }
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const uint4 u = row_units[(2 * h + j) * kUnitStride];
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+          out[16 * j + 4 * i + m] = dq_pair(((w[i] >> (4 * m)) & 0x000f000fu) | 0x64006400u, s2, z2);
+    }
+  } else if constexpr (BITS == 2) {
+    const uint4 u = row_units[h * kUnitStride];
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+        out[8 * i + m] = dq_pair(((w[i] >> (2 * m)) & 0x00030003u) | 0x64006400u, s2, z2);
+  } else {  // 3 bits: low planes in unit h, high-plane words 2h, 2h+1 of unit 2
+    const uint4 u = row_units[h * kUnitStride];
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    const uint2 hv = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + 2 * kUnitStride) + 2 * h);
+    const uint32_t wh[2] = {hv.x, hv.y};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int m = 0; m < 8; ++m) {
+        const int p = 8 * i + m;                 // pair index inside the half
+        const int hb = p & 15;                   // pair index inside its high-plane word
+        const uint32_t hw = wh[p >> 4];
+        const uint32_t hi = hb >= 2 ? (hw >> (hb - 2)) : (hw << (2 - hb));
+        const uint32_t lo = (w[i] >> (2 * m)) & 0x00030003u;
+        out[p] = dq_pair((hi & 0x00040004u) | lo | 0x64006400u, s2, z2);
+      }
+  }
+}
+
+}  // namespace pw

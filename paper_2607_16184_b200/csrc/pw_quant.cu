@@ -1,0 +1,369 @@
+// Group-wise quantize / demote of a linear-block into a weight page, and the TILED <-> CANONICAL
+// layout conversions.  One CTA per (128-row, one-group) tile, four threads per row, each owning a
+// 32-weight slice; HBM-bound: reads the source once, writes the page once.
+#include "pw_common.cuh"
+#include "pw_layout.cuh"
+
+namespace pw {
+
+enum SrcKind { SRC_RAW = 0, SRC_TILED = 1 };
+
+// The fp16 weight a stored code stands for, bit for bit: fp32 product (exact), fp32 add, one
+// rounding to fp16.
+__device__ __forceinline__ float dequant_exact(int code, float s, float z) {
+  return __half2float(__float2half_rn(__fadd_rn(__fmul_rn((float)code, s), z)));
+}
+
+
+// Words of slice q of row r of a tile image, fetched with the widest loads the layout allows.
+template <int BITS>
+__device__ __forceinline__ void load_slice_words(const char* tb, int r, int q, uint32_t* w) {
+  if constexpr (BITS == 16 || BITS == 8 || BITS == 4) {
+    constexpr int NU = BITS == 16 ? 4 : BITS == 8 ? 2 : 1;
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+      const uint4 u = __ldg(reinterpret_cast<const uint4*>(tb + slice_word_offset<BITS>(r, q, 4 * i)));
+      w[4 * i] = u.x;
+      w[4 * i + 1] = u.y;
+      w[4 * i + 2] = u.z;
+      w[4 * i + 3] = u.w;
+    }
+  } else {
+    const uint2 u = __ldg(reinterpret_cast<const uint2*>(tb + slice_word_offset<BITS>(r, q, 0)));
+    w[0] = u.x;
+    w[1] = u.y;
+    if constexpr (BITS == 3) w[2] = __ldg(reinterpret_cast<const uint32_t*>(tb + slice_word_offset<3>(r, q, 2)));
+  }
+}
+
+template <int SRC_KIND, int SRC_BITS, int DST_BITS>
+__global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict__ src_codes,
+                                                         const __half* __restrict__ src_scales,
+                                                         const __half* __restrict__ src_zps, uint32_t cols,
+                                                         void* __restrict__ dst_codes, __half* __restrict__ dst_scales,
+                                                         __half* __restrict__ dst_zps) {
+  const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
+  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
+  const size_t tile = (size_t)rt * ng + g;
+
+  float v[32];
+  if constexpr (SRC_KIND == SRC_RAW) {
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(src_codes) +
+                                                    ((size_t)rt * kTileRows + r) * cols + (size_t)g * kGroup + 32 * q);
+    uint4 u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) u[i] = __ldg(p + i);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __half2* h = reinterpret_cast<const __half2*>(&u[i]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float2 f = __half22float2(h[j]);
+        v[8 * i + 2 * j] = f.x;
+        v[8 * i + 2 * j + 1] = f.y;
+      }
+    }
+  } else {
+    const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_code_bytes(SRC_BITS);
+    constexpr int NW = SliceWords<SRC_BITS>::kWords;
+    uint32_t w[NW];
+    load_slice_words<SRC_BITS>(tb, r, q, w);
+    if constexpr (SRC_BITS == 16) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        float2 f = __half22float2(u32_as_h2(w[i]));
+        v[2 * i] = f.x;
+        v[2 * i + 1] = f.y;
+      }
+    } else {
+      int code[32];
+      unpack_slice<SRC_BITS>(w, code);
+      const float s = __half2float(src_scales[tile * kTileRows + r]);
+      const float z = __half2float(src_zps[tile * kTileRows + r]);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = dequant_exact(code[i], s, z);
+    }
+  }
+
+  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_code_bytes(DST_BITS);
+  if constexpr (DST_BITS == 16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint4 o;
+      __half2* h = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
+      *reinterpret_cast<uint4*>(db + slice_word_offset<16>(r, q, 4 * i)) = o;
+    }
+    return;
+  }
+
+  float lo = v[0], hi = v[0];
+#pragma unroll
+  for (int i = 1; i < 32; ++i) {
+    lo = fminf(lo, v[i]);
+    hi = fmaxf(hi, v[i]);
+  }
+#pragma unroll
+  for (int d = 1; d <= 2; d <<= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+  }
+  if (lo == 0.0f) lo = 0.0f;  // store -0 as +0
+  constexpr int L = (1 << DST_BITS) - 1;
+  const float rng = __fsub_rn(hi, lo);
+  __half sh;
+  if (rng == 0.0f) {
+    sh = __ushort_as_half((unsigned short)0x3c00);
+  } else {
+    sh = __float2half_rn(__fdiv_rn(rng, (float)L));
+    if ((__half_as_ushort(sh) & 0x7fff) == 0) sh = __ushort_as_half((unsigned short)0x0001);
+  }
+  const float rinv = __fdiv_rn(1.0f, __half2float(sh));
+  int code[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float c = rintf(__fmul_rn(__fsub_rn(v[i], lo), rinv));
+    c = fminf(fmaxf(c, 0.0f), (float)L);
+    code[i] = (int)c;
+  }
+  constexpr int NW = SliceWords<DST_BITS>::kWords;
+  uint32_t w[NW];
+  pack_slice<DST_BITS>(code, w);
+  if constexpr (DST_BITS == 8) {
+    *reinterpret_cast<uint4*>(db + slice_word_offset<8>(r, q, 0)) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(db + slice_word_offset<8>(r, q, 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+  } else if constexpr (DST_BITS == 4) {
+    *reinterpret_cast<uint4*>(db + slice_word_offset<4>(r, q, 0)) = make_uint4(w[0], w[1], w[2], w[3]);
+  } else {
+    *reinterpret_cast<uint2*>(db + slice_word_offset<DST_BITS>(r, q, 0)) = make_uint2(w[0], w[1]);
+    if constexpr (DST_BITS == 3) *reinterpret_cast<uint32_t*>(db + slice_word_offset<3>(r, q, 2)) = w[2];
+  }
+  if (q == 0) {
+    dst_scales[tile * kTileRows + r] = sh;
+    dst_zps[tile * kTileRows + r] = __float2half_rn(lo);
+  }
+}
+
+// TILED -> CANONICAL (EXPORT = true) or CANONICAL -> TILED, same bitwidth.
+template <int BITS, bool EXPORT>
+__global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ src_codes,
+                                                       const __half* __restrict__ src_scales,
+                                                       const __half* __restrict__ src_zps, uint32_t cols,
+                                                       void* __restrict__ dst_codes, __half* __restrict__ dst_scales,
+                                                       __half* __restrict__ dst_zps) {
+  const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
+  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
+  const size_t tile = (size_t)rt * ng + g;
+  const size_t row = (size_t)rt * kTileRows + r;
+  const size_t elem = row * cols + (size_t)g * kGroup + 32 * q;   // first element of the slice
+  constexpr int NW = SliceWords<BITS>::kWords;
+  // canonical side: the slice is BITS words of the bit stream (fp16: 16 words of the matrix)
+  const char* csrc = reinterpret_cast<const char*>(EXPORT ? dst_codes : src_codes);
+  char* cpos = const_cast<char*>(csrc) + elem * BITS / 8;
+  const char* tsrc = reinterpret_cast<const char*>(EXPORT ? src_codes : dst_codes);
+  char* tpos = const_cast<char*>(tsrc) + tile * tile_code_bytes(BITS);
+
+  uint32_t w[NW];
+  if constexpr (EXPORT) {
+#pragma unroll
+    for (int i = 0; i < NW; ++i) w[i] = *reinterpret_cast<const uint32_t*>(tpos + slice_word_offset<BITS>(r, q, i));
+    if constexpr (BITS == 16) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) reinterpret_cast<uint32_t*>(cpos)[i] = w[i];
+    } else {
+      int code[32];
+      unpack_slice<BITS>(w, code);
+      unsigned long long acc = 0;
+      int nb = 0, wi = 0;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        acc |= (unsigned long long)code[i] << nb;
+        nb += BITS;
+        if (nb >= 32) {
+          reinterpret_cast<uint32_t*>(cpos)[wi++] = (uint32_t)acc;
+          acc >>= 32;
+          nb -= 32;
+        }
+      }
+    }
+  } else {
+    if constexpr (BITS == 16) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) w[i] = reinterpret_cast<const uint32_t*>(cpos)[i];
+    } else {
+      int code[32];
+      unsigned long long acc = 0;
+      int nb = 0, wi = 0;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        if (nb < BITS) {
+          acc |= (unsigned long long)reinterpret_cast<const uint32_t*>(cpos)[wi++] << nb;
+          nb += 32;
+        }
+        code[i] = (int)(acc & ((1u << BITS) - 1));
+        acc >>= BITS;
+        nb -= BITS;
+      }
+      pack_slice<BITS>(code, w);
+    }
+#pragma unroll
+    for (int i = 0; i < NW; ++i) *reinterpret_cast<uint32_t*>(tpos + slice_word_offset<BITS>(r, q, i)) = w[i];
+  }
+  if (BITS < 16 && q == 0) {
+    const size_t ci = row * ng + g, ti = tile * kTileRows + r;
+    if constexpr (EXPORT) {
+      dst_scales[ci] = src_scales[ti];
+      dst_zps[ci] = src_zps[ti];
+    } else {
+      dst_scales[ti] = src_scales[ci];
+      dst_zps[ti] = src_zps[ci];
+    }
+  }
+}
+
+static bool bits_ok(int b) { return b == 16 || b == 8 || b == 4 || b == 3 || b == 2; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static pw_status check_page_buffers(const pw_page* p, int bits) {
+  if (!p->codes) return PW_ERR_INVALID_ARG;
+  if (!aligned16(p->codes)) return PW_ERR_ALIGN;
+  if (bits < 16) {
+    if (!p->scales || !p->zps) return PW_ERR_INVALID_ARG;
+    if (!aligned16(p->scales) || !aligned16(p->zps)) return PW_ERR_ALIGN;
+  }
+  return PW_OK;
+}
+
+template <int SK, int SB>
+static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void* sc, const __half* ss, const __half* sz,
+                             uint32_t cols, pw_page* d) {
+  __half* ds = reinterpret_cast<__half*>(d->scales);
+  __half* dz = reinterpret_cast<__half*>(d->zps);
+  switch (dst_bits) {
+    case 16:
+      if (SK == SRC_RAW) quant_tile_kernel<SK, SB, 16><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      break;
+    case 8:
+      if (SB > 8) quant_tile_kernel<SK, SB, (SB > 8 ? 8 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      break;
+    case 4:
+      if (SB > 4) quant_tile_kernel<SK, SB, (SB > 4 ? 4 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      break;
+    case 3:
+      if (SB > 3) quant_tile_kernel<SK, SB, (SB > 3 ? 3 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      break;
+    case 2:
+      quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      break;
+  }
+}
+
+}  // namespace pw
+
+using namespace pw;
+
+extern "C" size_t pw_page_bytes(uint32_t rows, uint32_t cols, int bits, int group, size_t* codes_b, size_t* scales_b,
+                                size_t* zps_b) {
+  if (!bits_ok(bits) || group != kGroup || rows == 0 || cols == 0 || cols % kGroup != 0) return 0;
+  const size_t n = (size_t)rows * cols;
+  const size_t cb = bits == 16 ? 2 * n : n * (size_t)bits / 8;
+  const size_t sb = bits == 16 ? 0 : 2 * (n / kGroup);
+  if (codes_b) *codes_b = cb;
+  if (scales_b) *scales_b = sb;
+  if (zps_b) *zps_b = sb;
+  return cb + 2 * sb;
+}
+
+extern "C" pw_status pw_quantize_block(pw_ctx* ctx, const void* w, uint32_t rows, uint32_t cols, int bits, pw_page* dst,
+                                       pw_stream stream) {
+  if (!ctx || !w || !dst) return PW_ERR_INVALID_ARG;
+  if (!bits_ok(bits)) return PW_ERR_BITS;
+  if (rows == 0 || cols == 0 || rows % kTileRows != 0 || cols % kGroup != 0) return PW_ERR_SHAPE;
+  if (!aligned16(w)) return PW_ERR_ALIGN;
+  pw_status st = check_page_buffers(dst, bits);
+  if (st != PW_OK) return st;
+  dst->rows = rows;
+  dst->cols = cols;
+  dst->group = kGroup;
+  dst->bits = (uint8_t)bits;
+  dst->layout = PW_LAYOUT_TILED;
+  dim3 grid(cols / kGroup, rows / kTileRows);
+  launch_quant_dst<SRC_RAW, 16>(bits, grid, stream, w, nullptr, nullptr, cols, dst);
+  ctx->launches++;
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
+extern "C" pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bits, pw_page* dst, pw_stream stream) {
+  if (!ctx || !src || !dst) return PW_ERR_INVALID_ARG;
+  if (!bits_ok(src->bits) || !bits_ok(dst_bits) || dst_bits >= src->bits) return PW_ERR_BITS;
+  if (src->layout != PW_LAYOUT_TILED) return PW_ERR_STATE;
+  if (src->rows == 0 || src->cols == 0 || src->rows % kTileRows != 0 || src->cols % kGroup != 0 ||
+      src->group != kGroup)
+    return PW_ERR_SHAPE;
+  pw_status st = check_page_buffers(src, src->bits);
+  if (st != PW_OK) return st;
+  st = check_page_buffers(dst, dst_bits);
+  if (st != PW_OK) return st;
+  if (dst->codes == src->codes) return PW_ERR_INVALID_ARG;  // a demote is out of place
+  dst->rows = src->rows;
+  dst->cols = src->cols;
+  dst->group = kGroup;
+  dst->bits = (uint8_t)dst_bits;
+  dst->layout = PW_LAYOUT_TILED;
+  dim3 grid(src->cols / kGroup, src->rows / kTileRows);
+  const __half* ss = reinterpret_cast<const __half*>(src->scales);
+  const __half* sz = reinterpret_cast<const __half*>(src->zps);
+  switch (src->bits) {
+    case 16: launch_quant_dst<SRC_TILED, 16>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
+    case 8: launch_quant_dst<SRC_TILED, 8>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
+    case 4: launch_quant_dst<SRC_TILED, 4>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
+    case 3: launch_quant_dst<SRC_TILED, 3>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
+  }
+  ctx->launches++;
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
+template <bool EXPORT>
+static pw_status relayout(pw_ctx* ctx, const pw_page* src, pw_page* dst, cudaStream_t stream) {
+  if (!ctx || !src || !dst) return PW_ERR_INVALID_ARG;
+  if (!bits_ok(src->bits)) return PW_ERR_BITS;
+  if (src->layout != (EXPORT ? PW_LAYOUT_TILED : PW_LAYOUT_CANONICAL)) return PW_ERR_STATE;
+  if (src->rows == 0 || src->cols == 0 || src->rows % kTileRows != 0 || src->cols % kGroup != 0 ||
+      src->group != kGroup)
+    return PW_ERR_SHAPE;
+  pw_status st = check_page_buffers(src, src->bits);
+  if (st != PW_OK) return st;
+  st = check_page_buffers(dst, src->bits);
+  if (st != PW_OK) return st;
+  if (dst->codes == src->codes) return PW_ERR_INVALID_ARG;
+  dst->rows = src->rows;
+  dst->cols = src->cols;
+  dst->group = kGroup;
+  dst->bits = src->bits;
+  dst->layout = EXPORT ? PW_LAYOUT_CANONICAL : PW_LAYOUT_TILED;
+  dim3 grid(src->cols / kGroup, src->rows / kTileRows);
+  const __half* ss = reinterpret_cast<const __half*>(src->scales);
+  const __half* sz = reinterpret_cast<const __half*>(src->zps);
+  __half* ds = reinterpret_cast<__half*>(dst->scales);
+  __half* dz = reinterpret_cast<__half*>(dst->zps);
+  switch (src->bits) {
+    case 16: relayout_kernel<16, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+    case 8: relayout_kernel<8, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+    case 4: relayout_kernel<4, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+    case 3: relayout_kernel<3, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+    case 2: relayout_kernel<2, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+  }
+  ctx->launches++;
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
+extern "C" pw_status pw_export_page(pw_ctx* ctx, const pw_page* src, pw_page* dst, pw_stream stream) {
+  return relayout<true>(ctx, src, dst, stream);
+}
+extern "C" pw_status pw_import_page(pw_ctx* ctx, const pw_page* src, pw_page* dst, pw_stream stream) {
+  return relayout<false>(ctx, src, dst, stream);
+}

@@ -1,0 +1,287 @@
+// Token router (top-k + renormalised softmax gates), stable grouping of (token, slot) pairs into
+// per-expert segments, operand gather, work-unit lists, and the gate-weighted combine.
+#include "pw_common.cuh"
+
+namespace pw {
+
+constexpr int kMaxExpertsPerLane = 8;  // E <= 256
+
+// One warp per token.  Slot j holds the j-th largest logit; equal logits: lower expert index first.
+__global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ logits, int T, int E, int k,
+                                                     int32_t* __restrict__ topk_ids, float* __restrict__ gates) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= T) return;
+  const float* l = logits + (size_t)warp * E;
+  float v[kMaxExpertsPerLane];
+#pragma unroll
+  for (int i = 0; i < kMaxExpertsPerLane; ++i) {
+    const int e = lane + 32 * i;
+    v[i] = e < E ? l[e] : -INFINITY;
+  }
+  uint32_t taken = 0;
+  float l0 = 0.f, S = 0.f, myp = 0.f;
+  int myid = 0;
+  for (int j = 0; j < k; ++j) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+#pragma unroll
+    for (int i = 0; i < kMaxExpertsPerLane; ++i) {
+      const int e = lane + 32 * i;
+      const bool ok = e < E && !((taken >> i) & 1u);
+      if (ok && (v[i] > bv || (v[i] == bv && e < bi))) {
+        bv = v[i];
+        bi = e;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+      if (ov > bv || (ov == bv && oi < bi)) {
+        bv = ov;
+        bi = oi;
+      }
+    }
+    if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+    if (j == 0) l0 = bv;
+    const float p = expf(__fsub_rn(bv, l0));
+    S = __fadd_rn(S, p);  // summed in slot order, identically on every lane
+    if (lane == j) {
+      myp = p;
+      myid = bi;
+    }
+  }
+  // k <= 32: lane j owns slot j
+  if (lane < k) {
+    topk_ids[(size_t)warp * k + lane] = myid;
+    gates[(size_t)warp * k + lane] = __fdiv_rn(myp, S);
+  }
+}
+
+// Single CTA.  Stable counting sort of the P = T*k pairs by expert (positions come from ordered
+// prefix counts, never from atomics), segment table including the shared experts, operand-row ->
+// token map, and the unit lists of the tensor-core kernels.
+__global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict__ topk_ids, int T, int k, int E,
+                                                       int n_shared, int32_t* __restrict__ counts,
+                                                       int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
+                                                       int32_t* __restrict__ inv_perm,
+                                                       int32_t* __restrict__ row_token, int32_t* __restrict__ counter,
+                                                       const DevRow* __restrict__ rows, int H, int F, int nt_tile,
+                                                       int ksplit, Unit* __restrict__ units_gu,
+                                                       Unit* __restrict__ units_dn, int32_t* __restrict__ n_units,
+                                                       int32_t* __restrict__ seg_order, int max_units,
+                                                       int32_t* __restrict__ status) {
+  extern __shared__ int32_t sm[];
+  const int S = E + n_shared;
+  int32_t* cnt = sm;                 // [S]
+  int32_t* off = cnt + S;            // [S + 1]
+  int32_t* run = off + S + 1;        // [E]   pairs of expert e placed so far
+  int32_t* wcnt = run + E;           // [32][E]
+  int32_t* ubase = wcnt + 32 * E;    // [S + 1] unit prefix (gate/up), reused for down
+  int32_t* order = ubase + S + 1;    // [S]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = T * k;
+
+  for (int e = tid; e < S; e += blockDim.x) cnt[e] = e < E ? 0 : T;
+  for (int e = tid; e < E; e += blockDim.x) run[e] = 0;
+  if (tid < 64) counter[tid] = 0;
+  __syncthreads();
+  for (int p = tid; p < P; p += blockDim.x) atomicAdd(&cnt[topk_ids[p]], 1);
+  __syncthreads();
+  if (tid == 0) {
+    int a = 0;
+    for (int e = 0; e < S; ++e) {
+      off[e] = a;
+      a += cnt[e];
+    }
+    off[S] = a;
+  }
+  __syncthreads();
+  for (int e = tid; e < S; e += blockDim.x) counts[e] = cnt[e];
+  for (int e = tid; e <= S; e += blockDim.x) offsets[e] = off[e];
+
+  for (int base = 0; base < P; base += blockDim.x) {
+    for (int i = tid; i < 32 * E; i += blockDim.x) wcnt[i] = 0;
+    __syncthreads();
+    const int p = base + tid;
+    const int e = p < P ? topk_ids[p] : -1;
+    const uint32_t same = __match_any_sync(0xffffffffu, e);
+    const int rank = __popc(same & ((1u << lane) - 1u));
+    if (e >= 0 && rank == 0) wcnt[warp * E + e] = __popc(same);
+    __syncthreads();
+    for (int x = tid; x < E; x += blockDim.x) {
+      int a = run[x];
+      for (int w = 0; w < 32; ++w) {
+        const int c = wcnt[w * E + x];
+        wcnt[w * E + x] = a;
+        a += c;
+      }
+      run[x] = a;
+    }
+    __syncthreads();
+    if (e >= 0) {
+      const int pos = off[e] + wcnt[warp * E + e] + rank;
+      perm[pos] = p;
+      inv_perm[p] = pos;
+      row_token[pos] = p / k;
+    }
+    __syncthreads();
+  }
+  const int R = off[S];
+  for (int i = tid; i < n_shared * T; i += blockDim.x) row_token[P + i] = i % T;
+  for (int i = tid; i < kPadRows; i += blockDim.x) row_token[R + i] = -1;
+
+  if (nt_tile <= 0) return;  // SIMT path: no unit lists
+
+  // Segments ordered by the bytes of their gate+up (resp. down) pages, largest first, so that the
+  // dynamically scheduled CTAs finish together.  Rank by counting (S is small).
+  for (int phase = 0; phase < 2; ++phase) {
+    __syncthreads();
+    for (int s = tid; s < S; s += blockDim.x) {
+      const uint32_t mine = phase == 0 ? rows[s * 3].bits + rows[s * 3 + 1].bits : rows[s * 3 + 2].bits;
+      int rk = 0;
+      for (int o = 0; o < S; ++o) {
+        const uint32_t other = phase == 0 ? rows[o * 3].bits + rows[o * 3 + 1].bits : rows[o * 3 + 2].bits;
+        rk += (other > mine) || (other == mine && o < s);
+      }
+      order[rk] = s;
+    }
+    __syncthreads();
+    const int row_tiles = (phase == 0 ? F : H) / kTileRows;
+    const int ng = (phase == 0 ? H : F) / kGroup;
+    const int splits = phase == 0 ? 1 : ksplit;
+    if (tid == 0) {
+      int a = 0;
+      for (int i = 0; i < S; ++i) {
+        ubase[i] = a;
+        const int n = cnt[order[i]];
+        a += ((n + nt_tile - 1) / nt_tile) * row_tiles * splits;
+      }
+      ubase[S] = a;
+      n_units[phase] = a <= max_units ? a : 0;
+      if (a > max_units) atomicMax(status, (int)PW_ERR_NOMEM);
+    }
+    __syncthreads();
+    if (ubase[S] > max_units) continue;
+    Unit* out = phase == 0 ? units_gu : units_dn;
+    if (phase == 0)
+      for (int i = tid; i < S; i += blockDim.x) seg_order[i] = order[i];
+    for (int i = 0; i < S; ++i) {
+      const int s = order[i];
+      const int n = cnt[s];
+      const int tt = (n + nt_tile - 1) / nt_tile;
+      const int total = tt * row_tiles * splits;
+      // order: row tile, then split, then token tile (innermost: tiles that share weights run together)
+      for (int u = tid; u < total; u += blockDim.x) {
+        const int ti = u % tt;
+        const int sp = (u / tt) % splits;
+        const int rt = u / (tt * splits);
+        Unit un;
+        un.seg = s;
+        un.row_tile = rt;
+        un.tok0 = off[s] + ti * nt_tile;
+        un.ntok = min(nt_tile, n - ti * nt_tile);
+        un.g0 = (int)(((long long)sp * ng) / splits);
+        un.g1 = (int)(((long long)(sp + 1) * ng) / splits);
+        un.split = sp;
+        un.pad_ = 0;
+        out[ubase[i] + u] = un;
+      }
+    }
+  }
+}
+
+// Xt[c][n][0..7] = hidden[row_token[n]][8c .. 8c+7], zero for padding rows.
+__global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
+                                                     const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
+                                                     uint4* __restrict__ xt) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int c = blockIdx.y;
+  const int R = offsets[S];
+  if (n >= R + kPadRows) return;
+  const int t = row_token[n];
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (t >= 0) v = __ldg(hidden + (size_t)t * H8 + c);
+  xt[(size_t)c * Rpad + n] = v;
+}
+
+// out[t] = sum_j gate[t,j] * (sum_s y[s][inv_perm[t*k+j]]) + sum over shared experts (sum_s y[s][row]).
+__global__ void __launch_bounds__(256) combine_kernel(const float4* __restrict__ y, const float* __restrict__ gates,
+                                                      const int32_t* __restrict__ inv_perm, int T, int k, int n_shared,
+                                                      int H4, int ksplit, size_t split_stride4,
+                                                      float4* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = blockIdx.y;
+  if (c >= H4) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j = 0; j < k + n_shared; ++j) {
+    int row;
+    float g;
+    if (j < k) {
+      row = inv_perm[(size_t)t * k + j];
+      g = gates[(size_t)t * k + j];
+    } else {
+      row = T * k + (j - k) * T + t;
+      g = 1.0f;
+    }
+    float4 a = y[(size_t)row * H4 + c];
+    for (int s = 1; s < ksplit; ++s) {
+      const float4 b = y[s * split_stride4 + (size_t)row * H4 + c];
+      a.x = __fadd_rn(a.x, b.x);
+      a.y = __fadd_rn(a.y, b.y);
+      a.z = __fadd_rn(a.z, b.z);
+      a.w = __fadd_rn(a.w, b.w);
+    }
+    acc.x = __fadd_rn(acc.x, __fmul_rn(g, a.x));
+    acc.y = __fadd_rn(acc.y, __fmul_rn(g, a.y));
+    acc.z = __fadd_rn(acc.z, __fmul_rn(g, a.z));
+    acc.w = __fadd_rn(acc.w, __fmul_rn(g, a.w));
+  }
+  out[(size_t)t * H4 + c] = acc;
+}
+
+pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
+                       int ksplit, cudaStream_t s) {
+  const pw_config& c = ctx->cfg;
+  const WsMap& w = ctx->ws;
+  char* b = ctx->base;
+  const int E = c.n_experts, S = w.S;
+  int32_t* ids = reinterpret_cast<int32_t*>(b + w.topk_ids);
+  router_kernel<<<(T * 32 + 255) / 256, 256, 0, s>>>(logits, T, E, k, ids, reinterpret_cast<float*>(b + w.gates));
+  const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + E + 32 * (size_t)E + (S + 1) + S);
+  const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * S * 3;
+  permute_kernel<<<1, 1024, smem, s>>>(
+      ids, T, k, E, c.n_shared, reinterpret_cast<int32_t*>(b + w.counts), reinterpret_cast<int32_t*>(b + w.offsets),
+      reinterpret_cast<int32_t*>(b + w.perm), reinterpret_cast<int32_t*>(b + w.inv_perm),
+      reinterpret_cast<int32_t*>(b + w.row_token), reinterpret_cast<int32_t*>(b + w.counter), rows, c.hidden, c.ffn,
+      nt_tile, ksplit, reinterpret_cast<Unit*>(b + w.units_gu), reinterpret_cast<Unit*>(b + w.units_dn),
+      reinterpret_cast<int32_t*>(b + w.n_units), reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units,
+      reinterpret_cast<int32_t*>(b + w.status));
+  const int R = T * k + c.n_shared * T;
+  dim3 grid((R + kPadRows + 255) / 256, c.hidden / 8);
+  gather_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(hidden),
+                                     reinterpret_cast<const int32_t*>(b + w.row_token),
+                                     reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
+                                     reinterpret_cast<uint4*>(b + w.xt));
+  ctx->launches += 3;
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
+pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cudaStream_t s) {
+  const pw_config& c = ctx->cfg;
+  const WsMap& w = ctx->ws;
+  char* b = ctx->base;
+  const int H4 = c.hidden / 4;
+  const int R = T * k + c.n_shared * T;
+  dim3 grid((H4 + 255) / 256, T);
+  combine_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const float4*>(b + w.y),
+                                      reinterpret_cast<const float*>(b + w.gates),
+                                      reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
+                                      (size_t)R * H4, reinterpret_cast<float4*>(out));
+  ctx->launches += 1;
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
+}  // namespace pw

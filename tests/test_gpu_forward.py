@@ -1,0 +1,189 @@
+"""GPU parity of pw_moe_forward against the oracle: routing bit-exact, outputs within tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_16184_b200 import binding as B
+from paper_2607_16184_b200 import synth
+
+from util_gpu import build_layer, error_metrics, export_to_oracle, import_from_oracle, make_ctx
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_F = 2e-2, 5e-3          # tolerance of the layer output (fp16 operands, fp32 accumulate)
+MODES = [B.PW_MODE_SIMT, B.PW_MODE_TENSOR]
+
+
+def check_routing(ctx, orc, logits, T, k, E):
+    r = {n: v.cpu().numpy() for n, v in ctx.pw_get_routing(T, k).items()}
+    ids, gates = orc.router(logits, k)
+    counts, offsets, perm, _ = orc.permute(ids, E)
+    assert np.array_equal(r["topk_ids"], ids)
+    assert np.array_equal(r["counts"], counts)
+    assert np.array_equal(r["offsets"], offsets)
+    assert np.array_equal(r["perm"], perm)
+    assert np.allclose(r["gates"], gates, rtol=1e-6, atol=1e-9)
+
+
+def run_case(orc, cfg, mode, tokens=None, bits=None, sample_tokens=None):
+    T = tokens or cfg.tokens
+    ctx = make_ctx(cfg, max_tokens=T, n_layers=1)
+    try:
+        pages, bits = build_layer(ctx, cfg, 0, bits)
+        x = synth.activations(cfg, device="cuda", tokens=T)
+        logits = synth.router_logits(cfg, device="cuda", tokens=T)
+        out = ctx.pw_moe_forward(0, x, logits, cfg.top_k, mode=mode)
+        torch.cuda.synchronize()
+        assert ctx.pw_last_device_status() == 0
+        check_routing(ctx, orc, logits.cpu().numpy(), T, cfg.top_k, cfg.n_experts)
+        opages = [export_to_oracle(ctx, p, orc) for p in pages]
+        ref = orc.moe_forward(x.cpu().numpy(), logits.cpu().numpy(), cfg.top_k, opages, n_shared=cfg.n_shared,
+                              tokens=sample_tokens)
+        got = out.cpu().numpy()
+        if sample_tokens is not None:
+            got, ref = got[sample_tokens], ref[sample_tokens]
+        assert np.isfinite(got).all()
+        max_abs, rel_f = error_metrics(got, ref)
+        assert max_abs <= MAX_ABS and rel_f <= REL_F, (max_abs, rel_f)
+        return max_abs, rel_f
+    finally:
+        ctx.close()
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("name", ["tiny", "tiny_cover"])
+def test_tiny_configs(orc, name, mode):
+    run_case(orc, synth.CONFIGS[name], mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("bits", [16, 8, 4, 3, 2])
+def test_uniform_bitwidth_table(orc, bits, mode):
+    cfg = synth.CONFIGS["tiny"]
+    run_case(orc, cfg, mode, bits=np.full((8, 3), bits, np.int32))
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("T", [1, 3, 17, 130])
+def test_ragged_token_counts(orc, T, mode):
+    run_case(orc, synth.CONFIGS["tiny_cover"], mode, tokens=T)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_shared_experts_and_many_experts(orc, mode):
+    cfg = synth.LayerConfig("fg_small", 64, 6, 256, 384, 96, n_shared=2, routing="zipf", zipf_a=1.2,
+                            bit_rule="int4_10fp16_20int2")
+    run_case(orc, cfg, mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_gate_and_up_sharing_one_bitwidth(orc, mode):
+    # the paper's block types are {gate_up, down}: gate and up of an expert always at the same bitwidth
+    cfg = synth.CONFIGS["tiny"]
+    rng = np.random.default_rng(3)
+    gu = rng.choice(synth.BITS, size=8)
+    dn = rng.choice(synth.BITS, size=8)
+    run_case(orc, cfg, mode, bits=np.stack([gu, gu, dn], axis=1).astype(np.int32))
+
+
+def test_forward_from_imported_oracle_pages(orc):
+    cfg = synth.CONFIGS["tiny_cover"]
+    ctx = make_ctx(cfg, n_layers=1)
+    bits = synth.assign_bits(cfg)
+    opages, entries, keep = [], [], []
+    for e in range(8):
+        for u in range(3):
+            op = orc.quantize_block(synth.block_weights(cfg, 0, e, u).numpy(), int(bits[e, u]))
+            opages.append(op)
+            keep.append(import_from_oracle(ctx, op))
+            entries.append((0, e, u, keep[-1]))
+    ctx.pw_set_page_table(entries)
+    x = synth.activations(cfg, device="cuda")
+    logits = synth.router_logits(cfg, device="cuda")
+    out = ctx.pw_moe_forward(0, x, logits, cfg.top_k, mode=B.PW_MODE_SIMT).cpu().numpy()
+    ref = orc.moe_forward(x.cpu().numpy(), logits.cpu().numpy(), cfg.top_k, opages)
+    max_abs, rel_f = error_metrics(out, ref)
+    assert max_abs <= MAX_ABS and rel_f <= REL_F
+    ctx.close()
+
+
+def test_router_ties_follow_the_index_rule(orc):
+    cfg = synth.CONFIGS["tiny"]
+    ctx = make_ctx(cfg, max_tokens=64, n_layers=1)
+    build_layer(ctx, cfg, 0, np.full((8, 3), 4, np.int32))
+    x = synth.activations(cfg, device="cuda", tokens=64)
+    logits = torch.round(synth.router_logits(cfg, device="cuda", tokens=64) * 2) / 2     # many exact ties
+    logits[0] = 0.0
+    ctx.pw_moe_forward(0, x, logits.contiguous(), 2, mode=B.PW_MODE_SIMT)
+    check_routing(ctx, orc, logits.cpu().numpy(), 64, 2, 8)
+    ctx.close()
+
+
+def test_commit_is_stream_ordered_and_forward_reads_the_committed_row(orc):
+    # demote one block, publish it between two forward calls: the first call sees the old page,
+    # the second the new one, and tokens not routed to that expert do not change
+    cfg = synth.CONFIGS["tiny"]
+    ctx = make_ctx(cfg, n_layers=1)
+    pages, bits = build_layer(ctx, cfg, 0, np.full((8, 3), 8, np.int32))
+    x = synth.activations(cfg, device="cuda")
+    logits = synth.router_logits(cfg, device="cuda")
+    e0 = ctx.pw_set_page_table([])
+    out_a = ctx.pw_moe_forward(0, x, logits, 2, mode=B.PW_MODE_SIMT)
+    side = torch.cuda.Stream()
+    low = ctx.pw_demote_block(pages[3 * 5 + 2], 2, stream=side)          # expert 5, down, 8 -> 2 on a side stream
+    done = torch.cuda.Event()
+    done.record(side)
+    out_b = ctx.pw_moe_forward(0, x, logits, 2, mode=B.PW_MODE_SIMT)     # still the old row
+    torch.cuda.current_stream().wait_event(done)
+    e1 = ctx.pw_set_page_table([(0, 5, 2, low)])
+    out_c = ctx.pw_moe_forward(0, x, logits, 2, mode=B.PW_MODE_SIMT)
+    torch.cuda.synchronize()
+    assert e1 == e0 + 1
+    assert ctx.pw_query_row(0, 5, 2).page.bits == 2
+    assert torch.equal(out_a, out_b)
+    ids, _ = orc.router(logits.cpu().numpy(), 2)
+    hit = torch.from_numpy((ids == 5).any(axis=1)).cuda()
+    assert hit.any() and (~hit).any()
+    assert torch.equal(out_a[~hit], out_c[~hit])
+    assert (out_a[hit] != out_c[hit]).any(dim=1).all()
+    opages = [export_to_oracle(ctx, p, orc) for p in pages]
+    opages[3 * 5 + 2] = export_to_oracle(ctx, low, orc)
+    ref = orc.moe_forward(x.cpu().numpy(), logits.cpu().numpy(), 2, opages)
+    max_abs, rel_f = error_metrics(out_c.cpu().numpy(), ref)
+    assert max_abs <= MAX_ABS and rel_f <= REL_F
+    ctx.close()
+
+
+def test_forward_argument_errors(orc):
+    cfg = synth.CONFIGS["tiny"]
+    ctx = make_ctx(cfg, n_layers=2)
+    x = synth.activations(cfg, device="cuda")
+    logits = synth.router_logits(cfg, device="cuda")
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_moe_forward(0, x, logits, 2)               # nothing published yet
+    assert e.value.status == 5
+    pages, _ = build_layer(ctx, cfg, 0)
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_moe_forward(1, x, logits, 2)               # layer 1 still unpublished
+    assert e.value.status == 5
+    for bad_k in (0, 3, 9):
+        with pytest.raises(B.PwError) as e:
+            ctx.pw_moe_forward(0, x, logits, bad_k)
+        assert e.value.status == 1
+    big = torch.zeros(17, 256, dtype=torch.float16, device="cuda")
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_moe_forward(0, big, torch.zeros(17, 8, device="cuda"), 2)
+    assert e.value.status == 1
+    wrong = B.Page(512, 256, 4)                           # a gate-shaped page offered as a down block
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_set_page_table([(0, 0, 2, wrong)])
+    assert e.value.status == 2
+    can = ctx.pw_export_page(pages[0])
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_set_page_table([(0, 0, 0, can)])           # canonical layout cannot be published
+    assert e.value.status == 5
+    with pytest.raises(B.PwError) as e:
+        ctx.pw_set_page_table([(0, 0, 0, pages[0])], state=B.PW_STATE_CPU_RESIDENT)
+    assert e.value.status == 5
+    assert ctx.pw_last_device_status() == 0
+    ctx.close()
