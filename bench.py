@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-weight MoE hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One "step" is one layer call of the whole forward path -- page-table commit of a row, router, stable
+permutation, page-table lookup, gate/up contraction with in-kernel dequantization, SwiGLU, down
+contraction, gate-weighted combine -- on a batch of synthetic decode tokens, with the layer's
+mixed-bitwidth weight pages already resident in HBM.  The quantize / demote kernels and their
+side-stream overlap with decode are timed in separate, shorter regions of the same run and reported
+under "demote"; the prefill configuration under "prefill".  N > 1 runs N independent replicas
+(the layer call does not shard and has no collective).
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import re
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2607_16184_b200 import replicas, synth
+
+METRIC = "MoE-layer decode tokens/s & HBM GB/s vs 8 TB/s; prefill TFLOP/s; demote GB/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+def profiled_traffic(name: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None."""
+    p = os.path.join(ROOT, "profiles", name)
+    if not os.path.exists(p):
+        return None
+    m = re.search(r"dram_bytes_per_launch_full_size:\s*([0-9.eE+]+)", open(p).read())
+    return float(m.group(1)) if m else None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs (read-only NVML queries)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self._stop = threading.Event()
+        self._thread = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {}
+        for n in dir(nv):
+            if n.startswith("nvmlClocksEventReason") or n.startswith("nvmlClocksThrottleReason"):
+                v = getattr(nv, n)
+                if isinstance(v, int) and v:
+                    names[v] = n.replace("nvmlClocksEventReason", "").replace("nvmlClocksThrottleReason", "")
+        while not self._stop.is_set():
+            try:
+                self.samples.append((time.time(), int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))))
+                try:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for v, n in names.items():
+                    if bits & v and n not in ("None", "All"):
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        self.t0 = time.time()
+
+    def stop(self):
+        self.t1 = time.time()
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=2)
+        mhz = [m for (t, m) in self.samples if self.t0 <= t <= self.t1] or [m for (_, m) in self.samples]
+        norm = {"SwPowerCap": "sw_power_cap", "HwSlowdown": "hw_slowdown", "HwThermalSlowdown": "hw_thermal_slowdown",
+                "SwThermalSlowdown": "sw_thermal_slowdown", "GpuIdle": "gpu_idle",
+                "ApplicationsClocksSetting": "applications_clocks_setting", "SyncBoost": "sync_boost",
+                "HwPowerBrakeSlowdown": "hw_power_brake_slowdown", "DisplayClockSetting": "display_clock_setting"}
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted({norm.get(r, r) for r in self.reasons} - {"gpu_idle"}), "samples": len(mhz)}
+
+
+def page_bytes_total(bits_table, cfg, active_mask=None):
+    """(gate+up bytes, down bytes) of the pages of the experts that hold at least one token."""
+    from paper_2607_16184_b200 import binding as B
+    gu = dn = 0
+    for e in range(bits_table.shape[0]):
+        if active_mask is not None and not active_mask[e]:
+            continue
+        for u in range(3):
+            rows, cols = cfg.block_shape(u)
+            n = B.pw_page_bytes(rows, cols, int(bits_table[e, u]))[0]
+            if u == 2:
+                dn += n
+            else:
+                gu += n
+    return gu, dn
+
+
+def build_layers(ctx, cfg, n_layers, device):
+    layers = []
+    for layer in range(n_layers):
+        bits = synth.assign_bits(cfg, layer)
+        pages, entries = [], []
+        for e in range(cfg.n_experts + cfg.n_shared):
+            for u in range(3):
+                w = synth.block_weights(cfg, layer, e, u, device=device)
+                pg = ctx.pw_quantize_block(w, int(bits[e, u]))
+                pages.append(pg)
+                entries.append((layer, e, u, pg))
+                del w
+        ctx.pw_set_page_table(entries)
+        layers.append({"bits": bits, "pages": pages, "entries": entries,
+                       "x": synth.activations(cfg, layer, device=device),
+                       "logits": synth.router_logits(cfg, layer, device=device)})
+    torch.cuda.synchronize(device)
+    return layers
+
+
+def time_region(fn, steps, device):
+    torch.cuda.synchronize(device)
+    replicas.barrier(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize(device)
+    replicas.barrier(device)
+    return e0.elapsed_time(e1)
+
+
+def cpu_oracle_sample(cfg, layer_pages_host, x, logits, n_tokens):
+    """Times the CPU oracle, as it stands, on the first n_tokens tokens of the batch."""
+    from oracle import oracle
+    t0 = time.time()
+    oracle.moe_forward(x, logits, cfg.top_k, layer_pages_host, n_shared=cfg.n_shared, tokens=list(range(n_tokens)))
+    dt = time.time() - t0
+    return n_tokens / dt, dt, oracle.num_threads()
+
+
+def export_layer_to_host(ctx, layer, cfg):
+    from oracle import oracle
+    out = []
+    for pg in layer["pages"]:
+        ex = ctx.pw_export_page(pg)
+        torch.cuda.synchronize()
+        ng = pg.cols // 128
+        if pg.bits == 16:
+            out.append(oracle.Page(ex.codes.cpu().numpy(), None, None, pg.rows, pg.cols, 16))
+        else:
+            out.append(oracle.Page(ex.codes.cpu().numpy(),
+                                   ex.scales.view(torch.int16).cpu().numpy().view(np.uint16).reshape(pg.rows, ng),
+                                   ex.zps.view(torch.int16).cpu().numpy().view(np.uint16).reshape(pg.rows, ng),
+                                   pg.rows, pg.cols, pg.bits))
+        del ex
+    return out
+
+
+def run_prefill(device, peaks, steps=3, warmup=1):
+    """Prefill configuration (4096 tokens, bits from {16,8,4}): useful TFLOP/s of one layer call."""
+    from paper_2607_16184_b200 import binding as B
+    cfg = synth.CONFIGS["mixtral_prefill"]
+    ctx = B.Context(1, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
+    layer = build_layers(ctx, cfg, 1, device)[0]
+    out = torch.empty(cfg.tokens, cfg.hidden, dtype=torch.float32, device=device)
+    fn = lambda i: ctx.pw_moe_forward(0, layer["x"], layer["logits"], cfg.top_k, out=out, mode=B.PW_MODE_TENSOR)
+    for i in range(warmup):
+        fn(i)
+    ms = time_region(fn, steps, device) / steps
+    status = ctx.pw_last_device_status()
+    flops = 2.0 * cfg.tokens * cfg.top_k * 3 * cfg.hidden * cfg.ffn
+    tf = flops / (ms * 1e-3) / 1e12
+    ctx.close()
+    return {"workload": "mixtral_prefill: T=4096, E=8, top-2, H=4096, F=14336, bits iid {16,8,4}", "ms_per_call": ms,
+            "tokens_per_s": cfg.tokens / (ms * 1e-3), "tflops": tf, "useful_flop_per_call": flops,
+            "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"],
+            "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS, "device_status": status, "steps": steps}
+
+
+def run_demote(ctx, cfg, layers, device, peaks, decode_fn, decode_ms):
+    """pw_demote_block alone (16->4 on distinct fp16 pages, then 4->2) and overlapped with decode on a side stream."""
+    from paper_2607_16184_b200 import binding as B
+    rows, cols = cfg.block_shape(0)
+    n_src = 6                                   # six 117 MB sources: well past L2 between reuses
+    srcs = [ctx.pw_quantize_block(synth.block_weights(cfg, 100, e, 0, device=device), 16) for e in range(n_src)]
+    dst4 = [B.Page(rows, cols, 4, device) for _ in range(n_src)]
+    dst2 = [B.Page(rows, cols, 2, device) for _ in range(n_src)]
+    b16, b4, b2 = (B.pw_page_bytes(rows, cols, b)[0] for b in (16, 4, 2))
+    for i in range(n_src):
+        ctx.pw_demote_block(srcs[i], 4, dst=dst4[i])
+        ctx.pw_demote_block(dst4[i], 2, dst=dst2[i])
+    reps = 18
+    ms164 = time_region(lambda i: ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src]), reps, device) / reps
+    ms42 = time_region(lambda i: ctx.pw_demote_block(dst4[i % n_src], 2, dst=dst2[i % n_src]), reps, device) / reps
+    # overlapped: decode on the current stream, one 16->4 demote per decode step on a side stream (never committed)
+    side = torch.cuda.Stream(device=device)
+    n_steps = 60
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    side.wait_stream(torch.cuda.current_stream(device))
+    e0.record()
+    s0.record(side)
+    for i in range(n_steps):
+        ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src], stream=side)
+        decode_fn(i)
+    e1.record()
+    s1.record(side)
+    torch.cuda.synchronize(device)
+    ms_dec = e0.elapsed_time(e1) / n_steps
+    ms_side = s0.elapsed_time(s1) / n_steps
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
+    return {"block": "%dx%d" % (rows, cols),
+            "16to4": {"ms": ms164, "gbs": gbs(b16 + b4, ms164), "frac_of_measured_hbm": gbs(b16 + b4, ms164) / peaks["hbm_gbs"],
+                      "frac_of_nominal_8000": gbs(b16 + b4, ms164) / NOMINAL_HBM_GBS, "bytes": b16 + b4},
+            "4to2": {"ms": ms42, "gbs": gbs(b4 + b2, ms42), "frac_of_measured_hbm": gbs(b4 + b2, ms42) / peaks["hbm_gbs"],
+                     "frac_of_nominal_8000": gbs(b4 + b2, ms42) / NOMINAL_HBM_GBS, "bytes": b4 + b2},
+            "under_decode": {"decode_ms_per_step": ms_dec, "decode_ms_alone": decode_ms,
+                             "decode_slowdown": 1.0 - decode_ms / ms_dec if ms_dec > 0 else None,
+                             "demote_16to4_gbs_side_stream": gbs(b16 + b4, ms_side), "steps": n_steps}}
+
+
+def run_gpu(args):
+    from paper_2607_16184_b200 import binding as B
+    from paper_2607_16184_b200 import build as pwbuild
+    rank, local_rank, world = replicas.init("nccl")
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    device = torch.device("cuda", local_rank if world > 1 else 0)
+    torch.cuda.set_device(device)
+    if rank == 0:
+        pwbuild.build()
+    replicas.barrier(device)
+    peaks = measured_peaks()
+    cfg = synth.CONFIGS[args.config]
+    L = args.layers
+    ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
+    layers = build_layers(ctx, cfg, L, device)
+    T, k = cfg.tokens, cfg.top_k
+    out = torch.empty(T, cfg.hidden, dtype=torch.float32, device=device)
+    mode = {"auto": B.PW_MODE_AUTO, "tensor": B.PW_MODE_TENSOR, "simt": B.PW_MODE_SIMT}[args.mode]
+
+    def step(i):
+        lay = layers[i % L]
+        ctx.pw_set_page_table(lay["entries"][(i // L) % len(lay["entries"]):][:1])      # commit one row (S10)
+        ctx.pw_moe_forward(i % L, lay["x"], lay["logits"], k, out=out, mode=mode)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(device.index or 0)
+    n0 = ctx.pw_launch_count()
+    sampler.start()
+    ms_total = time_region(step, args.steps, device)
+    clocks = sampler.stop()
+    launches = ctx.pw_launch_count() - n0
+    status = ctx.pw_last_device_status()
+    ms_max, tokens_all = replicas.aggregate(ms_total, float(T * args.steps), device)
+    value = tokens_all / (ms_max * 1e-3)
+
+    # per-kernel device times, same loop, events recorded around every kernel of the call
+    ctx.pw_kernel_timing(True)
+    ms_timed = time_region(step, args.steps, device)
+    ktimes, kcalls = ctx.pw_get_kernel_times()
+    ctx.pw_kernel_timing(False)
+    kavg = {n: v / max(kcalls, 1) for n, v in ktimes.items()}
+
+    # algorithmic bytes of a layer call: pages of experts that hold tokens + activations in/out
+    gu_bytes = dn_bytes = 0.0
+    for li, lay in enumerate(layers):
+        ctx.pw_moe_forward(li, lay["x"], lay["logits"], k, out=out, mode=mode)
+        counts = ctx.pw_get_routing(T, k)["counts"].cpu().numpy()
+        active = np.concatenate([counts > 0, np.ones(cfg.n_shared, bool)])
+        gu, dn = page_bytes_total(lay["bits"], cfg, active)
+        gu_bytes += gu / L
+        dn_bytes += dn / L
+    R = T * k + cfg.n_shared * T
+    io_bytes = 2 * T * cfg.hidden + 4 * T * cfg.n_experts + 4 * T * cfg.hidden
+    call_bytes = gu_bytes + dn_bytes + io_bytes
+    ms_step = ms_max / args.steps
+    gu_kernel_bytes = gu_bytes + 2.0 * R * cfg.hidden           # pages + the gathered fp16 token rows it reads
+    gu_gbs = gu_kernel_bytes / (kavg["ffn_gate_up"] * 1e-3) / 1e9 if kavg["ffn_gate_up"] > 0 else 0.0
+    dn_gbs = (dn_bytes + 2.0 * R * cfg.ffn) / (kavg["ffn_down"] * 1e-3) / 1e9 if kavg["ffn_down"] > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "ffn_tc_kernel<0> (gate/up + SwiGLU)", "achieved": gu_gbs,
+                "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": gu_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gu_gbs / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": gu_kernel_bytes, "avg_launch_ms": kavg["ffn_gate_up"],
+                "traffic": profiled_traffic("ffn_gate_up_mixtral_decode.md")}
+
+    # end to end: host buffers in, host buffer out, through the host-buffer entry point
+    xh = [lay["x"].cpu().pin_memory() for lay in layers]
+    lh = [lay["logits"].cpu().pin_memory() for lay in layers]
+    oh = torch.empty(T, cfg.hidden, dtype=torch.float32).pin_memory()
+
+    def step_e2e(i):
+        lay = layers[i % L]
+        ctx.pw_set_page_table(lay["entries"][(i // L) % len(lay["entries"]):][:1])
+        ctx.pw_moe_forward_host(i % L, xh[i % L], lh[i % L], k, oh, mode=mode)
+
+    for i in range(3):
+        step_e2e(i)
+    ms_e2e = time_region(step_e2e, args.steps, device)
+    ms_e2e_max, tok_e2e = replicas.aggregate(ms_e2e, float(T * args.steps), device)
+    e2e = {"value": tok_e2e / (ms_e2e_max * 1e-3), "unit": "tokens/s",
+           "h2d_bytes_per_step": int(xh[0].numel() * 2 + lh[0].numel() * 4), "d2h_bytes_per_step": int(oh.numel() * 4)}
+
+    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": "%s: one MoE layer call, E=%d top-%d H=%d F=%d T=%d, %s routing, bit mix %s; "
+                                   "rotating over %d distinct layers (%.2f GB of pages each, larger than L2)"
+                                   % (cfg.name, cfg.n_experts, k, cfg.hidden, cfg.ffn, T, cfg.routing, cfg.bit_rule, L,
+                                      (gu_bytes + dn_bytes) / 1e9),
+                       "mode": args.mode, "l2": "inputs larger than L2", "replicas": world,
+                       "bits_realised": {str(b): int((np.stack([l["bits"] for l in layers]) == b).sum()) for b in synth.BITS}},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": status,
+            "roofline": roofline,
+            "forward": {"algorithmic_bytes_per_call": call_bytes, "hbm_gbs": call_bytes / (ms_step * 1e-3) / 1e9,
+                        "frac_of_measured_hbm": call_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                        "frac_of_nominal_8000": call_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                        "kernel_ms": kavg, "kernel_timed_ms_per_step": ms_timed / args.steps,
+                        "ffn_down_gbs": dn_gbs}}
+
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        host_pages = export_layer_to_host(ctx, layers[0], cfg)
+        v, dt, cores = cpu_oracle_sample(cfg, host_pages, layers[0]["x"].cpu().numpy(),
+                                         layers[0]["logits"].cpu().numpy(), args.cpu_tokens)
+        line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                "sample": "first %d of %d tokens of layer 0, %.1f s" % (args.cpu_tokens, T, dt)}
+        del host_pages
+    else:
+        line["cpu_baseline"] = None
+    if rank == 0 and world == 1 and not args.skip_extra:
+        line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
+        del layers
+        ctx.close()
+        torch.cuda.empty_cache()
+        line["prefill"] = run_prefill(device, peaks)
+    if rank == 0:
+        print(json.dumps(line))
+    replicas.shutdown()
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: same config and metric, each step a bounded sample of the batch."""
+    rank, _, world = replicas.env_world()
+    if rank != 0:
+        return
+    from oracle import oracle
+    oracle.build()
+    cfg = synth.CONFIGS[args.config]
+    n_tok = args.ref_tokens
+    x = synth.activations(cfg, 0).numpy()
+    logits = synth.router_logits(cfg, 0).numpy()
+    bits = synth.assign_bits(cfg, 0)
+    ids, _ = oracle.router(logits, cfg.top_k)
+    need = set(int(e) for e in ids[:n_tok].reshape(-1)) | set(range(cfg.n_experts, cfg.n_experts + cfg.n_shared))
+    pages = []
+    for e in range(cfg.n_experts + cfg.n_shared):
+        for u in range(3):
+            rows, cols = cfg.block_shape(u)
+            if e in need:
+                pages.append(oracle.quantize_block(synth.block_weights(cfg, 0, e, u).numpy(), int(bits[e, u])))
+            else:   # never read: the sampled tokens are not routed here
+                pages.append(oracle.Page(np.zeros(16, np.uint8), None, None, rows, cols, 16))
+    toks = list(range(n_tok))
+    run = lambda: oracle.moe_forward(x, logits, cfg.top_k, pages, n_shared=cfg.n_shared, tokens=toks)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.time()
+    for _ in range(args.steps):
+        run()
+    dt = time.time() - t0
+    v = n_tok * args.steps / dt
+    cores = oracle.num_threads()
+    sample = "first %d of %d tokens of layer 0 per step" % (n_tok, cfg.tokens)
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": world,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                      "data": "synthetic", "config": {"workload": "%s (CPU oracle, %s)" % (cfg.name, sample)},
+                      "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                      "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode"])
+    ap.add_argument("--layers", type=int, default=3, help="distinct layer copies the decode loop rotates over")
+    ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
+    ap.add_argument("--cpu-tokens", type=int, default=8)
+    ap.add_argument("--ref-tokens", type=int, default=2)
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-extra", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 2000 if args.steps is None else args.steps
+        args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

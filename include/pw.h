@@ -112,8 +112,8 @@ typedef struct {
 /* Bytes of device workspace a context with this configuration needs (0 if cfg is invalid). */
 size_t pw_workspace_bytes(const pw_config* cfg);
 
-/* Creates a context on the current device.  cfg->workspace is zero-initialised on `the
- * legacy default stream` and the call returns after that has completed.
+/* Creates a context on the current device.  cfg->workspace is zero-initialised
+ * and the call returns after that has completed.
  * Errors: INVALID_ARG, SHAPE, ALIGN, NOMEM (workspace too small), CUDA. */
 pw_status pw_create(pw_ctx** ctx, const pw_config* cfg);
 
@@ -189,6 +189,15 @@ pw_status pw_query_row(pw_ctx* ctx, int layer, int expert, int kind, pw_table_en
 pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden_fp16, const float* router_logits, int T,
                          int top_k, const pw_page_table* table, float* out, pw_mode mode, pw_stream stream);
 
+/* The same layer call for callers whose activations live in host memory: copies hidden_host
+ * ([T, H] fp16) and logits_host ([T, E] fp32) to staging buffers in the workspace, runs
+ * pw_moe_forward on them and copies the fp32 result to out_host ([T, H]), all ordered on `stream`.
+ * The three host buffers should be pinned for the copies to be asynchronous, and must stay valid
+ * until the stream has passed this call.  Calls that overlap on different streams would share the
+ * staging buffers: use one stream per context.  Errors: as pw_moe_forward, plus CUDA. */
+pw_status pw_moe_forward_host(pw_ctx* ctx, int layer, const void* hidden_host, const float* logits_host, int T,
+                              int top_k, float* out_host, pw_mode mode, pw_stream stream);
+
 /* Copies the routing of the last forward call out of the workspace (device pointers, any may
  * be NULL): topk_ids int32 [T, k], gates fp32 [T, k], counts int32 [E], offsets int32 [E+1],
  * perm int32 [T*k] (pair ids p = t*k + j sorted by expert, then by p). */
@@ -198,6 +207,25 @@ pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* 
 /* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
  * then clears it. */
 pw_status pw_last_device_status(pw_ctx* ctx);
+
+/* Per-kernel device timing of pw_moe_forward (a measurement aid; off by default).  While enabled,
+ * every forward call records CUDA events around each of its kernels on the caller's stream.
+ * pw_kernel_timing(ctx, 1) enables and resets the sums, 0 disables.  pw_get_kernel_times waits for
+ * the recorded events, adds up the elapsed milliseconds per kernel since the last reset into
+ * ms_out[PW_NUM_KERNELS] (host) and returns the number of forward calls covered in calls_out (host).
+ * The paper reports no per-kernel profile; this exists so that a benchmark can put a roofline
+ * fraction on the dominant kernel. */
+enum {
+  PW_K_ROUTER = 0,
+  PW_K_PERMUTE = 1,
+  PW_K_GATHER = 2,
+  PW_K_FFN_GATE_UP = 3,
+  PW_K_FFN_DOWN = 4,
+  PW_K_COMBINE = 5,
+  PW_NUM_KERNELS = 6
+};
+pw_status pw_kernel_timing(pw_ctx* ctx, int enable);
+pw_status pw_get_kernel_times(pw_ctx* ctx, double* ms_out, uint64_t* calls_out);
 
 /* Number of kernels the library has launched through this context since creation. */
 uint64_t pw_launch_count(pw_ctx* ctx);

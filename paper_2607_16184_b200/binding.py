@@ -27,7 +27,9 @@ GROUP = 128
 # every symbol include/pw.h declares
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
-           "pw_moe_forward", "pw_get_routing", "pw_last_device_status", "pw_launch_count", "pw_status_str")
+           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_last_device_status", "pw_kernel_timing", "pw_get_kernel_times",
+           "pw_launch_count", "pw_status_str")
+KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine")
 
 
 class PwError(RuntimeError):
@@ -88,10 +90,16 @@ def load():
     L.pw_query_row.argtypes = [vp, i32, i32, i32, C.POINTER(pw_table_entry)]
     L.pw_moe_forward.restype = i32
     L.pw_moe_forward.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp]
+    L.pw_moe_forward_host.restype = i32
+    L.pw_moe_forward_host.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, vp]
     L.pw_get_routing.restype = i32
     L.pw_get_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.pw_last_device_status.restype = i32
     L.pw_last_device_status.argtypes = [vp]
+    L.pw_kernel_timing.restype = i32
+    L.pw_kernel_timing.argtypes = [vp, i32]
+    L.pw_get_kernel_times.restype = i32
+    L.pw_get_kernel_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     L.pw_launch_count.restype = C.c_uint64
     L.pw_launch_count.argtypes = [vp]
     L.pw_status_str.restype = C.c_char_p
@@ -237,6 +245,19 @@ class Context:
                                      table, out.data_ptr(), mode, _stream_ptr(stream)), "pw_moe_forward")
         return out
 
+    def pw_moe_forward_host(self, layer: int, hidden_host: torch.Tensor, logits_host: torch.Tensor, top_k: int,
+                            out_host: torch.Tensor, mode: int = PW_MODE_AUTO,
+                            stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Host-buffer variant: the three tensors are (preferably pinned) CPU tensors."""
+        assert not hidden_host.is_cuda and not logits_host.is_cuda and not out_host.is_cuda
+        assert hidden_host.dtype == torch.float16 and logits_host.dtype == torch.float32
+        assert out_host.dtype == torch.float32 and out_host.is_contiguous()
+        T = hidden_host.shape[0]
+        _check(self.L.pw_moe_forward_host(self.handle, layer, hidden_host.data_ptr(), logits_host.data_ptr(), T,
+                                          top_k, out_host.data_ptr(), mode, _stream_ptr(stream)),
+               "pw_moe_forward_host")
+        return out_host
+
     def pw_get_routing(self, T: int, top_k: int, stream: Optional[torch.cuda.Stream] = None) -> Dict[str, torch.Tensor]:
         E = self.cfg.n_experts
         d = self.device
@@ -252,6 +273,16 @@ class Context:
 
     def pw_last_device_status(self) -> int:
         return int(self.L.pw_last_device_status(self.handle))
+
+    def pw_kernel_timing(self, enable: bool):
+        _check(self.L.pw_kernel_timing(self.handle, 1 if enable else 0), "pw_kernel_timing")
+
+    def pw_get_kernel_times(self):
+        """({kernel name: summed ms}, forward calls covered) since timing was last enabled."""
+        ms = (C.c_double * len(KERNEL_NAMES))()
+        calls = C.c_uint64()
+        _check(self.L.pw_get_kernel_times(self.handle, ms, C.byref(calls)), "pw_get_kernel_times")
+        return {n: float(ms[i]) for i, n in enumerate(KERNEL_NAMES)}, int(calls.value)
 
     def pw_launch_count(self) -> int:
         return int(self.L.pw_launch_count(self.handle))

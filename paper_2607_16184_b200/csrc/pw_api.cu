@@ -51,8 +51,29 @@ WsMap make_wsmap(const pw_config& c) {
   m.xt = take((size_t)c.hidden * 2 * m.Rpad);
   m.ht = take((size_t)c.ffn * 2 * m.Rpad);
   m.y = take(m.y_slots * c.hidden * 4);
+  m.io_hidden = take((size_t)c.max_tokens * c.hidden * 2);
+  m.io_logits = take((size_t)c.max_tokens * c.n_experts * 4);
+  m.io_out = take((size_t)c.max_tokens * c.hidden * 4);
   m.total = o;
   return m;
+}
+
+static void timing_drain_slot(pw_ctx* ctx, int slot) {
+  if (!ctx->timing_busy[slot]) return;
+  cudaEvent_t* ev = ctx->timing_ev + (size_t)slot * (PW_NUM_KERNELS + 1);
+  if (cudaEventSynchronize(ev[PW_NUM_KERNELS]) == cudaSuccess) {
+    for (int i = 0; i < PW_NUM_KERNELS; ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ev[i], ev[i + 1]) == cudaSuccess) ctx->timing_ms[i] += ms;
+    }
+    ctx->timing_calls++;
+  }
+  ctx->timing_busy[slot] = false;
+}
+
+void timing_mark(pw_ctx* ctx, int i, cudaStream_t s) {
+  if (!ctx->timing_on) return;
+  cudaEventRecord(ctx->timing_ev[(size_t)ctx->timing_cur * (PW_NUM_KERNELS + 1) + i], s);
 }
 
 static size_t row_index(const pw_ctx* ctx, int layer, int expert, int kind) {
@@ -87,6 +108,12 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   ctx->last_T = ctx->last_k = 0;
   ctx->tc_state = nullptr;
   ctx->stage_next = 0;
+  ctx->timing_on = false;
+  ctx->timing_ev = nullptr;
+  ctx->timing_cur = 0;
+  ctx->timing_calls = 0;
+  for (int i = 0; i < pw_ctx::kTimingSlots; ++i) ctx->timing_busy[i] = false;
+  for (int i = 0; i < PW_NUM_KERNELS; ++i) ctx->timing_ms[i] = 0.0;
   const size_t nrows = (size_t)cfg->n_layers * m.S * 3;
   ctx->stage_rows = nrows;
   ctx->host_rows = new (std::nothrow) pw_table_entry[nrows]();
@@ -121,6 +148,11 @@ extern "C" pw_status pw_destroy(pw_ctx* ctx) {
   for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
     if (ctx->stage[i]) cudaFreeHost(ctx->stage[i]);
     if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+  }
+  if (ctx->timing_ev) {
+    for (int i = 0; i < pw_ctx::kTimingSlots * (PW_NUM_KERNELS + 1); ++i)
+      if (ctx->timing_ev[i]) cudaEventDestroy(ctx->timing_ev[i]);
+    delete[] ctx->timing_ev;
   }
   delete[] ctx->host_rows;
   delete[] ctx->host_valid;
@@ -233,6 +265,11 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
     while (want > 1 && (size_t)want * R > ctx->ws.y_slots) --want;
     ksplit = (int)want;
   }
+  if (ctx->timing_on) {
+    ctx->timing_cur = (ctx->timing_cur + 1) % pw_ctx::kTimingSlots;
+    timing_drain_slot(ctx, ctx->timing_cur);   // waits only when the ring has wrapped onto unfinished work
+    ctx->timing_busy[ctx->timing_cur] = true;
+  }
   pw_status st = launch_route(ctx, layer, hidden, logits, T, top_k, nt_tile, ksplit, stream);
   if (st != PW_OK) return st;
   st = mode == PW_MODE_SIMT ? launch_ffn_simt(ctx, layer, T, top_k, stream)
@@ -242,6 +279,22 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
   ctx->last_T = T;
   ctx->last_k = top_k;
   return st;
+}
+
+extern "C" pw_status pw_moe_forward_host(pw_ctx* ctx, int layer, const void* hidden_host, const float* logits_host, int T,
+                                         int top_k, float* out_host, pw_mode mode, pw_stream stream) {
+  if (!ctx || !hidden_host || !logits_host || !out_host) return PW_ERR_INVALID_ARG;
+  const pw_config& c = ctx->cfg;
+  if (T < 1 || T > c.max_tokens) return PW_ERR_INVALID_ARG;
+  char* b = ctx->base;
+  const WsMap& w = ctx->ws;
+  PW_CUDA_OK(cudaMemcpyAsync(b + w.io_hidden, hidden_host, (size_t)T * c.hidden * 2, cudaMemcpyHostToDevice, stream));
+  PW_CUDA_OK(cudaMemcpyAsync(b + w.io_logits, logits_host, (size_t)T * c.n_experts * 4, cudaMemcpyHostToDevice, stream));
+  pw_status st = pw_moe_forward(ctx, layer, b + w.io_hidden, reinterpret_cast<const float*>(b + w.io_logits), T, top_k,
+                                nullptr, reinterpret_cast<float*>(b + w.io_out), mode, stream);
+  if (st != PW_OK) return st;
+  PW_CUDA_OK(cudaMemcpyAsync(out_host, b + w.io_out, (size_t)T * c.hidden * 4, cudaMemcpyDeviceToHost, stream));
+  return PW_OK;
 }
 
 extern "C" pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
@@ -269,6 +322,33 @@ extern "C" pw_status pw_last_device_status(pw_ctx* ctx) {
     PW_CUDA_OK(cudaMemset(ctx->base + ctx->ws.status, 0, 4));
   }
   return (pw_status)v;
+}
+
+extern "C" pw_status pw_kernel_timing(pw_ctx* ctx, int enable) {
+  if (!ctx) return PW_ERR_INVALID_ARG;
+  if (enable && !ctx->timing_ev) {
+    const int n = pw_ctx::kTimingSlots * (PW_NUM_KERNELS + 1);
+    ctx->timing_ev = new (std::nothrow) cudaEvent_t[n]();
+    if (!ctx->timing_ev) return PW_ERR_NOMEM;
+    for (int i = 0; i < n; ++i) PW_CUDA_OK(cudaEventCreate(&ctx->timing_ev[i]));
+  }
+  if (ctx->timing_ev)
+    for (int i = 0; i < pw_ctx::kTimingSlots; ++i) timing_drain_slot(ctx, i);
+  ctx->timing_on = enable != 0;
+  if (enable) {
+    ctx->timing_calls = 0;
+    for (int i = 0; i < PW_NUM_KERNELS; ++i) ctx->timing_ms[i] = 0.0;
+  }
+  return PW_OK;
+}
+
+extern "C" pw_status pw_get_kernel_times(pw_ctx* ctx, double* ms_out, uint64_t* calls_out) {
+  if (!ctx || !ms_out) return PW_ERR_INVALID_ARG;
+  if (ctx->timing_ev)
+    for (int i = 0; i < pw_ctx::kTimingSlots; ++i) timing_drain_slot(ctx, i);
+  for (int i = 0; i < PW_NUM_KERNELS; ++i) ms_out[i] = ctx->timing_ms[i];
+  if (calls_out) *calls_out = ctx->timing_calls;
+  return PW_OK;
 }
 
 extern "C" uint64_t pw_launch_count(pw_ctx* ctx) { return ctx ? ctx->launches : 0; }

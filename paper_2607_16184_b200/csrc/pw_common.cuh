@@ -56,6 +56,9 @@ struct WsMap {
   size_t xt;          // fp16 operand rows, k-chunk major: [H/8][Rpad][8]
   size_t ht;          // fp16 SwiGLU output,  k-chunk major: [F/8][Rpad][8]
   size_t y;           // float [y_slots][H]  split-K partial outputs of the down projection
+  size_t io_hidden;   // fp16 [Tmax][H]   device staging of pw_moe_forward_host
+  size_t io_logits;   // float [Tmax][E]
+  size_t io_out;      // float [Tmax][H]
   size_t total;
   // derived sizes
   int S;              // segments = E + n_shared
@@ -94,6 +97,14 @@ struct pw_ctx {
   int last_T, last_k;
   int num_sms;
   void* tc_state;                 // tensor-core path state (set up lazily)
+  // optional per-kernel timing: a ring of call slots, PW_NUM_KERNELS + 1 events each
+  static constexpr int kTimingSlots = 256;
+  bool timing_on;
+  cudaEvent_t* timing_ev;         // [kTimingSlots][PW_NUM_KERNELS + 1], created on first enable
+  bool timing_busy[kTimingSlots];
+  int timing_cur;                 // slot of the forward call being enqueued
+  uint64_t timing_calls;
+  double timing_ms[PW_NUM_KERNELS];
 };
 
 #define PW_CUDA_OK(expr)                                   \
@@ -111,5 +122,7 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
 pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
 int tensor_token_tile(const pw_ctx* ctx, int T, int k);
+// records timing event `i` of the current forward call (no-op unless timing is enabled)
+void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 
 }  // namespace pw

@@ -105,9 +105,11 @@ pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s) 
   char* b = ctx->base;
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
   const int32_t* offsets = reinterpret_cast<const int32_t*>(b + w.offsets);
+  timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   ffn_simt_kernel<0><<<dim3(c.ffn / kTileRows, w.S), 128, 0, s>>>(rows, offsets, reinterpret_cast<const uint4*>(b + w.xt),
                                                                   w.Rpad, reinterpret_cast<__half*>(b + w.ht), nullptr,
                                                                   c.hidden);
+  timing_mark(ctx, PW_K_FFN_DOWN, s);
   ffn_simt_kernel<1><<<dim3(c.hidden / kTileRows, w.S), 128, 0, s>>>(rows, offsets,
                                                                      reinterpret_cast<const uint4*>(b + w.ht), w.Rpad,
                                                                      nullptr, reinterpret_cast<float*>(b + w.y),

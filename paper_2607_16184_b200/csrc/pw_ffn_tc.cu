@@ -413,10 +413,12 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const int R = T * k + c.n_shared * T;
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
+  timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
                                                         reinterpret_cast<const uint4*>(b + w.xt), w.Rpad, nt_tile,
                                                         n_bslots, reinterpret_cast<__half*>(b + w.ht), nullptr,
                                                         c.hidden, 0, status);
+  timing_mark(ctx, PW_K_FFN_DOWN, s);
   ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
                                                         reinterpret_cast<const uint4*>(b + w.ht), w.Rpad, nt_tile,
                                                         n_bslots, nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,

@@ -247,7 +247,9 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
   char* b = ctx->base;
   const int E = c.n_experts, S = w.S;
   int32_t* ids = reinterpret_cast<int32_t*>(b + w.topk_ids);
+  timing_mark(ctx, PW_K_ROUTER, s);
   router_kernel<<<(T * 32 + 255) / 256, 256, 0, s>>>(logits, T, E, k, ids, reinterpret_cast<float*>(b + w.gates));
+  timing_mark(ctx, PW_K_PERMUTE, s);
   const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + E + 32 * (size_t)E + (S + 1) + S);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * S * 3;
   permute_kernel<<<1, 1024, smem, s>>>(
@@ -258,6 +260,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
       reinterpret_cast<int32_t*>(b + w.n_units), reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units,
       reinterpret_cast<int32_t*>(b + w.status));
   const int R = T * k + c.n_shared * T;
+  timing_mark(ctx, PW_K_GATHER, s);
   dim3 grid((R + kPadRows + 255) / 256, c.hidden / 8);
   gather_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(hidden),
                                      reinterpret_cast<const int32_t*>(b + w.row_token),
@@ -275,10 +278,12 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
   const int H4 = c.hidden / 4;
   const int R = T * k + c.n_shared * T;
   dim3 grid((H4 + 255) / 256, T);
+  timing_mark(ctx, PW_K_COMBINE, s);
   combine_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const float4*>(b + w.y),
                                       reinterpret_cast<const float*>(b + w.gates),
                                       reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
                                       (size_t)R * H4, reinterpret_cast<float4*>(out));
+  timing_mark(ctx, PW_NUM_KERNELS, s);
   ctx->launches += 1;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
