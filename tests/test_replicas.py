@@ -24,7 +24,10 @@ SCRIPT = textwrap.dedent("""
 def test_two_replicas_aggregate_max_time_and_summed_units(tmp_path):
     script = tmp_path / "w.py"
     script.write_text(SCRIPT)
-    port = 29500 + os.getpid() % 2000
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
            "127.0.0.1", "--master-port", str(port), str(script)]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
