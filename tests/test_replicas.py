@@ -17,7 +17,8 @@ SCRIPT = textwrap.dedent("""
     assert world == 2 and t == 15.0 and u == 128.0, (world, t, u)
     replicas.barrier(dev)
     replicas.shutdown()
-    print("rank", rank, "ok")
+    sys.stdout.write("rank%d_ok\n" % rank)
+    sys.stdout.flush()
 """) % ROOT
 
 
@@ -32,7 +33,7 @@ def test_two_replicas_aggregate_max_time_and_summed_units(tmp_path):
            "127.0.0.1", "--master-port", str(port), str(script)]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
     assert out.returncode == 0, out.stdout + out.stderr
-    assert "rank 0 ok" in out.stdout and "rank 1 ok" in out.stdout
+    assert out.stdout.count("_ok") == 2 and "rank0" in out.stdout and "rank1" in out.stdout
 
 
 def test_single_process_is_identity():
