@@ -17,7 +17,7 @@ SCRIPT = textwrap.dedent("""
     assert world == 2 and t == 15.0 and u == 128.0, (world, t, u)
     replicas.barrier(dev)
     replicas.shutdown()
-    sys.stdout.write("rank%d_ok\n" % rank)
+    sys.stdout.write("rank" + str(rank) + "_ok" + chr(10))
     sys.stdout.flush()
 """) % ROOT
 
