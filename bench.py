@@ -273,6 +273,9 @@ def run_gpu(args):
     replicas.barrier(device)
     peaks = measured_peaks()
     cfg = synth.CONFIGS[args.config]
+    if args.uniform_bits:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, bit_rule="uniform%d" % args.uniform_bits)
     L = args.layers
     ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
     layers = build_layers(ctx, cfg, L, device)
@@ -434,6 +437,8 @@ def main():
     ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
     ap.add_argument("--cpu-tokens", type=int, default=8)
     ap.add_argument("--ref-tokens", type=int, default=2)
+    ap.add_argument("--uniform-bits", type=int, default=0, choices=[0, 16, 8, 4, 3, 2],
+                    help="diagnostic: give every routed block this bitwidth instead of the configured mix")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-extra", action="store_true")
     args = ap.parse_args()

@@ -149,6 +149,7 @@ extern "C" pw_status pw_destroy(pw_ctx* ctx) {
     if (ctx->stage[i]) cudaFreeHost(ctx->stage[i]);
     if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
   }
+  tc_teardown(ctx);
   if (ctx->timing_ev) {
     for (int i = 0; i < pw_ctx::kTimingSlots * (PW_NUM_KERNELS + 1); ++i)
       if (ctx->timing_ev[i]) cudaEventDestroy(ctx->timing_ev[i]);

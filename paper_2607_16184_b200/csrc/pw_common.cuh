@@ -122,6 +122,7 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
 pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
 int tensor_token_tile(const pw_ctx* ctx, int T, int k);
+void tc_teardown(pw_ctx* ctx);
 // records timing event `i` of the current forward call (no-op unless timing is enabled)
 void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 

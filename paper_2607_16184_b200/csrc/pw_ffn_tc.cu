@@ -1,43 +1,86 @@
-// Tensor-core expert FFN for sm_100a: weight pages stream HBM -> shared memory (bulk async copies),
-// are dequantized in registers straight into tensor memory (the A operand, one weight row per TMEM
-// lane), and tcgen05.mma contracts them against the token tile (B operand in shared memory), with
-// fp32 accumulators in tensor memory.  D[128 weight rows, N tokens] += W[128, 16] * X[N, 16]^T.
+// Tensor-core expert FFN for sm_100a.
 //
-// One persistent CTA per SM, 10 warps:
-//   warps 0-7  dequantize (two sets of four warps alternate groups; warp w owns TMEM lanes
-//              32*(w%4) .. +31) and run the epilogue (SwiGLU -> fp16 operand of the down projection,
-//              or the fp32 partial output of the down projection);
-//   warp 8     producer: one thread issues every bulk copy (weight stages and token tiles);
-//   warp 9     allocates tensor memory; one thread issues every MMA and commit.
-// Every wait on an mbarrier is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the
-// status word, stops issuing work, frees its tensor memory and returns.
+//   D[128 weight rows, N tokens] += W[128, 16] * X[N, 16]^T      (tcgen05.mma, kind::f16, fp32 in TMEM)
+//
+// Weight pages stream HBM -> shared memory with bulk async copies, one item (128 rows x one group of
+// one page, 4.5 .. 32 KB) at a time into a FIFO ring that holds as many items as fit, so that enough
+// bytes are in flight to cover the HBM latency whatever the bitwidth.  A 16-bit page tile is already in the tensor core's K-major core-matrix layout,
+// so the MMA reads it from shared memory as the A operand without any thread touching it.  A
+// quantized tile is unpacked and dequantized in registers (one weight row per thread) and written
+// to tensor memory, which the MMA then reads as its A operand.  The token tile (B operand) comes
+// from the k-chunk-major operand buffers with one 2-D TMA copy per group.
+//
+// One persistent CTA per SM, 25 warps:
+//   warps 0-15   dequantize: two groups of eight warps, each group takes every other quantized
+//                128x128 slab; warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
+//   warp 16      producer: one thread issues every copy (weight stages and token tiles);
+//   warps 17-20  MMA issuers (warp 17 also allocates tensor memory).  A tcgen05.mma holds its issuing
+//                thread for ~95 cycles whatever its size, so one issuer caps the SM at one 128x16
+//                weight slab per 95 cycles; four issuers in four warps overlap.  Each issuer owns the
+//                K-steps k = j mod (issuers per matrix) of one matrix and its own partial accumulator,
+//                so no two threads ever accumulate into the same columns; the epilogue adds the partials;
+//   warps 21-24  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
+//                split-K partial of the down projection (PHASE 1); accumulators are double-buffered
+//                when they fit so the next unit's MMAs overlap the epilogue.
+// Units are dealt to CTAs in snake order over a size-sorted list.  Every wait on an mbarrier is
+// bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <new>
+
 #include "pw_common.cuh"
 #include "pw_layout.cuh"
 
 namespace pw {
 
-constexpr int kWSlots = 4;                     // weight stages in shared memory
-constexpr int kWSlotCodes = 32768;             // code bytes of a stage (16 units x 2 KB)
-constexpr int kWSlotMeta = 2048;               // scale bytes, then zero-point bytes, of up to 8 groups
-constexpr int kWSlotBytes = kWSlotCodes + 2 * kWSlotMeta;
-constexpr int kASlots = 4;                     // dequantized groups in tensor memory (64 columns each)
+constexpr int kQDq = 16;                       // quantized items in flight (barrier pairs)
+constexpr int kQMma = 8;                       // 16-bit items in flight
+constexpr int kMaxASlots = 8;                  // dequantized groups in tensor memory (64 columns each)
 constexpr int kMaxBSlots = 4;
-constexpr int kCtrlBytes = 1024;
+constexpr int kCtrlBytes = 2048;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
-constexpr int kThreads = 320;
+constexpr int kDqWarps = 16;
+constexpr int kWarpProducer = 16, kWarpMma = 17, kIssuers = 4, kWarpEpi = 21;
+constexpr int kThreads = 800;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kColD0 = 0, kColD1 = 128, kColA = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct Ctrl {                                  // lives at the start of dynamic shared memory
-  unsigned long long w_full[kWSlots], w_empty[kWSlots];
+  // A weight item is consumed either by the dequantizers (quantized page) or by the MMA issuers (16-bit
+  // page); each kind has its own sequence of full / empty barriers so that every waiter sees every phase.
+  unsigned long long full_dq[kQDq], empty_dq[kQDq];
+  unsigned long long full_mma[2][kQMma], empty_mma[2][kQMma];   // per matrix of the unit (gate / up)
   unsigned long long b_full[kMaxBSlots], b_empty[kMaxBSlots];
-  unsigned long long a_full[kASlots], a_empty[kASlots];
+  unsigned long long a_full[kMaxASlots], a_empty[kMaxASlots];
   unsigned long long d_full, d_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
+  uint32_t q_off[64], q_seq[64];              // producer's queue of items in flight
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
+
+#ifdef PW_TC_PROFILE
+// Diagnostic build only: per-CTA cycle counters of where each role waits (kept in registers, flushed once).
+__device__ unsigned long long g_prof[2][160][24];
+#define PROF_DECL() unsigned long long pacc__[24] = {}
+#define PROF_T0() const long long pt0__ = clock64()
+#define PROF_ADD(slot) pacc__[slot] += (unsigned long long)(clock64() - pt0__)
+#define PROF_FLUSH()                                                                        \
+  if (lane == 0 && (warp == 0 || warp == kWarpProducer || warp == kWarpMma)) {              \
+    _Pragma("unroll") for (int i__ = 0; i__ < 24; ++i__) if (pacc__[i__])                   \
+        g_prof[PHASE][blockIdx.x][i__] += pacc__[i__];                                      \
+  }
+#else
+#define PROF_DECL()
+#define PROF_T0()
+#define PROF_ADD(slot)
+#define PROF_FLUSH()
+#endif
+
+struct TmapSet {                               // token-tile copies: one map per tile height 16, 32, .. 128
+  CUtensorMap m[8];
+};
 
 // ---- PTX wrappers ----------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -55,7 +98,11 @@ __device__ __forceinline__ bool mbar_try(unsigned long long* b, uint32_t parity)
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
+#ifdef PW_TC_PROFILE
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"   // non-blocking, so that waits are measured
+#else
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#endif
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(b)), "r"(parity)
@@ -68,11 +115,13 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting or the limit ran out (and then raises the abort).
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
   if (mbar_try(b, parity)) return true;
   const unsigned long long t0 = globaltimer();
   uint32_t spins = 0;
   while (true) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);       // leave the issue slots to the warps doing arithmetic
     if (mbar_try(b, parity)) return true;
     if (c->abort_flag) return false;
     if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
@@ -88,12 +137,20 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+__device__ __forceinline__ void tma_2d_g2s(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(unsigned long long* b) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(b))
                : "memory");
 }
+// A operand in tensor memory
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
@@ -101,6 +158,16 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// A operand in shared memory
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const __half2* v) {
@@ -114,23 +181,45 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const __half2* v) {
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const __half2* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+      "[%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// groups per weight stage: about 32 KB of codes whatever the bitwidth
-__device__ __forceinline__ int groups_per_stage(uint32_t bits) { return bits == 16 ? 1 : bits == 8 ? 2 : bits == 2 ? 8 : 4; }
+// Shared-memory footprint of one item (one 128-row x one-group tile of one page): codes, then the
+// 128 scales, then the 128 zero-points; rounded up to 1 KB.
+__device__ __forceinline__ uint32_t item_bytes(uint32_t bits) {
+  return bits == 16 ? 32768u : ((bits * 2048u + 512u + 1023u) & ~1023u);
+}
+// The weight ring is a FIFO of variable-sized items.  Every role replays the same allocation sequence.
+__device__ __forceinline__ uint32_t ring_take(uint32_t& head, uint32_t sz, uint32_t cap) {
+  if (head + sz > cap) head = 0;
+  const uint32_t off = head;
+  head += sz;
+  return off;
+}
 
-// Shared-memory matrix descriptor of the B operand: K-major, no swizzle.  A core matrix is 8 token
-// rows x 16 bytes (8 fp16 along K) stored as 128 contiguous bytes; 8-row groups are 128 bytes apart
-// (stride byte offset), the two K-halves of one MMA are `lbo_bytes` apart (leading byte offset).
-__device__ __forceinline__ uint64_t make_b_desc(uint32_t saddr, uint32_t lbo_bytes) {
+// Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
+// along K) stored as 128 contiguous bytes; 8-row groups are 128 bytes apart (stride byte offset),
+// the two K-halves of one MMA are `lbo_bytes` apart (leading byte offset).
+__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t saddr, uint32_t lbo_bytes) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr >> 4) & 0x3fffu);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
@@ -139,60 +228,66 @@ __device__ __forceinline__ uint64_t make_b_desc(uint32_t saddr, uint32_t lbo_byt
   return d;
 }
 
+// K-half `h` of one row of an item: shared memory -> 32 registers (half2 pairs in K order).
 template <int BITS>
-__device__ __forceinline__ void dequant_group_to_tmem(const char* slot, int sub, int r, uint32_t taddr) {
-  const uint4* row_units = reinterpret_cast<const uint4*>(slot + (size_t)sub * tile_code_bytes(BITS)) + r;
-  __half2 s2 = u32_as_h2(0x3c003c00u), z2 = s2;
-  if constexpr (BITS < 16) {
-    s2 = __half2half2(reinterpret_cast<const __half*>(slot + kWSlotCodes)[sub * kTileRows + r]);
-    z2 = __half2half2(reinterpret_cast<const __half*>(slot + kWSlotCodes + kWSlotMeta)[sub * kTileRows + r]);
-  }
-  __half2 w[32];
-  decode_half<BITS>(row_units, 0, s2, z2, w);
-  tmem_st32(taddr, w);
-  decode_half<BITS>(row_units, 1, s2, z2, w);
-  tmem_st32(taddr + 32, w);
+__device__ __forceinline__ void decode_item_half(const char* item, int r, int h, __half2* w) {
+  const uint4* row_units = reinterpret_cast<const uint4*>(item) + r;
+  const __half2 s2 = __half2half2(reinterpret_cast<const __half*>(item + BITS * 2048)[r]);
+  const __half2 z2 = __half2half2(reinterpret_cast<const __half*>(item + BITS * 2048 + 256)[r]);
+  decode_half<BITS>(row_units, h, s2, z2, w);
 }
 
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
 template <int PHASE>
-__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units,
-                                                             const int32_t* __restrict__ n_units_ptr,
-                                                             const uint4* __restrict__ bop, int Rpad, int nt_tile,
-                                                             int n_bslots, __half* __restrict__ ht,
-                                                             float* __restrict__ y, int H, size_t y_split_stride,
-                                                             int32_t* __restrict__ status) {
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, const int32_t* __restrict__ n_units_ptr,
+              const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, uint32_t wcap,
+              __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
+              int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
-  char* wslots = smem + kCtrlBytes;
-  char* bslots = wslots + kWSlots * kWSlotBytes;
+  char* wring = smem + kCtrlBytes;
+  char* bslots = wring + wcap;
   const int bslot_bytes = nt_tile * 256;
   constexpr int NMAT = PHASE == 0 ? 2 : 1;
-  constexpr int RING = kWSlots / NMAT;           // stages per matrix ring
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_units = n_units_ptr[PHASE];
+  // tensor-memory columns: partial accumulators first ([matrix][partial][nt_tile]), dequantized-operand
+  // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
+  constexpr int IPM = kIssuers / NMAT;           // issuers per matrix
+  int npart = IPM;
+  while (npart > 1 && NMAT * npart * nt_tile + 2 * 64 > kTmemCols) npart >>= 1;
+  const int n_issuers = NMAT * npart;            // active issuers
+  const int acol = NMAT * npart * nt_tile;
+  const int n_aslots = min(kMaxASlots, (kTmemCols - acol) / 64) & ~1;   // even: a slot always serves the same group
+  const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kWSlots; ++i) {
-      mbar_init(&c->w_full[i], 1);
-      mbar_init(&c->w_empty[i], 8);
+    for (int i = 0; i < kQDq; ++i) {
+      mbar_init(&c->full_dq[i], 1);
+      mbar_init(&c->empty_dq[i], 8);          // the eight warps of the group that owns the item
     }
+    for (int i = 0; i < kQMma; ++i)
+      for (int m = 0; m < 2; ++m) {
+        mbar_init(&c->full_mma[m][i], 1);
+        mbar_init(&c->empty_mma[m][i], npart);
+      }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
-      mbar_init(&c->b_empty[i], 1);
+      mbar_init(&c->b_empty[i], n_issuers);
     }
-    for (int i = 0; i < kASlots; ++i) {
-      mbar_init(&c->a_full[i], 4);
-      mbar_init(&c->a_empty[i], 1);
+    for (int i = 0; i < kMaxASlots; ++i) {
+      mbar_init(&c->a_full[i], 8);
+      mbar_init(&c->a_empty[i], npart);
     }
-    mbar_init(&c->d_full, 1);
-    mbar_init(&c->d_empty, 8);
+    mbar_init(&c->d_full, n_issuers);
+    mbar_init(&c->d_empty, 4);
     c->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c->tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
@@ -202,50 +297,127 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const DevRow* __res
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = c->tmem_base;
+  PROF_DECL();
+#ifdef PW_TC_PROFILE
+  const long long kernel_t0__ = clock64();
+#endif
 
-  if (warp == 8) {
+  // unit i of this CTA in snake order over the size-sorted list
+  auto unit_index = [&](int i) { return i * G + ((i & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x); };
+
+  if (warp == kWarpProducer) {
     // ---------------- producer ----------------
     if (lane == 0) {
-      uint32_t wcount[NMAT] = {};   // stages issued per ring
-      uint32_t bcount = 0;
+      // Items in flight, oldest first, in a small circular queue in shared memory: ring offset and the
+      // sequence tag that says which barrier frees the item (bits 30-31 = 1 + matrix for 16-bit items).
+      constexpr int NQ = 64;
+      uint32_t* q_off = c->q_off;
+      uint32_t* q_seq = c->q_seq;
+      int q_head = 0, q_count = 0;
+      uint32_t head = 0, dq_seq = 0, bcount = 0;
+      uint32_t mma_seq0 = 0, mma_seq1 = 0;
+      // releases are observed strictly in sequence per kind, so that no barrier phase is ever skipped
+      uint32_t rel_dq = 0, rel_mma0 = 0, rel_mma1 = 0;   // items 0 .. rel-1 of the kind are known to be released
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+#define PW_RELEASED_DQ(S)                                                                              \
+  while (ok && rel_dq <= (S)) {                                                                        \
+    ok = mbar_wait<64>(&c->empty_dq[rel_dq % kQDq], (rel_dq / kQDq) & 1, c, status);                   \
+    ++rel_dq;                                                                                          \
+  }
+#define PW_RELEASED_MMA(M, S)                                                                          \
+  {                                                                                                    \
+    uint32_t& rel__ = (M) == 0 ? rel_mma0 : rel_mma1;                                                  \
+    while (ok && rel__ <= (S)) {                                                                       \
+      ok = mbar_wait<64>(&c->empty_mma[M][rel__ % kQMma], (rel__ / kQMma) & 1, c, status);             \
+      ++rel__;                                                                                         \
+    }                                                                                                  \
+  }
+      for (int i = 0; ok; ++i) {
+        const int u = unit_index(i);
+        if (u >= n_units) break;
         const Unit un = units[u];
-        const DevRow* rr = rows + un.seg * 3;
+        DevRow urow[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) urow[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
         const int nb_rows = (un.ntok + 15) & ~15;
+        const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
         for (int g = un.g0; ok && g < un.g1; ++g) {
-          {  // token tile of this group: 16 K-chunks of nb_rows x 16 bytes
+          {  // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
             const int bs = bcount % n_bslots;
-            ok = mbar_wait(&c->b_empty[bs], ((bcount / n_bslots) & 1) ^ 1, c, status);
+            {
+              PROF_T0();
+              ok = mbar_wait<64>(&c->b_empty[bs], ((bcount / n_bslots) & 1) ^ 1, c, status);
+              PROF_ADD(0);
+            }
             if (!ok) break;
             mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
-            char* dst = bslots + (size_t)bs * bslot_bytes;
-            const uint4* src = bop + (size_t)(g * 16) * Rpad + un.tok0;
-            for (int kc = 0; kc < 16; ++kc)
-              bulk_g2s(dst + kc * nb_rows * 16, src + (size_t)kc * Rpad, nb_rows * 16, &c->b_full[bs]);
+            tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
             ++bcount;
           }
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            const DevRow& row = rr[PHASE == 0 ? m : 2];
-            const int gps = groups_per_stage(row.bits);
-            if ((g - un.g0) % gps != 0) continue;
-            const int ngr = min(gps, un.g1 - g);
-            const int ws = m * RING + (int)(wcount[m] % RING);
-            ok = mbar_wait(&c->w_empty[ws], ((wcount[m] / RING) & 1) ^ 1, c, status);
+            const DevRow& row = urow[m];
+            const uint32_t bits = row.bits;
+            const uint32_t sz = item_bytes(bits);
+            const uint32_t head_prev = head;
+            const uint32_t off = ring_take(head, sz, wcap);
+            // The items in flight occupy a circular span from the oldest item's offset (tail) up to
+            // head_prev.  Pop (wait for the release of) oldest items until [off, off+sz) is clear of it.
+            {
+              PROF_T0();
+              while (ok && q_count > 0) {
+                const uint32_t tail = q_off[q_head];
+                bool free_now;
+                if (tail < head_prev) free_now = (off == head_prev) || (sz <= tail);          // span [tail, head_prev)
+                else free_now = (off == head_prev) && (off + sz <= tail);                      // span wraps around
+                if (free_now && q_count < NQ) break;
+                const uint32_t sq = q_seq[q_head];
+                if (sq >> 30) {
+                  if ((sq >> 30) == 1) PW_RELEASED_MMA(0, sq & 0x3fffffffu) else PW_RELEASED_MMA(1, sq & 0x3fffffffu)
+                } else {
+                  PW_RELEASED_DQ(sq)
+                }
+                q_head = (q_head + 1) % NQ;
+                --q_count;
+              }
+              PROF_ADD(1);
+            }
             if (!ok) break;
+            // the barrier pair of this item must be free too: at most kQ* items of a kind in flight
+            unsigned long long* full;
+            uint32_t seqtag;
+            if (bits == 16) {
+              uint32_t& ms = m == 0 ? mma_seq0 : mma_seq1;
+              if (ms >= (uint32_t)kQMma) {
+                if (m == 0) PW_RELEASED_MMA(0, ms - kQMma) else PW_RELEASED_MMA(1, ms - kQMma)
+              }
+              full = &c->full_mma[m][ms % kQMma];
+              seqtag = ms | ((uint32_t)(m + 1) << 30);
+              ++ms;
+            } else {
+              if (dq_seq >= (uint32_t)kQDq) PW_RELEASED_DQ(dq_seq - kQDq)
+              full = &c->full_dq[dq_seq % kQDq];
+              seqtag = dq_seq;
+              ++dq_seq;
+            }
+            if (!ok) break;
+            const int qt = (q_head + q_count) % NQ;
+            q_off[qt] = off;
+            q_seq[qt] = seqtag;
+            ++q_count;
             const int ng = row.cols / kGroup;
             const size_t tile = (size_t)un.row_tile * ng + g;
-            const uint32_t cbytes = ngr * row.bits * 2048;
-            const uint32_t mbytes = row.bits < 16 ? ngr * 256 : 0;
-            mbar_expect_tx(&c->w_full[ws], cbytes + 2 * mbytes);
-            char* dst = wslots + (size_t)ws * kWSlotBytes;
-            bulk_g2s(dst, reinterpret_cast<const char*>(row.codes) + tile * row.bits * 2048, cbytes, &c->w_full[ws]);
-            if (mbytes) {
-              bulk_g2s(dst + kWSlotCodes, row.scales + tile * kTileRows, mbytes, &c->w_full[ws]);
-              bulk_g2s(dst + kWSlotCodes + kWSlotMeta, row.zps + tile * kTileRows, mbytes, &c->w_full[ws]);
+            const uint32_t cbytes = bits * 2048;
+            char* dst = wring + off;
+            if (bits == 16) {
+              mbar_expect_tx(full, cbytes);
+              bulk_g2s(dst, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, full);
+            } else {
+              mbar_expect_tx(full, cbytes + 512);
+              bulk_g2s(dst, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, full);
+              bulk_g2s(dst + cbytes, row.scales + tile * kTileRows, 256, full);
+              bulk_g2s(dst + cbytes + 256, row.zps + tile * kTileRows, 256, full);
             }
-            ++wcount[m];
           }
         }
       }
@@ -256,38 +428,86 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const DevRow* __res
         }
       }
     }
-  } else if (warp == 9) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+  } else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
+    // ---------------- MMA issuers ----------------
+    const int iss = warp - kWarpMma;
+    const int my_m = iss / IPM, my_p = iss % IPM;     // matrix and partial accumulator of this issuer
+    if (lane == 0 && my_p < npart) {
+      uint32_t head = 0, mma_seq = 0;               // mma_seq: 16-bit items of my matrix
       uint32_t acount = 0, bcount = 0, ucount = 0;
+      const uint32_t d_t = tmem + (my_m * npart + my_p) * nt_tile;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++ucount) {
+      for (int i = 0; ok; ++i, ++ucount) {
+        const int u = unit_index(i);
+        if (u >= n_units) break;
         const Unit un = units[u];
+        uint32_t ubits[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        ok = mbar_wait(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue of the previous unit is done
+        const uint32_t b_step = (uint32_t)(2 * nb_rows * 16) >> 4;    // descriptor advance per K-step
+        {
+          PROF_T0();
+          ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
+          PROF_ADD(4);
+        }
         if (!ok) break;
         tc_fence_after();
         for (int g = un.g0; ok && g < un.g1; ++g) {
           const int bs = bcount % n_bslots;
-          ok = mbar_wait(&c->b_full[bs], (bcount / n_bslots) & 1, c, status);
+          {
+            PROF_T0();
+            ok = mbar_wait(&c->b_full[bs], (bcount / n_bslots) & 1, c, status);
+            PROF_ADD(5);
+          }
           if (!ok) break;
-          const uint32_t baddr = smem_u32(bslots + (size_t)bs * bslot_bytes);
+          const uint64_t bd0 = make_kmajor_desc(smem_u32(bslots + (size_t)bs * bslot_bytes), nb_rows * 16);
+          const uint32_t later = (g > un.g0) ? 1u : 0u;   // accumulate onto earlier groups
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            const int as = acount % kASlots;
-            ok = mbar_wait(&c->a_full[as], (acount / kASlots) & 1, c, status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_t = tmem + (m == 0 ? kColD0 : kColD1);
-            const uint32_t a_t = tmem + kColA + as * 64;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint64_t bd = make_b_desc(baddr + kk * 2 * nb_rows * 16, nb_rows * 16);
-              tc_mma_ts(d_t, a_t + kk * 8, bd, idesc, (g > un.g0 || kk > 0) ? 1u : 0u);
+            const uint32_t bits = ubits[m];
+            const uint32_t off = ring_take(head, item_bytes(bits), wcap);
+            if (m != my_m) {
+              // The other matrix.  A quantized item still goes through the shared operand slots: watch its
+              // barrier phase go by, so that this thread never waits on a slot barrier it is a phase behind on.
+              if (bits != 16) {
+                const int as = acount % n_aslots;
+                ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
+                if (!ok) break;
+                ++acount;
+              }
+              continue;
             }
-            tc_commit(&c->a_empty[as]);
-            ++acount;
+            if (bits == 16) {
+              {
+                PROF_T0();
+                ok = mbar_wait(&c->full_mma[my_m][mma_seq % kQMma], (mma_seq / kQMma) & 1, c, status);
+                PROF_ADD(6);
+              }
+              if (!ok) break;
+              tc_fence_after();
+              const uint64_t ad0 = make_kmajor_desc(smem_u32(wring + off), 2048);
+              for (int kk = my_p; kk < 8; kk += npart)
+                tc_mma_ss(d_t, ad0 + (uint64_t)(kk * 256), bd0 + (uint64_t)(kk * b_step), idesc,
+                          (later || kk != my_p) ? 1u : 0u);
+              tc_commit(&c->empty_mma[my_m][mma_seq % kQMma]);
+              ++mma_seq;
+            } else {
+              const int as = acount % n_aslots;
+              {
+                PROF_T0();
+                ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
+                PROF_ADD(7);
+              }
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t a_t = tmem + acol + as * 64;
+              for (int kk = my_p; kk < 8; kk += npart)
+                tc_mma_ts(d_t, a_t + kk * 8, bd0 + (uint64_t)(kk * b_step), idesc, (later || kk != my_p) ? 1u : 0u);
+              tc_commit(&c->a_empty[as]);
+              ++acount;
+            }
           }
           if (!ok) break;
           tc_commit(&c->b_empty[bs]);
@@ -296,77 +516,135 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const DevRow* __res
         if (ok) tc_commit(&c->d_full);
       }
     }
-  } else {
-    // ---------------- dequantize + epilogue (warps 0..7) ----------------
-    const int set = warp >> 2, q = warp & 3;
+  } else if (warp < kDqWarps) {
+    // ---------------- dequantize ----------------
+    // Two warp-groups of eight warps; group j takes the quantized items j, j+2, j+4, .. (an item = one
+    // group of one matrix) so that each group alternates between two operand slots.  Inside a group,
+    // warp (q, h) owns rows (= TMEM lanes) 32q .. 32q+31, one row per thread, and K-half h of the item.
+    const int grp = warp >> 3, khalf = (warp >> 2) & 1, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
-    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    uint32_t wcount[NMAT] = {};
-    uint32_t acount = 0, ucount = 0;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + khalf * 32;
+    uint32_t head = 0, dq_seq = 0;
+    int pending = -1;                                // operand slot whose store has not been published yet
     bool ok = true;
-    for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++ucount) {
+    auto publish = [&]() {
+      if (pending >= 0) {
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&c->a_full[pending]);
+        pending = -1;
+      }
+    };
+    for (int i = 0; ok; ++i) {
+      const int u = unit_index(i);
+      if (u >= n_units) break;
       const Unit un = units[u];
-      const DevRow* rr = rows + un.seg * 3;
+      uint32_t ubits[NMAT];
+#pragma unroll
+      for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
       for (int g = un.g0; ok && g < un.g1; ++g) {
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
-          const uint32_t bits = rr[PHASE == 0 ? m : 2].bits;
-          const int gps = groups_per_stage(bits);
-          const int sub = (g - un.g0) % gps;
-          const int ws = m * RING + (int)(wcount[m] % RING);
-          if (sub == 0) {
-            ok = mbar_wait(&c->w_full[ws], (wcount[m] / RING) & 1, c, status);
-            if (!ok) break;
-          }
-          const int as = acount % kASlots;
-          if ((int)(acount & 1) == set) {
-            ok = mbar_wait(&c->a_empty[as], ((acount / kASlots) & 1) ^ 1, c, status);
+          const uint32_t bits = ubits[m];
+          const uint32_t off = ring_take(head, item_bytes(bits), wcap);
+          if (bits == 16) continue;                  // the MMA reads 16-bit tiles straight from shared memory
+          unsigned long long* full = &c->full_dq[dq_seq % kQDq];
+          const uint32_t par = (dq_seq / kQDq) & 1;
+          if ((int)(dq_seq & 1) == grp) {
+            if (!mbar_try(full, par)) {
+              PROF_T0();
+              publish();                             // do not sit on a finished item while waiting for HBM
+              ok = mbar_wait<20>(full, par, c, status);
+              PROF_ADD(14);
+              if (!ok) break;
+            }
+            const char* item = wring + off;
+            const int as = dq_seq % n_aslots;
+            __half2 w[32];
+            {
+              PROF_T0();
+              switch (bits) {
+                case 8: decode_item_half<8>(item, r, khalf, w); break;
+                case 4: decode_item_half<4>(item, r, khalf, w); break;
+                case 3: decode_item_half<3>(item, r, khalf, w); break;
+                default: decode_item_half<2>(item, r, khalf, w); break;
+              }
+              PROF_ADD(10);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&c->empty_dq[dq_seq % kQDq]);   // this warp has read its share of the item
+            {
+              PROF_T0();
+              publish();                             // previous item's store, overlapped with the decode above
+              PROF_ADD(11);
+            }
+            {
+              PROF_T0();
+              ok = mbar_wait<20>(&c->a_empty[as], ((dq_seq / n_aslots) & 1) ^ 1, c, status);
+              PROF_ADD(12);
+            }
             if (!ok) break;
             tc_fence_after();
-            const char* slot = wslots + (size_t)ws * kWSlotBytes;
-            const uint32_t taddr = lane_addr + kColA + as * 64;
-            switch (bits) {
-              case 16: dequant_group_to_tmem<16>(slot, sub, r, taddr); break;
-              case 8: dequant_group_to_tmem<8>(slot, sub, r, taddr); break;
-              case 4: dequant_group_to_tmem<4>(slot, sub, r, taddr); break;
-              case 3: dequant_group_to_tmem<3>(slot, sub, r, taddr); break;
-              default: dequant_group_to_tmem<2>(slot, sub, r, taddr); break;
+            {
+              PROF_T0();
+              tmem_st32(lane_addr + as * 64, w);
+              PROF_ADD(13);
             }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&c->a_full[as]);
+            pending = as;
           }
-          ++acount;
-          if (sub == gps - 1 || g == un.g1 - 1) {     // last group of this stage: hand the slot back
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&c->w_empty[ws]);
-            ++wcount[m];
-          }
+          ++dq_seq;
         }
       }
-      if (!ok) break;
-      // ---- epilogue of the unit ----
-      ok = mbar_wait(&c->d_full, ucount & 1, c, status);
+      if (ok) {
+        PROF_T0();
+        publish();
+        PROF_ADD(17);
+      }
+    }
+  } else if (warp >= kWarpEpi) {
+    // ---------------- epilogue ----------------
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    uint32_t ucount = 0;
+    bool ok = true;
+    for (int i = 0; ok; ++i, ++ucount) {
+      const int u = unit_index(i);
+      if (u >= n_units) break;
+      const Unit un = units[u];
+      ok = mbar_wait<200>(&c->d_full, ucount & 1, c, status);
       if (!ok) break;
       tc_fence_after();
       const int nb_rows = (un.ntok + 15) & ~15;
-      const int half_cols = nb_rows >> 1;              // multiple of 8
       const int row = un.row_tile * kTileRows + r;
-      for (int c0 = set * half_cols; c0 < (set + 1) * half_cols; c0 += 8) {
-        float a[8], b[8];
-        tmem_ld8(lane_addr + kColD0 + c0, a);
-        if (PHASE == 0) tmem_ld8(lane_addr + kColD1 + c0, b);
+      for (int c0 = 0; c0 < nb_rows; c0 += 16) {
+        float a[16], b[16];
+        tmem_ld16(lane_addr + c0, a);
+        if (PHASE == 0) tmem_ld16(lane_addr + npart * nt_tile + c0, b);
         tmem_wait_ld();
+        for (int p = 1; p < npart; ++p) {             // add the other issuers' partial sums, in order
+          float t[16];
+          tmem_ld16(lane_addr + p * nt_tile + c0, t);
+          tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int n = c0 + i;
+          for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
+          if (PHASE == 0) {
+            tmem_ld16(lane_addr + (npart + p) * nt_tile + c0, t);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int n = c0 + j;
           if (n < un.ntok) {
             if (PHASE == 0) {
-              const float hval = __fmul_rn(__fdiv_rn(a[i], __fadd_rn(1.0f, expf(-a[i]))), b[i]);
+              const float hval = __fmul_rn(__fdiv_rn(a[j], __fadd_rn(1.0f, expf(-a[j]))), b[j]);
               ht[((size_t)(row >> 3) * Rpad + un.tok0 + n) * 8 + (row & 7)] = __float2half_rn(hval);
             } else {
-              y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + n) * H + row] = a[i];
+              y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + n) * H + row] = a[j];
             }
           }
         }
@@ -377,19 +655,86 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const DevRow* __res
     }
   }
 
+#ifdef PW_TC_PROFILE
+  pacc__[20] += (unsigned long long)(clock64() - kernel_t0__);
+#endif
+  PROF_FLUSH();
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
 
+// ---- host side ---------------------------------------------------------------------------------
+#ifdef PW_TC_PROFILE
+extern "C" int pw_debug_read_prof(unsigned long long* host_out, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host_out, g_prof, sizeof(g_prof));
+  if (reset) {
+    static unsigned long long zeros[2][160][24];
+    cudaMemcpyToSymbol(g_prof, zeros, sizeof(g_prof));
+  }
+  return 0;
+}
+#endif
+
+struct TcState {
+  TmapSet xt, ht;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Maps over a k-chunk-major operand buffer [n_chunks][Rpad] of 16-byte units, seen as 8-byte
+// elements: box = (2 * rows) x 16 chunks, so that one copy lands [16][rows][16 B] in shared memory.
+static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, TmapSet* out) {
+  for (int i = 0; i < 8; ++i) {
+    const int rows = 16 * (i + 1);
+    cuuint64_t gdim[2] = {(cuuint64_t)Rpad * 2, (cuuint64_t)n_chunks};
+    cuuint64_t gstride[1] = {(cuuint64_t)Rpad * 16};
+    cuuint32_t box[2] = {(cuuint32_t)rows * 2, 16};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&out->m[i], CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+        CUDA_SUCCESS)
+      return false;
+  }
+  return true;
+}
+
+static pw_status tc_setup(pw_ctx* ctx) {
+  if (ctx->tc_state) return PW_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  PW_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return PW_ERR_CUDA;
+  TcState* st = new (std::nothrow) TcState();
+  if (!st) return PW_ERR_NOMEM;
+  const pw_config& c = ctx->cfg;
+  const WsMap& w = ctx->ws;
+  if (!make_maps(reinterpret_cast<EncodeTiledFn>(fn), ctx->base + w.xt, c.hidden / 8, w.Rpad, &st->xt) ||
+      !make_maps(reinterpret_cast<EncodeTiledFn>(fn), ctx->base + w.ht, c.ffn / 8, w.Rpad, &st->ht)) {
+    delete st;
+    return PW_ERR_CUDA;
+  }
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  ctx->tc_state = st;
+  return PW_OK;
+}
+
+void tc_teardown(pw_ctx* ctx) {
+  delete reinterpret_cast<TcState*>(ctx->tc_state);
+  ctx->tc_state = nullptr;
+}
+
 int tensor_token_tile(const pw_ctx* ctx, int T, int k) {
   (void)ctx;
   (void)k;
-  // an expert never holds more than T tokens; tiles of at most 128 tokens (two fp32 accumulators of
-  // 128 columns plus four 64-column operand slots fill the 512 tensor-memory columns)
+  // an expert never holds more than T tokens; tiles of at most 128 tokens
   int nt = (T + 15) & ~15;
   if (nt > 128) nt = 128;
   return nt;
@@ -399,29 +744,27 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const pw_config& c = ctx->cfg;
   const WsMap& w = ctx->ws;
   char* b = ctx->base;
+  pw_status pst = tc_setup(ctx);
+  if (pst != PW_OK) return pst;
+  const TcState* st = reinterpret_cast<const TcState*>(ctx->tc_state);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
   const int bslot_bytes = nt_tile * 256;
-  int n_bslots = (kMaxDynSmem - kCtrlBytes - kWSlots * kWSlotBytes) / bslot_bytes;
-  if (n_bslots > kMaxBSlots) n_bslots = kMaxBSlots;
-  if (n_bslots < 2) return PW_ERR_NOMEM;
-  const int smem = kCtrlBytes + kWSlots * kWSlotBytes + n_bslots * bslot_bytes;
-  if (!ctx->tc_state) {
-    PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-    ctx->tc_state = ctx;
-  }
+  const int n_bslots = nt_tile <= 64 ? 4 : 2;
+  const uint32_t wcap = (uint32_t)((kMaxDynSmem - kCtrlBytes - n_bslots * bslot_bytes) & ~1023);
+  if (wcap < 3 * 32768) return PW_ERR_NOMEM;
+  const int smem = kCtrlBytes + (int)wcap + n_bslots * bslot_bytes;
   const int R = T * k + c.n_shared * T;
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
-                                                        reinterpret_cast<const uint4*>(b + w.xt), w.Rpad, nt_tile,
-                                                        n_bslots, reinterpret_cast<__half*>(b + w.ht), nullptr,
-                                                        c.hidden, 0, status);
+                                                        st->xt, w.Rpad, nt_tile, n_bslots, wcap,
+                                                        reinterpret_cast<__half*>(b + w.ht), nullptr, c.hidden, 0,
+                                                        status);
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
-                                                        reinterpret_cast<const uint4*>(b + w.ht), w.Rpad, nt_tile,
-                                                        n_bslots, nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
+                                                        st->ht, w.Rpad, nt_tile, n_bslots, wcap, nullptr,
+                                                        reinterpret_cast<float*>(b + w.y), c.hidden,
                                                         (size_t)R * c.hidden, status);
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());

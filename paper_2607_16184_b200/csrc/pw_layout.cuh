@@ -134,17 +134,17 @@ __device__ inline __half2 dq_pair(uint32_t magic_or_code, __half2 s2, __half2 z2
   return __hfma2(__hsub2(u32_as_h2(magic_or_code), k1024), s2, z2);
 }
 
-// Half h (0 or 1) of a row-group: out[p] = weights (64h + 2p, 64h + 2p + 1), p = 0 .. 31.
+// Quarter t (0 .. 3) of a row-group: out[p] = weights (32t + 2p, 32t + 2p + 1), p = 0 .. 15.
 // `row_units` points at unit 0 of the row inside a tile image (shared or global memory); unit j
-// of the same row is kTileRowsStride uint4 further on.
+// of the same row is kUnitStride uint4 further on.
 constexpr int kUnitStride = 128;  // uint4 elements between consecutive units of one row
 
 template <int BITS>
-__device__ __forceinline__ void decode_half(const uint4* row_units, int h, __half2 s2, __half2 z2, __half2* out) {
+__device__ __forceinline__ void decode_quarter(const uint4* row_units, int t, __half2 s2, __half2 z2, __half2* out) {
   if constexpr (BITS == 16) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const uint4 u = row_units[(8 * h + j) * kUnitStride];
+    for (int j = 0; j < 4; ++j) {
+      const uint4 u = row_units[(4 * t + j) * kUnitStride];
       out[4 * j + 0] = u32_as_h2(u.x);
       out[4 * j + 1] = u32_as_h2(u.y);
       out[4 * j + 2] = u32_as_h2(u.z);
@@ -152,8 +152,8 @@ __device__ __forceinline__ void decode_half(const uint4* row_units, int h, __hal
     }
   } else if constexpr (BITS == 8) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint4 u = row_units[(4 * h + j) * kUnitStride];
+    for (int j = 0; j < 2; ++j) {
+      const uint4 u = row_units[(2 * t + j) * kUnitStride];
       const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -162,41 +162,40 @@ __device__ __forceinline__ void decode_half(const uint4* row_units, int h, __hal
       }
     }
   } else if constexpr (BITS == 4) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const uint4 u = row_units[(2 * h + j) * kUnitStride];
-      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int m = 0; m < 4; ++m)
-          out[16 * j + 4 * i + m] = dq_pair(((w[i] >> (4 * m)) & 0x000f000fu) | 0x64006400u, s2, z2);
-    }
-  } else if constexpr (BITS == 2) {
-    const uint4 u = row_units[h * kUnitStride];
+    const uint4 u = row_units[t * kUnitStride];
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int m = 0; m < 8; ++m)
-        out[8 * i + m] = dq_pair(((w[i] >> (2 * m)) & 0x00030003u) | 0x64006400u, s2, z2);
-  } else {  // 3 bits: low planes in unit h, high-plane words 2h, 2h+1 of unit 2
-    const uint4 u = row_units[h * kUnitStride];
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-    const uint2 hv = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + 2 * kUnitStride) + 2 * h);
-    const uint32_t wh[2] = {hv.x, hv.y};
+      for (int m = 0; m < 4; ++m)
+        out[4 * i + m] = dq_pair(((w[i] >> (4 * m)) & 0x000f000fu) | 0x64006400u, s2, z2);
+  } else {
+    // 2 bits: words 2(t%2), 2(t%2)+1 of unit t/2.  3 bits: the same low-plane words plus word t of unit 2.
+    const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + (t >> 1) * kUnitStride) +
+                                                     2 * (t & 1));
+    const uint32_t w[2] = {u.x, u.y};
+    uint32_t hw = 0;
+    if constexpr (BITS == 3) hw = reinterpret_cast<const uint32_t*>(row_units + 2 * kUnitStride)[t];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 2; ++i)
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
-        const int p = 8 * i + m;                 // pair index inside the half
-        const int hb = p & 15;                   // pair index inside its high-plane word
-        const uint32_t hw = wh[p >> 4];
-        const uint32_t hi = hb >= 2 ? (hw >> (hb - 2)) : (hw << (2 - hb));
-        const uint32_t lo = (w[i] >> (2 * m)) & 0x00030003u;
-        out[p] = dq_pair((hi & 0x00040004u) | lo | 0x64006400u, s2, z2);
+        const int p = 8 * i + m;                   // pair index inside the quarter = inside the high-plane word
+        uint32_t v = ((w[i] >> (2 * m)) & 0x00030003u) | 0x64006400u;
+        if constexpr (BITS == 3) {
+          const uint32_t hi = p >= 2 ? (hw >> (p - 2)) : (hw << (2 - p));
+          v |= hi & 0x00040004u;
+        }
+        out[p] = dq_pair(v, s2, z2);
       }
   }
+}
+
+// Half h (0 or 1) of a row-group: out[p] = weights (64h + 2p, 64h + 2p + 1), p = 0 .. 31.
+template <int BITS>
+__device__ __forceinline__ void decode_half(const uint4* row_units, int h, __half2 s2, __half2 z2, __half2* out) {
+  decode_quarter<BITS>(row_units, 2 * h, s2, z2, out);
+  decode_quarter<BITS>(row_units, 2 * h + 1, s2, z2, out + 16);
 }
 
 }  // namespace pw
