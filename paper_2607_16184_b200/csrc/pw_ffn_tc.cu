@@ -3,28 +3,32 @@
 //   D[128 weight rows, N tokens] += W[128, 16] * X[N, 16]^T      (tcgen05.mma, kind::f16, fp32 in TMEM)
 //
 // Weight pages stream HBM -> shared memory with bulk async copies, one item (128 rows x one group of
-// one page, 4.5 .. 32 KB) at a time into a FIFO ring that holds as many items as fit, so that enough
-// bytes are in flight to cover the HBM latency whatever the bitwidth.  A 16-bit page tile is already in the tensor core's K-major core-matrix layout,
-// so the MMA reads it from shared memory as the A operand without any thread touching it.  A
-// quantized tile is unpacked and dequantized in registers (one weight row per thread) and written
-// to tensor memory, which the MMA then reads as its A operand.  The token tile (B operand) comes
-// from the k-chunk-major operand buffers with one 2-D TMA copy per group.
+// one page, 4.5 .. 32 KB) at a time, into a ring of 17 KB slots (a 16-bit item takes two).  A 16-bit
+// tile is already in the tensor core's K-major core-matrix layout, so the MMA reads it from shared
+// memory as the A operand without any thread touching it.  A quantized tile is unpacked and
+// dequantized in registers (one weight row per thread) and written to tensor memory, which the MMA
+// then reads as its A operand.  The token tile (B operand) comes from the k-chunk-major operand
+// buffers with one 2-D TMA copy per group.
 //
-// One persistent CTA per SM, 25 warps:
-//   warps 0-15   dequantize: two groups of eight warps, each group takes every other quantized
-//                128x128 slab; warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
-//   warp 16      producer: one thread issues every copy (weight stages and token tiles);
-//   warps 17-20  MMA issuers (warp 17 also allocates tensor memory).  A tcgen05.mma holds its issuing
+// One persistent CTA per SM, 19 warps.  The control roles are single threads with short dependent
+// instruction chains: they share the schedulers with the arithmetic-heavy dequantizers, and every
+// instruction of theirs waits its turn.
+//   warps 0-7    dequantize: two groups of four warps, group j takes the quantized items j, j+2, ..;
+//                warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
+//   warp 8       weight producer: arms an item's barrier and copies its codes, as far ahead as the
+//                slot ring allows;
+//   warp 9       copies scales and zero-points of the items the weight producer has armed;
+//   warp 10      token-tile producer (its own few slots, never holds back the weight stream);
+//   warps 11-14  MMA issuers (warp 11 also allocates tensor memory).  A tcgen05.mma holds its issuing
 //                thread for ~95 cycles whatever its size, so one issuer caps the SM at one 128x16
 //                weight slab per 95 cycles; four issuers in four warps overlap.  Each issuer owns the
 //                K-steps k = j mod (issuers per matrix) of one matrix and its own partial accumulator,
 //                so no two threads ever accumulate into the same columns; the epilogue adds the partials;
-//   warps 21-24  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
-//                split-K partial of the down projection (PHASE 1); accumulators are double-buffered
-//                when they fit so the next unit's MMAs overlap the epilogue.
-// Units are dealt to CTAs in snake order over a size-sorted list.  Every wait on an mbarrier is
-// bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work,
-// frees its tensor memory and returns.
+//   warps 15-18  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
+//                split-K partial of the down projection (PHASE 1).
+// Units are dealt to CTAs in snake order over a size-sorted list.  Every wait is bounded; when one
+// runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
+// memory and returns.
 #include <cuda.h>
 
 #include <new>
@@ -34,48 +38,39 @@
 
 namespace pw {
 
-constexpr int kQDq = 16;                       // quantized items in flight (barrier pairs)
-constexpr int kQMma = 8;                       // 16-bit items in flight
+constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item (16 KB codes + 512 B) fits
+constexpr int kMaxSlots = 16;
 constexpr int kMaxASlots = 8;                  // dequantized groups in tensor memory (64 columns each)
 constexpr int kMaxBSlots = 4;
-constexpr int kCtrlBytes = 2048;
+constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
-constexpr int kDqWarps = 16;
-constexpr int kWarpProducer = 16, kWarpMma = 17, kIssuers = 4, kWarpEpi = 21;
-constexpr int kThreads = 800;
+constexpr int kDqWarps = 8;
+constexpr int kWarpCodes = 8, kWarpMeta = 9, kWarpTokens = 10, kWarpMma = 11, kIssuers = 4, kWarpEpi = 15;
+constexpr int kThreads = 608;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct Ctrl {                                  // lives at the start of dynamic shared memory
-  // A weight item is consumed either by the dequantizers (quantized page) or by the MMA issuers (16-bit
-  // page); each kind has its own sequence of full / empty barriers so that every waiter sees every phase.
-  unsigned long long full_dq[kQDq], empty_dq[kQDq];
-  unsigned long long full_mma[2][kQMma], empty_mma[2][kQMma];   // per matrix of the unit (gate / up)
+  // One full barrier per ring slot (armed by the weight producer).  A slot is handed back either by the
+  // four warps of the dequantizer group that read it (empty_dq) or by the MMA issuers of its matrix
+  // (empty_mma, through tcgen05.commit); the weight producer remembers which.
+  unsigned long long full[kMaxSlots], empty_dq[kMaxSlots], empty_mma[kMaxSlots];
   unsigned long long b_full[kMaxBSlots], b_empty[kMaxBSlots];
   unsigned long long a_full[kMaxASlots], a_empty[kMaxASlots];
   unsigned long long d_full, d_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
-  uint32_t q_off[64], q_seq[64];              // producer's queue of items in flight
+  volatile uint32_t issued;                    // items 0 .. issued-1 have been armed by the weight producer
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
 #ifdef PW_TC_PROFILE
-// Diagnostic build only: per-CTA cycle counters of where each role waits (kept in registers, flushed once).
-__device__ unsigned long long g_prof[2][160][24];
-#define PROF_DECL() unsigned long long pacc__[24] = {}
-#define PROF_T0() const long long pt0__ = clock64()
-#define PROF_ADD(slot) pacc__[slot] += (unsigned long long)(clock64() - pt0__)
-#define PROF_FLUSH()                                                                        \
-  if (lane == 0 && (warp == 0 || warp == kWarpProducer || warp == kWarpMma)) {              \
-    _Pragma("unroll") for (int i__ = 0; i__ < 24; ++i__) if (pacc__[i__])                   \
-        g_prof[PHASE][blockIdx.x][i__] += pacc__[i__];                                      \
-  }
+// Diagnostic build only: time stamps of the first few hundred items of CTA 0.
+__device__ long long g_trace[16][512];
+#define TRACE(ev, n) \
+  if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
 #else
-#define PROF_DECL()
-#define PROF_T0()
-#define PROF_ADD(slot)
-#define PROF_FLUSH()
+#define TRACE(ev, n)
 #endif
 
 struct TmapSet {                               // token-tile copies: one map per tile height 16, 32, .. 128
@@ -98,11 +93,7 @@ __device__ __forceinline__ bool mbar_try(unsigned long long* b, uint32_t parity)
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-#ifdef PW_TC_PROFILE
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"   // non-blocking, so that waits are measured
-#else
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#endif
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(b)), "r"(parity)
@@ -203,17 +194,33 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Shared-memory footprint of one item (one 128-row x one-group tile of one page): codes, then the
-// 128 scales, then the 128 zero-points; rounded up to 1 KB.
-__device__ __forceinline__ uint32_t item_bytes(uint32_t bits) {
-  return bits == 16 ? 32768u : ((bits * 2048u + 512u + 1023u) & ~1023u);
+// Ring slots an item needs: a 16-bit tile is 32 KB, every quantized tile (codes, then its 128 scales,
+// then its 128 zero-points) fits one slot.
+__device__ __forceinline__ int item_slots(uint32_t bits) { return bits == 16 ? 2 : 1; }
+// Slots are handed out cyclically; an item never wraps (a two-slot item skips a lone last slot).
+// Every role replays the same sequence.
+__device__ __forceinline__ int slot_take(int& head, int k, int n_slots) {
+  if (head + k > n_slots) head = 0;
+  const int s = head;
+  head += k;
+  return s;
 }
-// The weight ring is a FIFO of variable-sized items.  Every role replays the same allocation sequence.
-__device__ __forceinline__ uint32_t ring_take(uint32_t& head, uint32_t sz, uint32_t cap) {
-  if (head + sz > cap) head = 0;
-  const uint32_t off = head;
-  head += sz;
-  return off;
+// Bounded wait until the weight producer has armed item n.  A consumer looks at an item's full barrier
+// only after this, so it can never mistake an older phase of the slot's barrier for the item's.
+__device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
+  if (c->issued > n) return true;
+  const unsigned long long t0 = globaltimer();
+  uint32_t spins = 0;
+  while (true) {
+    __nanosleep(32);
+    if (c->issued > n) return true;
+    if (c->abort_flag) return false;
+    if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
+      c->abort_flag = 1;
+      atomicMax(status, (int)PW_ERR_TIMEOUT);
+      return false;
+    }
+  }
 }
 
 // Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
@@ -242,13 +249,13 @@ __device__ __forceinline__ void decode_item_half(const char* item, int r, int h,
 template <int PHASE>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, const int32_t* __restrict__ n_units_ptr,
-              const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, uint32_t wcap,
+              const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
               __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
               int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   char* wring = smem + kCtrlBytes;
-  char* bslots = wring + wcap;
+  char* bslots = wring + n_slots * kSlotBytes;
   const int bslot_bytes = nt_tile * 256;
   constexpr int NMAT = PHASE == 0 ? 2 : 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -264,26 +271,23 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kQDq; ++i) {
-      mbar_init(&c->full_dq[i], 1);
-      mbar_init(&c->empty_dq[i], 8);          // the eight warps of the group that owns the item
+    for (int i = 0; i < kMaxSlots; ++i) {
+      mbar_init(&c->full[i], 1);
+      mbar_init(&c->empty_dq[i], 4);             // the four warps of the group that owns the item
+      mbar_init(&c->empty_mma[i], npart);
     }
-    for (int i = 0; i < kQMma; ++i)
-      for (int m = 0; m < 2; ++m) {
-        mbar_init(&c->full_mma[m][i], 1);
-        mbar_init(&c->empty_mma[m][i], npart);
-      }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
       mbar_init(&c->b_empty[i], n_issuers);
     }
     for (int i = 0; i < kMaxASlots; ++i) {
-      mbar_init(&c->a_full[i], 8);
-      mbar_init(&c->a_empty[i], npart);
+      mbar_init(&c->a_full[i], 4);
+      mbar_init(&c->a_empty[i], n_issuers);      // every issuer lets go of an operand slot, see below
     }
     mbar_init(&c->d_full, n_issuers);
     mbar_init(&c->d_empty, 4);
     c->abort_flag = 0;
+    c->issued = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -297,143 +301,120 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = c->tmem_base;
-  PROF_DECL();
-#ifdef PW_TC_PROFILE
-  const long long kernel_t0__ = clock64();
-#endif
 
   // unit i of this CTA in snake order over the size-sorted list
   auto unit_index = [&](int i) { return i * G + ((i & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x); };
 
-  if (warp == kWarpProducer) {
-    // ---------------- producer ----------------
+  if (warp == kWarpCodes) {
+    // ---------------- weight producer ----------------
     if (lane == 0) {
-      // Items in flight, oldest first, in a small circular queue in shared memory: ring offset and the
-      // sequence tag that says which barrier frees the item (bits 30-31 = 1 + matrix for 16-bit items).
-      constexpr int NQ = 64;
-      uint32_t* q_off = c->q_off;
-      uint32_t* q_seq = c->q_seq;
-      int q_head = 0, q_count = 0;
-      uint32_t head = 0, dq_seq = 0, bcount = 0;
-      uint32_t mma_seq0 = 0, mma_seq1 = 0;
-      // releases are observed strictly in sequence per kind, so that no barrier phase is ever skipped
-      uint32_t rel_dq = 0, rel_mma0 = 0, rel_mma1 = 0;   // items 0 .. rel-1 of the kind are known to be released
+      int head = 0;
+      uint32_t n = 0;                              // item sequence number
+      // Per-slot state, one bit per slot.  lk_*: who hands the slot back (a dequantizer group, the MMA
+      // issuers, or the MMA issuers through the barrier of the slot before it, for the second slot of a
+      // 16-bit item).  ed_par / em_par: parity of the next phase of empty_dq / empty_mma of the slot.
+      uint32_t lk_dq = 0, lk_mma = 0, lk_mma2 = 0, ed_par = 0, em_par = 0;
       bool ok = true;
-#define PW_RELEASED_DQ(S)                                                                              \
-  while (ok && rel_dq <= (S)) {                                                                        \
-    ok = mbar_wait<64>(&c->empty_dq[rel_dq % kQDq], (rel_dq / kQDq) & 1, c, status);                   \
-    ++rel_dq;                                                                                          \
-  }
-#define PW_RELEASED_MMA(M, S)                                                                          \
-  {                                                                                                    \
-    uint32_t& rel__ = (M) == 0 ? rel_mma0 : rel_mma1;                                                  \
-    while (ok && rel__ <= (S)) {                                                                       \
-      ok = mbar_wait<64>(&c->empty_mma[M][rel__ % kQMma], (rel__ / kQMma) & 1, c, status);             \
-      ++rel__;                                                                                         \
-    }                                                                                                  \
-  }
       for (int i = 0; ok; ++i) {
         const int u = unit_index(i);
         if (u >= n_units) break;
         const Unit un = units[u];
-        DevRow urow[NMAT];
-#pragma unroll
-        for (int m = 0; m < NMAT; ++m) urow[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
-        const int nb_rows = (un.ntok + 15) & ~15;
-        const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
         for (int g = un.g0; ok && g < un.g1; ++g) {
-          {  // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
-            const int bs = bcount % n_bslots;
-            {
-              PROF_T0();
-              ok = mbar_wait<64>(&c->b_empty[bs], ((bcount / n_bslots) & 1) ^ 1, c, status);
-              PROF_ADD(0);
-            }
-            if (!ok) break;
-            mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
-            tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
-            ++bcount;
-          }
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            const DevRow& row = urow[m];
+            const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
             const uint32_t bits = row.bits;
-            const uint32_t sz = item_bytes(bits);
-            const uint32_t head_prev = head;
-            const uint32_t off = ring_take(head, sz, wcap);
-            // The items in flight occupy a circular span from the oldest item's offset (tail) up to
-            // head_prev.  Pop (wait for the release of) oldest items until [off, off+sz) is clear of it.
-            {
-              PROF_T0();
-              while (ok && q_count > 0) {
-                const uint32_t tail = q_off[q_head];
-                bool free_now;
-                if (tail < head_prev) free_now = (off == head_prev) || (sz <= tail);          // span [tail, head_prev)
-                else free_now = (off == head_prev) && (off + sz <= tail);                      // span wraps around
-                if (free_now && q_count < NQ) break;
-                const uint32_t sq = q_seq[q_head];
-                if (sq >> 30) {
-                  if ((sq >> 30) == 1) PW_RELEASED_MMA(0, sq & 0x3fffffffu) else PW_RELEASED_MMA(1, sq & 0x3fffffffu)
-                } else {
-                  PW_RELEASED_DQ(sq)
-                }
-                q_head = (q_head + 1) % NQ;
-                --q_count;
-              }
-              PROF_ADD(1);
+            const int k = item_slots(bits);
+            const int s = slot_take(head, k, n_slots);
+            // every slot the item covers must have been handed back by its last occupant
+            for (int j = s; ok && j < s + k; ++j) {
+              const uint32_t bit = 1u << j;
+              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
+              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
+              else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
+              lk_dq &= ~bit;
+              lk_mma &= ~bit;
+              lk_mma2 &= ~bit;
             }
             if (!ok) break;
-            // the barrier pair of this item must be free too: at most kQ* items of a kind in flight
-            unsigned long long* full;
-            uint32_t seqtag;
-            if (bits == 16) {
-              uint32_t& ms = m == 0 ? mma_seq0 : mma_seq1;
-              if (ms >= (uint32_t)kQMma) {
-                if (m == 0) PW_RELEASED_MMA(0, ms - kQMma) else PW_RELEASED_MMA(1, ms - kQMma)
-              }
-              full = &c->full_mma[m][ms % kQMma];
-              seqtag = ms | ((uint32_t)(m + 1) << 30);
-              ++ms;
-            } else {
-              if (dq_seq >= (uint32_t)kQDq) PW_RELEASED_DQ(dq_seq - kQDq)
-              full = &c->full_dq[dq_seq % kQDq];
-              seqtag = dq_seq;
-              ++dq_seq;
-            }
-            if (!ok) break;
-            const int qt = (q_head + q_count) % NQ;
-            q_off[qt] = off;
-            q_seq[qt] = seqtag;
-            ++q_count;
-            const int ng = row.cols / kGroup;
-            const size_t tile = (size_t)un.row_tile * ng + g;
             const uint32_t cbytes = bits * 2048;
-            char* dst = wring + off;
+            const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + g;
+            TRACE(0, n);
+            mbar_expect_tx(&c->full[s], bits == 16 ? cbytes : cbytes + 512);
+            bulk_g2s(wring + s * kSlotBytes, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, &c->full[s]);
             if (bits == 16) {
-              mbar_expect_tx(full, cbytes);
-              bulk_g2s(dst, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, full);
+              lk_mma |= 1u << s;
+              lk_mma2 |= 1u << (s + 1);
+              em_par ^= 1u << s;
             } else {
-              mbar_expect_tx(full, cbytes + 512);
-              bulk_g2s(dst, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, full);
-              bulk_g2s(dst + cbytes, row.scales + tile * kTileRows, 256, full);
-              bulk_g2s(dst + cbytes + 256, row.zps + tile * kTileRows, 256, full);
+              lk_dq |= 1u << s;
+              ed_par ^= 1u << s;
             }
+            ++n;
+            c->issued = n;
           }
-        }
-      }
-      if (!ok) {
-        // let copies already in flight land before the CTA leaves (bounded)
-        const unsigned long long t0 = globaltimer();
-        while (globaltimer() - t0 < 200000ull) {
         }
       }
     }
-  } else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
+  } else if (warp == kWarpMeta) {
+    // ---------------- scales / zero-points producer ----------------
+    if (lane == 0) {
+      int head = 0;
+      uint32_t n = 0;
+      bool ok = true;
+      for (int i = 0; ok; ++i) {
+        const int u = unit_index(i);
+        if (u >= n_units) break;
+        const Unit un = units[u];
+        for (int g = un.g0; ok && g < un.g1; ++g) {
+#pragma unroll
+          for (int m = 0; m < NMAT; ++m) {
+            const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+            const uint32_t bits = row.bits;
+            const int s = slot_take(head, item_slots(bits), n_slots);
+            if (bits != 16) {
+              ok = wait_issued(n, c, status);        // the slot is free and its barrier armed for this item
+              if (!ok) break;
+              const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + g;
+              char* dst = wring + s * kSlotBytes + bits * 2048;
+              bulk_g2s(dst, row.scales + tile * kTileRows, 256, &c->full[s]);
+              bulk_g2s(dst + 256, row.zps + tile * kTileRows, 256, &c->full[s]);
+            }
+            ++n;
+          }
+        }
+      }
+    }
+  } else if (warp == kWarpTokens) {
+    // ---------------- token-tile producer ----------------
+    if (lane == 0) {
+      uint32_t bcount = 0;
+      bool ok = true;
+      for (int i = 0; ok; ++i) {
+        const int u = unit_index(i);
+        if (u >= n_units) break;
+        const Unit un = units[u];
+        const int nb_rows = (un.ntok + 15) & ~15;
+        const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
+        for (int g = un.g0; ok && g < un.g1; ++g) {
+          // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
+          const int bs = bcount % n_bslots;
+          ok = mbar_wait<64>(&c->b_empty[bs], ((bcount / n_bslots) & 1) ^ 1, c, status);
+          if (!ok) break;
+          mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
+          tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
+          ++bcount;
+        }
+      }
+    }
+  }
+  else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
     // ---------------- MMA issuers ----------------
     const int iss = warp - kWarpMma;
     const int my_m = iss / IPM, my_p = iss % IPM;     // matrix and partial accumulator of this issuer
     if (lane == 0 && my_p < npart) {
-      uint32_t head = 0, mma_seq = 0;               // mma_seq: 16-bit items of my matrix
+      int head = 0;
+      uint32_t n = 0, full_par = 0;                 // item sequence number; per-slot parity of the full barrier
       uint32_t acount = 0, bcount = 0, ucount = 0;
       const uint32_t d_t = tmem + (my_m * npart + my_p) * nt_tile;
       bool ok = true;
@@ -447,65 +428,55 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         const uint32_t b_step = (uint32_t)(2 * nb_rows * 16) >> 4;    // descriptor advance per K-step
-        {
-          PROF_T0();
-          ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
-          PROF_ADD(4);
-        }
+        ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
         if (!ok) break;
         tc_fence_after();
         for (int g = un.g0; ok && g < un.g1; ++g) {
           const int bs = bcount % n_bslots;
-          {
-            PROF_T0();
-            ok = mbar_wait(&c->b_full[bs], (bcount / n_bslots) & 1, c, status);
-            PROF_ADD(5);
-          }
+          ok = mbar_wait(&c->b_full[bs], (bcount / n_bslots) & 1, c, status);
           if (!ok) break;
           const uint64_t bd0 = make_kmajor_desc(smem_u32(bslots + (size_t)bs * bslot_bytes), nb_rows * 16);
           const uint32_t later = (g > un.g0) ? 1u : 0u;   // accumulate onto earlier groups
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
             const uint32_t bits = ubits[m];
-            const uint32_t off = ring_take(head, item_bytes(bits), wcap);
+            const int s = slot_take(head, item_slots(bits), n_slots);
+            const uint32_t par = (full_par >> s) & 1;
+            full_par ^= 1u << s;
+            const uint32_t item_n = n++;
             if (m != my_m) {
               // The other matrix.  A quantized item still goes through the shared operand slots: watch its
-              // barrier phase go by, so that this thread never waits on a slot barrier it is a phase behind on.
+              // barrier phase go by and let go of the slot, so that the slot is never refilled before every
+              // issuer has seen this phase (a thread that misses a phase would wait on the wrong one for ever).
               if (bits != 16) {
                 const int as = acount % n_aslots;
                 ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
                 if (!ok) break;
+                mbar_arrive(&c->a_empty[as]);
                 ++acount;
               }
               continue;
             }
             if (bits == 16) {
-              {
-                PROF_T0();
-                ok = mbar_wait(&c->full_mma[my_m][mma_seq % kQMma], (mma_seq / kQMma) & 1, c, status);
-                PROF_ADD(6);
-              }
+              ok = wait_issued(item_n, c, status) && mbar_wait(&c->full[s], par, c, status);
               if (!ok) break;
               tc_fence_after();
-              const uint64_t ad0 = make_kmajor_desc(smem_u32(wring + off), 2048);
+              const uint64_t ad0 = make_kmajor_desc(smem_u32(wring + s * kSlotBytes), 2048);
               for (int kk = my_p; kk < 8; kk += npart)
                 tc_mma_ss(d_t, ad0 + (uint64_t)(kk * 256), bd0 + (uint64_t)(kk * b_step), idesc,
                           (later || kk != my_p) ? 1u : 0u);
-              tc_commit(&c->empty_mma[my_m][mma_seq % kQMma]);
-              ++mma_seq;
+              tc_commit(&c->empty_mma[s]);
             } else {
               const int as = acount % n_aslots;
-              {
-                PROF_T0();
-                ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
-                PROF_ADD(7);
-              }
+              ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
               if (!ok) break;
               tc_fence_after();
+              if (my_p == 0) { TRACE(8, item_n); }
               const uint32_t a_t = tmem + acol + as * 64;
               for (int kk = my_p; kk < 8; kk += npart)
                 tc_mma_ts(d_t, a_t + kk * 8, bd0 + (uint64_t)(kk * b_step), idesc, (later || kk != my_p) ? 1u : 0u);
               tc_commit(&c->a_empty[as]);
+              if (my_p == 0) { TRACE(9, item_n); }
               ++acount;
             }
           }
@@ -518,13 +489,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     }
   } else if (warp < kDqWarps) {
     // ---------------- dequantize ----------------
-    // Two warp-groups of eight warps; group j takes the quantized items j, j+2, j+4, .. (an item = one
-    // group of one matrix) so that each group alternates between two operand slots.  Inside a group,
-    // warp (q, h) owns rows (= TMEM lanes) 32q .. 32q+31, one row per thread, and K-half h of the item.
-    const int grp = warp >> 3, khalf = (warp >> 2) & 1, q = warp & 3;
+    // Two groups of four warps; group j takes the quantized items j, j+2, j+4, .. (an item = one group of
+    // one matrix), so each group alternates between two operand slots.  Warp q of a group owns rows
+    // (= TMEM lanes) 32q .. 32q+31 of the item, one row per thread, all 128 weights of the row.
+    const int grp = warp >> 2, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
-    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + khalf * 32;
-    uint32_t head = 0, dq_seq = 0;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol;
+    int head = 0;
+    uint32_t n = 0, full_par = 0, dq_seq = 0;
     int pending = -1;                                // operand slot whose store has not been published yet
     bool ok = true;
     auto publish = [&]() {
@@ -547,60 +519,54 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
           const uint32_t bits = ubits[m];
-          const uint32_t off = ring_take(head, item_bytes(bits), wcap);
+          const int s = slot_take(head, item_slots(bits), n_slots);
+          const uint32_t par = (full_par >> s) & 1;
+          full_par ^= 1u << s;
+          const uint32_t item_n = n++;
           if (bits == 16) continue;                  // the MMA reads 16-bit tiles straight from shared memory
-          unsigned long long* full = &c->full_dq[dq_seq % kQDq];
-          const uint32_t par = (dq_seq / kQDq) & 1;
           if ((int)(dq_seq & 1) == grp) {
-            if (!mbar_try(full, par)) {
-              PROF_T0();
+            if (c->issued <= item_n || !mbar_try(&c->full[s], par)) {
               publish();                             // do not sit on a finished item while waiting for HBM
-              ok = mbar_wait<20>(full, par, c, status);
-              PROF_ADD(14);
+              ok = wait_issued(item_n, c, status) && mbar_wait<20>(&c->full[s], par, c, status);
               if (!ok) break;
             }
-            const char* item = wring + off;
+            if (q == 0) { TRACE(1, item_n); }
+            const char* item = wring + s * kSlotBytes;
             const int as = dq_seq % n_aslots;
+            const uint32_t taddr = lane_addr + as * 64;
             __half2 w[32];
-            {
-              PROF_T0();
-              switch (bits) {
-                case 8: decode_item_half<8>(item, r, khalf, w); break;
-                case 4: decode_item_half<4>(item, r, khalf, w); break;
-                case 3: decode_item_half<3>(item, r, khalf, w); break;
-                default: decode_item_half<2>(item, r, khalf, w); break;
-              }
-              PROF_ADD(10);
+            switch (bits) {
+              case 8: decode_item_half<8>(item, r, 0, w); break;
+              case 4: decode_item_half<4>(item, r, 0, w); break;
+              case 3: decode_item_half<3>(item, r, 0, w); break;
+              default: decode_item_half<2>(item, r, 0, w); break;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&c->empty_dq[dq_seq % kQDq]);   // this warp has read its share of the item
-            {
-              PROF_T0();
-              publish();                             // previous item's store, overlapped with the decode above
-              PROF_ADD(11);
-            }
-            {
-              PROF_T0();
-              ok = mbar_wait<20>(&c->a_empty[as], ((dq_seq / n_aslots) & 1) ^ 1, c, status);
-              PROF_ADD(12);
-            }
+            if (q == 0) { TRACE(2, item_n); }
+            publish();                               // previous item's store, overlapped with the decode above
+            if (q == 0) { TRACE(3, item_n); }
+            ok = mbar_wait<20>(&c->a_empty[as], ((dq_seq / n_aslots) & 1) ^ 1, c, status);
             if (!ok) break;
             tc_fence_after();
-            {
-              PROF_T0();
-              tmem_st32(lane_addr + as * 64, w);
-              PROF_ADD(13);
+            if (q == 0) { TRACE(4, item_n); }
+            tmem_st32(taddr, w);
+            if (q == 0) { TRACE(5, item_n); }
+            switch (bits) {
+              case 8: decode_item_half<8>(item, r, 1, w); break;
+              case 4: decode_item_half<4>(item, r, 1, w); break;
+              case 3: decode_item_half<3>(item, r, 1, w); break;
+              default: decode_item_half<2>(item, r, 1, w); break;
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
+            if (q == 0) { TRACE(6, item_n); }
+            tmem_st32(taddr + 32, w);
+            if (q == 0) { TRACE(7, item_n); }
             pending = as;
           }
           ++dq_seq;
         }
       }
-      if (ok) {
-        PROF_T0();
-        publish();
-        PROF_ADD(17);
-      }
+      if (ok) publish();
     }
   } else if (warp >= kWarpEpi) {
     // ---------------- epilogue ----------------
@@ -638,13 +604,13 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const int n = c0 + j;
-          if (n < un.ntok) {
+          const int nn = c0 + j;
+          if (nn < un.ntok) {
             if (PHASE == 0) {
               const float hval = __fmul_rn(__fdiv_rn(a[j], __fadd_rn(1.0f, expf(-a[j]))), b[j]);
-              ht[((size_t)(row >> 3) * Rpad + un.tok0 + n) * 8 + (row & 7)] = __float2half_rn(hval);
+              ht[((size_t)(row >> 3) * Rpad + un.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
             } else {
-              y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + n) * H + row] = a[j];
+              y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + nn) * H + row] = a[j];
             }
           }
         }
@@ -655,10 +621,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     }
   }
 
-#ifdef PW_TC_PROFILE
-  pacc__[20] += (unsigned long long)(clock64() - kernel_t0__);
-#endif
-  PROF_FLUSH();
   tc_fence_before();
   __syncthreads();
   if (warp == kWarpMma) {
@@ -669,17 +631,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 
 // ---- host side ---------------------------------------------------------------------------------
 #ifdef PW_TC_PROFILE
-extern "C" int pw_debug_read_prof(unsigned long long* host_out, int reset) {
+extern "C" int pw_debug_read_trace(long long* host_out) {
   cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, g_prof, sizeof(g_prof));
-  if (reset) {
-    static unsigned long long zeros[2][160][24];
-    cudaMemcpyToSymbol(g_prof, zeros, sizeof(g_prof));
-  }
+  cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace));
   return 0;
 }
 #endif
-
 struct TcState {
   TmapSet xt, ht;
 };
@@ -750,20 +707,21 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
   const int bslot_bytes = nt_tile * 256;
   const int n_bslots = nt_tile <= 64 ? 4 : 2;
-  const uint32_t wcap = (uint32_t)((kMaxDynSmem - kCtrlBytes - n_bslots * bslot_bytes) & ~1023);
-  if (wcap < 3 * 32768) return PW_ERR_NOMEM;
-  const int smem = kCtrlBytes + (int)wcap + n_bslots * bslot_bytes;
+  int n_slots = (kMaxDynSmem - kCtrlBytes - n_bslots * bslot_bytes) / kSlotBytes;
+  if (n_slots > kMaxSlots) n_slots = kMaxSlots;
+  if (n_slots < 4) return PW_ERR_NOMEM;
+  const int smem = kCtrlBytes + n_slots * kSlotBytes + n_bslots * bslot_bytes;
   const int R = T * k + c.n_shared * T;
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
-                                                        st->xt, w.Rpad, nt_tile, n_bslots, wcap,
+                                                        st->xt, w.Rpad, nt_tile, n_bslots, n_slots,
                                                         reinterpret_cast<__half*>(b + w.ht), nullptr, c.hidden, 0,
                                                         status);
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
-                                                        st->ht, w.Rpad, nt_tile, n_bslots, wcap, nullptr,
+                                                        st->ht, w.Rpad, nt_tile, n_bslots, n_slots, nullptr,
                                                         reinterpret_cast<float*>(b + w.y), c.hidden,
                                                         (size_t)R * c.hidden, status);
   ctx->launches += 2;
