@@ -15,10 +15,10 @@
 // instruction of theirs waits its turn.
 //   warps 0-7    dequantize: two groups of four warps, group j takes the quantized items j, j+2, ..;
 //                warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
-//   warp 8       weight producer: arms an item's barrier and copies its codes, as far ahead as the
-//                slot ring allows;
-//   warp 9       copies scales and zero-points of the items the weight producer has armed;
-//   warp 10      token-tile producer (its own few slots, never holds back the weight stream);
+//   warp 8       weight producer: arms an item's barrier and copies its codes, scales and zero-points,
+//                as far ahead as the slot ring allows;
+//   warp 9       token-tile producer (its own few slots, never holds back the weight stream);
+//   warp 10      idle (keeps the issuers on four different schedulers);
 //   warps 11-14  MMA issuers (warp 11 also allocates tensor memory).  A tcgen05.mma holds its issuing
 //                thread for ~95 cycles whatever its size, so one issuer caps the SM at one 128x16
 //                weight slab per 95 cycles; four issuers in four warps overlap.  Each issuer owns the
@@ -45,7 +45,7 @@ constexpr int kMaxBSlots = 4;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
 constexpr int kDqWarps = 8;
-constexpr int kWarpCodes = 8, kWarpMeta = 9, kWarpTokens = 10, kWarpMma = 11, kIssuers = 4, kWarpEpi = 15;
+constexpr int kWarpCodes = 8, kWarpTokens = 9, kWarpMma = 11, kIssuers = 4, kWarpEpi = 15;
 constexpr int kThreads = 608;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
@@ -342,6 +342,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             TRACE(0, n);
             mbar_expect_tx(&c->full[s], bits == 16 ? cbytes : cbytes + 512);
             bulk_g2s(wring + s * kSlotBytes, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, &c->full[s]);
+            if (bits != 16) {
+              bulk_g2s(wring + s * kSlotBytes + cbytes, row.scales + tile * kTileRows, 256, &c->full[s]);
+              bulk_g2s(wring + s * kSlotBytes + cbytes + 256, row.zps + tile * kTileRows, 256, &c->full[s]);
+            }
             if (bits == 16) {
               lk_mma |= 1u << s;
               lk_mma2 |= 1u << (s + 1);
@@ -352,35 +356,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             }
             ++n;
             c->issued = n;
-          }
-        }
-      }
-    }
-  } else if (warp == kWarpMeta) {
-    // ---------------- scales / zero-points producer ----------------
-    if (lane == 0) {
-      int head = 0;
-      uint32_t n = 0;
-      bool ok = true;
-      for (int i = 0; ok; ++i) {
-        const int u = unit_index(i);
-        if (u >= n_units) break;
-        const Unit un = units[u];
-        for (int g = un.g0; ok && g < un.g1; ++g) {
-#pragma unroll
-          for (int m = 0; m < NMAT; ++m) {
-            const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
-            const uint32_t bits = row.bits;
-            const int s = slot_take(head, item_slots(bits), n_slots);
-            if (bits != 16) {
-              ok = wait_issued(n, c, status);        // the slot is free and its barrier armed for this item
-              if (!ok) break;
-              const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + g;
-              char* dst = wring + s * kSlotBytes + bits * 2048;
-              bulk_g2s(dst, row.scales + tile * kTileRows, 256, &c->full[s]);
-              bulk_g2s(dst + 256, row.zps + tile * kTileRows, 256, &c->full[s]);
-            }
-            ++n;
           }
         }
       }
