@@ -204,6 +204,28 @@ pw_status pw_moe_forward_host(pw_ctx* ctx, int layer, const void* hidden_host, c
 pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
                          int32_t* perm, pw_stream stream);
 
+/* Routing for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a convenience of this library.)  Some hosts of this code must not call cudaMalloc at all -- a
+ * plug-in running inside another engine's memory pool, a process that has handed all device memory
+ * to a caching allocator, code between the begin and end of a stream capture.  They cannot create a
+ * context, because a context needs a workspace.  This call does the router and the stable grouping
+ * of pw_moe_forward (same kernels, same results) and needs no context and no workspace: its scratch
+ * (inverse permutation, row map, counters; about 0.5 MB) is a fixed array inside the library image,
+ * which every GPU that has loaded the library holds until the process exits.
+ *   router_logits: device [T, n_experts] fp32.  Outputs, all device and caller-allocated: topk_ids
+ *   int32 [T, top_k], gates fp32 [T, top_k], counts int32 [n_experts], offsets int32 [n_experts + 1],
+ *   perm int32 [T * top_k].
+ * Limits: T * top_k <= 65536 and n_experts <= 256, else PW_ERR_NOMEM; top_k <= 32.
+ * The first call on a device looks up the device address of the scratch array (one
+ * cudaGetSymbolAddress with that device current); make that first call outside any stream capture.
+ * The call allocates nothing, frees nothing and calls no allocating library routine.  All calls on a
+ * device share the one scratch array: two calls that may run at the same time on the GPU (different
+ * streams) race and must be ordered by the caller.  Calls on one stream are safe back to back; the
+ * array keeps the previous call's contents and the kernels clear what they need to start from zero.
+ * Errors: INVALID_ARG, ALIGN, NOMEM (over the limits), CUDA. */
+pw_status pw_route_tokens_static(const float* router_logits, int T, int n_experts, int top_k, int32_t* topk_ids,
+                                 float* gates, int32_t* counts, int32_t* offsets, int32_t* perm, pw_stream stream);
+
 /* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
  * then clears it. */
 pw_status pw_last_device_status(pw_ctx* ctx);

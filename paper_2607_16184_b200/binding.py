@@ -27,7 +27,7 @@ GROUP = 128
 # every symbol include/pw.h declares
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
-           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_last_device_status", "pw_kernel_timing", "pw_get_kernel_times",
+           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_last_device_status", "pw_kernel_timing", "pw_get_kernel_times",
            "pw_launch_count", "pw_status_str")
 KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine")
 
@@ -92,6 +92,8 @@ def load():
     L.pw_moe_forward.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp]
     L.pw_moe_forward_host.restype = i32
     L.pw_moe_forward_host.argtypes = [vp, i32, vp, vp, i32, i32, vp, i32, vp]
+    L.pw_route_tokens_static.restype = i32
+    L.pw_route_tokens_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     L.pw_get_routing.restype = i32
     L.pw_get_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.pw_last_device_status.restype = i32
@@ -124,6 +126,25 @@ def pw_page_bytes(rows: int, cols: int, bits: int, group: int = GROUP) -> Tuple[
     a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
     tot = load().pw_page_bytes(rows, cols, bits, group, C.byref(a), C.byref(b), C.byref(c))
     return int(tot), int(a.value), int(b.value), int(c.value)
+
+
+def pw_route_tokens_static(router_logits: torch.Tensor, top_k: int,
+                           stream: Optional[torch.cuda.Stream] = None) -> Dict[str, torch.Tensor]:
+    """Router + stable grouping without a context or workspace (for callers that must not allocate
+    device memory inside the call; the output tensors here are made by the caller's allocator, torch)."""
+    assert router_logits.dtype == torch.float32 and router_logits.is_contiguous() and router_logits.is_cuda
+    T, E = router_logits.shape
+    d = router_logits.device
+    r = {"topk_ids": torch.empty(T, top_k, dtype=torch.int32, device=d),
+         "gates": torch.empty(T, top_k, dtype=torch.float32, device=d),
+         "counts": torch.empty(E, dtype=torch.int32, device=d),
+         "offsets": torch.empty(E + 1, dtype=torch.int32, device=d),
+         "perm": torch.empty(T * top_k, dtype=torch.int32, device=d)}
+    with torch.cuda.device(d):
+        _check(load().pw_route_tokens_static(router_logits.data_ptr(), T, E, top_k, r["topk_ids"].data_ptr(),
+                                             r["gates"].data_ptr(), r["counts"].data_ptr(), r["offsets"].data_ptr(),
+                                             r["perm"].data_ptr(), _stream_ptr(stream)), "pw_route_tokens_static")
+    return r
 
 
 class Page:

@@ -290,3 +290,56 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
 }
 
 }  // namespace pw
+
+// ---- routing without any allocation ------------------------------------------------------------
+// Scratch of pw_route_tokens_static: inverse permutation, operand-row map and counters of the
+// grouping kernel.  Lives in the library image, so every GPU that loads the library holds it until
+// the process exits.  In host code `g_route_scratch` is only a handle of the symbol, not a device
+// address: the address a kernel may use comes from cudaGetSymbolAddress, once per device.
+namespace {
+constexpr int kStaticMaxPairs = 65536;        // T * top_k
+constexpr int kStaticMaxExperts = 256;
+constexpr size_t kStaticInvPerm = 0;                                            // int32[kStaticMaxPairs]
+constexpr size_t kStaticRowToken = kStaticInvPerm + 4 * (size_t)kStaticMaxPairs;   // int32[kStaticMaxPairs + kPadRows]
+constexpr size_t kStaticCounter = kStaticRowToken + 4 * (size_t)(kStaticMaxPairs + pw::kPadRows);   // int32[64]
+constexpr size_t kStaticStatus = kStaticCounter + 256;                          // int32[64]
+constexpr size_t kStaticBytes = kStaticStatus + 256;
+static __device__ __align__(256) unsigned char g_route_scratch[kStaticBytes];
+constexpr int kMaxDevices = 64;
+static void* g_route_scratch_addr[kMaxDevices];   // device address of the array, per device, once resolved
+}  // namespace
+
+extern "C" pw_status pw_route_tokens_static(const float* router_logits, int T, int n_experts, int top_k,
+                                            int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
+                                            int32_t* perm, pw_stream stream) {
+  using namespace pw;
+  if (!router_logits || !topk_ids || !gates || !counts || !offsets || !perm) return PW_ERR_INVALID_ARG;
+  if (T < 1 || n_experts < 1 || top_k < 1 || top_k > n_experts || top_k > 32) return PW_ERR_INVALID_ARG;
+  if (n_experts > kStaticMaxExperts || (long long)T * top_k > kStaticMaxPairs) return PW_ERR_NOMEM;
+  const void* ptrs[6] = {router_logits, topk_ids, gates, counts, offsets, perm};
+  for (const void* q : ptrs)
+    if (reinterpret_cast<uintptr_t>(q) & 15) return PW_ERR_ALIGN;
+  int dev = -1;
+  PW_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return PW_ERR_INVALID_ARG;
+  if (!g_route_scratch_addr[dev]) {   // first call on this device: resolve the symbol with this device current
+    void* addr = nullptr;
+    PW_CUDA_OK(cudaGetSymbolAddress(&addr, g_route_scratch));
+    if (!addr) return PW_ERR_CUDA;
+    g_route_scratch_addr[dev] = addr;
+  }
+  char* sc = reinterpret_cast<char*>(g_route_scratch_addr[dev]);
+  router_kernel<<<(T * 32 + 255) / 256, 256, 0, stream>>>(router_logits, T, n_experts, top_k, topk_ids, gates);
+  const int S = n_experts;
+  const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + n_experts + 32 * (size_t)n_experts + (S + 1) + S);
+  // the grouping kernel clears the counters it uses; everything else in the scratch is overwritten before it is read
+  permute_kernel<<<1, 1024, smem, stream>>>(topk_ids, T, top_k, n_experts, 0, counts, offsets, perm,
+                                            reinterpret_cast<int32_t*>(sc + kStaticInvPerm),
+                                            reinterpret_cast<int32_t*>(sc + kStaticRowToken),
+                                            reinterpret_cast<int32_t*>(sc + kStaticCounter), nullptr, 0, 0, 0, 1, nullptr,
+                                            nullptr, nullptr, nullptr, 0,
+                                            reinterpret_cast<int32_t*>(sc + kStaticStatus));
+  PW_CUDA_OK(cudaGetLastError());
+  return PW_OK;
+}
+
