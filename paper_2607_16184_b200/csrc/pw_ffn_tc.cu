@@ -10,21 +10,21 @@
 // then reads as its A operand.  The token tile (B operand) comes from the k-chunk-major operand
 // buffers with one 2-D TMA copy per group.
 //
-// One persistent CTA per SM, 19 warps.  The control roles are single threads with short dependent
+// One persistent CTA per SM, 27 warps.  The control roles are single threads with short dependent
 // instruction chains: they share the schedulers with the arithmetic-heavy dequantizers, and every
 // instruction of theirs waits its turn.
-//   warps 0-7    dequantize: two groups of four warps, group j takes the quantized items j, j+2, ..;
+//   warps 0-15   dequantize: four groups of four warps, group j takes the quantized items j, j+4, ..;
 //                warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
-//   warp 8       weight producer: arms an item's barrier and copies its codes, scales and zero-points,
+//   warp 16      weight producer: arms an item's barrier and copies its codes, scales and zero-points,
 //                as far ahead as the slot ring allows;
-//   warp 9       token-tile producer (its own few slots, never holds back the weight stream);
-//   warp 10      idle (keeps the issuers on four different schedulers);
-//   warps 11-14  MMA issuers (warp 11 also allocates tensor memory).  A tcgen05.mma holds its issuing
+//   warp 17      token-tile producer (its own few slots, never holds back the weight stream);
+//   warp 18      idle;
+//   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  A tcgen05.mma holds its issuing
 //                thread for ~95 cycles whatever its size, so one issuer caps the SM at one 128x16
 //                weight slab per 95 cycles; four issuers in four warps overlap.  Each issuer owns the
 //                K-steps k = j mod (issuers per matrix) of one matrix and its own partial accumulator,
 //                so no two threads ever accumulate into the same columns; the epilogue adds the partials;
-//   warps 15-18  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
+//   warps 23-26  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
 //                split-K partial of the down projection (PHASE 1).
 // Units are dealt to CTAs in snake order over a size-sorted list.  Every wait is bounded; when one
 // runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
@@ -40,13 +40,13 @@ namespace pw {
 
 constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item (16 KB codes + 512 B) fits
 constexpr int kMaxSlots = 16;
-constexpr int kMaxASlots = 8;                  // dequantized groups in tensor memory (64 columns each)
+constexpr int kMaxASlots = 8;                  // operand half-slots in tensor memory (32 columns = 64 K each)
 constexpr int kMaxBSlots = 4;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
-constexpr int kDqWarps = 8;
-constexpr int kWarpCodes = 8, kWarpTokens = 9, kWarpMma = 11, kIssuers = 4, kWarpEpi = 15;
-constexpr int kThreads = 608;
+constexpr int kDqWarps = 16;
+constexpr int kWarpCodes = 16, kWarpTokens = 17, kWarpMma = 19, kIssuers = 4, kWarpEpi = 23;
+constexpr int kThreads = 864;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
@@ -264,10 +264,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
   constexpr int IPM = kIssuers / NMAT;           // issuers per matrix
   int npart = IPM;
-  while (npart > 1 && NMAT * npart * nt_tile + 2 * 64 > kTmemCols) npart >>= 1;
+  while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 32 > kTmemCols) npart >>= 1;
   const int n_issuers = NMAT * npart;            // active issuers
-  const int acol = NMAT * npart * nt_tile;
-  const int n_aslots = min(kMaxASlots, (kTmemCols - acol) / 64) & ~1;   // even: a slot always serves the same group
+  const int acol = NMAT * npart * nt_tile;       // operand half-slot hs = 2 * group + K-half sits at acol + 32 * hs
+  const int per_half = npart >= 2 ? npart / 2 : 1;   // issuers per (matrix, K-half)
   const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
@@ -281,8 +281,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       mbar_init(&c->b_empty[i], n_issuers);
     }
     for (int i = 0; i < kMaxASlots; ++i) {
-      mbar_init(&c->a_full[i], 4);
-      mbar_init(&c->a_empty[i], n_issuers);      // every issuer lets go of an operand slot, see below
+      mbar_init(&c->a_full[i], 4);                // the four warps of the group that owns the half-slot
+      mbar_init(&c->a_empty[i], per_half);       // the issuers that read this K-half
     }
     mbar_init(&c->d_full, n_issuers);
     mbar_init(&c->d_empty, 4);
@@ -319,10 +319,13 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         const int u = unit_index(i);
         if (u >= n_units) break;
         const Unit un = units[u];
+        DevRow urow[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) urow[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
         for (int g = un.g0; ok && g < un.g1; ++g) {
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+            const DevRow& row = urow[m];
             const uint32_t bits = row.bits;
             const int k = item_slots(bits);
             const int s = slot_take(head, k, n_slots);
@@ -385,13 +388,20 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   }
   else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
     // ---------------- MMA issuers ----------------
+    // Issuer j of matrix m owns partial accumulator j.  With two or more issuers per matrix, each reads
+    // one K-half of every item (k-steps 4h .. 4h+3, strided over the issuers of that half), so it
+    // waits on one operand half-slot per item; a lone issuer walks both halves.
     const int iss = warp - kWarpMma;
-    const int my_m = iss / IPM, my_p = iss % IPM;     // matrix and partial accumulator of this issuer
-    if (lane == 0 && my_p < npart) {
+    const int my_m = iss / IPM, my_j = iss % IPM;
+    if (lane == 0 && my_j < npart) {
+      const int my_h0 = npart >= 2 ? my_j / per_half : 0;
+      const int n_h = npart >= 2 ? 1 : 2;
+      const int my_p = npart >= 2 ? my_j % per_half : 0;
+      const int kk_first = 4 * my_h0 + my_p;          // my first k-step of an item
       int head = 0;
       uint32_t n = 0, full_par = 0;                 // item sequence number; per-slot parity of the full barrier
-      uint32_t acount = 0, bcount = 0, ucount = 0;
-      const uint32_t d_t = tmem + (my_m * npart + my_p) * nt_tile;
+      uint32_t cnt = 0, bcount = 0, ucount = 0;     // cnt: quantized items of my matrix so far
+      const uint32_t d_t = tmem + (my_m * npart + my_j) * nt_tile;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = unit_index(i);
@@ -419,40 +429,37 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const uint32_t par = (full_par >> s) & 1;
             full_par ^= 1u << s;
             const uint32_t item_n = n++;
-            if (m != my_m) {
-              // The other matrix.  A quantized item still goes through the shared operand slots: watch its
-              // barrier phase go by and let go of the slot, so that the slot is never refilled before every
-              // issuer has seen this phase (a thread that misses a phase would wait on the wrong one for ever).
-              if (bits != 16) {
-                const int as = acount % n_aslots;
-                ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
-                if (!ok) break;
-                mbar_arrive(&c->a_empty[as]);
-                ++acount;
-              }
-              continue;
-            }
+            if (m != my_m) continue;                 // the other matrix has its own issuers and operand slots
             if (bits == 16) {
               ok = wait_issued(item_n, c, status) && mbar_wait(&c->full[s], par, c, status);
               if (!ok) break;
               tc_fence_after();
               const uint64_t ad0 = make_kmajor_desc(smem_u32(wring + s * kSlotBytes), 2048);
-              for (int kk = my_p; kk < 8; kk += npart)
-                tc_mma_ss(d_t, ad0 + (uint64_t)(kk * 256), bd0 + (uint64_t)(kk * b_step), idesc,
-                          (later || kk != my_p) ? 1u : 0u);
+              for (int hh = 0; hh < n_h; ++hh)
+                for (int kk = 4 * (my_h0 + hh) + my_p; kk < 4 * (my_h0 + hh) + 4; kk += per_half)
+                  tc_mma_ss(d_t, ad0 + (uint64_t)(kk * 256), bd0 + (uint64_t)(kk * b_step), idesc,
+                            (later || kk != kk_first) ? 1u : 0u);
               tc_commit(&c->empty_mma[s]);
             } else {
-              const int as = acount % n_aslots;
-              ok = mbar_wait(&c->a_full[as], (acount / n_aslots) & 1, c, status);
+              // the group that dequantizes this item, and the parity of this use of its half-slots
+              const int grp = NMAT == 2 ? 2 * my_m + (int)(cnt & 1) : (int)(cnt & 3);
+              const uint32_t use_par = NMAT == 2 ? (cnt >> 1) & 1 : (cnt >> 2) & 1;
+              for (int hh = 0; hh < n_h; ++hh) {
+                const int h = my_h0 + hh;
+                const int hs = 2 * grp + h;
+                ok = mbar_wait(&c->a_full[hs], use_par, c, status);
+                if (!ok) break;
+                tc_fence_after();
+                if (my_j == 0) { TRACE(8, item_n); }
+                const uint32_t a_t = tmem + acol + hs * 32;
+                for (int kk = 4 * h + my_p; kk < 4 * h + 4; kk += per_half)
+                  tc_mma_ts(d_t, a_t + (kk - 4 * h) * 8, bd0 + (uint64_t)(kk * b_step), idesc,
+                            (later || kk != kk_first) ? 1u : 0u);
+                tc_commit(&c->a_empty[hs]);
+              }
               if (!ok) break;
-              tc_fence_after();
-              if (my_p == 0) { TRACE(8, item_n); }
-              const uint32_t a_t = tmem + acol + as * 64;
-              for (int kk = my_p; kk < 8; kk += npart)
-                tc_mma_ts(d_t, a_t + kk * 8, bd0 + (uint64_t)(kk * b_step), idesc, (later || kk != my_p) ? 1u : 0u);
-              tc_commit(&c->a_empty[as]);
-              if (my_p == 0) { TRACE(9, item_n); }
-              ++acount;
+              if (my_j == 0) { TRACE(9, item_n); }
+              ++cnt;
             }
           }
           if (!ok) break;
@@ -464,15 +471,17 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     }
   } else if (warp < kDqWarps) {
     // ---------------- dequantize ----------------
-    // Two groups of four warps; group j takes the quantized items j, j+2, j+4, .. (an item = one group of
-    // one matrix), so each group alternates between two operand slots.  Warp q of a group owns rows
-    // (= TMEM lanes) 32q .. 32q+31 of the item, one row per thread, all 128 weights of the row.
+    // Four groups of four warps, each taking every other quantized item of one matrix (every fourth when
+    // the unit has a single matrix; an item = one group of one matrix).  Warp q of a group owns rows (= TMEM lanes) 32q .. 32q+31 of the item, one row per
+    // thread.  Each group has two operand half-slots (K 0..63 and K 64..127 of its item): while the
+    // issuers consume one half the group decodes the other.
     const int grp = warp >> 2, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
-    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + grp * 64;
     int head = 0;
-    uint32_t n = 0, full_par = 0, dq_seq = 0;
-    int pending = -1;                                // operand slot whose store has not been published yet
+    uint32_t n = 0, full_par = 0;
+    uint32_t cnt[NMAT] = {};                          // quantized items per matrix so far
+    int pending = -1;                                // operand half-slot whose store has not been published yet
     bool ok = true;
     auto publish = [&]() {
       if (pending >= 0) {
@@ -499,46 +508,44 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           full_par ^= 1u << s;
           const uint32_t item_n = n++;
           if (bits == 16) continue;                  // the MMA reads 16-bit tiles straight from shared memory
-          if ((int)(dq_seq & 1) == grp) {
+          // gate items go to groups 0, 1 and up items to groups 2, 3 (a single matrix uses all four), so that
+          // the issuers of one matrix never share an operand slot with the other's
+          const int owner = NMAT == 2 ? 2 * m + (int)(cnt[m] & 1) : (int)(cnt[m] & 3);
+          const uint32_t use_par = NMAT == 2 ? (cnt[m] >> 1) & 1 : (cnt[m] >> 2) & 1;
+          ++cnt[m];
+          if (owner == grp) {
             if (c->issued <= item_n || !mbar_try(&c->full[s], par)) {
-              publish();                             // do not sit on a finished item while waiting for HBM
+              publish();                             // do not sit on a finished half while waiting for HBM
               ok = wait_issued(item_n, c, status) && mbar_wait<20>(&c->full[s], par, c, status);
               if (!ok) break;
             }
             if (q == 0) { TRACE(1, item_n); }
             const char* item = wring + s * kSlotBytes;
-            const int as = dq_seq % n_aslots;
-            const uint32_t taddr = lane_addr + as * 64;
-            __half2 w[32];
-            switch (bits) {
-              case 8: decode_item_half<8>(item, r, 0, w); break;
-              case 4: decode_item_half<4>(item, r, 0, w); break;
-              case 3: decode_item_half<3>(item, r, 0, w); break;
-              default: decode_item_half<2>(item, r, 0, w); break;
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+              __half2 w[32];
+              switch (bits) {
+                case 8: decode_item_half<8>(item, r, h, w); break;
+                case 4: decode_item_half<4>(item, r, h, w); break;
+                case 3: decode_item_half<3>(item, r, h, w); break;
+                default: decode_item_half<2>(item, r, h, w); break;
+              }
+              if (q == 0) { TRACE(2 + 3 * h, item_n); }
+              if (h == 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
+              }
+              publish();                             // the previous half's store, overlapped with the decode above
+              const int hs = 2 * grp + h;
+              ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
+              if (!ok) break;
+              tc_fence_after();
+              tmem_st32(lane_addr + h * 32, w);
+              if (q == 0) { TRACE(3 + 3 * h, item_n); }
+              pending = hs;
             }
-            if (q == 0) { TRACE(2, item_n); }
-            publish();                               // previous item's store, overlapped with the decode above
-            if (q == 0) { TRACE(3, item_n); }
-            ok = mbar_wait<20>(&c->a_empty[as], ((dq_seq / n_aslots) & 1) ^ 1, c, status);
             if (!ok) break;
-            tc_fence_after();
-            if (q == 0) { TRACE(4, item_n); }
-            tmem_st32(taddr, w);
-            if (q == 0) { TRACE(5, item_n); }
-            switch (bits) {
-              case 8: decode_item_half<8>(item, r, 1, w); break;
-              case 4: decode_item_half<4>(item, r, 1, w); break;
-              case 3: decode_item_half<3>(item, r, 1, w); break;
-              default: decode_item_half<2>(item, r, 1, w); break;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
-            if (q == 0) { TRACE(6, item_n); }
-            tmem_st32(taddr + 32, w);
-            if (q == 0) { TRACE(7, item_n); }
-            pending = as;
           }
-          ++dq_seq;
         }
       }
       if (ok) publish();
