@@ -161,6 +161,65 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// NK consecutive k-steps of one item issued from one asm block (the issuing thread gets few issue slots,
+// so every instruction around an MMA counts).  Descriptors are passed as (lo, hi) words; only lo moves.
+// TS: A in tensor memory at a_tmem (+a_step per k-step).  `acc0`: accumulate flag of the first k-step.
+template <int NK>
+__device__ __forceinline__ void tc_mma_ts_burst(uint32_t d_tmem, uint32_t a_tmem, uint32_t a_step, uint32_t b_lo,
+                                                uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t acc0) {
+  asm volatile(
+      "{\n\t.reg .pred p, t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
+      "setp.ne.b32 p, %7, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "mov.b64 bd, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %6, p;\n\t"
+      "add.u32 lo, %3, %5;\n\tadd.u32 a, %1, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
+      : "memory");
+  if (NK == 4) {
+    asm volatile(
+        "{\n\t.reg .pred t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "mad.lo.u32 lo, %5, 2, %3;\n\tmad.lo.u32 a, %2, 2, %1;\n\tmov.b64 bd, {lo, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "add.u32 lo, lo, %5;\n\tadd.u32 a, a, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        : "memory");
+  }
+}
+// SS: A in shared memory, descriptor (a_lo, a_hi), +a_step per k-step.
+template <int NK>
+__device__ __forceinline__ void tc_mma_ss_burst(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step,
+                                                uint32_t b_lo, uint32_t b_hi, uint32_t b_step, uint32_t idesc,
+                                                uint32_t acc0) {
+  asm volatile(
+      "{\n\t.reg .pred p, t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
+      "setp.ne.b32 p, %8, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "mov.b64 ad, {%1, %2};\n\tmov.b64 bd, {%4, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, p;\n\t"
+      "add.u32 la, %1, %3;\n\tadd.u32 lb, %4, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
+      : "memory");
+  if (NK == 4) {
+    asm volatile(
+        "{\n\t.reg .pred t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "mad.lo.u32 la, %3, 2, %1;\n\tmad.lo.u32 lb, %6, 2, %4;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "add.u32 la, la, %3;\n\tadd.u32 lb, lb, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        : "memory");
+  }
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const __half2* v) {
   const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
   asm volatile(
@@ -397,11 +456,15 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const int my_h0 = npart >= 2 ? my_j / per_half : 0;
       const int n_h = npart >= 2 ? 1 : 2;
       const int my_p = npart >= 2 ? my_j % per_half : 0;
-      const int kk_first = 4 * my_h0 + my_p;          // my first k-step of an item
       int head = 0;
       uint32_t n = 0, full_par = 0;                 // item sequence number; per-slot parity of the full barrier
-      uint32_t cnt = 0, bcount = 0, ucount = 0;     // cnt: quantized items of my matrix so far
+      uint32_t cnt = 0, ucount = 0;                 // cnt: quantized items of my matrix so far
+      int bs = 0;                                   // token-tile slot and its barrier parity, kept incrementally
+      uint32_t bpar = 0;
       const uint32_t d_t = tmem + (my_m * npart + my_j) * nt_tile;
+      const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
+      const uint32_t b_lo_base = smem_u32(bslots) >> 4;
+      const uint32_t w_lo_base = smem_u32(wring) >> 4;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = unit_index(i);
@@ -412,16 +475,20 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const uint32_t b_step = (uint32_t)(2 * nb_rows * 16) >> 4;    // descriptor advance per K-step
+        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
+        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
+        const uint32_t b_step = (uint32_t)(2 * nb_rows) * per_half;
+        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
         ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
         if (!ok) break;
         tc_fence_after();
+        uint32_t later = 0;                          // becomes 1 after the first group: accumulate onto earlier groups
         for (int g = un.g0; ok && g < un.g1; ++g) {
-          const int bs = bcount % n_bslots;
-          ok = mbar_wait(&c->b_full[bs], (bcount / n_bslots) & 1, c, status);
+          if (my_m == 0 && my_j == 0) { TRACE(10, n); }
+          ok = mbar_wait(&c->b_full[bs], bpar, c, status);
           if (!ok) break;
-          const uint64_t bd0 = make_kmajor_desc(smem_u32(bslots + (size_t)bs * bslot_bytes), nb_rows * 16);
-          const uint32_t later = (g > un.g0) ? 1u : 0u;   // accumulate onto earlier groups
+          if (my_m == 0 && my_j == 0) { TRACE(11, n); }
+          const uint32_t b_lo = b_lo_unit + (uint32_t)bs * (uint32_t)(bslot_bytes >> 4);
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
             const uint32_t bits = ubits[m];
@@ -434,11 +501,16 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               ok = wait_issued(item_n, c, status) && mbar_wait(&c->full[s], par, c, status);
               if (!ok) break;
               tc_fence_after();
-              const uint64_t ad0 = make_kmajor_desc(smem_u32(wring + s * kSlotBytes), 2048);
-              for (int hh = 0; hh < n_h; ++hh)
-                for (int kk = 4 * (my_h0 + hh) + my_p; kk < 4 * (my_h0 + hh) + 4; kk += per_half)
-                  tc_mma_ss(d_t, ad0 + (uint64_t)(kk * 256), bd0 + (uint64_t)(kk * b_step), idesc,
-                            (later || kk != kk_first) ? 1u : 0u);
+              const uint32_t a_lo = (w_lo_base + (uint32_t)s * (kSlotBytes >> 4)) | a_lo_lbo;
+              for (int hh = 0; hh < n_h; ++hh) {
+                const uint32_t k0 = 4 * (my_h0 + hh) + my_p;
+                if (per_half == 1)
+                  tc_mma_ss_burst<4>(d_t, a_lo + k0 * 256, desc_hi, 256, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
+                                     later | (uint32_t)hh);
+                else
+                  tc_mma_ss_burst<2>(d_t, a_lo + k0 * 256, desc_hi, 512, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
+                                     later);
+              }
               tc_commit(&c->empty_mma[s]);
             } else {
               // the group that dequantizes this item, and the parity of this use of its half-slots
@@ -447,14 +519,17 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               for (int hh = 0; hh < n_h; ++hh) {
                 const int h = my_h0 + hh;
                 const int hs = 2 * grp + h;
+                if (my_j == 0) { TRACE(12, item_n); }
                 ok = mbar_wait(&c->a_full[hs], use_par, c, status);
                 if (!ok) break;
                 tc_fence_after();
                 if (my_j == 0) { TRACE(8, item_n); }
-                const uint32_t a_t = tmem + acol + hs * 32;
-                for (int kk = 4 * h + my_p; kk < 4 * h + 4; kk += per_half)
-                  tc_mma_ts(d_t, a_t + (kk - 4 * h) * 8, bd0 + (uint64_t)(kk * b_step), idesc,
-                            (later || kk != kk_first) ? 1u : 0u);
+                const uint32_t a_t = tmem + acol + hs * 32 + my_p * 8;
+                const uint32_t k0 = 4 * h + my_p;
+                if (per_half == 1)
+                  tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later | (uint32_t)hh);
+                else
+                  tc_mma_ts_burst<2>(d_t, a_t, 16, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later);
                 tc_commit(&c->a_empty[hs]);
               }
               if (!ok) break;
@@ -464,7 +539,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           }
           if (!ok) break;
           tc_commit(&c->b_empty[bs]);
-          ++bcount;
+          later = 1;
+          if (++bs == n_bslots) {
+            bs = 0;
+            bpar ^= 1;
+          }
         }
         if (ok) tc_commit(&c->d_full);
       }
