@@ -128,6 +128,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+// the same with shared-memory addresses already in hand (saves the address conversions in a hot control loop)
+__device__ __forceinline__ void mbar_expect_tx_s(uint32_t bar_s, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_s(uint32_t dst_s, const void* src, uint32_t bytes, uint32_t bar_s) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_s),
+               "l"(src), "r"(bytes), "r"(bar_s)
+               : "memory");
+}
 __device__ __forceinline__ void tma_2d_g2s(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
@@ -373,49 +382,78 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       // issuers, or the MMA issuers through the barrier of the slot before it, for the second slot of a
       // 16-bit item).  ed_par / em_par: parity of the next phase of empty_dq / empty_mma of the slot.
       uint32_t lk_dq = 0, lk_mma = 0, lk_mma2 = 0, ed_par = 0, em_par = 0;
+      const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]);
       bool ok = true;
       for (int i = 0; ok; ++i) {
         const int u = unit_index(i);
         if (u >= n_units) break;
         const Unit un = units[u];
-        DevRow urow[NMAT];
+        // per matrix of the unit: bitwidth, bytes of a code tile, and the source addresses of the unit's
+        // first item; consecutive groups of a row tile are consecutive tiles of the page
+        uint32_t ubits[NMAT], ucb[NMAT];
+        const char* usrc[NMAT];
+        const __half* uscl[NMAT];
+        const __half* uzp[NMAT];
 #pragma unroll
-        for (int m = 0; m < NMAT; ++m) urow[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+        for (int m = 0; m < NMAT; ++m) {
+          const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+          ubits[m] = row.bits;
+          ucb[m] = row.bits * 2048;
+          const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + un.g0;
+          usrc[m] = reinterpret_cast<const char*>(row.codes) + tile * ucb[m];
+          uscl[m] = row.scales + tile * kTileRows;
+          uzp[m] = row.zps + tile * kTileRows;
+        }
         for (int g = un.g0; ok && g < un.g1; ++g) {
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            const DevRow& row = urow[m];
-            const uint32_t bits = row.bits;
-            const int k = item_slots(bits);
-            const int s = slot_take(head, k, n_slots);
-            // every slot the item covers must have been handed back by its last occupant
-            for (int j = s; ok && j < s + k; ++j) {
-              const uint32_t bit = 1u << j;
-              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
-              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
-              else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
-              lk_dq &= ~bit;
-              lk_mma &= ~bit;
-              lk_mma2 &= ~bit;
-            }
-            if (!ok) break;
-            const uint32_t cbytes = bits * 2048;
-            const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + g;
-            TRACE(0, n);
-            mbar_expect_tx(&c->full[s], bits == 16 ? cbytes : cbytes + 512);
-            bulk_g2s(wring + s * kSlotBytes, reinterpret_cast<const char*>(row.codes) + tile * cbytes, cbytes, &c->full[s]);
-            if (bits != 16) {
-              bulk_g2s(wring + s * kSlotBytes + cbytes, row.scales + tile * kTileRows, 256, &c->full[s]);
-              bulk_g2s(wring + s * kSlotBytes + cbytes + 256, row.zps + tile * kTileRows, 256, &c->full[s]);
-            }
+            const uint32_t bits = ubits[m];
+            const uint32_t cbytes = ucb[m];
+            uint32_t bar_s, dst_s;
             if (bits == 16) {
+              const int s = slot_take(head, 2, n_slots);
+              const uint32_t two = 3u << s;          // both slots must have been handed back
+              if ((lk_dq | lk_mma | lk_mma2) & two) {
+                for (int j = s; ok && j < s + 2; ++j) {
+                  const uint32_t bit = 1u << j;
+                  if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
+                  else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
+                  else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
+                }
+                if (!ok) break;
+                lk_dq &= ~two;
+                lk_mma &= ~two;
+                lk_mma2 &= ~two;
+              }
+              bar_s = full_s + 8 * s;
+              dst_s = wring_s + s * kSlotBytes;
+              mbar_expect_tx_s(bar_s, cbytes);
+              bulk_g2s_s(dst_s, usrc[m], cbytes, bar_s);
               lk_mma |= 1u << s;
-              lk_mma2 |= 1u << (s + 1);
+              lk_mma2 |= 2u << s;
               em_par ^= 1u << s;
             } else {
-              lk_dq |= 1u << s;
-              ed_par ^= 1u << s;
+              const int s = slot_take(head, 1, n_slots);
+              const uint32_t bit = 1u << s;
+              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
+              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
+              else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[s - 1], ((em_par >> (s - 1)) & 1) ^ 1, c, status);
+              if (!ok) break;
+              lk_mma &= ~bit;
+              lk_mma2 &= ~bit;
+              bar_s = full_s + 8 * s;
+              dst_s = wring_s + s * kSlotBytes;
+              TRACE(0, n);
+              mbar_expect_tx_s(bar_s, cbytes + 512);
+              bulk_g2s_s(dst_s, usrc[m], cbytes, bar_s);
+              bulk_g2s_s(dst_s + cbytes, uscl[m], 256, bar_s);
+              bulk_g2s_s(dst_s + cbytes + 256, uzp[m], 256, bar_s);
+              uscl[m] += kTileRows;
+              uzp[m] += kTileRows;
+              lk_dq |= bit;
+              ed_par ^= bit;
             }
+            usrc[m] += cbytes;
             ++n;
             c->issued = n;
           }
