@@ -258,12 +258,23 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
     const int R = T * top_k + c.n_shared * T;
     const int active = ctx->ws.S < R ? ctx->ws.S : R;
     const long long tiles = (long long)active * ((R / active + nt_tile - 1) / nt_tile) * (c.hidden / kTileRows);
-    long long want = (4ll * ctx->num_sms + tiles - 1) / tiles;
+    // Pick the split (1..8) whose unit count fills whole rounds of one CTA per SM best; at least three
+    // rounds so that the pipeline of a CTA stays fed, and on ties the smaller split (less partial traffic).
     const int ng = c.ffn / kGroup;
-    if (want > 8) want = 8;
-    if (want > ng) want = ng;
-    if (want < 1) want = 1;
-    while (want > 1 && (size_t)want * R > ctx->ws.y_slots) --want;
+    const long long G = ctx->num_sms;
+    long long want = 1;
+    double best = -1.0;
+    for (int ks = 1; ks <= 8 && ks <= ng; ++ks) {
+      if ((size_t)ks * R > ctx->ws.y_slots) break;
+      const long long units = tiles * ks;
+      const long long rounds = (units + G - 1) / G;
+      double eff = (double)units / (double)(rounds * G);
+      if (rounds < 3) eff *= 0.5 + 0.15 * (double)rounds;       // too few units per SM: prefer a finer split
+      if (eff > best + 1e-9) {
+        best = eff;
+        want = ks;
+      }
+    }
     ksplit = (int)want;
   }
   if (ctx->timing_on) {

@@ -517,8 +517,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
         const uint32_t b_step = (uint32_t)(2 * nb_rows) * per_half;
         const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
         ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
         if (!ok) break;
+        if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
         tc_fence_after();
         uint32_t later = 0;                          // becomes 1 after the first group: accumulate onto earlier groups
         for (int g = un.g0; ok && g < un.g1; ++g) {
@@ -680,6 +682,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const Unit un = units[u];
       ok = mbar_wait<200>(&c->d_full, ucount & 1, c, status);
       if (!ok) break;
+      if (q == 0) { TRACE(13, ucount); }
       tc_fence_after();
       const int nb_rows = (un.ntok + 15) & ~15;
       const int row = un.row_tile * kTileRows + r;
@@ -716,6 +719,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       }
       tc_fence_before();
       __syncwarp();
+      if (q == 0) { TRACE(14, ucount); }
       if (lane == 0) mbar_arrive(&c->d_empty);
     }
   }
