@@ -61,7 +61,11 @@ typedef enum {
  * fp16 [rows, cols/group] row-major; a 16-bit page is the fp16 matrix itself.
  * TILED: the same bytes regrouped per (128-row, one-group) tile so that a kernel reads a
  * tile with contiguous 16-byte loads; produced by pw_quantize_block / pw_demote_block /
- * pw_import_page and required by pw_moe_forward.  Both layouts have identical sizes. */
+ * pw_import_page and required by pw_moe_forward.  A TILED page is ONE buffer of the total
+ * size pw_page_bytes returns, at `codes`: every tile is stored as its packed codes followed by
+ * the 128 scales and the 128 zero-points of its rows, so a tile travels in a single copy;
+ * `scales` and `zps` of a TILED page are ignored (may be NULL).  Both layouts have the same
+ * total size. */
 enum { PW_LAYOUT_CANONICAL = 0, PW_LAYOUT_TILED = 1 };
 
 /* Residency state of a page-table row (Sec. 3.1).  Only GPU_RESIDENT rows can be used. */
@@ -87,9 +91,10 @@ typedef struct {
 
 /* One weight page = one linear-block at one bitwidth (Sec. 3.1).  All pointers device. */
 typedef struct {
-  void* codes;    /* bits < 16: packed codes, rows*cols*bits/8 bytes; bits == 16: fp16 weights   */
-  void* scales;   /* fp16, rows*cols/group values; ignored (may be NULL) when bits == 16         */
-  void* zps;      /* fp16, rows*cols/group values; ignored (may be NULL) when bits == 16         */
+  void* codes;    /* CANONICAL: packed codes, rows*cols*bits/8 bytes (bits == 16: fp16 weights);
+                     TILED: the whole page, pw_page_bytes(...) bytes                             */
+  void* scales;   /* CANONICAL, bits < 16: fp16, rows*cols/group values; otherwise ignored        */
+  void* zps;      /* CANONICAL, bits < 16: fp16, rows*cols/group values; otherwise ignored        */
   uint32_t rows;  /* output features                                                            */
   uint32_t cols;  /* input features (the grouped, contracted dimension)                         */
   uint16_t group; /* 128                                                                        */
@@ -129,8 +134,9 @@ size_t pw_page_bytes(uint32_t rows, uint32_t cols, int bits, int group, size_t* 
 /* ---- pages -------------------------------------------------------------------------- */
 
 /* Group-quantizes an fp16 block into a new page.  w_fp16: device, [rows, cols] row-major.
- * dst: host struct whose codes / scales / zps point to caller-allocated device buffers of the
- * sizes pw_page_bytes reports; the call fills rows, cols, group, bits, layout (TILED).
+ * dst: host struct whose `codes` points to a caller-allocated device buffer of the total size
+ * pw_page_bytes reports (a TILED page is one buffer); the call fills rows, cols, group, bits,
+ * layout (TILED).
  * bits == 16 stores the weights unchanged (a re-tiled copy).  Per group of 128 along cols, in
  * fp32 with one rounding per operation: lo = min, hi = max, scale = fp16((hi-lo)/(2^bits-1))
  * (1.0 if hi == lo, 2^-24 if it rounds to zero), zero-point = fp16(lo),

@@ -148,7 +148,11 @@ def pw_route_tokens_static(router_logits: torch.Tensor, top_k: int,
 
 
 class Page:
-    """Device buffers of one weight page plus its ``pw_page`` header."""
+    """Device buffers of one weight page plus its ``pw_page`` header.
+
+    A TILED page is one buffer (``codes``) of the total page size; a CANONICAL page below 16 bits has
+    separate ``codes``, ``scales`` and ``zps`` buffers.
+    """
 
     def __init__(self, rows: int, cols: int, bits: int, device="cuda", layout: int = PW_LAYOUT_TILED):
         tot, cb, sb, zb = pw_page_bytes(rows, cols, bits)
@@ -158,6 +162,8 @@ class Page:
             self.c = pw_page(None, None, None, rows, cols, GROUP, bits & 0xff, layout)
             self.nbytes = 0
             return
+        if layout == PW_LAYOUT_TILED:
+            cb, sb, zb = tot, 0, 0
         self.codes = torch.empty(cb, dtype=torch.uint8, device=device)
         self.scales = torch.empty(sb // 2, dtype=torch.float16, device=device) if sb else None
         self.zps = torch.empty(zb // 2, dtype=torch.float16, device=device) if zb else None

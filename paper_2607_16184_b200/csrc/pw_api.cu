@@ -175,8 +175,8 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
     if (!bits_ok(p.bits)) return PW_ERR_BITS;
     const uint32_t er = e.kind == PW_DOWN ? c.hidden : c.ffn, ec = e.kind == PW_DOWN ? c.ffn : c.hidden;
     if (p.rows != er || p.cols != ec || p.group != kGroup) return PW_ERR_SHAPE;
-    if (!p.codes || (p.bits < 16 && (!p.scales || !p.zps))) return PW_ERR_INVALID_ARG;
-    if (!aligned16(p.codes) || (p.bits < 16 && (!aligned16(p.scales) || !aligned16(p.zps)))) return PW_ERR_ALIGN;
+    if (!p.codes) return PW_ERR_INVALID_ARG;   // a TILED page is one buffer: scales and zero-points sit inside it
+    if (!aligned16(p.codes)) return PW_ERR_ALIGN;
     if (p.layout != PW_LAYOUT_TILED || e.state != PW_STATE_GPU_RESIDENT) return PW_ERR_STATE;
     if (e.expert >= c.n_experts && p.bits != 16) return PW_ERR_STATE;
     if (e.desired_bits != 0 && !bits_ok(e.desired_bits)) return PW_ERR_BITS;
@@ -192,8 +192,6 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       const pw_table_entry& e = entries[i];
       DevRow r{};
       r.codes = e.page.codes;
-      r.scales = reinterpret_cast<const __half*>(e.page.scales);
-      r.zps = reinterpret_cast<const __half*>(e.page.zps);
       r.rows = e.page.rows;
       r.cols = e.page.cols;
       r.bits = e.page.bits;

@@ -16,13 +16,11 @@ constexpr int kPadRows = 256;    // zero rows appended to the token-major operan
 
 // One row of the device-resident page table (48 bytes).
 struct DevRow {
-  const void* codes;
-  const __half* scales;
-  const __half* zps;
+  const void* codes;             // the TILED page buffer (tile images: codes, scales, zero-points)
   uint32_t rows, cols;
   uint32_t bits;
   uint32_t valid;
-  uint64_t pad_;
+  uint64_t reserved[3];
 };
 static_assert(sizeof(DevRow) == 48, "DevRow layout");
 

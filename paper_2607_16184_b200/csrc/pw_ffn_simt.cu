@@ -11,12 +11,12 @@ constexpr int kSimtTok = 8;  // tokens per pass over the weights
 
 template <int BITS>
 __device__ __forceinline__ void load_decode_group(const DevRow& row, size_t tile, int r, __half2* w) {
-  const uint4* tb =
-      reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row.codes) + tile * tile_code_bytes(BITS)) + r;
+  const char* tile_base = reinterpret_cast<const char*>(row.codes) + tile * tile_bytes(BITS);
+  const uint4* tb = reinterpret_cast<const uint4*>(tile_base) + r;
   __half2 s2 = __half2half2(__ushort_as_half((unsigned short)0x3c00)), z2 = s2;
   if constexpr (BITS < 16) {
-    s2 = __half2half2(row.scales[tile * kTileRows + r]);
-    z2 = __half2half2(row.zps[tile * kTileRows + r]);
+    s2 = __half2half2(*reinterpret_cast<const __half*>(tile_base + tile_scale_offset(BITS, r)));
+    z2 = __half2half2(*reinterpret_cast<const __half*>(tile_base + tile_zp_offset(BITS, r)));
   }
   decode_half<BITS>(tb, 0, s2, z2, w);
   decode_half<BITS>(tb, 1, s2, z2, w + 32);

@@ -67,6 +67,7 @@ static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 #ifdef PW_TC_PROFILE
 // Diagnostic build only: time stamps of the first few hundred items of CTA 0.
 __device__ long long g_trace[16][512];
+__device__ unsigned long long g_spins[32];      // polling-loop iterations per warp index, all CTAs
 #define TRACE(ev, n) \
   if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
 #else
@@ -106,14 +107,25 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting or the limit ran out (and then raises the abort).
-template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
-  if (mbar_try(b, parity)) return true;
+// The polling loop is kept out of line so that the hot loops of every role stay short.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_s, uint32_t parity, uint32_t sleep_ns, Ctrl* c,
+                                            int32_t* status) {
   const unsigned long long t0 = globaltimer();
   uint32_t spins = 0;
   while (true) {
-    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);       // leave the issue slots to the warps doing arithmetic
-    if (mbar_try(b, parity)) return true;
+    if (sleep_ns > 0) __nanosleep(sleep_ns);       // leave the issue slots to the warps doing arithmetic
+#ifdef PW_TC_PROFILE
+    if ((threadIdx.x & 31) == 0) atomicAdd(&g_spins[threadIdx.x >> 5], 1ull);
+#endif
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_s), "r"(parity)
+        : "memory");
+    if (ok) return true;
     if (c->abort_flag) return false;
     if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
       c->abort_flag = 1;
@@ -121,6 +133,35 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity
       return false;
     }
   }
+}
+// Fast path: a short loop around try_wait with a suspend-time hint, so that a waiting thread sleeps inside the
+// barrier unit instead of spending issue slots (an arrival that does not complete the phase still wakes it, hence
+// the loop).  After kFastPolls wake-ups it falls into the bounded out-of-line loop above.
+constexpr uint32_t kFastPolls = 64;
+constexpr uint32_t kSuspendHintNs = 20000;
+template <int SLEEP_NS = 0>
+__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
+  const uint32_t bar_s = smem_u32(b);
+  uint32_t ok, polls;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "mov.u32 %1, 0;\n"
+      "PW_WAIT:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%2], %3, %4;\n\t"
+      "@p bra PW_DONE;\n\t"
+      "add.u32 %1, %1, 1;\n\t"
+      "setp.lt.u32 q, %1, %5;\n\t"
+      "@q bra PW_WAIT;\n"
+      "PW_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok), "=&r"(polls)
+      : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "r"(kFastPolls)
+      : "memory");
+#ifdef PW_TC_PROFILE
+  if ((threadIdx.x & 31) == 0 && polls) atomicAdd(&g_spins[threadIdx.x >> 5], (unsigned long long)polls);
+#endif
+  if (ok) return true;
+  return mbar_wait_slow(bar_s, parity, SLEEP_NS, c, status);
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -275,8 +316,7 @@ __device__ __forceinline__ int slot_take(int& head, int k, int n_slots) {
 }
 // Bounded wait until the weight producer has armed item n.  A consumer looks at an item's full barrier
 // only after this, so it can never mistake an older phase of the slot's barrier for the item's.
-__device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
-  if (c->issued > n) return true;
+__device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* status) {
   const unsigned long long t0 = globaltimer();
   uint32_t spins = 0;
   while (true) {
@@ -290,6 +330,10 @@ __device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status
     }
   }
 }
+__device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
+  if (c->issued > n) return true;
+  return wait_issued_slow(n, c, status);
+}
 
 // Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
 // along K) stored as 128 contiguous bytes; 8-row groups are 128 bytes apart (stride byte offset),
@@ -302,6 +346,12 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t saddr, uint32_t lb
   d |= (uint64_t)1 << 46;  // descriptor version of sm_100
   return d;
 }
+
+// Source of the next item of one matrix of a unit (weight producer).
+struct MatSrc {
+  uint32_t bits, tb;                              // bitwidth; bytes of a tile image
+  const char* src;
+};
 
 // K-half `h` of one row of an item: shared memory -> 32 registers (half2 pairs in K order).
 template <int BITS>
@@ -389,73 +439,72 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         if (u >= n_units) break;
         const Unit un = units[u];
         // per matrix of the unit: bitwidth, bytes of a code tile, and the source addresses of the unit's
-        // first item; consecutive groups of a row tile are consecutive tiles of the page
-        uint32_t ubits[NMAT], ucb[NMAT];
-        const char* usrc[NMAT];
-        const __half* uscl[NMAT];
-        const __half* uzp[NMAT];
+        // first item; consecutive groups of a row tile are consecutive tiles of the page.  Items alternate
+        // between the matrices, so the state of the matrix whose turn it is sits in `cur` and the two swap
+        // after every item (one copy of the issue code instead of one per matrix).
+        MatSrc cur, oth;
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
           const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
-          ubits[m] = row.bits;
-          ucb[m] = row.bits * 2048;
+          MatSrc t;
+          t.bits = row.bits;
+          t.tb = (uint32_t)tile_bytes((int)row.bits);
           const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + un.g0;
-          usrc[m] = reinterpret_cast<const char*>(row.codes) + tile * ucb[m];
-          uscl[m] = row.scales + tile * kTileRows;
-          uzp[m] = row.zps + tile * kTileRows;
+          t.src = reinterpret_cast<const char*>(row.codes) + tile * t.tb;
+          if (m == 0) cur = t;
+          else oth = t;
         }
-        for (int g = un.g0; ok && g < un.g1; ++g) {
-#pragma unroll
-          for (int m = 0; m < NMAT; ++m) {
-            const uint32_t bits = ubits[m];
-            const uint32_t cbytes = ucb[m];
-            uint32_t bar_s, dst_s;
-            if (bits == 16) {
-              const int s = slot_take(head, 2, n_slots);
-              const uint32_t two = 3u << s;          // both slots must have been handed back
-              if ((lk_dq | lk_mma | lk_mma2) & two) {
-                for (int j = s; ok && j < s + 2; ++j) {
-                  const uint32_t bit = 1u << j;
-                  if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
-                  else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
-                  else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
-                }
-                if (!ok) break;
-                lk_dq &= ~two;
-                lk_mma &= ~two;
-                lk_mma2 &= ~two;
+        const int n_items = (un.g1 - un.g0) * NMAT;
+#pragma unroll 1
+        for (int it = 0; ok && it < n_items; ++it) {
+          const uint32_t cbytes = cur.tb;             // the whole tile image travels in one copy
+          uint32_t bar_s, dst_s;
+          if (cur.bits == 16) {
+            const int s = slot_take(head, 2, n_slots);
+            const uint32_t two = 3u << s;          // both slots must have been handed back
+            if ((lk_dq | lk_mma | lk_mma2) & two) {
+              for (int j = s; ok && j < s + 2; ++j) {
+                const uint32_t bit = 1u << j;
+                if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
+                else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
+                else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
               }
-              bar_s = full_s + 8 * s;
-              dst_s = wring_s + s * kSlotBytes;
-              mbar_expect_tx_s(bar_s, cbytes);
-              bulk_g2s_s(dst_s, usrc[m], cbytes, bar_s);
-              lk_mma |= 1u << s;
-              lk_mma2 |= 2u << s;
-              em_par ^= 1u << s;
-            } else {
-              const int s = slot_take(head, 1, n_slots);
-              const uint32_t bit = 1u << s;
-              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
-              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
-              else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[s - 1], ((em_par >> (s - 1)) & 1) ^ 1, c, status);
               if (!ok) break;
-              lk_mma &= ~bit;
-              lk_mma2 &= ~bit;
-              bar_s = full_s + 8 * s;
-              dst_s = wring_s + s * kSlotBytes;
-              TRACE(0, n);
-              mbar_expect_tx_s(bar_s, cbytes + 512);
-              bulk_g2s_s(dst_s, usrc[m], cbytes, bar_s);
-              bulk_g2s_s(dst_s + cbytes, uscl[m], 256, bar_s);
-              bulk_g2s_s(dst_s + cbytes + 256, uzp[m], 256, bar_s);
-              uscl[m] += kTileRows;
-              uzp[m] += kTileRows;
-              lk_dq |= bit;
-              ed_par ^= bit;
+              lk_dq &= ~two;
+              lk_mma &= ~two;
+              lk_mma2 &= ~two;
             }
-            usrc[m] += cbytes;
-            ++n;
-            c->issued = n;
+            bar_s = full_s + 8 * s;
+            dst_s = wring_s + s * kSlotBytes;
+            mbar_expect_tx_s(bar_s, cbytes);
+            bulk_g2s_s(dst_s, cur.src, cbytes, bar_s);
+            lk_mma |= 1u << s;
+            lk_mma2 |= 2u << s;
+            em_par ^= 1u << s;
+          } else {
+            const int s = slot_take(head, 1, n_slots);
+            const uint32_t bit = 1u << s;
+            if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
+            else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
+            else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[s - 1], ((em_par >> (s - 1)) & 1) ^ 1, c, status);
+            if (!ok) break;
+            lk_mma &= ~bit;
+            lk_mma2 &= ~bit;
+            bar_s = full_s + 8 * s;
+            dst_s = wring_s + s * kSlotBytes;
+            TRACE(0, n);
+            mbar_expect_tx_s(bar_s, cbytes);
+            bulk_g2s_s(dst_s, cur.src, cbytes, bar_s);
+            lk_dq |= bit;
+            ed_par ^= bit;
+          }
+          cur.src += cbytes;
+          ++n;
+          c->issued = n;
+          if (NMAT == 2) {
+            const MatSrc t = cur;
+            cur = oth;
+            oth = t;
           }
         }
       }
@@ -511,6 +560,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         uint32_t ubits[NMAT];
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
+        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
@@ -529,14 +579,18 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, n); }
           const uint32_t b_lo = b_lo_unit + (uint32_t)bs * (uint32_t)(bslot_bytes >> 4);
-#pragma unroll
-          for (int m = 0; m < NMAT; ++m) {
-            const uint32_t bits = ubits[m];
+          // the other matrix has its own issuers and operand slots: only replay its ring slot
+          if (NMAT == 2 && my_m == 1) {
+            const int so = slot_take(head, item_slots(ubits[0]), n_slots);
+            full_par ^= 1u << so;
+            ++n;
+          }
+          {
+            const uint32_t bits = my_bits;
             const int s = slot_take(head, item_slots(bits), n_slots);
             const uint32_t par = (full_par >> s) & 1;
             full_par ^= 1u << s;
             const uint32_t item_n = n++;
-            if (m != my_m) continue;                 // the other matrix has its own issuers and operand slots
             if (bits == 16) {
               ok = wait_issued(item_n, c, status) && mbar_wait(&c->full[s], par, c, status);
               if (!ok) break;
@@ -577,6 +631,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               ++cnt;
             }
           }
+          if (NMAT == 2 && my_m == 0) {
+            const int so = slot_take(head, item_slots(ubits[NMAT - 1]), n_slots);
+            full_par ^= 1u << so;
+            ++n;
+          }
           if (!ok) break;
           tc_commit(&c->b_empty[bs]);
           later = 1;
@@ -599,7 +658,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + grp * 64;
     int head = 0;
     uint32_t n = 0, full_par = 0;
-    uint32_t cnt[NMAT] = {};                          // quantized items per matrix so far
+    uint32_t cnt0 = 0, cnt1 = 0;                     // quantized items per matrix so far
     int pending = -1;                                // operand half-slot whose store has not been published yet
     bool ok = true;
     auto publish = [&]() {
@@ -618,53 +677,64 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       uint32_t ubits[NMAT];
 #pragma unroll
       for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
-      for (int g = un.g0; ok && g < un.g1; ++g) {
-#pragma unroll
-        for (int m = 0; m < NMAT; ++m) {
-          const uint32_t bits = ubits[m];
-          const int s = slot_take(head, item_slots(bits), n_slots);
-          const uint32_t par = (full_par >> s) & 1;
-          full_par ^= 1u << s;
-          const uint32_t item_n = n++;
-          if (bits == 16) continue;                  // the MMA reads 16-bit tiles straight from shared memory
-          // gate items go to groups 0, 1 and up items to groups 2, 3 (a single matrix uses all four), so that
-          // the issuers of one matrix never share an operand slot with the other's
-          const int owner = NMAT == 2 ? 2 * m + (int)(cnt[m] & 1) : (int)(cnt[m] & 3);
-          const uint32_t use_par = NMAT == 2 ? (cnt[m] >> 1) & 1 : (cnt[m] >> 2) & 1;
-          ++cnt[m];
-          if (owner == grp) {
-            if (c->issued <= item_n || !mbar_try(&c->full[s], par)) {
-              publish();                             // do not sit on a finished half while waiting for HBM
-              ok = wait_issued(item_n, c, status) && mbar_wait<20>(&c->full[s], par, c, status);
-              if (!ok) break;
-            }
-            if (q == 0) { TRACE(1, item_n); }
-            const char* item = wring + s * kSlotBytes;
+      const int n_items = (un.g1 - un.g0) * NMAT;
 #pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-              __half2 w[32];
-              switch (bits) {
-                case 8: decode_item_half<8>(item, r, h, w); break;
-                case 4: decode_item_half<4>(item, r, h, w); break;
-                case 3: decode_item_half<3>(item, r, h, w); break;
-                default: decode_item_half<2>(item, r, h, w); break;
-              }
-              if (q == 0) { TRACE(2 + 3 * h, item_n); }
-              if (h == 1) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
-              }
-              publish();                             // the previous half's store, overlapped with the decode above
-              const int hs = 2 * grp + h;
-              ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
-              if (!ok) break;
-              tc_fence_after();
-              tmem_st32(lane_addr + h * 32, w);
-              if (q == 0) { TRACE(3 + 3 * h, item_n); }
-              pending = hs;
+      for (int it = 0; ok && it < n_items; ++it) {
+        // items alternate between the matrices of the unit; one copy of the code serves both
+        const int m = NMAT == 2 ? (it & 1) : 0;
+        const uint32_t bits = m ? ubits[NMAT - 1] : ubits[0];
+        const int s = slot_take(head, item_slots(bits), n_slots);
+        const uint32_t par = (full_par >> s) & 1;
+        full_par ^= 1u << s;
+        const uint32_t item_n = n++;
+        if (bits == 16) continue;                    // the MMA reads 16-bit tiles straight from shared memory
+        // gate items go to groups 0, 1 and up items to groups 2, 3 (a single matrix uses all four), so that
+        // the issuers of one matrix never share an operand slot with the other's
+        const uint32_t cm = m ? cnt1 : cnt0;
+        const int owner = NMAT == 2 ? 2 * m + (int)(cm & 1) : (int)(cm & 3);
+        const uint32_t use_par = NMAT == 2 ? (cm >> 1) & 1 : (cm >> 2) & 1;
+        if (m) ++cnt1;
+        else ++cnt0;
+        if (owner != grp) continue;
+        if (c->issued <= item_n || !mbar_try(&c->full[s], par)) {
+          publish();                                 // do not sit on a finished half while waiting for HBM
+          ok = wait_issued(item_n, c, status) && mbar_wait<20>(&c->full[s], par, c, status);
+          if (!ok) break;
+        }
+        if (q == 0) { TRACE(1, item_n); }
+        const char* item = wring + s * kSlotBytes;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          __half2 w[32];
+#ifdef PW_EXP_NODECODE
+          {
+            const uint4 t = reinterpret_cast<const uint4*>(item)[r + h * 128];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              w[j] = u32_as_h2(t.x); w[j + 1] = u32_as_h2(t.y); w[j + 2] = u32_as_h2(t.z); w[j + 3] = u32_as_h2(t.w);
             }
-            if (!ok) break;
           }
+          if (false)
+#endif
+          switch (bits) {
+            case 8: decode_item_half<8>(item, r, h, w); break;
+            case 4: decode_item_half<4>(item, r, h, w); break;
+            case 3: decode_item_half<3>(item, r, h, w); break;
+            default: decode_item_half<2>(item, r, h, w); break;
+          }
+          if (q == 0) { TRACE(2 + 3 * h, item_n); }
+          if (h == 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
+          }
+          publish();                                 // the previous half's store, overlapped with the decode above
+          const int hs = 2 * grp + h;
+          ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
+          if (!ok) break;
+          tc_fence_after();
+          tmem_st32(lane_addr + h * 32, w);
+          if (q == 0) { TRACE(3 + 3 * h, item_n); }
+          pending = hs;
         }
       }
       if (ok) publish();
@@ -737,6 +807,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 extern "C" int pw_debug_read_trace(long long* host_out) {
   cudaDeviceSynchronize();
   cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace));
+  cudaMemcpyFromSymbol(host_out + 16 * 512, g_spins, sizeof(g_spins));
+  static unsigned long long zeros[32];
+  cudaMemcpyToSymbol(g_spins, zeros, sizeof(zeros));
   return 0;
 }
 #endif

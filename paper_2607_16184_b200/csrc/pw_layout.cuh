@@ -1,11 +1,12 @@
 // The TILED page layout and the bit-level packing of codes inside it.
 //
 // A page of `rows x cols` at `bits` is cut into tiles of 128 rows x one group (128 columns).
-// Tile (rt, g) is stored contiguously at byte offset (rt * n_groups + g) * bits * 2048 of the
-// codes buffer.  A row of a tile owns bits * 16 bytes = `bits` units of 16 bytes; unit j of row r
+// Tile (rt, g) is one contiguous image at byte offset (rt * n_groups + g) * tile_bytes(bits) of the
+// page buffer: bits * 2048 bytes of codes, then (below 16 bits) the 128 fp16 scales of its rows and
+// the 128 fp16 zero-points, so that a forward kernel fetches everything it needs of a tile with one
+// bulk copy.  A row of a tile owns bits * 16 bytes = `bits` units of 16 bytes; unit j of row r
 // sits at ((j * 128) + r) * 16 inside the tile, so that the 128 threads of a row-per-thread kernel
-// read unit j with one contiguous 2 KB access.  Scales and zero-points are stored
-// [(rt * n_groups + g) * 128 + r].
+// read unit j with one contiguous 2 KB access.
 //
 // Inside a row's units the 128 codes are ordered for cheap unpacking to half2 pairs
 // (k, k+1), k even:
@@ -25,6 +26,11 @@
 namespace pw {
 
 __host__ __device__ inline size_t tile_code_bytes(int bits) { return (size_t)bits * 2048; }
+// bytes of a whole tile image: codes, then the scales and zero-points of its 128 rows
+__host__ __device__ inline size_t tile_bytes(int bits) { return (size_t)bits * 2048 + (bits < 16 ? 512 : 0); }
+// scale / zero-point of row r inside a tile image
+__host__ __device__ inline size_t tile_scale_offset(int bits, int r) { return (size_t)bits * 2048 + 2 * (size_t)r; }
+__host__ __device__ inline size_t tile_zp_offset(int bits, int r) { return (size_t)bits * 2048 + 256 + 2 * (size_t)r; }
 
 // ---- integer codes of a 32-weight slice (quarter of a row-group) -----------------------------
 // Slice q (0..3) of a row covers k = 32q .. 32q+31.  Word addresses inside a tile image:
@@ -134,6 +140,11 @@ __device__ inline __half2 dq_pair(uint32_t magic_or_code, __half2 s2, __half2 z2
   return __hfma2(__hsub2(u32_as_h2(magic_or_code), k1024), s2, z2);
 }
 
+// the same with the bias to subtract given as a half2 bit pattern (the constant whose mantissa carried the code)
+__device__ inline __half2 dq_pair_k(uint32_t biased, uint32_t bias, __half2 s2, __half2 z2) {
+  return __hfma2(__hsub2(u32_as_h2(biased), u32_as_h2(bias)), s2, z2);
+}
+
 // Quarter t (0 .. 3) of a row-group: out[p] = weights (32t + 2p, 32t + 2p + 1), p = 0 .. 15.
 // `row_units` points at unit 0 of the row inside a tile image (shared or global memory); unit j
 // of the same row is kUnitStride uint4 further on.
@@ -162,13 +173,18 @@ __device__ __forceinline__ void decode_quarter(const uint4* row_units, int t, __
       }
     }
   } else if constexpr (BITS == 4) {
+    // A nibble at mantissa bits 0-3 of 0x6400 reads 1024 + code; at bits 4-7 of 0x5400 it reads 64 + code.  One
+    // shift by 8 per word brings the other two nibbles of each half-word to those positions.
     const uint4 u = row_units[t * kUnitStride];
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int m = 0; m < 4; ++m)
-        out[4 * i + m] = dq_pair(((w[i] >> (4 * m)) & 0x000f000fu) | 0x64006400u, s2, z2);
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t w8 = w[i] >> 8;
+      out[4 * i + 0] = dq_pair_k((w[i] & 0x000f000fu) | 0x64006400u, 0x64006400u, s2, z2);
+      out[4 * i + 1] = dq_pair_k((w[i] & 0x00f000f0u) | 0x54005400u, 0x54005400u, s2, z2);
+      out[4 * i + 2] = dq_pair_k((w8 & 0x000f000fu) | 0x64006400u, 0x64006400u, s2, z2);
+      out[4 * i + 3] = dq_pair_k((w8 & 0x00f000f0u) | 0x54005400u, 0x54005400u, s2, z2);
+    }
   } else {
     // 2 bits: words 2(t%2), 2(t%2)+1 of unit t/2.  3 bits: the same low-plane words plus word t of unit 2.
     const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + (t >> 1) * kUnitStride) +

@@ -37,11 +37,8 @@ __device__ __forceinline__ void load_slice_words(const char* tb, int r, int q, u
 }
 
 template <int SRC_KIND, int SRC_BITS, int DST_BITS>
-__global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict__ src_codes,
-                                                         const __half* __restrict__ src_scales,
-                                                         const __half* __restrict__ src_zps, uint32_t cols,
-                                                         void* __restrict__ dst_codes, __half* __restrict__ dst_scales,
-                                                         __half* __restrict__ dst_zps) {
+__global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict__ src_codes, uint32_t cols,
+                                                         void* __restrict__ dst_codes) {
   const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
   const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
   const size_t tile = (size_t)rt * ng + g;
@@ -64,7 +61,7 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
       }
     }
   } else {
-    const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_code_bytes(SRC_BITS);
+    const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_bytes(SRC_BITS);
     constexpr int NW = SliceWords<SRC_BITS>::kWords;
     uint32_t w[NW];
     load_slice_words<SRC_BITS>(tb, r, q, w);
@@ -78,14 +75,14 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
     } else {
       int code[32];
       unpack_slice<SRC_BITS>(w, code);
-      const float s = __half2float(src_scales[tile * kTileRows + r]);
-      const float z = __half2float(src_zps[tile * kTileRows + r]);
+      const float s = __half2float(*reinterpret_cast<const __half*>(tb + tile_scale_offset(SRC_BITS, r)));
+      const float z = __half2float(*reinterpret_cast<const __half*>(tb + tile_zp_offset(SRC_BITS, r)));
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = dequant_exact(code[i], s, z);
     }
   }
 
-  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_code_bytes(DST_BITS);
+  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(DST_BITS);
   if constexpr (DST_BITS == 16) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -140,18 +137,17 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
     if constexpr (DST_BITS == 3) *reinterpret_cast<uint32_t*>(db + slice_word_offset<3>(r, q, 2)) = w[2];
   }
   if (q == 0) {
-    dst_scales[tile * kTileRows + r] = sh;
-    dst_zps[tile * kTileRows + r] = __float2half_rn(lo);
+    *reinterpret_cast<__half*>(db + tile_scale_offset(DST_BITS, r)) = sh;
+    *reinterpret_cast<__half*>(db + tile_zp_offset(DST_BITS, r)) = __float2half_rn(lo);
   }
 }
 
 // TILED -> CANONICAL (EXPORT = true) or CANONICAL -> TILED, same bitwidth.
 template <int BITS, bool EXPORT>
-__global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ src_codes,
-                                                       const __half* __restrict__ src_scales,
-                                                       const __half* __restrict__ src_zps, uint32_t cols,
-                                                       void* __restrict__ dst_codes, __half* __restrict__ dst_scales,
-                                                       __half* __restrict__ dst_zps) {
+__global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ src_codes, uint32_t cols,
+                                                       void* __restrict__ dst_codes,
+                                                       __half* __restrict__ can_scales,   // canonical side
+                                                       __half* __restrict__ can_zps) {
   const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
   const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
   const size_t tile = (size_t)rt * ng + g;
@@ -162,7 +158,7 @@ __global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ 
   const char* csrc = reinterpret_cast<const char*>(EXPORT ? dst_codes : src_codes);
   char* cpos = const_cast<char*>(csrc) + elem * BITS / 8;
   const char* tsrc = reinterpret_cast<const char*>(EXPORT ? src_codes : dst_codes);
-  char* tpos = const_cast<char*>(tsrc) + tile * tile_code_bytes(BITS);
+  char* tpos = const_cast<char*>(tsrc) + tile * tile_bytes(BITS);
 
   uint32_t w[NW];
   if constexpr (EXPORT) {
@@ -211,13 +207,15 @@ __global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ 
     for (int i = 0; i < NW; ++i) *reinterpret_cast<uint32_t*>(tpos + slice_word_offset<BITS>(r, q, i)) = w[i];
   }
   if (BITS < 16 && q == 0) {
-    const size_t ci = row * ng + g, ti = tile * kTileRows + r;
+    const size_t ci = row * ng + g;
+    __half* ts = reinterpret_cast<__half*>(tpos + tile_scale_offset(BITS, r));
+    __half* tz = reinterpret_cast<__half*>(tpos + tile_zp_offset(BITS, r));
     if constexpr (EXPORT) {
-      dst_scales[ci] = src_scales[ti];
-      dst_zps[ci] = src_zps[ti];
+      can_scales[ci] = *ts;
+      can_zps[ci] = *tz;
     } else {
-      dst_scales[ti] = src_scales[ci];
-      dst_zps[ti] = src_zps[ci];
+      *ts = can_scales[ci];
+      *tz = can_zps[ci];
     }
   }
 }
@@ -225,10 +223,12 @@ __global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ 
 static bool bits_ok(int b) { return b == 16 || b == 8 || b == 4 || b == 3 || b == 2; }
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-static pw_status check_page_buffers(const pw_page* p, int bits) {
+// A TILED page is one buffer (codes, scales and zero-points of a tile stored together); a CANONICAL page
+// below 16 bits has three.
+static pw_status check_page_buffers(const pw_page* p, int bits, int layout) {
   if (!p->codes) return PW_ERR_INVALID_ARG;
   if (!aligned16(p->codes)) return PW_ERR_ALIGN;
-  if (bits < 16) {
+  if (bits < 16 && layout == PW_LAYOUT_CANONICAL) {
     if (!p->scales || !p->zps) return PW_ERR_INVALID_ARG;
     if (!aligned16(p->scales) || !aligned16(p->zps)) return PW_ERR_ALIGN;
   }
@@ -236,25 +236,22 @@ static pw_status check_page_buffers(const pw_page* p, int bits) {
 }
 
 template <int SK, int SB>
-static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void* sc, const __half* ss, const __half* sz,
-                             uint32_t cols, pw_page* d) {
-  __half* ds = reinterpret_cast<__half*>(d->scales);
-  __half* dz = reinterpret_cast<__half*>(d->zps);
+static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void* sc, uint32_t cols, pw_page* d) {
   switch (dst_bits) {
     case 16:
-      if (SK == SRC_RAW) quant_tile_kernel<SK, SB, 16><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      if (SK == SRC_RAW) quant_tile_kernel<SK, SB, 16><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
     case 8:
-      if (SB > 8) quant_tile_kernel<SK, SB, (SB > 8 ? 8 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      if (SB > 8) quant_tile_kernel<SK, SB, (SB > 8 ? 8 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
     case 4:
-      if (SB > 4) quant_tile_kernel<SK, SB, (SB > 4 ? 4 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      if (SB > 4) quant_tile_kernel<SK, SB, (SB > 4 ? 4 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
     case 3:
-      if (SB > 3) quant_tile_kernel<SK, SB, (SB > 3 ? 3 : 2)><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      if (SB > 3) quant_tile_kernel<SK, SB, (SB > 3 ? 3 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
     case 2:
-      quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, ss, sz, cols, d->codes, ds, dz);
+      quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
   }
 }
@@ -281,7 +278,7 @@ extern "C" pw_status pw_quantize_block(pw_ctx* ctx, const void* w, uint32_t rows
   if (!bits_ok(bits)) return PW_ERR_BITS;
   if (rows == 0 || cols == 0 || rows % kTileRows != 0 || cols % kGroup != 0) return PW_ERR_SHAPE;
   if (!aligned16(w)) return PW_ERR_ALIGN;
-  pw_status st = check_page_buffers(dst, bits);
+  pw_status st = check_page_buffers(dst, bits, PW_LAYOUT_TILED);
   if (st != PW_OK) return st;
   dst->rows = rows;
   dst->cols = cols;
@@ -289,7 +286,7 @@ extern "C" pw_status pw_quantize_block(pw_ctx* ctx, const void* w, uint32_t rows
   dst->bits = (uint8_t)bits;
   dst->layout = PW_LAYOUT_TILED;
   dim3 grid(cols / kGroup, rows / kTileRows);
-  launch_quant_dst<SRC_RAW, 16>(bits, grid, stream, w, nullptr, nullptr, cols, dst);
+  launch_quant_dst<SRC_RAW, 16>(bits, grid, stream, w, cols, dst);
   ctx->launches++;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
@@ -302,9 +299,9 @@ extern "C" pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bi
   if (src->rows == 0 || src->cols == 0 || src->rows % kTileRows != 0 || src->cols % kGroup != 0 ||
       src->group != kGroup)
     return PW_ERR_SHAPE;
-  pw_status st = check_page_buffers(src, src->bits);
+  pw_status st = check_page_buffers(src, src->bits, PW_LAYOUT_TILED);
   if (st != PW_OK) return st;
-  st = check_page_buffers(dst, dst_bits);
+  st = check_page_buffers(dst, dst_bits, PW_LAYOUT_TILED);
   if (st != PW_OK) return st;
   if (dst->codes == src->codes) return PW_ERR_INVALID_ARG;  // a demote is out of place
   dst->rows = src->rows;
@@ -313,13 +310,11 @@ extern "C" pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bi
   dst->bits = (uint8_t)dst_bits;
   dst->layout = PW_LAYOUT_TILED;
   dim3 grid(src->cols / kGroup, src->rows / kTileRows);
-  const __half* ss = reinterpret_cast<const __half*>(src->scales);
-  const __half* sz = reinterpret_cast<const __half*>(src->zps);
   switch (src->bits) {
-    case 16: launch_quant_dst<SRC_TILED, 16>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
-    case 8: launch_quant_dst<SRC_TILED, 8>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
-    case 4: launch_quant_dst<SRC_TILED, 4>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
-    case 3: launch_quant_dst<SRC_TILED, 3>(dst_bits, grid, stream, src->codes, ss, sz, src->cols, dst); break;
+    case 16: launch_quant_dst<SRC_TILED, 16>(dst_bits, grid, stream, src->codes, src->cols, dst); break;
+    case 8: launch_quant_dst<SRC_TILED, 8>(dst_bits, grid, stream, src->codes, src->cols, dst); break;
+    case 4: launch_quant_dst<SRC_TILED, 4>(dst_bits, grid, stream, src->codes, src->cols, dst); break;
+    case 3: launch_quant_dst<SRC_TILED, 3>(dst_bits, grid, stream, src->codes, src->cols, dst); break;
   }
   ctx->launches++;
   PW_CUDA_OK(cudaGetLastError());
@@ -334,9 +329,9 @@ static pw_status relayout(pw_ctx* ctx, const pw_page* src, pw_page* dst, cudaStr
   if (src->rows == 0 || src->cols == 0 || src->rows % kTileRows != 0 || src->cols % kGroup != 0 ||
       src->group != kGroup)
     return PW_ERR_SHAPE;
-  pw_status st = check_page_buffers(src, src->bits);
+  pw_status st = check_page_buffers(src, src->bits, src->layout);
   if (st != PW_OK) return st;
-  st = check_page_buffers(dst, src->bits);
+  st = check_page_buffers(dst, src->bits, EXPORT ? PW_LAYOUT_CANONICAL : PW_LAYOUT_TILED);
   if (st != PW_OK) return st;
   if (dst->codes == src->codes) return PW_ERR_INVALID_ARG;
   dst->rows = src->rows;
@@ -345,16 +340,16 @@ static pw_status relayout(pw_ctx* ctx, const pw_page* src, pw_page* dst, cudaStr
   dst->bits = src->bits;
   dst->layout = EXPORT ? PW_LAYOUT_CANONICAL : PW_LAYOUT_TILED;
   dim3 grid(src->cols / kGroup, src->rows / kTileRows);
-  const __half* ss = reinterpret_cast<const __half*>(src->scales);
-  const __half* sz = reinterpret_cast<const __half*>(src->zps);
-  __half* ds = reinterpret_cast<__half*>(dst->scales);
-  __half* dz = reinterpret_cast<__half*>(dst->zps);
+  // scales / zero-points of the canonical side (read on import, written on export)
+  const pw_page* can = EXPORT ? dst : src;
+  __half* cs = reinterpret_cast<__half*>(can->scales);
+  __half* cz = reinterpret_cast<__half*>(can->zps);
   switch (src->bits) {
-    case 16: relayout_kernel<16, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
-    case 8: relayout_kernel<8, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
-    case 4: relayout_kernel<4, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
-    case 3: relayout_kernel<3, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
-    case 2: relayout_kernel<2, EXPORT><<<grid, 512, 0, stream>>>(src->codes, ss, sz, src->cols, dst->codes, ds, dz); break;
+    case 16: relayout_kernel<16, EXPORT><<<grid, 512, 0, stream>>>(src->codes, src->cols, dst->codes, cs, cz); break;
+    case 8: relayout_kernel<8, EXPORT><<<grid, 512, 0, stream>>>(src->codes, src->cols, dst->codes, cs, cz); break;
+    case 4: relayout_kernel<4, EXPORT><<<grid, 512, 0, stream>>>(src->codes, src->cols, dst->codes, cs, cz); break;
+    case 3: relayout_kernel<3, EXPORT><<<grid, 512, 0, stream>>>(src->codes, src->cols, dst->codes, cs, cz); break;
+    case 2: relayout_kernel<2, EXPORT><<<grid, 512, 0, stream>>>(src->codes, src->cols, dst->codes, cs, cz); break;
   }
   ctx->launches++;
   PW_CUDA_OK(cudaGetLastError());
