@@ -61,6 +61,10 @@ struct Ctrl {                                  // lives at the start of dynamic 
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile uint32_t issued;                    // items 0 .. issued-1 have been armed by the weight producer
+  // Work list of this CTA: the weight producer claims units from a global counter and posts them here;
+  // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
+  volatile uint32_t sched_n;
+  volatile int32_t sched_unit[32];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
@@ -70,8 +74,11 @@ __device__ long long g_trace[16][512];
 __device__ unsigned long long g_spins[32];      // polling-loop iterations per warp index, all CTAs
 #define TRACE(ev, n) \
   if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
+#define TRACEV(ev, n, v) \
+  if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = (long long)(v)
 #else
 #define TRACE(ev, n)
+#define TRACEV(ev, n, v)
 #endif
 
 struct TmapSet {                               // token-tile copies: one map per tile height 16, 32, .. 128
@@ -303,18 +310,30 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Ring slots an item needs: a 16-bit tile is 32 KB, every quantized tile (codes, then its 128 scales,
-// then its 128 zero-points) fits one slot.
-__device__ __forceinline__ int item_slots(uint32_t bits) { return bits == 16 ? 2 : 1; }
-// Slots are handed out cyclically; an item never wraps (a two-slot item skips a lone last slot).
-// Every role replays the same sequence.
-__device__ __forceinline__ int slot_take(int& head, int k, int n_slots) {
-  if (head + k > n_slots) head = 0;
-  const int s = head;
-  head += k;
-  return s;
+// The slot ring.  Everything that travels through it is one "slot item" of at most kSlotBytes: a quantized
+// tile image (codes, scales, zero-points), or one K-half (64 columns, 16 KB) of a 16-bit tile -- the two halves
+// of a 16-bit tile are consecutive slot items.  Slot items are numbered in issue order; number `seq` sits in
+// slot seq % n_slots and uses phase seq / n_slots of that slot's barriers, so every role finds its own slot
+// items without replaying anybody else's.
+struct RingPos {
+  uint32_t s, par;                               // slot, parity of the full-barrier phase
+};
+__device__ __forceinline__ RingPos ring_pos(uint32_t seq, uint32_t n_slots) {
+  const uint32_t q = seq / n_slots;
+  RingPos p;
+  p.s = seq - q * n_slots;
+  p.par = q & 1u;
+  return p;
 }
-// Bounded wait until the weight producer has armed item n.  A consumer looks at an item's full barrier
+__device__ __forceinline__ void ring_advance(RingPos& p, uint32_t step, uint32_t n_slots) {
+  p.s += step;
+  while (p.s >= n_slots) {
+    p.s -= n_slots;
+    p.par ^= 1u;
+  }
+}
+__device__ __forceinline__ uint32_t slot_items(uint32_t bits) { return bits == 16 ? 2u : 1u; }
+// Bounded wait until the weight producer has armed slot item n.  A consumer looks at a slot item's full barrier
 // only after this, so it can never mistake an older phase of the slot's barrier for the item's.
 __device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* status) {
   const unsigned long long t0 = globaltimer();
@@ -333,6 +352,26 @@ __device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* stat
 __device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
   if (c->issued > n) return true;
   return wait_issued_slow(n, c, status);
+}
+// Unit i of this CTA's work list (bounded wait until the weight producer has posted it); -1 = no more work,
+// -2 = the CTA is aborting.
+__device__ __noinline__ int next_unit_slow(uint32_t i, Ctrl* c, int32_t* status) {
+  const unsigned long long t0 = globaltimer();
+  uint32_t spins = 0;
+  while (true) {
+    __nanosleep(64);
+    if (c->sched_n > i) return c->sched_unit[i & 31];
+    if (c->abort_flag) return -2;
+    if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
+      c->abort_flag = 1;
+      atomicMax(status, (int)PW_ERR_TIMEOUT);
+      return -2;
+    }
+  }
+}
+__device__ __forceinline__ int next_unit(uint32_t i, Ctrl* c, int32_t* status) {
+  if (c->sched_n > i) return c->sched_unit[i & 31];
+  return next_unit_slow(i, c, status);
 }
 
 // Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
@@ -369,7 +408,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, const int32_t* __restrict__ n_units_ptr,
               const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
               __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
-              int32_t* __restrict__ status) {
+              int32_t* __restrict__ work_counter, int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   char* wring = smem + kCtrlBytes;
@@ -392,7 +431,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(&c->full[i], 1);
       mbar_init(&c->empty_dq[i], 4);             // the four warps of the group that owns the item
-      mbar_init(&c->empty_mma[i], npart);
+      mbar_init(&c->empty_mma[i], per_half);      // the issuers that read this K-half of a 16-bit tile
     }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
@@ -406,6 +445,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     mbar_init(&c->d_empty, 4);
     c->abort_flag = 0;
     c->issued = 0;
+    c->sched_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -420,28 +460,31 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   tc_fence_after();
   const uint32_t tmem = c->tmem_base;
 
-  // unit i of this CTA in snake order over the size-sorted list
-  auto unit_index = [&](int i) { return i * G + ((i & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x); };
+  // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
+  // (the weight producer claims, the other roles follow its list).
 
   if (warp == kWarpCodes) {
     // ---------------- weight producer ----------------
     if (lane == 0) {
-      int head = 0;
-      uint32_t n = 0;                              // item sequence number
-      // Per-slot state, one bit per slot.  lk_*: who hands the slot back (a dequantizer group, the MMA
-      // issuers, or the MMA issuers through the barrier of the slot before it, for the second slot of a
-      // 16-bit item).  ed_par / em_par: parity of the next phase of empty_dq / empty_mma of the slot.
-      uint32_t lk_dq = 0, lk_mma = 0, lk_mma2 = 0, ed_par = 0, em_par = 0;
+      uint32_t seq = 0, s = 0;                     // slot items armed so far; slot of the next one
+      // Per-slot state, one bit per slot.  lk_dq / lk_mma: who hands the slot back (the dequantizer group
+      // that read it, or the MMA issuers that read a 16-bit half).  ed_par / em_par: parity of the next
+      // phase of empty_dq / empty_mma of the slot.
+      uint32_t lk_dq = 0, lk_mma = 0, ed_par = 0, em_par = 0;
       const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]);
       bool ok = true;
-      for (int i = 0; ok; ++i) {
-        const int u = unit_index(i);
-        if (u >= n_units) break;
+      // the work list: unit blockIdx.x first, then whatever the global counter hands out
+      int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
+      c->sched_unit[0] = u;
+      __threadfence_block();
+      c->sched_n = 1;
+      for (int i = 0; ok && u >= 0; ++i) {
         const Unit un = units[u];
-        // per matrix of the unit: bitwidth, bytes of a code tile, and the source addresses of the unit's
-        // first item; consecutive groups of a row tile are consecutive tiles of the page.  Items alternate
-        // between the matrices, so the state of the matrix whose turn it is sits in `cur` and the two swap
-        // after every item (one copy of the issue code instead of one per matrix).
+        int claimed = 0;
+        // per matrix of the unit: bitwidth, bytes of a tile image, address of the unit's first tile;
+        // consecutive groups of a row tile are consecutive tiles of the page.  Tiles alternate between the
+        // matrices, so the state of the matrix whose turn it is sits in `cur` and the two swap after every
+        // tile (one copy of the issue code instead of one per matrix).
         MatSrc cur, oth;
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
@@ -454,59 +497,48 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           if (m == 0) cur = t;
           else oth = t;
         }
-        const int n_items = (un.g1 - un.g0) * NMAT;
+        const int n_tiles = (un.g1 - un.g0) * NMAT;
+        const int claim_at = n_tiles >> 1;
 #pragma unroll 1
-        for (int it = 0; ok && it < n_items; ++it) {
-          const uint32_t cbytes = cur.tb;             // the whole tile image travels in one copy
-          uint32_t bar_s, dst_s;
-          if (cur.bits == 16) {
-            const int s = slot_take(head, 2, n_slots);
-            const uint32_t two = 3u << s;          // both slots must have been handed back
-            if ((lk_dq | lk_mma | lk_mma2) & two) {
-              for (int j = s; ok && j < s + 2; ++j) {
-                const uint32_t bit = 1u << j;
-                if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[j], ((ed_par >> j) & 1) ^ 1, c, status);
-                else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[j], ((em_par >> j) & 1) ^ 1, c, status);
-                else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[j - 1], ((em_par >> (j - 1)) & 1) ^ 1, c, status);
-              }
-              if (!ok) break;
-              lk_dq &= ~two;
-              lk_mma &= ~two;
-              lk_mma2 &= ~two;
-            }
-            bar_s = full_s + 8 * s;
-            dst_s = wring_s + s * kSlotBytes;
-            mbar_expect_tx_s(bar_s, cbytes);
-            bulk_g2s_s(dst_s, cur.src, cbytes, bar_s);
-            lk_mma |= 1u << s;
-            lk_mma2 |= 2u << s;
-            em_par ^= 1u << s;
-          } else {
-            const int s = slot_take(head, 1, n_slots);
+        for (int it = 0; ok && it < n_tiles; ++it) {
+          // claim the next unit half-way through this one: the answer is back long before it is needed
+          if (it == claim_at) claimed = atomicAdd(work_counter, 1) + G;
+          const bool f16 = cur.bits == 16;
+          const uint32_t bytes = f16 ? 16384u : cur.tb;   // a 16-bit tile goes as two K-halves
+          const int nsub = f16 ? 2 : 1;
+          for (int sub = 0; sub < nsub; ++sub) {
             const uint32_t bit = 1u << s;
             if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
             else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
-            else if (lk_mma2 & bit) ok = mbar_wait<32>(&c->empty_mma[s - 1], ((em_par >> (s - 1)) & 1) ^ 1, c, status);
             if (!ok) break;
-            lk_mma &= ~bit;
-            lk_mma2 &= ~bit;
-            bar_s = full_s + 8 * s;
-            dst_s = wring_s + s * kSlotBytes;
-            TRACE(0, n);
-            mbar_expect_tx_s(bar_s, cbytes);
-            bulk_g2s_s(dst_s, cur.src, cbytes, bar_s);
-            lk_dq |= bit;
-            ed_par ^= bit;
+            const uint32_t bar_s = full_s + 8 * s;
+            TRACE(0, seq);
+            mbar_expect_tx_s(bar_s, bytes);
+            bulk_g2s_s(wring_s + s * kSlotBytes, cur.src, bytes, bar_s);
+            if (f16) {
+              lk_mma |= bit;
+              lk_dq &= ~bit;
+              em_par ^= bit;
+            } else {
+              lk_dq |= bit;
+              lk_mma &= ~bit;
+              ed_par ^= bit;
+            }
+            cur.src += bytes;
+            ++seq;
+            c->issued = seq;
+            if (++s == (uint32_t)n_slots) s = 0;
           }
-          cur.src += cbytes;
-          ++n;
-          c->issued = n;
           if (NMAT == 2) {
             const MatSrc t = cur;
             cur = oth;
             oth = t;
           }
         }
+        u = claimed < n_units ? claimed : -1;
+        c->sched_unit[(i + 1) & 31] = u;
+        __threadfence_block();
+        c->sched_n = (uint32_t)i + 2;
       }
     }
   } else if (warp == kWarpTokens) {
@@ -515,8 +547,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       uint32_t bcount = 0;
       bool ok = true;
       for (int i = 0; ok; ++i) {
-        const int u = unit_index(i);
-        if (u >= n_units) break;
+        const int u = next_unit((uint32_t)i, c, status);
+        if (u < 0) break;
         const Unit un = units[u];
         const int nb_rows = (un.ntok + 15) & ~15;
         const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
@@ -543,9 +575,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const int my_h0 = npart >= 2 ? my_j / per_half : 0;
       const int n_h = npart >= 2 ? 1 : 2;
       const int my_p = npart >= 2 ? my_j % per_half : 0;
-      int head = 0;
-      uint32_t n = 0, full_par = 0;                 // item sequence number; per-slot parity of the full barrier
-      uint32_t cnt = 0, ucount = 0;                 // cnt: quantized items of my matrix so far
+      uint32_t seq_unit = 0;                        // slot items before the current unit
+      uint32_t cnt = 0, ucount = 0;                 // cnt: quantized tiles of my matrix so far
       int bs = 0;                                   // token-tile slot and its barrier parity, kept incrementally
       uint32_t bpar = 0;
       const uint32_t d_t = tmem + (my_m * npart + my_j) * nt_tile;
@@ -554,19 +585,25 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const uint32_t w_lo_base = smem_u32(wring) >> 4;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
-        const int u = unit_index(i);
-        if (u >= n_units) break;
+        const int u = next_unit((uint32_t)i, c, status);
+        if (u < 0) break;
         const Unit un = units[u];
         uint32_t ubits[NMAT];
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
         const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
+        // slot items per group of the unit (W) and the offset of my matrix's inside a group
+        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
         const uint32_t b_step = (uint32_t)(2 * nb_rows) * per_half;
         const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        // my first 16-bit slot item of the unit: K-half my_h0 of my matrix's tile of the first group
+        uint32_t sq = seq_unit + my_off + (uint32_t)my_h0;
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
         ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
         if (!ok) break;
@@ -574,69 +611,59 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         tc_fence_after();
         uint32_t later = 0;                          // becomes 1 after the first group: accumulate onto earlier groups
         for (int g = un.g0; ok && g < un.g1; ++g) {
-          if (my_m == 0 && my_j == 0) { TRACE(10, n); }
+          if (my_m == 0 && my_j == 0) { TRACE(10, sq); }
           ok = mbar_wait(&c->b_full[bs], bpar, c, status);
           if (!ok) break;
-          if (my_m == 0 && my_j == 0) { TRACE(11, n); }
+          if (my_m == 0 && my_j == 0) { TRACE(11, sq); }
           const uint32_t b_lo = b_lo_unit + (uint32_t)bs * (uint32_t)(bslot_bytes >> 4);
-          // the other matrix has its own issuers and operand slots: only replay its ring slot
-          if (NMAT == 2 && my_m == 1) {
-            const int so = slot_take(head, item_slots(ubits[0]), n_slots);
-            full_par ^= 1u << so;
-            ++n;
-          }
-          {
-            const uint32_t bits = my_bits;
-            const int s = slot_take(head, item_slots(bits), n_slots);
-            const uint32_t par = (full_par >> s) & 1;
-            full_par ^= 1u << s;
-            const uint32_t item_n = n++;
-            if (bits == 16) {
-              ok = wait_issued(item_n, c, status) && mbar_wait(&c->full[s], par, c, status);
+          if (my_bits == 16) {
+            // the K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3 at 4 KB)
+            RingPos hp = rp;
+            for (int hh = 0; hh < n_h; ++hh) {
+              if (my_j == 0) { TRACE(12, sq + hh); }
+              ok = wait_issued(sq + (uint32_t)hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
-              const uint32_t a_lo = (w_lo_base + (uint32_t)s * (kSlotBytes >> 4)) | a_lo_lbo;
-              for (int hh = 0; hh < n_h; ++hh) {
-                const uint32_t k0 = 4 * (my_h0 + hh) + my_p;
-                if (per_half == 1)
-                  tc_mma_ss_burst<4>(d_t, a_lo + k0 * 256, desc_hi, 256, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
-                                     later | (uint32_t)hh);
-                else
-                  tc_mma_ss_burst<2>(d_t, a_lo + k0 * 256, desc_hi, 512, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
-                                     later);
-              }
-              tc_commit(&c->empty_mma[s]);
-            } else {
-              // the group that dequantizes this item, and the parity of this use of its half-slots
-              const int grp = NMAT == 2 ? 2 * my_m + (int)(cnt & 1) : (int)(cnt & 3);
-              const uint32_t use_par = NMAT == 2 ? (cnt >> 1) & 1 : (cnt >> 2) & 1;
-              for (int hh = 0; hh < n_h; ++hh) {
-                const int h = my_h0 + hh;
-                const int hs = 2 * grp + h;
-                if (my_j == 0) { TRACE(12, item_n); }
-                ok = mbar_wait(&c->a_full[hs], use_par, c, status);
-                if (!ok) break;
-                tc_fence_after();
-                if (my_j == 0) { TRACE(8, item_n); }
-                const uint32_t a_t = tmem + acol + hs * 32 + my_p * 8;
-                const uint32_t k0 = 4 * h + my_p;
-                if (per_half == 1)
-                  tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later | (uint32_t)hh);
-                else
-                  tc_mma_ts_burst<2>(d_t, a_t, 16, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later);
-                tc_commit(&c->a_empty[hs]);
-              }
-              if (!ok) break;
-              if (my_j == 0) { TRACE(9, item_n); }
-              ++cnt;
+              if (my_j == 0) { TRACE(8, sq + hh); }
+              const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
+              const uint32_t k0 = 4 * (my_h0 + hh) + my_p;
+              if (per_half == 1)
+                tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
+                                   later | (uint32_t)hh);
+              else
+                tc_mma_ss_burst<2>(d_t, a_lo + my_p * 256, desc_hi, 512, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
+                                   later);
+              tc_commit(&c->empty_mma[hp.s]);
+              if (my_j == 0) { TRACE(9, sq + hh); }
+              if (n_h == 2) ring_advance(hp, 1, (uint32_t)n_slots);
             }
+            if (!ok) break;
+          } else {
+            // the group that dequantizes this tile, and the parity of this use of its half-slots
+            const int grp = NMAT == 2 ? 2 * my_m + (int)(cnt & 1) : (int)(cnt & 3);
+            const uint32_t use_par = NMAT == 2 ? (cnt >> 1) & 1 : (cnt >> 2) & 1;
+            for (int hh = 0; hh < n_h; ++hh) {
+              const int h = my_h0 + hh;
+              const int hs = 2 * grp + h;
+              if (my_j == 0) { TRACE(12, sq); }
+              ok = mbar_wait(&c->a_full[hs], use_par, c, status);
+              if (!ok) break;
+              tc_fence_after();
+              if (my_j == 0) { TRACE(8, sq); }
+              const uint32_t a_t = tmem + acol + hs * 32 + my_p * 8;
+              const uint32_t k0 = 4 * h + my_p;
+              if (per_half == 1)
+                tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later | (uint32_t)hh);
+              else
+                tc_mma_ts_burst<2>(d_t, a_t, 16, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later);
+              tc_commit(&c->a_empty[hs]);
+            }
+            if (!ok) break;
+            if (my_j == 0) { TRACE(9, sq); }
+            ++cnt;
           }
-          if (NMAT == 2 && my_m == 0) {
-            const int so = slot_take(head, item_slots(ubits[NMAT - 1]), n_slots);
-            full_par ^= 1u << so;
-            ++n;
-          }
-          if (!ok) break;
+          sq += W;
+          ring_advance(rp, W, (uint32_t)n_slots);
           tc_commit(&c->b_empty[bs]);
           later = 1;
           if (++bs == n_bslots) {
@@ -645,6 +672,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           }
         }
         if (ok) tc_commit(&c->d_full);
+        TRACE(4, ucount * 4 + iss);
+        seq_unit += (uint32_t)(un.g1 - un.g0) * W;
       }
     }
   } else if (warp < kDqWarps) {
@@ -656,9 +685,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     const int grp = warp >> 2, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + grp * 64;
-    int head = 0;
-    uint32_t n = 0, full_par = 0;
-    uint32_t cnt0 = 0, cnt1 = 0;                     // quantized items per matrix so far
+    const int qm = NMAT == 2 ? grp >> 1 : 0;         // the matrix this group serves
+    const uint32_t gsub = NMAT == 2 ? (uint32_t)(grp & 1) : (uint32_t)grp;   // which of that matrix's groups
+    constexpr uint32_t kStride = NMAT == 2 ? 2 : 4;  // groups per matrix = distance between my tiles
+    uint32_t seq_unit = 0;                           // slot items before the current unit
+    uint32_t cntm = 0;                               // quantized tiles of my matrix so far
+    uint32_t uses = 0;                               // tiles I have taken so far (parity of my half-slots' use)
     int pending = -1;                                // operand half-slot whose store has not been published yet
     bool ok = true;
     auto publish = [&]() {
@@ -671,74 +703,76 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       }
     };
     for (int i = 0; ok; ++i) {
-      const int u = unit_index(i);
-      if (u >= n_units) break;
+      const int u = next_unit((uint32_t)i, c, status);
+      if (u < 0) break;
       const Unit un = units[u];
       uint32_t ubits[NMAT];
 #pragma unroll
       for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
-      const int n_items = (un.g1 - un.g0) * NMAT;
+      const uint32_t bits = qm ? ubits[NMAT - 1] : ubits[0];
+      const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+      const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+      if (bits != 16) {                              // the MMA reads 16-bit tiles straight from shared memory
+        // Quantized tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my
+        // first one in this unit is group j0, then every kStride-th.
+        const uint32_t j0 = (gsub - cntm) & (kStride - 1);
+        const uint32_t step = kStride * W;
+        uint32_t sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
 #pragma unroll 1
-      for (int it = 0; ok && it < n_items; ++it) {
-        // items alternate between the matrices of the unit; one copy of the code serves both
-        const int m = NMAT == 2 ? (it & 1) : 0;
-        const uint32_t bits = m ? ubits[NMAT - 1] : ubits[0];
-        const int s = slot_take(head, item_slots(bits), n_slots);
-        const uint32_t par = (full_par >> s) & 1;
-        full_par ^= 1u << s;
-        const uint32_t item_n = n++;
-        if (bits == 16) continue;                    // the MMA reads 16-bit tiles straight from shared memory
-        // gate items go to groups 0, 1 and up items to groups 2, 3 (a single matrix uses all four), so that
-        // the issuers of one matrix never share an operand slot with the other's
-        const uint32_t cm = m ? cnt1 : cnt0;
-        const int owner = NMAT == 2 ? 2 * m + (int)(cm & 1) : (int)(cm & 3);
-        const uint32_t use_par = NMAT == 2 ? (cm >> 1) & 1 : (cm >> 2) & 1;
-        if (m) ++cnt1;
-        else ++cnt0;
-        if (owner != grp) continue;
-        if (c->issued <= item_n || !mbar_try(&c->full[s], par)) {
-          publish();                                 // do not sit on a finished half while waiting for HBM
-          ok = wait_issued(item_n, c, status) && mbar_wait<20>(&c->full[s], par, c, status);
-          if (!ok) break;
-        }
-        if (q == 0) { TRACE(1, item_n); }
-        const char* item = wring + s * kSlotBytes;
+        for (uint32_t j = j0; ok && j < ng; j += kStride) {
+          const uint32_t use_par = uses & 1u;
+          ++uses;
+          if (c->issued <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
+            publish();                               // do not sit on a finished half while waiting for HBM
+            ok = wait_issued(sq, c, status) && mbar_wait<20>(&c->full[rp.s], rp.par, c, status);
+            if (!ok) break;
+          }
+          if (q == 0) { TRACE(1, sq); }
+          const char* item = wring + rp.s * kSlotBytes;
 #pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          __half2 w[32];
+          for (int h = 0; h < 2; ++h) {
+            __half2 w[32];
 #ifdef PW_EXP_NODECODE
-          {
-            const uint4 t = reinterpret_cast<const uint4*>(item)[r + h * 128];
+            {
+              const uint4 t = reinterpret_cast<const uint4*>(item)[r + h * 128];
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              w[j] = u32_as_h2(t.x); w[j + 1] = u32_as_h2(t.y); w[j + 2] = u32_as_h2(t.z); w[j + 3] = u32_as_h2(t.w);
+              for (int jj = 0; jj < 32; jj += 4) {
+                w[jj] = u32_as_h2(t.x); w[jj + 1] = u32_as_h2(t.y); w[jj + 2] = u32_as_h2(t.z); w[jj + 3] = u32_as_h2(t.w);
+              }
             }
-          }
-          if (false)
+            if (false)
 #endif
-          switch (bits) {
-            case 8: decode_item_half<8>(item, r, h, w); break;
-            case 4: decode_item_half<4>(item, r, h, w); break;
-            case 3: decode_item_half<3>(item, r, h, w); break;
-            default: decode_item_half<2>(item, r, h, w); break;
+            switch (bits) {
+              case 8: decode_item_half<8>(item, r, h, w); break;
+              case 4: decode_item_half<4>(item, r, h, w); break;
+              case 3: decode_item_half<3>(item, r, h, w); break;
+              default: decode_item_half<2>(item, r, h, w); break;
+            }
+            if (q == 0) { TRACE(2 + 3 * h, sq); }
+            if (h == 1) {
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&c->empty_dq[rp.s]);   // this warp has read its rows of the tile
+            }
+            publish();                               // the previous half's store, overlapped with the decode above
+            const int hs = 2 * grp + h;
+            ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
+            if (!ok) break;
+            tc_fence_after();
+            tmem_st32(lane_addr + h * 32, w);
+            if (q == 0) { TRACE(3 + 3 * h, sq); }
+            pending = hs;
           }
-          if (q == 0) { TRACE(2 + 3 * h, item_n); }
-          if (h == 1) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&c->empty_dq[s]);   // this warp has read its rows of the item
-          }
-          publish();                                 // the previous half's store, overlapped with the decode above
-          const int hs = 2 * grp + h;
-          ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
           if (!ok) break;
-          tc_fence_after();
-          tmem_st32(lane_addr + h * 32, w);
-          if (q == 0) { TRACE(3 + 3 * h, item_n); }
-          pending = hs;
+          if (j + kStride >= ng) publish();          // my last tile of the unit: the issuers are waiting to finish it
+          sq += step;
+          ring_advance(rp, step, (uint32_t)n_slots);
         }
+        cntm += ng;
       }
-      if (ok) publish();
+      seq_unit += ng * W;
     }
+    publish();
   } else if (warp >= kWarpEpi) {
     // ---------------- epilogue ----------------
     const int q = warp & 3;
@@ -747,12 +781,13 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     uint32_t ucount = 0;
     bool ok = true;
     for (int i = 0; ok; ++i, ++ucount) {
-      const int u = unit_index(i);
-      if (u >= n_units) break;
+      const int u = next_unit((uint32_t)i, c, status);
+      if (u < 0) break;
       const Unit un = units[u];
       ok = mbar_wait<200>(&c->d_full, ucount & 1, c, status);
       if (!ok) break;
       if (q == 0) { TRACE(13, ucount); }
+      if (q == 0) { TRACEV(7, ucount, rows[un.seg * 3].bits * 100 + rows[un.seg * 3 + 1].bits + 10000 * un.ntok); }
       tc_fence_after();
       const int nb_rows = (un.ntok + 15) & ~15;
       const int row = un.row_tile * kTileRows + r;
@@ -890,16 +925,17 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const int R = T * k + c.n_shared * T;
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
+  int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
                                                         st->xt, w.Rpad, nt_tile, n_bslots, n_slots,
                                                         reinterpret_cast<__half*>(b + w.ht), nullptr, c.hidden, 0,
-                                                        status);
+                                                        work_counter, status);
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
                                                         st->ht, w.Rpad, nt_tile, n_bslots, n_slots, nullptr,
                                                         reinterpret_cast<float*>(b + w.y), c.hidden,
-                                                        (size_t)R * c.hidden, status);
+                                                        (size_t)R * c.hidden, work_counter + 1, status);
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   (void)ksplit;

@@ -133,8 +133,11 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
 
   if (nt_tile <= 0) return;  // SIMT path: no unit lists
 
-  // Segments ordered by the bytes of their gate+up (resp. down) pages, largest first, so that the
-  // dynamically scheduled CTAs finish together.  Rank by counting (S is small).
+  // Unit lists.  The CTAs of the FFN kernels claim units in list order, so the list is laid out for that:
+  // row tile outermost, K split next, then every segment's token tiles (segments with the widest pages
+  // first).  Consecutive units therefore belong to different experts -- pages of different bitwidths are
+  // in flight together, the ones bound by HBM beside the ones bound by unpacking -- and the tiles that
+  // share weights are adjacent.  Rank segments by counting (S is small).
   for (int phase = 0; phase < 2; ++phase) {
     __syncthreads();
     for (int s = tid; s < S; s += blockDim.x) {
@@ -151,18 +154,19 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
     const int ng = (phase == 0 ? H : F) / kGroup;
     const int splits = phase == 0 ? 1 : ksplit;
     if (tid == 0) {
-      int a = 0;
+      int a = 0;                                   // token tiles of the segments before i, in rank order
       for (int i = 0; i < S; ++i) {
         ubase[i] = a;
-        const int n = cnt[order[i]];
-        a += ((n + nt_tile - 1) / nt_tile) * row_tiles * splits;
+        a += (cnt[order[i]] + nt_tile - 1) / nt_tile;
       }
       ubase[S] = a;
-      n_units[phase] = a <= max_units ? a : 0;
-      if (a > max_units) atomicMax(status, (int)PW_ERR_NOMEM);
+      const long long total = (long long)a * row_tiles * splits;
+      n_units[phase] = total <= max_units ? (int)total : 0;
+      if (total > max_units) atomicMax(status, (int)PW_ERR_NOMEM);
     }
     __syncthreads();
-    if (ubase[S] > max_units) continue;
+    const int TT = ubase[S];
+    if ((long long)TT * row_tiles * splits > max_units) continue;
     Unit* out = phase == 0 ? units_gu : units_dn;
     if (phase == 0)
       for (int i = tid; i < S; i += blockDim.x) seg_order[i] = order[i];
@@ -171,11 +175,11 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
       const int n = cnt[s];
       const int tt = (n + nt_tile - 1) / nt_tile;
       const int total = tt * row_tiles * splits;
-      // order: row tile, then split, then token tile (innermost: tiles that share weights run together)
       for (int u = tid; u < total; u += blockDim.x) {
         const int ti = u % tt;
-        const int sp = (u / tt) % splits;
-        const int rt = u / (tt * splits);
+        const int rs = u / tt;                       // row tile * splits + split
+        const int sp = rs % splits;
+        const int rt = rs / splits;
         Unit un;
         un.seg = s;
         un.row_tile = rt;
@@ -185,7 +189,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
         un.g1 = (int)(((long long)(sp + 1) * ng) / splits);
         un.split = sp;
         un.pad_ = 0;
-        out[ubase[i] + u] = un;
+        out[(size_t)rs * TT + ubase[i] + ti] = un;
       }
     }
   }
