@@ -45,7 +45,7 @@ constexpr int kMaxBSlots = 4;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
 constexpr int kDqWarps = 16;
-constexpr int kWarpCodes = 16, kWarpTokens = 17, kWarpMma = 19, kIssuers = 4, kWarpEpi = 23;
+constexpr int kWarpCodes = 16, kWarpTokens = 17, kWarpCodes2 = 18, kWarpMma = 19, kIssuers = 4, kWarpEpi = 23;
 constexpr int kThreads = 864;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
@@ -60,7 +60,10 @@ struct Ctrl {                                  // lives at the start of dynamic 
   unsigned long long d_full, d_empty;
   uint32_t tmem_base;
   volatile int abort_flag;
-  volatile uint32_t issued;                    // items 0 .. issued-1 have been armed by the weight producer
+  // Slot items with an even number are armed by weight producer 0, odd ones by producer 1 (the number of
+  // slots is even, so each producer also owns every other slot).  issued[p]: producer p has armed all of
+  // its slot items below this number.
+  volatile uint32_t issued[2];
   // Work list of this CTA: the weight producer claims units from a global counter and posts them here;
   // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
@@ -340,7 +343,7 @@ __device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* stat
   uint32_t spins = 0;
   while (true) {
     __nanosleep(32);
-    if (c->issued > n) return true;
+    if (c->issued[n & 1] > n) return true;
     if (c->abort_flag) return false;
     if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
       c->abort_flag = 1;
@@ -350,7 +353,7 @@ __device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* stat
   }
 }
 __device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
-  if (c->issued > n) return true;
+  if (c->issued[n & 1] > n) return true;
   return wait_issued_slow(n, c, status);
 }
 // Unit i of this CTA's work list (bounded wait until the weight producer has posted it); -1 = no more work,
@@ -444,7 +447,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     mbar_init(&c->d_full, n_issuers);
     mbar_init(&c->d_empty, 4);
     c->abort_flag = 0;
-    c->issued = 0;
+    c->issued[0] = c->issued[1] = 0;
     c->sched_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -463,10 +466,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
   // (the weight producer claims, the other roles follow its list).
 
-  if (warp == kWarpCodes) {
-    // ---------------- weight producer ----------------
+  if (warp == kWarpCodes || warp == kWarpCodes2) {
+    // ---------------- weight producers ----------------
+    // Two single-thread producers share the stream: producer P arms the slot items with number = P mod 2,
+    // which (even slot count) always land in the slots = P mod 2, so each keeps the state of its own slots.
+    // Producer 0 also claims the units.
     if (lane == 0) {
-      uint32_t seq = 0, s = 0;                     // slot items armed so far; slot of the next one
+      const uint32_t P = warp == kWarpCodes ? 0u : 1u;
+      uint32_t seq = 0, s = 0;                     // number and slot of the next slot item of the stream
       // Per-slot state, one bit per slot.  lk_dq / lk_mma: who hands the slot back (the dequantizer group
       // that read it, or the MMA issuers that read a 16-bit half).  ed_par / em_par: parity of the next
       // phase of empty_dq / empty_mma of the slot.
@@ -475,9 +482,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       bool ok = true;
       // the work list: unit blockIdx.x first, then whatever the global counter hands out
       int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
-      c->sched_unit[0] = u;
-      __threadfence_block();
-      c->sched_n = 1;
+      if (P == 0) {
+        c->sched_unit[0] = u;
+        __threadfence_block();
+        c->sched_n = 1;
+      }
       for (int i = 0; ok && u >= 0; ++i) {
         const Unit un = units[u];
         int claimed = 0;
@@ -502,31 +511,33 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 #pragma unroll 1
         for (int it = 0; ok && it < n_tiles; ++it) {
           // claim the next unit half-way through this one: the answer is back long before it is needed
-          if (it == claim_at) claimed = atomicAdd(work_counter, 1) + G;
+          if (P == 0 && it == claim_at) claimed = atomicAdd(work_counter, 1) + G;
           const bool f16 = cur.bits == 16;
           const uint32_t bytes = f16 ? 16384u : cur.tb;   // a 16-bit tile goes as two K-halves
           const int nsub = f16 ? 2 : 1;
           for (int sub = 0; sub < nsub; ++sub) {
-            const uint32_t bit = 1u << s;
-            if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
-            else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
-            if (!ok) break;
-            const uint32_t bar_s = full_s + 8 * s;
-            TRACE(0, seq);
-            mbar_expect_tx_s(bar_s, bytes);
-            bulk_g2s_s(wring_s + s * kSlotBytes, cur.src, bytes, bar_s);
-            if (f16) {
-              lk_mma |= bit;
-              lk_dq &= ~bit;
-              em_par ^= bit;
-            } else {
-              lk_dq |= bit;
-              lk_mma &= ~bit;
-              ed_par ^= bit;
+            if ((seq & 1u) == P) {
+              const uint32_t bit = 1u << s;
+              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
+              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
+              if (!ok) break;
+              const uint32_t bar_s = full_s + 8 * s;
+              if (P == 0) { TRACE(0, seq); }
+              mbar_expect_tx_s(bar_s, bytes);
+              bulk_g2s_s(wring_s + s * kSlotBytes, cur.src, bytes, bar_s);
+              if (f16) {
+                lk_mma |= bit;
+                lk_dq &= ~bit;
+                em_par ^= bit;
+              } else {
+                lk_dq |= bit;
+                lk_mma &= ~bit;
+                ed_par ^= bit;
+              }
+              c->issued[P] = seq + 2;                  // my next slot item is seq + 2
             }
             cur.src += bytes;
             ++seq;
-            c->issued = seq;
             if (++s == (uint32_t)n_slots) s = 0;
           }
           if (NMAT == 2) {
@@ -535,10 +546,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             oth = t;
           }
         }
-        u = claimed < n_units ? claimed : -1;
-        c->sched_unit[(i + 1) & 31] = u;
-        __threadfence_block();
-        c->sched_n = (uint32_t)i + 2;
+        if (P == 0) {
+          u = claimed < n_units ? claimed : -1;
+          c->sched_unit[(i + 1) & 31] = u;
+          __threadfence_block();
+          c->sched_n = (uint32_t)i + 2;
+        } else {
+          u = next_unit((uint32_t)i + 1, c, status);
+        }
       }
     }
   } else if (warp == kWarpTokens) {
@@ -723,7 +738,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         for (uint32_t j = j0; ok && j < ng; j += kStride) {
           const uint32_t use_par = uses & 1u;
           ++uses;
-          if (c->issued <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
+          if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
             publish();                               // do not sit on a finished half while waiting for HBM
             ok = wait_issued(sq, c, status) && mbar_wait<20>(&c->full[rp.s], rp.par, c, status);
             if (!ok) break;
@@ -917,9 +932,10 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const TcState* st = reinterpret_cast<const TcState*>(ctx->tc_state);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
   const int bslot_bytes = nt_tile * 256;
-  const int n_bslots = nt_tile <= 64 ? 4 : 2;
+  const int n_bslots = nt_tile <= 64 ? 3 : 2;
   int n_slots = (kMaxDynSmem - kCtrlBytes - n_bslots * bslot_bytes) / kSlotBytes;
   if (n_slots > kMaxSlots) n_slots = kMaxSlots;
+  n_slots &= ~1;                                   // even: the two weight producers own every other slot
   if (n_slots < 4) return PW_ERR_NOMEM;
   const int smem = kCtrlBytes + n_slots * kSlotBytes + n_bslots * bslot_bytes;
   const int R = T * k + c.n_shared * T;
