@@ -64,6 +64,7 @@ struct Ctrl {                                  // lives at the start of dynamic 
   // slots is even, so each producer also owns every other slot).  issued[p]: producer p has armed all of
   // its slot items below this number.
   volatile uint32_t issued[2];
+  volatile uint32_t b_issued;                  // token tiles armed so far (same purpose, for the token-tile slots)
   // Work list of this CTA: the weight producer claims units from a global counter and posts them here;
   // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
@@ -422,32 +423,32 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   const int n_units = n_units_ptr[PHASE];
   // tensor-memory columns: partial accumulators first ([matrix][partial][nt_tile]), dequantized-operand
   // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
-  constexpr int IPM = kIssuers / NMAT;           // issuers per matrix
+  constexpr int IPM = kIssuers / NMAT;           // issuers per matrix = dequantizer groups per matrix
   int npart = IPM;
   while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 32 > kTmemCols) npart >>= 1;
   const int n_issuers = NMAT * npart;            // active issuers
   const int acol = NMAT * npart * nt_tile;       // operand half-slot hs = 2 * group + K-half sits at acol + 32 * hs
-  const int per_half = npart >= 2 ? npart / 2 : 1;   // issuers per (matrix, K-half)
   const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(&c->full[i], 1);
       mbar_init(&c->empty_dq[i], 4);             // the four warps of the group that owns the item
-      mbar_init(&c->empty_mma[i], per_half);      // the issuers that read this K-half of a 16-bit tile
+      mbar_init(&c->empty_mma[i], 1);             // the issuer that read this K-half of a 16-bit tile
     }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
-      mbar_init(&c->b_empty[i], n_issuers);
+      mbar_init(&c->b_empty[i], NMAT);             // one issuer per matrix multiplies a token tile
     }
     for (int i = 0; i < kMaxASlots; ++i) {
       mbar_init(&c->a_full[i], 4);                // the four warps of the group that owns the half-slot
-      mbar_init(&c->a_empty[i], per_half);       // the issuers that read this K-half
+      mbar_init(&c->a_empty[i], 1);                // the issuer that serves the group
     }
     mbar_init(&c->d_full, n_issuers);
     mbar_init(&c->d_empty, 4);
     c->abort_flag = 0;
     c->issued[0] = c->issued[1] = 0;
+    c->b_issued = 0;
     c->sched_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -575,25 +576,24 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
           tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
           ++bcount;
+          c->b_issued = bcount;
         }
       }
     }
   }
   else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
     // ---------------- MMA issuers ----------------
-    // Issuer j of matrix m owns partial accumulator j.  With two or more issuers per matrix, each reads
-    // one K-half of every item (k-steps 4h .. 4h+3, strided over the issuers of that half), so it
-    // waits on one operand half-slot per item; a lone issuer walks both halves.
+    // Tile k of a matrix (counted over all units) belongs to issuer k mod npart of that matrix, which issues
+    // all eight k-steps of it into its own partial accumulator; a quantized tile k is dequantized by the
+    // matrix's group k mod IPM, so with npart == IPM every dequantizer group has an issuer of its own.
+    // The epilogue adds the partials.
     const int iss = warp - kWarpMma;
     const int my_m = iss / IPM, my_j = iss % IPM;
     if (lane == 0 && my_j < npart) {
-      const int my_h0 = npart >= 2 ? my_j / per_half : 0;
-      const int n_h = npart >= 2 ? 1 : 2;
-      const int my_p = npart >= 2 ? my_j % per_half : 0;
       uint32_t seq_unit = 0;                        // slot items before the current unit
-      uint32_t cnt = 0, ucount = 0;                 // cnt: quantized tiles of my matrix so far
-      int bs = 0;                                   // token-tile slot and its barrier parity, kept incrementally
-      uint32_t bpar = 0;
+      uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand half-slots
+      uint32_t ucount = 0;
       const uint32_t d_t = tmem + (my_m * npart + my_j) * nt_tile;
       const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
       const uint32_t b_lo_base = smem_u32(bslots) >> 4;
@@ -610,85 +610,95 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         // slot items per group of the unit (W) and the offset of my matrix's inside a group
         const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
         const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
+        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
         const int nb_rows = (un.ntok + 15) & ~15;
         const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
-        const uint32_t b_step = (uint32_t)(2 * nb_rows) * per_half;
+        const uint32_t b_step = (uint32_t)(2 * nb_rows);
         const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
-        // my first 16-bit slot item of the unit: K-half my_h0 of my matrix's tile of the first group
-        uint32_t sq = seq_unit + my_off + (uint32_t)my_h0;
+        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        uint32_t bt = base + j0;                     // token-tile number
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
         RingPos rp = ring_pos(sq, (uint32_t)n_slots);
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
         ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
         if (!ok) break;
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
         tc_fence_after();
-        uint32_t later = 0;                          // becomes 1 after the first group: accumulate onto earlier groups
-        for (int g = un.g0; ok && g < un.g1; ++g) {
-          if (my_m == 0 && my_j == 0) { TRACE(10, sq); }
-          ok = mbar_wait(&c->b_full[bs], bpar, c, status);
+        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
+#pragma unroll 1
+        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
+          if (my_m == 0 && my_j == 0) { TRACE(10, bt); }
+          // the token tile of this group (a tile is looked at only once it is known to have been armed)
+          if (c->b_issued <= bt) {
+            const unsigned long long t0 = globaltimer();
+            while (c->b_issued <= bt && !c->abort_flag) {
+              __nanosleep(32);
+              if (globaltimer() - t0 > kWaitLimitNs) {
+                c->abort_flag = 1;
+                atomicMax(status, (int)PW_ERR_TIMEOUT);
+              }
+            }
+            if (c->abort_flag) {
+              ok = false;
+              break;
+            }
+          }
+          ok = mbar_wait(&c->b_full[bp.s], bp.par, c, status);
           if (!ok) break;
-          if (my_m == 0 && my_j == 0) { TRACE(11, sq); }
-          const uint32_t b_lo = b_lo_unit + (uint32_t)bs * (uint32_t)(bslot_bytes >> 4);
+          if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
+          const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
           if (my_bits == 16) {
-            // the K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3 at 4 KB)
+            // each K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3, 4 KB apart)
             RingPos hp = rp;
-            for (int hh = 0; hh < n_h; ++hh) {
+#pragma unroll 1
+            for (uint32_t hh = 0; hh < 2; ++hh) {
               if (my_j == 0) { TRACE(12, sq + hh); }
-              ok = wait_issued(sq + (uint32_t)hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
+              ok = wait_issued(sq + hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
               if (my_j == 0) { TRACE(8, sq + hh); }
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
-              const uint32_t k0 = 4 * (my_h0 + hh) + my_p;
-              if (per_half == 1)
-                tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
-                                   later | (uint32_t)hh);
-              else
-                tc_mma_ss_burst<2>(d_t, a_lo + my_p * 256, desc_hi, 512, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc,
-                                   later);
+              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
               tc_commit(&c->empty_mma[hp.s]);
               if (my_j == 0) { TRACE(9, sq + hh); }
-              if (n_h == 2) ring_advance(hp, 1, (uint32_t)n_slots);
+              ring_advance(hp, 1, (uint32_t)n_slots);
             }
             if (!ok) break;
           } else {
             // the group that dequantizes this tile, and the parity of this use of its half-slots
-            const int grp = NMAT == 2 ? 2 * my_m + (int)(cnt & 1) : (int)(cnt & 3);
-            const uint32_t use_par = NMAT == 2 ? (cnt >> 1) & 1 : (cnt >> 2) & 1;
-            for (int hh = 0; hh < n_h; ++hh) {
-              const int h = my_h0 + hh;
-              const int hs = 2 * grp + h;
-              if (my_j == 0) { TRACE(12, sq); }
+            const uint32_t k = base + j;
+            const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
+            const uint32_t use_par = (upar >> grp) & 1u;
+            upar ^= 1u << grp;
+#pragma unroll 1
+            for (uint32_t hh = 0; hh < 2; ++hh) {
+              const uint32_t hs = 2 * grp + hh;
+              if (my_j == 0) { TRACE(12, sq + hh * 256); }
               ok = mbar_wait(&c->a_full[hs], use_par, c, status);
               if (!ok) break;
               tc_fence_after();
-              if (my_j == 0) { TRACE(8, sq); }
-              const uint32_t a_t = tmem + acol + hs * 32 + my_p * 8;
-              const uint32_t k0 = 4 * h + my_p;
-              if (per_half == 1)
-                tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later | (uint32_t)hh);
-              else
-                tc_mma_ts_burst<2>(d_t, a_t, 16, b_lo + k0 * (2 * nb_rows), desc_hi, b_step, idesc, later);
+              if (my_j == 0) { TRACE(8, sq + hh * 256); }
+              tc_mma_ts_burst<4>(d_t, tmem + acol + hs * 32, 8, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
               tc_commit(&c->a_empty[hs]);
+              if (my_j == 0) { TRACE(9, sq + hh * 256); }
             }
             if (!ok) break;
-            if (my_j == 0) { TRACE(9, sq); }
-            ++cnt;
           }
-          sq += W;
-          ring_advance(rp, W, (uint32_t)n_slots);
-          tc_commit(&c->b_empty[bs]);
+          tc_commit(&c->b_empty[bp.s]);
           later = 1;
-          if (++bs == n_bslots) {
-            bs = 0;
-            bpar ^= 1;
-          }
+          bt += (uint32_t)npart;
+          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
+          sq += (uint32_t)npart * W;
+          ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
         }
         if (ok) tc_commit(&c->d_full);
         TRACE(4, ucount * 4 + iss);
-        seq_unit += (uint32_t)(un.g1 - un.g0) * W;
+        base += ng;
+        seq_unit += ng * W;
       }
     }
   } else if (warp < kDqWarps) {
@@ -704,7 +714,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     const uint32_t gsub = NMAT == 2 ? (uint32_t)(grp & 1) : (uint32_t)grp;   // which of that matrix's groups
     constexpr uint32_t kStride = NMAT == 2 ? 2 : 4;  // groups per matrix = distance between my tiles
     uint32_t seq_unit = 0;                           // slot items before the current unit
-    uint32_t cntm = 0;                               // quantized tiles of my matrix so far
+    uint32_t base = 0;                               // tiles of one matrix before the current unit
     uint32_t uses = 0;                               // tiles I have taken so far (parity of my half-slots' use)
     int pending = -1;                                // operand half-slot whose store has not been published yet
     bool ok = true;
@@ -728,9 +738,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
       if (bits != 16) {                              // the MMA reads 16-bit tiles straight from shared memory
-        // Quantized tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my
-        // first one in this unit is group j0, then every kStride-th.
-        const uint32_t j0 = (gsub - cntm) & (kStride - 1);
+        // Tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my first one
+        // in this unit is group j0, then every kStride-th.
+        const uint32_t j0 = (gsub - base) & (kStride - 1);
         const uint32_t step = kStride * W;
         uint32_t sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
         RingPos rp = ring_pos(sq, (uint32_t)n_slots);
@@ -779,12 +789,15 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             pending = hs;
           }
           if (!ok) break;
-          if (j + kStride >= ng) publish();          // my last tile of the unit: the issuers are waiting to finish it
+          // The second half goes out at once: its half-slot is the one this group needs back soonest (for the
+          // second half of its next tile), and holding it over the next tile's first decode would delay that.
+          // The first half's store stays overlapped with the decode of the second.
+          publish();
           sq += step;
           ring_advance(rp, step, (uint32_t)n_slots);
         }
-        cntm += ng;
       }
+      base += ng;
       seq_unit += ng * W;
     }
     publish();
@@ -793,7 +806,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     const int q = warp & 3;
     const int r = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    uint32_t ucount = 0;
+    uint32_t ucount = 0, base = 0;                   // base: tiles of one matrix before the current unit
     bool ok = true;
     for (int i = 0; ok; ++i, ++ucount) {
       const int u = next_unit((uint32_t)i, c, status);
@@ -806,12 +819,19 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       tc_fence_after();
       const int nb_rows = (un.ntok + 15) & ~15;
       const int row = un.row_tile * kTileRows + r;
+      // partial accumulator p holds the tiles base + j with (base + j) mod npart == p: it has been written in
+      // this unit only if there is such a j below the unit's group count
+      const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+      uint32_t written = 0;
+      for (int p = 0; p < npart; ++p)
+        if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
+      base += ng;
       for (int c0 = 0; c0 < nb_rows; c0 += 16) {
         float a[16], b[16];
-        tmem_ld16(lane_addr + c0, a);
-        if (PHASE == 0) tmem_ld16(lane_addr + npart * nt_tile + c0, b);
-        tmem_wait_ld();
-        for (int p = 1; p < npart; ++p) {             // add the other issuers' partial sums, in order
+#pragma unroll
+        for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
+        for (int p = 0; p < npart; ++p) {              // add the issuers' partial sums, in order
+          if (!((written >> p) & 1u)) continue;
           float t[16];
           tmem_ld16(lane_addr + p * nt_tile + c0, t);
           tmem_wait_ld();
@@ -829,7 +849,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           const int nn = c0 + j;
           if (nn < un.ntok) {
             if (PHASE == 0) {
-              const float hval = __fmul_rn(__fdiv_rn(a[j], __fadd_rn(1.0f, expf(-a[j]))), b[j]);
+              // SwiGLU: silu(gate) * up; the result is rounded to fp16, so the fast exponential and
+              // division (relative error ~1e-6) change nothing that survives the rounding
+              const float hval = __fmul_rn(__fdividef(a[j], __fadd_rn(1.0f, __expf(-a[j]))), b[j]);
               ht[((size_t)(row >> 3) * Rpad + un.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
             } else {
               y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + nn) * H + row] = a[j];
