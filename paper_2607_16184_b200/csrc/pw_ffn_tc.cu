@@ -57,7 +57,7 @@ struct Ctrl {                                  // lives at the start of dynamic 
   unsigned long long full[kMaxSlots], empty_dq[kMaxSlots], empty_mma[kMaxSlots];
   unsigned long long b_full[kMaxBSlots], b_empty[kMaxBSlots];
   unsigned long long a_full[kMaxASlots], a_empty[kMaxASlots];
-  unsigned long long d_full, d_empty;
+  unsigned long long d_full[2], d_empty[2];     // two accumulator buffers (a wide token tile takes both)
   uint32_t tmem_base;
   volatile int abort_flag;
   // Slot items with an even number are armed by weight producer 0, odd ones by producer 1 (the number of
@@ -444,8 +444,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       mbar_init(&c->a_full[i], 4);                // the four warps of the group that owns the half-slot
       mbar_init(&c->a_empty[i], 1);                // the issuer that serves the group
     }
-    mbar_init(&c->d_full, n_issuers);
-    mbar_init(&c->d_empty, 4);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&c->d_full[i], n_issuers);
+      mbar_init(&c->d_empty[i], 4);
+    }
     c->abort_flag = 0;
     c->issued[0] = c->issued[1] = 0;
     c->b_issued = 0;
@@ -594,7 +596,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
       uint32_t upar = 0;                            // per group: parity of the next use of its operand half-slots
       uint32_t ucount = 0;
-      const uint32_t d_t = tmem + (my_m * npart + my_j) * nt_tile;
+      // Accumulators: partial (m, j) of a unit sits at buffer base + (m * npart + j) * nb_rows.  A unit whose
+      // accumulators fit half of the accumulator columns takes one of two buffers in turn, so that its MMAs
+      // overlap the epilogue of the unit before it; a wider unit takes both.
+      uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
       const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
       const uint32_t b_lo_base = smem_u32(bslots) >> 4;
       const uint32_t w_lo_base = smem_u32(wring) >> 4;
@@ -623,8 +628,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
         RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const uint32_t dbuf = wide ? 0u : dtoggle;
+        if (!wide) dtoggle ^= 1u;
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
-        ok = mbar_wait<32>(&c->d_empty, (ucount & 1) ^ 1, c, status);   // epilogue has drained the accumulators
+        // the epilogue has drained the buffer(s) this unit accumulates into
+        if (wide || dbuf == 0) ok = mbar_wait<32>(&c->d_empty[0], (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait<32>(&c->d_empty[1], (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
         tc_fence_after();
@@ -695,7 +706,16 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           sq += (uint32_t)npart * W;
           ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
         }
-        if (ok) tc_commit(&c->d_full);
+        if (ok) {
+          if (wide || dbuf == 0) {
+            tc_commit(&c->d_full[0]);
+            ++duse0;
+          }
+          if (wide || dbuf == 1) {
+            tc_commit(&c->d_full[1]);
+            ++duse1;
+          }
+        }
         TRACE(4, ucount * 4 + iss);
         base += ng;
         seq_unit += ng * W;
@@ -807,18 +827,24 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     const int r = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     uint32_t ucount = 0, base = 0;                   // base: tiles of one matrix before the current unit
+    uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;      // accumulator buffers: the issuers' rule, replayed
     bool ok = true;
     for (int i = 0; ok; ++i, ++ucount) {
       const int u = next_unit((uint32_t)i, c, status);
       if (u < 0) break;
       const Unit un = units[u];
-      ok = mbar_wait<200>(&c->d_full, ucount & 1, c, status);
+      const int nb_rows = (un.ntok + 15) & ~15;
+      const bool wide = NMAT * npart * nb_rows > acol / 2;
+      const uint32_t dbuf = wide ? 0u : dtoggle;
+      if (!wide) dtoggle ^= 1u;
+      if (wide || dbuf == 0) ok = mbar_wait<200>(&c->d_full[0], duse0 & 1, c, status);
+      if (ok && (wide || dbuf == 1)) ok = mbar_wait<200>(&c->d_full[1], duse1 & 1, c, status);
       if (!ok) break;
       if (q == 0) { TRACE(13, ucount); }
       if (q == 0) { TRACEV(7, ucount, rows[un.seg * 3].bits * 100 + rows[un.seg * 3 + 1].bits + 10000 * un.ntok); }
       tc_fence_after();
-      const int nb_rows = (un.ntok + 15) & ~15;
       const int row = un.row_tile * kTileRows + r;
+      const uint32_t dbase = lane_addr + dbuf * (uint32_t)(acol / 2);
       // partial accumulator p holds the tiles base + j with (base + j) mod npart == p: it has been written in
       // this unit only if there is such a j below the unit's group count
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
@@ -833,12 +859,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         for (int p = 0; p < npart; ++p) {              // add the issuers' partial sums, in order
           if (!((written >> p) & 1u)) continue;
           float t[16];
-          tmem_ld16(lane_addr + p * nt_tile + c0, t);
+          tmem_ld16(dbase + p * nb_rows + c0, t);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
           if (PHASE == 0) {
-            tmem_ld16(lane_addr + (npart + p) * nt_tile + c0, t);
+            tmem_ld16(dbase + (npart + p) * nb_rows + c0, t);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
@@ -862,7 +888,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       tc_fence_before();
       __syncwarp();
       if (q == 0) { TRACE(14, ucount); }
-      if (lane == 0) mbar_arrive(&c->d_empty);
+      if (lane == 0) {
+        if (wide || dbuf == 0) mbar_arrive(&c->d_empty[0]);
+        if (wide || dbuf == 1) mbar_arrive(&c->d_empty[1]);
+      }
+      if (wide || dbuf == 0) ++duse0;
+      if (wide || dbuf == 1) ++duse1;
     }
   }
 
