@@ -41,7 +41,7 @@ namespace pw {
 constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item (16 KB codes + 512 B) fits
 constexpr int kMaxSlots = 16;
 constexpr int kMaxASlots = 8;                  // operand half-slots in tensor memory (32 columns = 64 K each)
-constexpr int kMaxBSlots = 4;
+constexpr int kMaxBSlots = 5;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
 constexpr int kDqWarps = 16;
@@ -985,24 +985,34 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const TcState* st = reinterpret_cast<const TcState*>(ctx->tc_state);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
   const int bslot_bytes = nt_tile * 256;
-  const int n_bslots = nt_tile <= 64 ? 3 : 2;
-  int n_slots = (kMaxDynSmem - kCtrlBytes - n_bslots * bslot_bytes) / kSlotBytes;
-  if (n_slots > kMaxSlots) n_slots = kMaxSlots;
-  n_slots &= ~1;                                   // even: the two weight producers own every other slot
-  if (n_slots < 4) return PW_ERR_NOMEM;
-  const int smem = kCtrlBytes + n_slots * kSlotBytes + n_bslots * bslot_bytes;
+  // Shared-memory plan per kernel.  The issuers of a matrix work on as many token tiles at once as there are
+  // partial accumulators per matrix (the kernel's own rule, repeated here); one more slot keeps a tile on its
+  // way.  The rest of the 227 KB goes to the weight ring (an even number of slots, one set per producer).
+  int n_bslots[2], n_slots[2], smem[2];
+  for (int phase = 0; phase < 2; ++phase) {
+    const int nmat = phase == 0 ? 2 : 1;
+    int npart = kIssuers / nmat;
+    while (npart > 1 && nmat * npart * nt_tile + kMaxASlots * 32 > kTmemCols) npart >>= 1;
+    n_bslots[phase] = npart + 1 > kMaxBSlots ? kMaxBSlots : npart + 1;
+    int ns = (kMaxDynSmem - kCtrlBytes - n_bslots[phase] * bslot_bytes) / kSlotBytes;
+    if (ns > kMaxSlots) ns = kMaxSlots;
+    ns &= ~1;
+    if (ns < 4) return PW_ERR_NOMEM;
+    n_slots[phase] = ns;
+    smem[phase] = kCtrlBytes + ns * kSlotBytes + n_bslots[phase] * bslot_bytes;
+  }
   const int R = T * k + c.n_shared * T;
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
-  ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
-                                                        st->xt, w.Rpad, nt_tile, n_bslots, n_slots,
+  ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem[0], s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
+                                                        st->xt, w.Rpad, nt_tile, n_bslots[0], n_slots[0],
                                                         reinterpret_cast<__half*>(b + w.ht), nullptr, c.hidden, 0,
                                                         work_counter, status);
   timing_mark(ctx, PW_K_FFN_DOWN, s);
-  ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem, s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
-                                                        st->ht, w.Rpad, nt_tile, n_bslots, n_slots, nullptr,
+  ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem[1], s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
+                                                        st->ht, w.Rpad, nt_tile, n_bslots[1], n_slots[1], nullptr,
                                                         reinterpret_cast<float*>(b + w.y), c.hidden,
                                                         (size_t)R * c.hidden, work_counter + 1, status);
   ctx->launches += 2;
