@@ -58,6 +58,13 @@ __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ l
   }
 }
 
+#ifdef PW_TC_PROFILE
+__device__ long long g_ptrace[32];
+#define PSTAMP(i) if (threadIdx.x == 0) g_ptrace[i] = clock64()
+#else
+#define PSTAMP(i)
+#endif
+
 // Single CTA.  Stable counting sort of the P = T*k pairs by expert (positions come from ordered
 // prefix counts, never from atomics), segment table including the shared experts, operand-row ->
 // token map, and the unit lists of the tensor-core kernels.
@@ -82,12 +89,14 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = T * k;
 
+  PSTAMP(0);
   for (int e = tid; e < S; e += blockDim.x) cnt[e] = e < E ? 0 : T;
   for (int e = tid; e < E; e += blockDim.x) run[e] = 0;
   if (tid < 64) counter[tid] = 0;
   __syncthreads();
   for (int p = tid; p < P; p += blockDim.x) atomicAdd(&cnt[topk_ids[p]], 1);
   __syncthreads();
+  PSTAMP(1);
   if (tid == 0) {
     int a = 0;
     for (int e = 0; e < S; ++e) {
@@ -99,6 +108,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
   __syncthreads();
   for (int e = tid; e < S; e += blockDim.x) counts[e] = cnt[e];
   for (int e = tid; e <= S; e += blockDim.x) offsets[e] = off[e];
+  PSTAMP(2);
 
   for (int base = 0; base < P; base += blockDim.x) {
     for (int i = tid; i < 32 * E; i += blockDim.x) wcnt[i] = 0;
@@ -127,11 +137,13 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
     }
     __syncthreads();
   }
+  PSTAMP(3);
   const int R = off[S];
   for (int i = tid; i < n_shared * T; i += blockDim.x) row_token[P + i] = i % T;
   for (int i = tid; i < kPadRows; i += blockDim.x) row_token[R + i] = -1;
 
   if (nt_tile <= 0) return;  // SIMT path: no unit lists
+  PSTAMP(4);
 
   // Unit lists.  The CTAs of the FFN kernels claim units in list order, so the list is laid out for that:
   // row tile outermost, K split next, then every segment's token tiles (segments with the widest pages
@@ -150,6 +162,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
       order[rk] = s;
     }
     __syncthreads();
+    PSTAMP(5 + 4 * phase);
     const int row_tiles = (phase == 0 ? F : H) / kTileRows;
     const int ng = (phase == 0 ? H : F) / kGroup;
     const int splits = phase == 0 ? 1 : ksplit;
@@ -165,35 +178,67 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
       if (total > max_units) atomicMax(status, (int)PW_ERR_NOMEM);
     }
     __syncthreads();
+    PSTAMP(6 + 4 * phase);
     const int TT = ubase[S];
     if ((long long)TT * row_tiles * splits > max_units) continue;
     Unit* out = phase == 0 ? units_gu : units_dn;
     if (phase == 0)
       for (int i = tid; i < S; i += blockDim.x) seg_order[i] = order[i];
-    for (int i = 0; i < S; ++i) {
-      const int s = order[i];
-      const int n = cnt[s];
-      const int tt = (n + nt_tile - 1) / nt_tile;
-      const int total = tt * row_tiles * splits;
-      for (int u = tid; u < total; u += blockDim.x) {
-        const int ti = u % tt;
-        const int rs = u / tt;                       // row tile * splits + split
-        const int sp = rs % splits;
-        const int rt = rs / splits;
+    // token tile j of the list -> rank of its segment (the sort's scratch is free by now; a layer with more
+    // token tiles than fit there searches the prefix instead), and the group range of every K split
+    int32_t* tseg = wcnt;
+    const bool use_table = TT + splits + 1 <= 32 * E;
+    int32_t* gtab = wcnt + (use_table ? TT : 0);     // [splits + 1] when it fits
+    if (use_table) {
+      for (int i = tid; i < S; i += blockDim.x)
+        for (int j = ubase[i]; j < ubase[i + 1]; ++j) tseg[j] = i;
+      for (int sp = tid; sp <= splits; sp += blockDim.x) gtab[sp] = (sp * ng) / splits;
+    }
+    __syncthreads();
+    // warp w writes the units of (row tile, split) pairs w, w + 32, ..; its lanes walk the token tiles: no
+    // per-unit division, consecutive lanes write consecutive units
+    const int n_rs = row_tiles * splits;
+    for (int rs = warp; rs < n_rs; rs += 32) {
+      int sp = 0, rt = rs;
+      if (splits > 1) {
+        rt = rs / splits;
+        sp = rs - rt * splits;
+      }
+      const int g0 = use_table ? gtab[sp] : (sp * ng) / splits;
+      const int g1 = use_table ? gtab[sp + 1] : ((sp + 1) * ng) / splits;
+      for (int j = lane; j < TT; j += 32) {
+        int i;
+        if (use_table) {
+          i = tseg[j];
+        } else {
+          i = 0;
+          while (ubase[i + 1] <= j) ++i;
+        }
+        const int s = order[i];
+        const int n = cnt[s];
+        const int ti = j - ubase[i];
         Unit un;
         un.seg = s;
         un.row_tile = rt;
         un.tok0 = off[s] + ti * nt_tile;
         un.ntok = min(nt_tile, n - ti * nt_tile);
-        un.g0 = (int)(((long long)sp * ng) / splits);
-        un.g1 = (int)(((long long)(sp + 1) * ng) / splits);
+        un.g0 = g0;
+        un.g1 = g1;
         un.split = sp;
         un.pad_ = 0;
-        out[(size_t)rs * TT + ubase[i] + ti] = un;
+        out[(size_t)rs * TT + j] = un;
       }
     }
+    PSTAMP(7 + 4 * phase);
   }
 }
+#ifdef PW_TC_PROFILE
+extern "C" int pw_debug_read_ptrace(long long* out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, g_ptrace, sizeof(g_ptrace));
+  return 0;
+}
+#endif
 
 // Xt[c][n][0..7] = hidden[row_token[n]][8c .. 8c+7], zero for padding rows.
 __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
