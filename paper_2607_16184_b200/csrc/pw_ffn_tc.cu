@@ -494,59 +494,54 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         const Unit un = units[u];
         int claimed = 0;
         // per matrix of the unit: bitwidth, bytes of a tile image, address of the unit's first tile;
-        // consecutive groups of a row tile are consecutive tiles of the page.  Tiles alternate between the
-        // matrices, so the state of the matrix whose turn it is sits in `cur` and the two swap after every
-        // tile (one copy of the issue code instead of one per matrix).
-        MatSrc cur, oth;
+        // consecutive groups of a row tile are consecutive tiles of the page
+        MatSrc ms[NMAT];
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
           const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
-          MatSrc t;
-          t.bits = row.bits;
-          t.tb = (uint32_t)tile_bytes((int)row.bits);
+          ms[m].bits = row.bits;
+          ms[m].tb = (uint32_t)tile_bytes((int)row.bits);
           const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + un.g0;
-          t.src = reinterpret_cast<const char*>(row.codes) + tile * t.tb;
-          if (m == 0) cur = t;
-          else oth = t;
+          ms[m].src = reinterpret_cast<const char*>(row.codes) + tile * ms[m].tb;
         }
-        const int n_tiles = (un.g1 - un.g0) * NMAT;
-        const int claim_at = n_tiles >> 1;
+        const int ng = un.g1 - un.g0;
+        const int claim_at = ng >> 1;
 #pragma unroll 1
-        for (int it = 0; ok && it < n_tiles; ++it) {
+        for (int g = 0; ok && g < ng; ++g) {
           // claim the next unit half-way through this one: the answer is back long before it is needed
-          if (P == 0 && it == claim_at) claimed = atomicAdd(work_counter, 1) + G;
-          const bool f16 = cur.bits == 16;
-          const uint32_t bytes = f16 ? 16384u : cur.tb;   // a 16-bit tile goes as two K-halves
-          const int nsub = f16 ? 2 : 1;
-          for (int sub = 0; sub < nsub; ++sub) {
-            if ((seq & 1u) == P) {
-              const uint32_t bit = 1u << s;
-              if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
-              else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
-              if (!ok) break;
-              const uint32_t bar_s = full_s + 8 * s;
-              if (P == 0) { TRACE(0, seq); }
-              mbar_expect_tx_s(bar_s, bytes);
-              bulk_g2s_s(wring_s + s * kSlotBytes, cur.src, bytes, bar_s);
-              if (f16) {
-                lk_mma |= bit;
-                lk_dq &= ~bit;
-                em_par ^= bit;
-              } else {
-                lk_dq |= bit;
-                lk_mma &= ~bit;
-                ed_par ^= bit;
+          if (P == 0 && g == claim_at) claimed = atomicAdd(work_counter, 1) + G;
+#pragma unroll
+          for (int m = 0; m < NMAT; ++m) {
+            const bool f16 = ms[m].bits == 16;
+            const uint32_t bytes = f16 ? 16384u : ms[m].tb;   // a 16-bit tile goes as two K-halves
+            const int nsub = f16 ? 2 : 1;
+            const char* src = ms[m].src;
+            ms[m].src += ms[m].tb;
+            for (int sub = 0; sub < nsub; ++sub, src += 16384) {
+              if ((seq & 1u) == P) {
+                const uint32_t bit = 1u << s;
+                if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
+                else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
+                if (!ok) break;
+                const uint32_t bar_s = full_s + 8 * s;
+                if (P == 0) { TRACE(0, seq); }
+                mbar_expect_tx_s(bar_s, bytes);
+                bulk_g2s_s(wring_s + s * kSlotBytes, src, bytes, bar_s);
+                if (f16) {
+                  lk_mma |= bit;
+                  lk_dq &= ~bit;
+                  em_par ^= bit;
+                } else {
+                  lk_dq |= bit;
+                  lk_mma &= ~bit;
+                  ed_par ^= bit;
+                }
+                c->issued[P] = seq + 2;                // my next slot item is seq + 2
               }
-              c->issued[P] = seq + 2;                  // my next slot item is seq + 2
+              ++seq;
+              if (++s == (uint32_t)n_slots) s = 0;
             }
-            cur.src += bytes;
-            ++seq;
-            if (++s == (uint32_t)n_slots) s = 0;
-          }
-          if (NMAT == 2) {
-            const MatSrc t = cur;
-            cur = oth;
-            oth = t;
+            if (!ok) break;
           }
         }
         if (P == 0) {
