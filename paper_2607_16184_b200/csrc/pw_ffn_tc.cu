@@ -52,9 +52,10 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct Ctrl {                                  // lives at the start of dynamic shared memory
   // One full barrier per ring slot (armed by the weight producer).  A slot is handed back either by the
-  // four warps of the dequantizer group that read it (empty_dq) or by the MMA issuers of its matrix
-  // (empty_mma, through tcgen05.commit); the weight producer remembers which.
-  unsigned long long full[kMaxSlots], empty_dq[kMaxSlots], empty_mma[kMaxSlots];
+  // four warps of the dequantizer group that read it, or by the MMA issuer that read a 16-bit half from it
+  // (one tcgen05.commit plus three plain arrivals, so that both kinds complete the same four-arrival phase
+  // and the weight producers need not remember who holds a slot).
+  unsigned long long full[kMaxSlots], empty[kMaxSlots];
   unsigned long long b_full[kMaxBSlots], b_empty[kMaxBSlots];
   unsigned long long a_full[kMaxASlots], a_empty[kMaxASlots];
   unsigned long long d_full[2], d_empty[2];     // two accumulator buffers (a wide token tile takes both)
@@ -97,6 +98,9 @@ __device__ __forceinline__ void mbar_init(unsigned long long* b, uint32_t count)
 }
 __device__ __forceinline__ void mbar_arrive(unsigned long long* b) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(unsigned long long* b, uint32_t n) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(n) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(unsigned long long* b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
@@ -433,8 +437,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(&c->full[i], 1);
-      mbar_init(&c->empty_dq[i], 4);             // the four warps of the group that owns the item
-      mbar_init(&c->empty_mma[i], 1);             // the issuer that read this K-half of a 16-bit tile
+      mbar_init(&c->empty[i], 4);                 // four dequantizer warps, or an issuer's commit + 3 arrivals
     }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
@@ -477,10 +480,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     if (lane == 0) {
       const uint32_t P = warp == kWarpCodes ? 0u : 1u;
       uint32_t seq = 0, s = 0;                     // number and slot of the next slot item of the stream
-      // Per-slot state, one bit per slot.  lk_dq / lk_mma: who hands the slot back (the dequantizer group
-      // that read it, or the MMA issuers that read a 16-bit half).  ed_par / em_par: parity of the next
-      // phase of empty_dq / empty_mma of the slot.
-      uint32_t lk_dq = 0, lk_mma = 0, ed_par = 0, em_par = 0;
+      // A slot is free for slot item seq once the phase seq / n_slots - 1 of its empty barrier has completed
+      // (nothing to wait for during the first pass over the ring).
+      uint32_t pass = 0;                           // seq / n_slots
       const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]);
       bool ok = true;
       // the work list: unit blockIdx.x first, then whatever the global counter hands out
@@ -519,27 +521,19 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             ms[m].src += ms[m].tb;
             for (int sub = 0; sub < nsub; ++sub, src += 16384) {
               if ((seq & 1u) == P) {
-                const uint32_t bit = 1u << s;
-                if (lk_dq & bit) ok = mbar_wait<32>(&c->empty_dq[s], ((ed_par >> s) & 1) ^ 1, c, status);
-                else if (lk_mma & bit) ok = mbar_wait<32>(&c->empty_mma[s], ((em_par >> s) & 1) ^ 1, c, status);
+                if (pass) ok = mbar_wait<32>(&c->empty[s], (pass - 1) & 1, c, status);
                 if (!ok) break;
                 const uint32_t bar_s = full_s + 8 * s;
                 if (P == 0) { TRACE(0, seq); }
                 mbar_expect_tx_s(bar_s, bytes);
                 bulk_g2s_s(wring_s + s * kSlotBytes, src, bytes, bar_s);
-                if (f16) {
-                  lk_mma |= bit;
-                  lk_dq &= ~bit;
-                  em_par ^= bit;
-                } else {
-                  lk_dq |= bit;
-                  lk_mma &= ~bit;
-                  ed_par ^= bit;
-                }
                 c->issued[P] = seq + 2;                // my next slot item is seq + 2
               }
               ++seq;
-              if (++s == (uint32_t)n_slots) s = 0;
+              if (++s == (uint32_t)n_slots) {
+                s = 0;
+                ++pass;
+              }
             }
             if (!ok) break;
           }
@@ -669,7 +663,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               if (my_j == 0) { TRACE(8, sq + hh); }
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
               tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
-              tc_commit(&c->empty_mma[hp.s]);
+              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
+              tc_commit(&c->empty[hp.s]);
               if (my_j == 0) { TRACE(9, sq + hh); }
               ring_advance(hp, 1, (uint32_t)n_slots);
             }
@@ -792,7 +787,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             if (q == 0) { TRACE(2 + 3 * h, sq); }
             if (h == 1) {
               __syncwarp();
-              if (lane == 0) mbar_arrive(&c->empty_dq[rp.s]);   // this warp has read its rows of the tile
+              if (lane == 0) mbar_arrive(&c->empty[rp.s]);   // this warp has read its rows of the tile
             }
             publish();                               // the previous half's store, overlapped with the decode above
             const int hs = 2 * grp + h;
