@@ -154,9 +154,9 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_s, uint32_t parity, uin
 // the loop).  After kFastPolls wake-ups it falls into the bounded out-of-line loop above.
 constexpr uint32_t kFastPolls = 64;
 constexpr uint32_t kSuspendHintNs = 20000;
+// (the barrier is given by its shared-memory address: the control loops keep those in registers)
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
-  const uint32_t bar_s = smem_u32(b);
+__device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, Ctrl* c, int32_t* status) {
   uint32_t ok, polls;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
@@ -177,6 +177,10 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity
 #endif
   if (ok) return true;
   return mbar_wait_slow(bar_s, parity, SLEEP_NS, c, status);
+}
+template <int SLEEP_NS = 0>
+__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
+  return mbar_wait_s<SLEEP_NS>(smem_u32(b), parity, c, status);
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -205,6 +209,9 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(unsigned long long* b) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(b))
                : "memory");
+}
+__device__ __forceinline__ void tc_commit_s(uint32_t bar_s) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_s) : "memory");
 }
 // A operand in tensor memory
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
@@ -592,6 +599,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
       const uint32_t b_lo_base = smem_u32(bslots) >> 4;
       const uint32_t w_lo_base = smem_u32(wring) >> 4;
+      const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
+      const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
+      const uint32_t a_base = tmem + acol;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = next_unit((uint32_t)i, c, status);
@@ -647,7 +657,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               break;
             }
           }
-          ok = mbar_wait(&c->b_full[bp.s], bp.par, c, status);
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
@@ -669,32 +679,34 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               ring_advance(hp, 1, (uint32_t)n_slots);
             }
             if (!ok) break;
+            sq += (uint32_t)npart * W;
+            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
           } else {
             // the group that dequantizes this tile, and the parity of this use of its half-slots
             const uint32_t k = base + j;
             const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
             const uint32_t use_par = (upar >> grp) & 1u;
             upar ^= 1u << grp;
-#pragma unroll 1
-            for (uint32_t hh = 0; hh < 2; ++hh) {
-              const uint32_t hs = 2 * grp + hh;
-              if (my_j == 0) { TRACE(12, sq + hh * 256); }
-              ok = mbar_wait(&c->a_full[hs], use_par, c, status);
-              if (!ok) break;
-              tc_fence_after();
-              if (my_j == 0) { TRACE(8, sq + hh * 256); }
-              tc_mma_ts_burst<4>(d_t, tmem + acol + hs * 32, 8, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
-              tc_commit(&c->a_empty[hs]);
-              if (my_j == 0) { TRACE(9, sq + hh * 256); }
-            }
+            const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
+            const uint32_t a_t = a_base + grp * 64;
+            if (my_j == 0) { TRACE(12, k); }
+            ok = mbar_wait_s(f0, use_par, c, status);
             if (!ok) break;
+            tc_fence_after();
+            if (my_j == 0) { TRACE(8, k); }
+            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_commit_s(e0);
+            if (my_j == 0) { TRACE(9, k); }
+            ok = mbar_wait_s(f0 + 8, use_par, c, status);
+            if (!ok) break;
+            tc_fence_after();
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            tc_commit_s(e0 + 8);
           }
-          tc_commit(&c->b_empty[bp.s]);
+          tc_commit_s(be_s + 8 * bp.s);
           later = 1;
           bt += (uint32_t)npart;
           ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
-          sq += (uint32_t)npart * W;
-          ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
         }
         if (ok) {
           if (wide || dbuf == 0) {
