@@ -780,16 +780,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 #pragma unroll 1
           for (int h = 0; h < 2; ++h) {
             __half2 w[32];
-#ifdef PW_EXP_NODECODE
-            {
-              const uint4 t = reinterpret_cast<const uint4*>(item)[r + h * 128];
-#pragma unroll
-              for (int jj = 0; jj < 32; jj += 4) {
-                w[jj] = u32_as_h2(t.x); w[jj + 1] = u32_as_h2(t.y); w[jj + 2] = u32_as_h2(t.z); w[jj + 3] = u32_as_h2(t.w);
-              }
-            }
-            if (false)
-#endif
             switch (bits) {
               case 8: decode_item_half<8>(item, r, h, w); break;
               case 4: decode_item_half<4>(item, r, h, w); break;

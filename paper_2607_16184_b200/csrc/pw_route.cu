@@ -240,14 +240,14 @@ extern "C" int pw_debug_read_ptrace(long long* out) {
 }
 #endif
 
-// Xt[c][n][0..7] = hidden[row_token[n]][8c .. 8c+7], zero for padding rows.
+// Xt[c][n][0..7] = hidden[row_token[n]][8c .. 8c+7] for the operand rows n < R.  Rows past R only ever feed
+// accumulator columns that nobody reads, so they keep whatever they hold.
 __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
                                                      const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
                                                      uint4* __restrict__ xt) {
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   const int c = blockIdx.y;
-  const int R = offsets[S];
-  if (n >= R + kPadRows) return;
+  if (n >= offsets[S]) return;
   const int t = row_token[n];
   uint4 v = make_uint4(0, 0, 0, 0);
   if (t >= 0) v = __ldg(hidden + (size_t)t * H8 + c);
@@ -310,7 +310,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
       reinterpret_cast<int32_t*>(b + w.status));
   const int R = T * k + c.n_shared * T;
   timing_mark(ctx, PW_K_GATHER, s);
-  dim3 grid((R + kPadRows + 255) / 256, c.hidden / 8);
+  dim3 grid((R + 255) / 256, c.hidden / 8);
   gather_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(hidden),
                                      reinterpret_cast<const int32_t*>(b + w.row_token),
                                      reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
