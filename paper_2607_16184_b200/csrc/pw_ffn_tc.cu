@@ -2,33 +2,35 @@
 //
 //   D[128 weight rows, N tokens] += W[128, 16] * X[N, 16]^T      (tcgen05.mma, kind::f16, fp32 in TMEM)
 //
-// Weight pages stream HBM -> shared memory with bulk async copies, one item (128 rows x one group of
-// one page, 4.5 .. 32 KB) at a time, into a ring of 17 KB slots (a 16-bit item takes two).  A 16-bit
-// tile is already in the tensor core's K-major core-matrix layout, so the MMA reads it from shared
-// memory as the A operand without any thread touching it.  A quantized tile is unpacked and
-// dequantized in registers (one weight row per thread) and written to tensor memory, which the MMA
-// then reads as its A operand.  The token tile (B operand) comes from the k-chunk-major operand
-// buffers with one 2-D TMA copy per group.
+// Weight pages stream HBM -> shared memory with bulk async copies into a ring of 17 KB slots.  A "slot item"
+// is one tile image of a quantized page (128 rows x one group: codes, scales, zero-points, 4.5 .. 16.5 KB,
+// one copy) or one K-half (16 KB) of a 16-bit tile; slot item number seq lives in slot seq mod n_slots, so
+// every role finds its own items from their numbers alone.  A 16-bit half is already in the tensor core's
+// K-major core-matrix layout: the MMA reads it from shared memory as the A operand without any thread
+// touching it.  A quantized tile is unpacked and dequantized in registers (one weight row per thread) and
+// written to tensor memory, which the MMA then reads as its A operand.  The token tile (B operand) comes
+// from the k-chunk-major operand buffers with one 2-D TMA copy per group.
 //
 // One persistent CTA per SM, 27 warps.  The control roles are single threads with short dependent
 // instruction chains: they share the schedulers with the arithmetic-heavy dequantizers, and every
-// instruction of theirs waits its turn.
-//   warps 0-15   dequantize: four groups of four warps, group j takes the quantized items j, j+4, ..;
-//                warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
-//   warp 16      weight producer: arms an item's barrier and copies its codes, scales and zero-points,
-//                as far ahead as the slot ring allows;
+// instruction of theirs waits its turn, so each of them does as little per item as possible.
+//   warps 0-15   dequantize: four groups of four warps; tile k of a matrix goes to that matrix's group
+//                k mod (groups per matrix); warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
+//                a group has two operand half-slots in tensor memory (K 0..63 / 64..127 of its tile);
+//   warps 16,18  weight producers: producer P arms the slot items with number = P mod 2 (which sit in the
+//                slots = P mod 2) and issues their copies, as far ahead as the ring allows; producer 0 also
+//                claims the CTA's units from a global counter and posts them on the CTA's work list;
 //   warp 17      token-tile producer (its own few slots, never holds back the weight stream);
-//   warp 18      idle;
 //   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  A tcgen05.mma holds its issuing
-//                thread for ~95 cycles whatever its size, so one issuer caps the SM at one 128x16
-//                weight slab per 95 cycles; four issuers in four warps overlap.  Each issuer owns the
-//                K-steps k = j mod (issuers per matrix) of one matrix and its own partial accumulator,
-//                so no two threads ever accumulate into the same columns; the epilogue adds the partials;
-//   warps 23-26  epilogue: SwiGLU -> fp16 operand of the down projection (PHASE 0), or the fp32
-//                split-K partial of the down projection (PHASE 1).
-// Units are dealt to CTAs in snake order over a size-sorted list.  Every wait is bounded; when one
-// runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
-// memory and returns.
+//                thread for ~100 cycles whatever its size, so the issuers work in parallel: issuer j of a
+//                matrix issues all eight k-steps of the tiles k = j mod (issuers per matrix) into its own
+//                partial accumulator -- with as many issuers as groups, each dequantizer group has an
+//                issuer of its own -- and no two threads ever accumulate into the same columns;
+//   warps 23-26  epilogue: adds the partials; SwiGLU -> fp16 operand of the down projection (PHASE 0), or the
+//                fp32 split-K partial of the down projection (PHASE 1).  Narrow token tiles alternate
+//                between two accumulator buffers, so the next unit's MMAs overlap the epilogue.
+// Every wait is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing
+// work, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include <new>
