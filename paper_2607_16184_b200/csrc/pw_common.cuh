@@ -124,4 +124,34 @@ void tc_teardown(pw_ctx* ctx);
 // records timing event `i` of the current forward call (no-op unless timing is enabled)
 void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 
+
+// ---- programmatic dependent launch -------------------------------------------------------------
+// The kernels of one forward call run back to back on one stream.  Each is launched with programmatic
+// stream serialization: its CTAs may be placed on an SM, and start, while the kernel before it is still
+// finishing elsewhere.  grid_dep_sync() returns once the kernel before this one has completed and its writes
+// are visible; a thread calls it before it reads anything that kernel wrote.  grid_dep_trigger() lets the
+// kernel after this one be placed as soon as SMs free up; a kernel calls it only after its own
+// grid_dep_sync(), so "my CTA has been placed" implies that every kernel two or more steps back in the chain
+// has completed.  That is what allows the FFN kernels to start streaming weight pages at once (unit lists
+// and page-table rows are written two steps back or earlier) and to wait only before their first token tile.
+// With the timing events between the kernels the attribute has no effect.
+__device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 }  // namespace pw

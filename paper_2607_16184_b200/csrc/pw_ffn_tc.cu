@@ -477,6 +477,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = c->tmem_base;
+  // This CTA may have been placed while the kernel before this one is still finishing on other SMs.  Unit
+  // lists, work counters and page-table rows were written earlier in the chain and are final (see
+  // grid_dep_sync); the token rows are not: the token-tile producer waits for them, everybody else starts.
 
   // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
   // (the weight producer claims, the other roles follow its list).
@@ -560,6 +563,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   } else if (warp == kWarpTokens) {
     // ---------------- token-tile producer ----------------
     if (lane == 0) {
+      grid_dep_sync();
+      grid_dep_trigger();
       uint32_t bcount = 0;
       bool ok = true;
       for (int i = 0; ok; ++i) {
@@ -1000,15 +1005,15 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
-  ffn_tc_kernel<0><<<ctx->num_sms, kThreads, smem[0], s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_gu), n_units,
-                                                        st->xt, w.Rpad, nt_tile, n_bslots[0], n_slots[0],
-                                                        reinterpret_cast<__half*>(b + w.ht), nullptr, c.hidden, 0,
-                                                        work_counter, status);
+  PW_CUDA_OK(launch_dependent(ffn_tc_kernel<0>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[0], s, rows,
+                              reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
+                              n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
+                              work_counter, status));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
-  ffn_tc_kernel<1><<<ctx->num_sms, kThreads, smem[1], s>>>(rows, reinterpret_cast<const Unit*>(b + w.units_dn), n_units,
-                                                        st->ht, w.Rpad, nt_tile, n_bslots[1], n_slots[1], nullptr,
-                                                        reinterpret_cast<float*>(b + w.y), c.hidden,
-                                                        (size_t)R * c.hidden, work_counter + 1, status);
+  PW_CUDA_OK(launch_dependent(ffn_tc_kernel<1>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
+                              reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
+                              n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
+                              (size_t)R * c.hidden, work_counter + 1, status));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   (void)ksplit;

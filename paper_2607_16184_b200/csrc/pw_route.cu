@@ -9,6 +9,8 @@ constexpr int kMaxExpertsPerLane = 8;  // E <= 256
 // One warp per token.  Slot j holds the j-th largest logit; equal logits: lower expert index first.
 __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ logits, int T, int E, int k,
                                                      int32_t* __restrict__ topk_ids, float* __restrict__ gates) {
+  grid_dep_sync();   // the gates of the call before this one may still be read by its combine kernel
+  grid_dep_trigger();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= T) return;
   const float* l = logits + (size_t)warp * E;
@@ -78,6 +80,8 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
                                                        Unit* __restrict__ units_dn, int32_t* __restrict__ n_units,
                                                        int32_t* __restrict__ seg_order, int max_units,
                                                        int32_t* __restrict__ status) {
+  grid_dep_sync();
+  grid_dep_trigger();
   extern __shared__ int32_t sm[];
   const int S = E + n_shared;
   int32_t* cnt = sm;                 // [S]
@@ -245,6 +249,8 @@ extern "C" int pw_debug_read_ptrace(long long* out) {
 __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
                                                      const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
                                                      uint4* __restrict__ xt) {
+  grid_dep_sync();
+  grid_dep_trigger();
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   const int c = blockIdx.y;
   if (n >= offsets[S]) return;
@@ -259,6 +265,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4* __restrict__
                                                       const int32_t* __restrict__ inv_perm, int T, int k, int n_shared,
                                                       int H4, int ksplit, size_t split_stride4,
                                                       float4* __restrict__ out) {
+  grid_dep_sync();
+  grid_dep_trigger();
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   const int t = blockIdx.y;
   if (c >= H4) return;
@@ -297,24 +305,26 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
   const int E = c.n_experts, S = w.S;
   int32_t* ids = reinterpret_cast<int32_t*>(b + w.topk_ids);
   timing_mark(ctx, PW_K_ROUTER, s);
-  router_kernel<<<(T * 32 + 255) / 256, 256, 0, s>>>(logits, T, E, k, ids, reinterpret_cast<float*>(b + w.gates));
+  PW_CUDA_OK(launch_dependent(router_kernel, dim3((T * 32 + 255) / 256), dim3(256), 0, s, logits, T, E, k, ids,
+                              reinterpret_cast<float*>(b + w.gates)));
   timing_mark(ctx, PW_K_PERMUTE, s);
   const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + E + 32 * (size_t)E + (S + 1) + S);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * S * 3;
-  permute_kernel<<<1, 1024, smem, s>>>(
-      ids, T, k, E, c.n_shared, reinterpret_cast<int32_t*>(b + w.counts), reinterpret_cast<int32_t*>(b + w.offsets),
-      reinterpret_cast<int32_t*>(b + w.perm), reinterpret_cast<int32_t*>(b + w.inv_perm),
-      reinterpret_cast<int32_t*>(b + w.row_token), reinterpret_cast<int32_t*>(b + w.counter), rows, c.hidden, c.ffn,
-      nt_tile, ksplit, reinterpret_cast<Unit*>(b + w.units_gu), reinterpret_cast<Unit*>(b + w.units_dn),
+  PW_CUDA_OK(launch_dependent(
+      permute_kernel, dim3(1), dim3(1024), smem, s, ids, T, k, E, c.n_shared, reinterpret_cast<int32_t*>(b + w.counts),
+      reinterpret_cast<int32_t*>(b + w.offsets), reinterpret_cast<int32_t*>(b + w.perm),
+      reinterpret_cast<int32_t*>(b + w.inv_perm), reinterpret_cast<int32_t*>(b + w.row_token),
+      reinterpret_cast<int32_t*>(b + w.counter), rows, c.hidden, c.ffn, nt_tile, ksplit,
+      reinterpret_cast<Unit*>(b + w.units_gu), reinterpret_cast<Unit*>(b + w.units_dn),
       reinterpret_cast<int32_t*>(b + w.n_units), reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units,
-      reinterpret_cast<int32_t*>(b + w.status));
+      reinterpret_cast<int32_t*>(b + w.status)));
   const int R = T * k + c.n_shared * T;
   timing_mark(ctx, PW_K_GATHER, s);
   dim3 grid((R + 255) / 256, c.hidden / 8);
-  gather_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(hidden),
-                                     reinterpret_cast<const int32_t*>(b + w.row_token),
-                                     reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
-                                     reinterpret_cast<uint4*>(b + w.xt));
+  PW_CUDA_OK(launch_dependent(gather_kernel, grid, dim3(256), 0, s, reinterpret_cast<const uint4*>(hidden),
+                              reinterpret_cast<const int32_t*>(b + w.row_token),
+                              reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
+                              reinterpret_cast<uint4*>(b + w.xt)));
   ctx->launches += 3;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
@@ -328,10 +338,10 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
   const int R = T * k + c.n_shared * T;
   dim3 grid((H4 + 255) / 256, T);
   timing_mark(ctx, PW_K_COMBINE, s);
-  combine_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const float4*>(b + w.y),
-                                      reinterpret_cast<const float*>(b + w.gates),
-                                      reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
-                                      (size_t)R * H4, reinterpret_cast<float4*>(out));
+  PW_CUDA_OK(launch_dependent(combine_kernel, grid, dim3(256), 0, s, reinterpret_cast<const float4*>(b + w.y),
+                              reinterpret_cast<const float*>(b + w.gates),
+                              reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
+                              (size_t)R * H4, reinterpret_cast<float4*>(out)));
   timing_mark(ctx, PW_NUM_KERNELS, s);
   ctx->launches += 1;
   PW_CUDA_OK(cudaGetLastError());
