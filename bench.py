@@ -435,7 +435,7 @@ def main():
     ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode"])
     ap.add_argument("--layers", type=int, default=3, help="distinct layer copies the decode loop rotates over")
     ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
-    ap.add_argument("--cpu-tokens", type=int, default=8)
+    ap.add_argument("--cpu-tokens", type=int, default=48)
     ap.add_argument("--ref-tokens", type=int, default=2)
     ap.add_argument("--uniform-bits", type=int, default=0, choices=[0, 16, 8, 4, 3, 2],
                     help="diagnostic: give every routed block this bitwidth instead of the configured mix")
