@@ -967,11 +967,14 @@ void tc_teardown(pw_ctx* ctx) {
 }
 
 int tensor_token_tile(const pw_ctx* ctx, int T, int k) {
-  (void)ctx;
-  (void)k;
-  // an expert never holds more than T tokens; tiles of at most 128 tokens
+  // An expert never holds more than T tokens.  Tiles of 128 tokens leave tensor memory for one partial
+  // accumulator per matrix only (one MMA issuer per matrix): right when experts hold hundreds of tokens and
+  // the MMAs are wide, wrong when most experts hold a few dozen.  So: 128 only if the average routed expert
+  // holds more than 64 tokens, otherwise at most 64 (a busier expert then takes several tiles).
   int nt = (T + 15) & ~15;
-  if (nt > 128) nt = 128;
+  const long long avg = ((long long)T * k) / (ctx->cfg.n_experts > 0 ? ctx->cfg.n_experts : 1);
+  const int cap = avg > 64 ? 128 : 64;
+  if (nt > cap) nt = cap;
   return nt;
 }
 
