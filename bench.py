@@ -384,6 +384,165 @@ def run_gpu(args):
     replicas.shutdown()
 
 
+def run_d5(args):
+    """The demotion-under-load configuration at full size: 32 stacked Mixtral-shaped layers, all 16-bit at the
+    start (90 GB of pages), a seeded third of the blocks demoted 16->4 and then 4->2 on a side stream while
+    batch-64 decode steps (one call per layer) keep running.  Three runs: decode alone; "shadow" (demotes run
+    but are never committed: pure interference); "committed" (every finished demote is published at the next
+    call boundary and the page it replaces is released)."""
+    from paper_2607_16184_b200 import binding as B
+    from paper_2607_16184_b200 import build as pwbuild
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    pwbuild.build()
+    peaks = measured_peaks()
+    cfg = synth.CONFIGS["demote_under_load"]
+    T, k = cfg.tokens, cfg.top_k
+    per_layer = sum(B.pw_page_bytes(*cfg.block_shape(u), 16)[0] for u in range(3)) * cfg.n_experts
+    free, _ = torch.cuda.mem_get_info(device)
+    L = int(min(cfg.n_layers, (free - 14e9) // (per_layer * 1.1)))          # demoted copies add < 10 %
+    if L < 2:
+        raise RuntimeError("not enough free device memory for two layers of %.1f GB" % (per_layer / 1e9))
+    ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, T, k, device=device)
+    pages, xs, lgs = {}, [], []
+    for layer in range(L):
+        ents = []
+        for e in range(cfg.n_experts):
+            for u in range(3):
+                w = synth.block_weights(cfg, layer, e, u, device=device)
+                pages[(layer, e, u)] = ctx.pw_quantize_block(w, 16)
+                ents.append((layer, e, u, pages[(layer, e, u)]))
+                del w
+        ctx.pw_set_page_table(ents)
+        xs.append(synth.activations(cfg, layer, device=device))
+        lgs.append(synth.router_logits(cfg, layer, device=device))
+    torch.cuda.synchronize(device)
+    sched = [key for key in synth.demote_schedule(cfg) if key[0] < L]
+    out = torch.empty(T, cfg.hidden, dtype=torch.float32, device=device)
+    main = torch.cuda.current_stream(device)
+    side = torch.cuda.Stream(device=device)
+
+    def decode_step():
+        for layer in range(L):
+            ctx.pw_moe_forward(layer, xs[layer], lgs[layer], k, out=out)
+
+    def timed(fn, n):
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize(device)
+        return e0.elapsed_time(e1)
+
+    for _ in range(2):
+        decode_step()
+    sampler = ClockSampler(0)
+    sampler.start()
+    n0 = ctx.pw_launch_count()
+    n_base = 6
+    ms_base = timed(lambda i: decode_step(), n_base) / n_base
+
+    # shadow run: one chunk of 16->4 demotes per decode step into a small pool of scratch pages, never committed
+    per_step = 8
+    rows_cols = [cfg.block_shape(u) for u in range(3)]
+    pool = {u: [B.Page(rows_cols[u][0], rows_cols[u][1], 4, device) for _ in range(per_step)] for u in range(3)}
+    n_shadow = min(12, max(1, len(sched) // per_step))
+    moved = [0]
+
+    def shadow_step(i):
+        side.wait_stream(main)
+        used = {0: 0, 1: 0, 2: 0}
+        for key in sched[i * per_step:(i + 1) * per_step]:
+            u = key[2]
+            ctx.pw_demote_block(pages[key], 4, dst=pool[u][used[u] % per_step], stream=side)
+            used[u] += 1
+            moved[0] += B.pw_page_bytes(*rows_cols[u], 16)[0] + B.pw_page_bytes(*rows_cols[u], 4)[0]
+        decode_step()
+
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(device)
+    s0.record(side)
+    ms_shadow = timed(shadow_step, n_shadow) / n_shadow
+    s1.record(side)
+    torch.cuda.synchronize(device)
+    shadow_side_ms = s0.elapsed_time(s1)
+    shadow_gbs = moved[0] / (shadow_side_ms * 1e-3) / 1e9
+    del pool
+
+    # committed run: phase 1 (16->4) then phase 2 (4->2) over the same blocks
+    def page_total():
+        return sum(B.pw_page_bytes(p.rows, p.cols, p.bits)[0] for p in pages.values())
+
+    bytes_start = page_total()
+    phases = []
+    for dst_bits in (4, 2):
+        todo = list(sched)
+        inflight = []
+        steps = 0
+        moved_b = 0
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        while todo or inflight:
+            done = [x for x in inflight if x[2].query()]
+            if done:
+                for key, pg, ev in done:
+                    main.wait_event(ev)
+                    # The page it replaces is released here.  Its last readers are already enqueued on the main
+                    # stream, and whoever gets its memory next (a demote destination, written on the side stream)
+                    # starts only after side.wait_stream(main) below.
+                    pages[key] = pg
+                ctx.pw_set_page_table([(key[0], key[1], key[2], pg) for key, pg, _ in done])
+                inflight = [x for x in inflight if not any(x is d for d in done)]
+            side.wait_stream(main)
+            for key in todo[:per_step]:
+                src = pages[key]
+                dst = ctx.pw_demote_block(src, dst_bits, stream=side)
+                ev = torch.cuda.Event()
+                ev.record(side)
+                inflight.append((key, dst, ev))
+                moved_b += B.pw_page_bytes(src.rows, src.cols, src.bits)[0] + B.pw_page_bytes(src.rows, src.cols, dst_bits)[0]
+            todo = todo[per_step:]
+            decode_step()
+            steps += 1
+        e1.record()
+        torch.cuda.synchronize(device)
+        ms = e0.elapsed_time(e1)
+        phases.append({"dst_bits": dst_bits, "blocks": len(sched), "decode_steps": steps, "ms": ms,
+                       "tokens_per_s": T * steps / (ms * 1e-3), "demote_bytes_moved": moved_b,
+                       "demote_gbs_over_phase": moved_b / (ms * 1e-3) / 1e9, "page_bytes_after": page_total()})
+    clocks = sampler.stop()
+    launches = ctx.pw_launch_count() - n0
+    status = ctx.pw_last_device_status()
+    tot_steps = sum(p["decode_steps"] for p in phases)
+    tot_ms = sum(p["ms"] for p in phases)
+    tok_base = T / (ms_base * 1e-3)
+    line = {"metric": METRIC, "value": T * tot_steps / (tot_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+            "steps": tot_steps, "warmup": 2, "ms_per_step": tot_ms / tot_steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": "demote_under_load: %d stacked layers (E=8 top-2 H=4096 F=14336, T=64), all 16-bit at "
+                                   "the start (%.1f GB of pages); a step = one forward call per layer; %d blocks demoted "
+                                   "16->4 then 4->2 on a side stream, %d per step, committed between calls"
+                                   % (L, bytes_start / 1e9, len(sched), per_step),
+                       "l2": "inputs larger than L2", "layers": L, "layers_of_config": cfg.n_layers},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches), "device_status": status,
+            "roofline": {"bound": "hbm", "kernel": "whole decode step, all 16-bit", "unit": "GB/s",
+                         "achieved": (L * per_layer) / (ms_base * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "peak_source": peaks["source"],
+                         "frac": (L * per_layer) / (ms_base * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None},
+            "cpu_baseline": None,
+            "d5": {"baseline": {"ms_per_step": ms_base, "tokens_per_s": tok_base},
+                   "shadow": {"ms_per_step": ms_shadow, "tokens_per_s": T / (ms_shadow * 1e-3),
+                              "slowdown": 1.0 - ms_base / ms_shadow, "demotes_per_step": per_step,
+                              "demote_gbs_side_stream": shadow_gbs},
+                   "committed": phases, "page_bytes_start": bytes_start}}
+    print(json.dumps(line), flush=True)
+
+
 def run_reference(args):
     """The CPU oracle as the reference arm: same config and metric, each step a bounded sample of the batch."""
     rank, _, world = replicas.env_world()
@@ -432,7 +591,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode"])
+    ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode", "demote_under_load"])
     ap.add_argument("--layers", type=int, default=3, help="distinct layer copies the decode loop rotates over")
     ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
     ap.add_argument("--cpu-tokens", type=int, default=48)
@@ -449,7 +608,10 @@ def main():
     else:
         args.steps = 2000 if args.steps is None else args.steps
         args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
-        run_gpu(args)
+        if args.config == "demote_under_load":
+            run_d5(args)
+        else:
+            run_gpu(args)
 
 
 if __name__ == "__main__":
