@@ -328,7 +328,8 @@ def run_gpu(args):
                 "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": gu_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gu_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": gu_kernel_bytes, "avg_launch_ms": kavg["ffn_gate_up"],
-                "traffic": profiled_traffic("ffn_gate_up_mixtral_decode.md")}
+                "traffic": profiled_traffic("ffn_gate_up_mixtral_decode.md")
+                if cfg.name == "mixtral_decode" and not args.uniform_bits else None}
 
     # end to end: host buffers in, host buffer out, through the host-buffer entry point
     xh = [lay["x"].cpu().pin_memory() for lay in layers]
