@@ -154,13 +154,20 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
   // first).  Consecutive units therefore belong to different experts -- pages of different bitwidths are
   // in flight together, the ones bound by HBM beside the ones bound by unpacking -- and the tiles that
   // share weights are adjacent.  Rank segments by counting (S is small).
+  // (the sort's scratch is free by now: its tail holds the page bits of every segment for the ranking, its
+  // head the per-list tables below)
+  int32_t* sbits = wcnt + 32 * E - S;              // gate + up bits | down bits << 16
+  __syncthreads();
+  for (int s = tid; s < S; s += blockDim.x)
+    sbits[s] = (int32_t)((rows[s * 3].bits + rows[s * 3 + 1].bits) | (rows[s * 3 + 2].bits << 16));
   for (int phase = 0; phase < 2; ++phase) {
     __syncthreads();
     for (int s = tid; s < S; s += blockDim.x) {
-      const uint32_t mine = phase == 0 ? rows[s * 3].bits + rows[s * 3 + 1].bits : rows[s * 3 + 2].bits;
+      const int sh = phase == 0 ? 0 : 16;
+      const uint32_t mine = ((uint32_t)sbits[s] >> sh) & 0xffffu;
       int rk = 0;
       for (int o = 0; o < S; ++o) {
-        const uint32_t other = phase == 0 ? rows[o * 3].bits + rows[o * 3 + 1].bits : rows[o * 3 + 2].bits;
+        const uint32_t other = ((uint32_t)sbits[o] >> sh) & 0xffffu;
         rk += (other > mine) || (other == mine && o < s);
       }
       order[rk] = s;
@@ -170,11 +177,15 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
     const int row_tiles = (phase == 0 ? F : H) / kTileRows;
     const int ng = (phase == 0 ? H : F) / kGroup;
     const int splits = phase == 0 ? 1 : ksplit;
+    // token tiles per segment in rank order (in parallel), then their prefix (S additions by one thread)
+    for (int i = tid; i < S; i += blockDim.x) ubase[i + 1] = (cnt[order[i]] + nt_tile - 1) / nt_tile;
+    __syncthreads();
     if (tid == 0) {
-      int a = 0;                                   // token tiles of the segments before i, in rank order
+      int a = 0;
       for (int i = 0; i < S; ++i) {
+        const int tt = ubase[i + 1];
         ubase[i] = a;
-        a += (cnt[order[i]] + nt_tile - 1) / nt_tile;
+        a += tt;
       }
       ubase[S] = a;
       const long long total = (long long)a * row_tiles * splits;
@@ -191,7 +202,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
     // token tile j of the list -> rank of its segment (the sort's scratch is free by now; a layer with more
     // token tiles than fit there searches the prefix instead), and the group range of every K split
     int32_t* tseg = wcnt;
-    const bool use_table = TT + splits + 1 <= 32 * E;
+    const bool use_table = TT + splits + 1 <= 32 * E - S;
     int32_t* gtab = wcnt + (use_table ? TT : 0);     // [splits + 1] when it fits
     if (use_table) {
       for (int i = tid; i < S; i += blockDim.x)
