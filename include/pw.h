@@ -48,11 +48,11 @@ typedef enum {
 
 typedef enum { PW_GATE = 0, PW_UP = 1, PW_DOWN = 2 } pw_kind;
 
-/* Which expert-FFN kernel family pw_moe_forward uses.
- * AUTO picks TENSOR unless every expert holds at most a few tokens. */
+/* Which expert-FFN kernel family pw_moe_forward uses.  AUTO is TENSOR: the tensor-core kernels are the
+ * faster ones at every batch size, one token included. */
 typedef enum {
   PW_MODE_AUTO = 0,
-  PW_MODE_SIMT = 1,  /* CUDA-core kernel, thread per weight row; right for a handful of tokens */
+  PW_MODE_SIMT = 1,  /* CUDA-core kernel, thread per weight row: an independent second implementation */
   PW_MODE_TENSOR = 2 /* tcgen05 tensor-core kernel, pages dequantized into tensor memory      */
 } pw_mode;
 

@@ -244,11 +244,10 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
     for (int u = 0; u < 3; ++u)
       if (!ctx->host_valid[row_index(ctx, layer, e, u)]) return PW_ERR_STATE;
 
-  if (mode == PW_MODE_AUTO) {
-    // a handful of tokens per expert at most: the CUDA-core kernel streams the pages once and is done
-    const long long pairs = (long long)T * top_k;
-    mode = (pairs <= 8 && c.n_shared == 0) ? PW_MODE_SIMT : PW_MODE_TENSOR;
-  }
+  // The tensor-core kernels win at every batch size measured (one token of a Mixtral-shaped layer: 0.12 ms
+  // against 1.96 ms for the CUDA-core kernel), so AUTO means TENSOR; the CUDA-core kernel stays selectable as
+  // an independent second implementation.
+  if (mode == PW_MODE_AUTO) mode = PW_MODE_TENSOR;
   int nt_tile = 0, ksplit = 1;
   if (mode == PW_MODE_TENSOR) {
     nt_tile = tensor_token_tile(ctx, T, top_k);

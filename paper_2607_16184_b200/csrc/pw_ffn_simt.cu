@@ -1,7 +1,7 @@
 // CUDA-core expert FFN: one thread per weight row, pages read tile by tile with contiguous 16-byte
-// loads, dequantized in registers, fp32 accumulation against up to eight tokens at a time.  The
-// right kernel when an expert holds only a handful of tokens (latency decode); for larger batches
-// the tensor-core kernel takes over.
+// loads, dequantized in registers, fp32 accumulation against up to eight tokens at a time.  An
+// independent second implementation of the expert FFN (PW_MODE_SIMT): the tests run it beside the
+// tensor-core kernels.  It is far slower than those at every batch size, so PW_MODE_AUTO never picks it.
 #include "pw_common.cuh"
 #include "pw_layout.cuh"
 
