@@ -45,6 +45,8 @@ WsMap make_wsmap(const pw_config& c) {
   m.inv_perm = take(4 * (size_t)P);
   m.row_token = take(4 * (size_t)m.Rpad);
   m.seg_order = take(4 * (size_t)m.S);
+  m.max_tiles = m.Rmax / 16 + m.S + 8;
+  m.tile_tab = take(2 * 8 * (size_t)m.max_tiles);
   m.units_gu = take(sizeof(Unit) * (size_t)m.max_units);
   m.units_dn = take(sizeof(Unit) * (size_t)m.max_units);
   m.n_units = take(16);

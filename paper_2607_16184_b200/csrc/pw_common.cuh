@@ -48,6 +48,7 @@ struct WsMap {
   size_t inv_perm;    // int32[Pmax]
   size_t row_token;   // int32[Rpad]    operand row -> token (-1 for padding)
   size_t seg_order;   // int32[S]
+  size_t tile_tab;    // int2[2][max_tiles]: (segment, token tile of the segment) of every token tile of the two unit lists
   size_t units_gu;    // Unit[max_units]
   size_t units_dn;    // Unit[max_units]
   size_t n_units;     // int32[4]
@@ -63,6 +64,7 @@ struct WsMap {
   int Rmax;           // max operand rows = Tmax*kmax + n_shared*Tmax
   int Rpad;           // Rmax + kPadRows
   int max_units;
+  int max_tiles;
   size_t y_slots;     // rows of the y buffer (split * R must fit)
 };
 

@@ -76,8 +76,8 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
                                                        int32_t* __restrict__ inv_perm,
                                                        int32_t* __restrict__ row_token, int32_t* __restrict__ counter,
                                                        const DevRow* __restrict__ rows, int H, int F, int nt_tile,
-                                                       int ksplit, Unit* __restrict__ units_gu,
-                                                       Unit* __restrict__ units_dn, int32_t* __restrict__ n_units,
+                                                       int ksplit, int2* __restrict__ tile_tab, int max_tiles,
+                                                       int32_t* __restrict__ n_units,
                                                        int32_t* __restrict__ seg_order, int max_units,
                                                        int32_t* __restrict__ status) {
   grid_dep_sync();
@@ -149,14 +149,13 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
   if (nt_tile <= 0) return;  // SIMT path: no unit lists
   PSTAMP(4);
 
-  // Unit lists.  The CTAs of the FFN kernels claim units in list order, so the list is laid out for that:
-  // row tile outermost, K split next, then every segment's token tiles (segments with the widest pages
-  // first).  Consecutive units therefore belong to different experts -- pages of different bitwidths are
-  // in flight together, the ones bound by HBM beside the ones bound by unpacking -- and the tiles that
-  // share weights are adjacent.  Rank segments by counting (S is small).
-  // (the sort's scratch is free by now: its tail holds the page bits of every segment for the ranking, its
-  // head the per-list tables below)
-  int32_t* sbits = wcnt + 32 * E - S;              // gate + up bits | down bits << 16
+  // Tables of the unit lists (the lists themselves are written by the gather kernel, which has the threads
+  // for it).  The CTAs of the FFN kernels claim units in list order, so the lists are laid out for that: row
+  // tile outermost, K split next, then every segment's token tiles (segments with the widest pages first).
+  // Consecutive units therefore belong to different experts -- pages of different bitwidths are in flight
+  // together -- and the tiles that share weights are adjacent.  Here: per list, the token tiles in that
+  // order.  Rank segments by counting (S is small); the sort's scratch is free by now and holds the bits.
+  int32_t* sbits = wcnt;                           // gate + up bits | down bits << 16
   __syncthreads();
   for (int s = tid; s < S; s += blockDim.x)
     sbits[s] = (int32_t)((rows[s * 3].bits + rows[s * 3 + 1].bits) | (rows[s * 3 + 2].bits << 16));
@@ -175,7 +174,6 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
     __syncthreads();
     PSTAMP(5 + 4 * phase);
     const int row_tiles = (phase == 0 ? F : H) / kTileRows;
-    const int ng = (phase == 0 ? H : F) / kGroup;
     const int splits = phase == 0 ? 1 : ksplit;
     // token tiles per segment in rank order (in parallel), then their prefix (S additions by one thread)
     for (int i = tid; i < S; i += blockDim.x) ubase[i + 1] = (cnt[order[i]] + nt_tile - 1) / nt_tile;
@@ -189,79 +187,63 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
       }
       ubase[S] = a;
       const long long total = (long long)a * row_tiles * splits;
-      n_units[phase] = total <= max_units ? (int)total : 0;
-      if (total > max_units) atomicMax(status, (int)PW_ERR_NOMEM);
+      const bool fits = total <= max_units && a <= max_tiles;
+      n_units[phase] = fits ? (int)total : 0;
+      n_units[2 + phase] = a;                      // token tiles of the list
+      if (!fits) atomicMax(status, (int)PW_ERR_NOMEM);
     }
     __syncthreads();
     PSTAMP(6 + 4 * phase);
-    const int TT = ubase[S];
-    if ((long long)TT * row_tiles * splits > max_units) continue;
-    Unit* out = phase == 0 ? units_gu : units_dn;
+    if (ubase[S] > max_tiles) continue;
     if (phase == 0)
       for (int i = tid; i < S; i += blockDim.x) seg_order[i] = order[i];
-    // token tile j of the list -> rank of its segment (the sort's scratch is free by now; a layer with more
-    // token tiles than fit there searches the prefix instead), and the group range of every K split
-    int32_t* tseg = wcnt;
-    const bool use_table = TT + splits + 1 <= 32 * E - S;
-    int32_t* gtab = wcnt + (use_table ? TT : 0);     // [splits + 1] when it fits
-    if (use_table) {
-      for (int i = tid; i < S; i += blockDim.x)
-        for (int j = ubase[i]; j < ubase[i + 1]; ++j) tseg[j] = i;
-      for (int sp = tid; sp <= splits; sp += blockDim.x) gtab[sp] = (sp * ng) / splits;
-    }
-    __syncthreads();
-    // warp w writes the units of (row tile, split) pairs w, w + 32, ..; its lanes walk the token tiles: no
-    // per-unit division, consecutive lanes write consecutive units
-    const int n_rs = row_tiles * splits;
-    for (int rs = warp; rs < n_rs; rs += 32) {
-      int sp = 0, rt = rs;
-      if (splits > 1) {
-        rt = rs / splits;
-        sp = rs - rt * splits;
-      }
-      const int g0 = use_table ? gtab[sp] : (sp * ng) / splits;
-      const int g1 = use_table ? gtab[sp + 1] : ((sp + 1) * ng) / splits;
-      for (int j = lane; j < TT; j += 32) {
-        int i;
-        if (use_table) {
-          i = tseg[j];
-        } else {
-          i = 0;
-          while (ubase[i + 1] <= j) ++i;
-        }
-        const int s = order[i];
-        const int n = cnt[s];
-        const int ti = j - ubase[i];
-        Unit un;
-        un.seg = s;
-        un.row_tile = rt;
-        un.tok0 = off[s] + ti * nt_tile;
-        un.ntok = min(nt_tile, n - ti * nt_tile);
-        un.g0 = g0;
-        un.g1 = g1;
-        un.split = sp;
-        un.pad_ = 0;
-        out[(size_t)rs * TT + j] = un;
-      }
-    }
+    int2* tab = tile_tab + (size_t)phase * max_tiles;
+    for (int i = tid; i < S; i += blockDim.x)
+      for (int j = ubase[i]; j < ubase[i + 1]; ++j) tab[j] = make_int2(order[i], j - ubase[i]);
     PSTAMP(7 + 4 * phase);
   }
 }
-#ifdef PW_TC_PROFILE
-extern "C" int pw_debug_read_ptrace(long long* out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, g_ptrace, sizeof(g_ptrace));
-  return 0;
-}
-#endif
 
 // Xt[c][n][0..7] = hidden[row_token[n]][8c .. 8c+7] for the operand rows n < R.  Rows past R only ever feed
 // accumulator columns that nobody reads, so they keep whatever they hold.
+// The same grid first writes the two unit lists from the tables of the permute kernel: unit u of a list is
+// (row tile, K split) pair u / TT and token tile u mod TT.
 __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
                                                      const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
-                                                     uint4* __restrict__ xt) {
+                                                     uint4* __restrict__ xt, const int32_t* __restrict__ counts,
+                                                     const int2* __restrict__ tile_tab, int max_tiles,
+                                                     const int32_t* __restrict__ n_units, int nt_tile, int ksplit,
+                                                     int ng_gu, int ng_dn, Unit* __restrict__ units_gu,
+                                                     Unit* __restrict__ units_dn) {
   grid_dep_sync();
   grid_dep_trigger();
+  if (nt_tile > 0) {
+    const int gt = (blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
+    const int n_threads = gridDim.x * gridDim.y * blockDim.x;
+    for (int phase = 0; phase < 2; ++phase) {
+      const int total = n_units[phase], TT = n_units[2 + phase];
+      const int splits = phase == 0 ? 1 : ksplit;
+      const int ng = phase == 0 ? ng_gu : ng_dn;
+      const int2* tab = tile_tab + (size_t)phase * max_tiles;
+      Unit* out = phase == 0 ? units_gu : units_dn;
+      for (int u = gt; u < total; u += n_threads) {
+        const int rs = u / TT, j = u - rs * TT;
+        const int rt = rs / splits, sp = rs - rt * splits;
+        const int2 t = tab[j];
+        const int n = counts[t.x];
+        Unit un;
+        un.seg = t.x;
+        un.row_tile = rt;
+        un.tok0 = offsets[t.x] + t.y * nt_tile;
+        un.ntok = min(nt_tile, n - t.y * nt_tile);
+        un.g0 = (sp * ng) / splits;
+        un.g1 = ((sp + 1) * ng) / splits;
+        un.split = sp;
+        un.pad_ = 0;
+        out[u] = un;
+      }
+    }
+  }
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   const int c = blockIdx.y;
   if (n >= offsets[S]) return;
@@ -326,16 +308,19 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
       reinterpret_cast<int32_t*>(b + w.offsets), reinterpret_cast<int32_t*>(b + w.perm),
       reinterpret_cast<int32_t*>(b + w.inv_perm), reinterpret_cast<int32_t*>(b + w.row_token),
       reinterpret_cast<int32_t*>(b + w.counter), rows, c.hidden, c.ffn, nt_tile, ksplit,
-      reinterpret_cast<Unit*>(b + w.units_gu), reinterpret_cast<Unit*>(b + w.units_dn),
-      reinterpret_cast<int32_t*>(b + w.n_units), reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units,
-      reinterpret_cast<int32_t*>(b + w.status)));
+      reinterpret_cast<int2*>(b + w.tile_tab), w.max_tiles, reinterpret_cast<int32_t*>(b + w.n_units),
+      reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units, reinterpret_cast<int32_t*>(b + w.status)));
   const int R = T * k + c.n_shared * T;
   timing_mark(ctx, PW_K_GATHER, s);
   dim3 grid((R + 255) / 256, c.hidden / 8);
   PW_CUDA_OK(launch_dependent(gather_kernel, grid, dim3(256), 0, s, reinterpret_cast<const uint4*>(hidden),
                               reinterpret_cast<const int32_t*>(b + w.row_token),
                               reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
-                              reinterpret_cast<uint4*>(b + w.xt)));
+                              reinterpret_cast<uint4*>(b + w.xt), reinterpret_cast<const int32_t*>(b + w.counts),
+                              reinterpret_cast<const int2*>(b + w.tile_tab), w.max_tiles,
+                              reinterpret_cast<const int32_t*>(b + w.n_units), nt_tile, ksplit, c.hidden / kGroup,
+                              c.ffn / kGroup, reinterpret_cast<Unit*>(b + w.units_gu),
+                              reinterpret_cast<Unit*>(b + w.units_dn)));
   ctx->launches += 3;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
@@ -407,7 +392,7 @@ extern "C" pw_status pw_route_tokens_static(const float* router_logits, int T, i
                                             reinterpret_cast<int32_t*>(sc + kStaticInvPerm),
                                             reinterpret_cast<int32_t*>(sc + kStaticRowToken),
                                             reinterpret_cast<int32_t*>(sc + kStaticCounter), nullptr, 0, 0, 0, 1, nullptr,
-                                            nullptr, nullptr, nullptr, 0,
+                                            0, nullptr, nullptr, 0,
                                             reinterpret_cast<int32_t*>(sc + kStaticStatus));
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
