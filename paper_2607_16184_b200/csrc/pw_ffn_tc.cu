@@ -29,6 +29,8 @@
 //   warps 23-26  epilogue: adds the partials; SwiGLU -> fp16 operand of the down projection (PHASE 0), or the
 //                fp32 split-K partial of the down projection (PHASE 1).  Narrow token tiles alternate
 //                between two accumulator buffers, so the next unit's MMAs overlap the epilogue.
+//                Token tiles wider than 64 leave no second buffer: the HELP instantiation, launched for
+//                those, has the four issuer warps share the epilogue of every wide unit.
 // Every wait is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing
 // work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -420,7 +422,7 @@ __device__ __forceinline__ void decode_item_half(const char* item, int r, int h,
 
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
-template <int PHASE>
+template <int PHASE, bool HELP>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, const int32_t* __restrict__ n_units_ptr,
               const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
@@ -458,7 +460,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&c->d_full[i], n_issuers);
-      mbar_init(&c->d_empty[i], 4);
+      mbar_init(&c->d_empty[i], HELP ? 8 : 4);    // epilogue warps (+ the issuer warps when they share the epilogue)
     }
     c->abort_flag = 0;
     c->issued[0] = c->issued[1] = 0;
@@ -592,6 +594,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     // all eight k-steps of it into its own partial accumulator; a quantized tile k is dequantized by the
     // matrix's group k mod IPM, so with npart == IPM every dequantizer group has an issuer of its own.
     // The epilogue adds the partials.
+    if constexpr (!HELP) {
     const int iss = warp - kWarpMma;
     const int my_m = iss / IPM, my_j = iss % IPM;
     if (lane == 0 && my_j < npart) {
@@ -730,8 +733,204 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         seq_unit += ng * W;
       }
     }
-  } else if (warp < kDqWarps) {
-    // ---------------- dequantize ----------------
+    } else {
+    const int iss = warp - kWarpMma;
+    const int my_m = iss / IPM, my_j = iss % IPM;
+    // Wide token tiles leave no room for a second accumulator buffer, so the epilogue of a unit is not
+    // overlapped: here the four issuer warps share it with the four epilogue warps (they take the upper
+    // half of the token columns of their lane quarter), lane 0 of the warps with an accumulator of their own
+    // issuing the unit's MMAs first.  Every lane tracks the per-unit state; only lane 0 uses the issuing part.
+    const bool issuing = my_j < npart;
+    const int hq = warp & 3;
+    const int hr = hq * 32 + lane;
+    const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
+    {
+      uint32_t seq_unit = 0;                        // slot items before the current unit
+      uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand half-slots
+      uint32_t ucount = 0;
+      uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
+      const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
+      const uint32_t b_lo_base = smem_u32(bslots) >> 4;
+      const uint32_t w_lo_base = smem_u32(wring) >> 4;
+      const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
+      const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
+      const uint32_t a_base = tmem + acol;
+      bool ok = true;
+      for (int i = 0; ok; ++i, ++ucount) {
+        const int u = next_unit((uint32_t)i, c, status);
+        if (u < 0) break;
+        const Unit un = units[u];
+        uint32_t ubits[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) ubits[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)].bits;
+        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
+        // slot items per group of the unit (W) and the offset of my matrix's inside a group
+        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
+        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+        const int nb_rows = (un.ntok + 15) & ~15;
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
+        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
+        const uint32_t b_step = (uint32_t)(2 * nb_rows);
+        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        uint32_t bt = base + j0;                     // token-tile number
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const uint32_t dbuf = wide ? 0u : dtoggle;
+        if (!wide) dtoggle ^= 1u;
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        if (lane == 0 && issuing) {
+          do {
+        if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
+        // the epilogue has drained the buffer(s) this unit accumulates into
+        if (wide || dbuf == 0) ok = mbar_wait<32>(&c->d_empty[0], (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait<32>(&c->d_empty[1], (duse1 & 1) ^ 1, c, status);
+        if (!ok) break;
+        if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
+        tc_fence_after();
+        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
+#pragma unroll 1
+        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
+          if (my_m == 0 && my_j == 0) { TRACE(10, bt); }
+          // the token tile of this group (a tile is looked at only once it is known to have been armed)
+          if (c->b_issued <= bt) {
+            const unsigned long long t0 = globaltimer();
+            while (c->b_issued <= bt && !c->abort_flag) {
+              __nanosleep(32);
+              if (globaltimer() - t0 > kWaitLimitNs) {
+                c->abort_flag = 1;
+                atomicMax(status, (int)PW_ERR_TIMEOUT);
+              }
+            }
+            if (c->abort_flag) {
+              ok = false;
+              break;
+            }
+          }
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
+          if (!ok) break;
+          if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
+          const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
+          if (my_bits == 16) {
+            // each K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3, 4 KB apart)
+            RingPos hp = rp;
+#pragma unroll 1
+            for (uint32_t hh = 0; hh < 2; ++hh) {
+              if (my_j == 0) { TRACE(12, sq + hh); }
+              ok = wait_issued(sq + hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
+              if (!ok) break;
+              tc_fence_after();
+              if (my_j == 0) { TRACE(8, sq + hh); }
+              const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
+              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
+              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
+              tc_commit(&c->empty[hp.s]);
+              if (my_j == 0) { TRACE(9, sq + hh); }
+              ring_advance(hp, 1, (uint32_t)n_slots);
+            }
+            if (!ok) break;
+            sq += (uint32_t)npart * W;
+            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
+          } else {
+            // the group that dequantizes this tile, and the parity of this use of its half-slots
+            const uint32_t k = base + j;
+            const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
+            const uint32_t use_par = (upar >> grp) & 1u;
+            upar ^= 1u << grp;
+            const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
+            const uint32_t a_t = a_base + grp * 64;
+            if (my_j == 0) { TRACE(12, k); }
+            ok = mbar_wait_s(f0, use_par, c, status);
+            if (!ok) break;
+            tc_fence_after();
+            if (my_j == 0) { TRACE(8, k); }
+            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_commit_s(e0);
+            if (my_j == 0) { TRACE(9, k); }
+            ok = mbar_wait_s(f0 + 8, use_par, c, status);
+            if (!ok) break;
+            tc_fence_after();
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            tc_commit_s(e0 + 8);
+          }
+          tc_commit_s(be_s + 8 * bp.s);
+          later = 1;
+          bt += (uint32_t)npart;
+          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
+        }
+            if (ok) {
+              if (wide || dbuf == 0) tc_commit(&c->d_full[0]);
+              if (wide || dbuf == 1) tc_commit(&c->d_full[1]);
+            }
+          } while (false);
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        const uint32_t par0 = duse0 & 1u, par1 = duse1 & 1u;     // phases of d_full this unit completes
+        if (wide || dbuf == 0) ++duse0;
+        if (wide || dbuf == 1) ++duse1;
+        // every issuer warp sees every phase of the accumulator barriers, also of the narrow units it has no
+        // part in: it must not run ahead of the epilogue by more than the phase parity can tell apart
+        if (wide || dbuf == 0) ok = mbar_wait<200>(&c->d_full[0], par0, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait<200>(&c->d_full[1], par1, c, status);
+        if (!ok) break;
+        if (wide) {
+          tc_fence_after();
+          uint32_t written = 0;
+          for (int p = 0; p < npart; ++p)
+            if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
+          const int row = un.row_tile * kTileRows + hr;
+          const int half = ((nb_rows / 16 + 1) / 2) * 16;         // the epilogue warps take [0, half)
+          for (int c0 = half; c0 < nb_rows; c0 += 16) {
+            float a[16], b[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
+            for (int p = 0; p < npart; ++p) {
+              if (!((written >> p) & 1u)) continue;
+              float t[16];
+              tmem_ld16(hlane_addr + p * nb_rows + c0, t);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
+              if (PHASE == 0) {
+                tmem_ld16(hlane_addr + (npart + p) * nb_rows + c0, t);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int nn = c0 + j;
+              if (nn < un.ntok) {
+                if (PHASE == 0) {
+                  const float hval = __fmul_rn(__fdividef(a[j], __fadd_rn(1.0f, __expf(-a[j]))), b[j]);
+                  ht[((size_t)(row >> 3) * Rpad + un.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
+                } else {
+                  y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + nn) * H + row] = a[j];
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&c->d_empty[0]);
+            mbar_arrive(&c->d_empty[1]);
+          }
+        }
+        base += ng;
+        seq_unit += ng * W;
+      }
+    }
+    }
+  } else if (warp < kDqWarps) {    // ---------------- dequantize ----------------
     // Four groups of four warps, each taking every other quantized item of one matrix (every fourth when
     // the unit has a single matrix; an item = one group of one matrix).  Warp q of a group owns rows (= TMEM lanes) 32q .. 32q+31 of the item, one row per
     // thread.  Each group has two operand half-slots (K 0..63 and K 64..127 of its item): while the
@@ -851,7 +1050,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       for (int p = 0; p < npart; ++p)
         if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
       base += ng;
-      for (int c0 = 0; c0 < nb_rows; c0 += 16) {
+      // with helpers, the issuer warps take the upper half of the token columns of a wide unit
+      const int c_end = HELP && wide ? ((nb_rows / 16 + 1) / 2) * 16 : nb_rows;
+      for (int c0 = 0; c0 < c_end; c0 += 16) {
         float a[16], b[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
@@ -888,8 +1089,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       __syncwarp();
       if (q == 0) { TRACE(14, ucount); }
       if (lane == 0) {
-        if (wide || dbuf == 0) mbar_arrive(&c->d_empty[0]);
-        if (wide || dbuf == 1) mbar_arrive(&c->d_empty[1]);
+        // (a narrow unit has no helpers: this warp arrives for the issuer warp of its lane quarter as well)
+        const uint32_t n_arr = HELP && !wide ? 2u : 1u;
+        if (wide || dbuf == 0) mbar_arrive_n(&c->d_empty[0], n_arr);
+        if (wide || dbuf == 1) mbar_arrive_n(&c->d_empty[1], n_arr);
       }
       if (wide || dbuf == 0) ++duse0;
       if (wide || dbuf == 1) ++duse1;
@@ -955,8 +1158,10 @@ static pw_status tc_setup(pw_ctx* ctx) {
     delete st;
     return PW_ERR_CUDA;
   }
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
   ctx->tc_state = st;
   return PW_OK;
 }
@@ -1008,12 +1213,14 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
-  PW_CUDA_OK(launch_dependent(ffn_tc_kernel<0>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[0], s, rows,
+  // token tiles of 128 leave no second accumulator buffer: the variant whose issuer warps share the epilogue
+  const bool help = nt_tile > 64;
+  PW_CUDA_OK(launch_dependent(help ? ffn_tc_kernel<0, true> : ffn_tc_kernel<0, false>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[0], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
                               n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
                               work_counter, status));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
-  PW_CUDA_OK(launch_dependent(ffn_tc_kernel<1>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
+  PW_CUDA_OK(launch_dependent(help ? ffn_tc_kernel<1, true> : ffn_tc_kernel<1, false>, dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
                               n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
                               (size_t)R * c.hidden, work_counter + 1, status));
