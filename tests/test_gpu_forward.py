@@ -236,3 +236,10 @@ def test_back_to_back_calls_with_different_routing(orc):
             assert max_abs <= MAX_ABS and rel_f <= REL_F, (i, max_abs, rel_f)
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("tokens", [600, 1100])
+def test_wide_and_narrow_token_tiles_together(orc, tokens):
+    """Enough tokens per expert for 128-token tiles (the kernel variant whose issuer warps share the epilogue),
+    with remainders that make narrow, double-buffered units in the same launch."""
+    run_case(orc, synth.CONFIGS["tiny_cover"], B.PW_MODE_TENSOR, tokens=tokens)
