@@ -78,13 +78,17 @@ struct Ctrl {                                  // lives at the start of dynamic 
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
 #ifdef PW_TC_PROFILE
-// Diagnostic build only: time stamps of the first few hundred items of CTA 0.
+// Diagnostic build only: time stamps of the first few hundred items of CTA 0 (of the gate/up kernel, or of the
+// down kernel with -DPW_TRACE_PHASE=1).
+#ifndef PW_TRACE_PHASE
+#define PW_TRACE_PHASE 0
+#endif
 __device__ long long g_trace[16][512];
 __device__ unsigned long long g_spins[32];      // polling-loop iterations per warp index, all CTAs
 #define TRACE(ev, n) \
-  if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
+  if (PHASE == PW_TRACE_PHASE && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
 #define TRACEV(ev, n, v) \
-  if (PHASE == 0 && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = (long long)(v)
+  if (PHASE == PW_TRACE_PHASE && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = (long long)(v)
 #else
 #define TRACE(ev, n)
 #define TRACEV(ev, n, v)
