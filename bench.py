@@ -384,6 +384,22 @@ def run_gpu(args):
     else:
         line["cpu_baseline"] = None
     if rank == 0 and world == 1 and not args.skip_extra:
+        # observation taps (routing mass, routed-input features): the same timed loop with the taps on
+        ctx.pw_observe(True)
+        for i in range(3):
+            step(i)
+        ms_obs = time_region(step, args.steps, device) / args.steps
+        ctx.pw_kernel_timing(True)
+        time_region(step, args.steps, device)
+        kt, kc = ctx.pw_get_kernel_times()
+        ctx.pw_kernel_timing(False)
+        mass, _ = ctx.pw_observation_summary(0)
+        R = T * k + cfg.n_shared * T
+        line["observe"] = {"ms_per_step_taps_on": ms_obs, "ms_per_step_taps_off": ms_step,
+                           "taps_kernels_ms": kt["observe"] / max(kc, 1),
+                           "bytes_read_per_call": 2.0 * R * (cfg.hidden + cfg.ffn),
+                           "mass_layer0_sum": float(mass.sum().item())}
+        ctx.pw_observe(False)
         line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
         del layers
         ctx.close()

@@ -232,6 +232,50 @@ pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* 
 pw_status pw_route_tokens_static(const float* router_logits, int T, int n_experts, int top_k, int32_t* topk_ids,
                                  float* gates, int32_t* counts, int32_t* offsets, int32_t* perm, pw_stream stream);
 
+/* ---- observation taps ---------------------------------------------------------------- */
+
+/* What a planner watches while the layer runs (Sec. 2.1, Sec. 3.2): the routing mass of every expert,
+ * Eq. 1, and for every linear-block the three routed-input features -- routing-weighted mean input norm,
+ * routing-weighted RMS input norm, maximum input norm -- of the tokens routed to the block's expert.
+ * Both are ratios of sums over the observed (token, choice) pairs, so the library keeps the sums: per
+ * layer and per expert segment s (routed experts, then shared experts) PW_OBS_FIELDS floats,
+ *   SUM_R     sum of the routing weights r (the gates) of the pairs routed to s; a shared expert takes
+ *             every token with r = 1
+ *   PAIRS     number of those pairs
+ *   SUM_R_NX, SUM_R_NX2, MAX_NX   sum r*|x|, sum r*|x|^2, max |x| with x the token's hidden state, the
+ *             input of the gate and up blocks
+ *   SUM_R_NH, SUM_R_NH2, MAX_NH   the same with h = silu(W_gate x) * (W_up x), the input of the down
+ *             block, as the forward call computed it (fp16)
+ * (the paper names the three features without a formula; |.| is the Euclidean norm).
+ *
+ * pw_observe(ctx, accumulators, stream): accumulators is a device array of
+ * n_layers * (n_experts + n_shared) * PW_OBS_FIELDS floats owned by the caller; the call zeroes it on
+ * `stream` and from then on every forward call of the context adds its tokens to the rows of its layer
+ * (two small kernels at the end of the call, ordered on the call's stream; sums in a fixed order).
+ * NULL switches the taps off.  The array must stay valid while the taps are on.
+ * Errors: INVALID_ARG, ALIGN, CUDA. */
+enum {
+  PW_OBS_SUM_R = 0,
+  PW_OBS_PAIRS = 1,
+  PW_OBS_SUM_R_NX = 2,
+  PW_OBS_SUM_R_NX2 = 3,
+  PW_OBS_MAX_NX = 4,
+  PW_OBS_SUM_R_NH = 5,
+  PW_OBS_SUM_R_NH2 = 6,
+  PW_OBS_MAX_NH = 7,
+  PW_OBS_FIELDS = 8
+};
+pw_status pw_observe(pw_ctx* ctx, float* accumulators, pw_stream stream);
+
+/* Turns the sums of one layer into the quantities themselves, on the device:
+ *   mass (device, [n_experts] fp32, may be NULL): m_e = SUM_R[e] / sum over the routed experts (Eq. 1),
+ *     zeros while nothing has been observed;
+ *   phi (device, [(n_experts + n_shared) * 3 * 3] fp32, may be NULL): for segment s and kind u the triple
+ *     (SUM_R_N / SUM_R, sqrt(SUM_R_N2 / SUM_R), MAX_N) at index (s * 3 + u) * 3, with the x sums for
+ *     PW_GATE and PW_UP and the h sums for PW_DOWN; zeros for an expert without tokens.
+ * Errors: INVALID_ARG, ALIGN, STATE (taps are off), CUDA. */
+pw_status pw_observation_summary(pw_ctx* ctx, int layer, float* mass, float* phi, pw_stream stream);
+
 /* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
  * then clears it. */
 pw_status pw_last_device_status(pw_ctx* ctx);
@@ -250,7 +294,8 @@ enum {
   PW_K_FFN_GATE_UP = 3,
   PW_K_FFN_DOWN = 4,
   PW_K_COMBINE = 5,
-  PW_NUM_KERNELS = 6
+  PW_K_OBSERVE = 6, /* the two kernels of the observation taps; ~0 while the taps are off */
+  PW_NUM_KERNELS = 7
 };
 pw_status pw_kernel_timing(pw_ctx* ctx, int enable);
 pw_status pw_get_kernel_times(pw_ctx* ctx, double* ms_out, uint64_t* calls_out);

@@ -27,9 +27,11 @@ GROUP = 128
 # every symbol include/pw.h declares
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
-           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_last_device_status", "pw_kernel_timing", "pw_get_kernel_times",
-           "pw_launch_count", "pw_status_str")
-KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine")
+           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_last_device_status",
+           "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_status_str")
+KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "observe")
+PW_OBS_FIELDS = 8
+OBS_FIELD_NAMES = ("sum_r", "pairs", "sum_r_nx", "sum_r_nx2", "max_nx", "sum_r_nh", "sum_r_nh2", "max_nh")
 
 
 class PwError(RuntimeError):
@@ -96,6 +98,10 @@ def load():
     L.pw_route_tokens_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     L.pw_get_routing.restype = i32
     L.pw_get_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.pw_observe.restype = i32
+    L.pw_observe.argtypes = [vp, vp, vp]
+    L.pw_observation_summary.restype = i32
+    L.pw_observation_summary.argtypes = [vp, i32, vp, vp, vp]
     L.pw_last_device_status.restype = i32
     L.pw_last_device_status.argtypes = [vp]
     L.pw_kernel_timing.restype = i32
@@ -196,11 +202,15 @@ class Context:
         with torch.cuda.device(self.device):
             _check(self.L.pw_create(C.byref(self.handle), C.byref(cfg)), "pw_create")
         self.n_segments = n_experts + n_shared
+        self._committed = {}          # (layer, expert, kind) -> the page the row points to
+        self.obs = None               # accumulators of the observation taps while they are on
 
     def close(self):
         if self.handle:
-            self.L.pw_destroy(self.handle)
+            self.L.pw_destroy(self.handle)      # waits for the device: nothing reads the pages any more
             self.handle = C.c_void_p()
+            self._committed = {}
+            self.obs = None
 
     def __del__(self):
         try:
@@ -251,6 +261,9 @@ class Context:
         epoch = C.c_uint64()
         _check(self.L.pw_set_page_table(self.handle, arr, len(entries), _stream_ptr(stream), C.byref(epoch)),
                "pw_set_page_table")
+        # the library only borrows page buffers: keep every committed page alive until its row is replaced
+        for layer, expert, kind, page in entries:
+            self._committed[(layer, expert, kind)] = page
         return int(epoch.value)
 
     def pw_query_row(self, layer: int, expert: int, kind: int) -> pw_table_entry:
@@ -297,6 +310,26 @@ class Context:
                                      r["counts"].data_ptr(), r["offsets"].data_ptr(), r["perm"].data_ptr(),
                                      _stream_ptr(stream)), "pw_get_routing")
         return r
+
+    def pw_observe(self, enable: bool = True, stream: Optional[torch.cuda.Stream] = None) -> Optional[torch.Tensor]:
+        """Switches the observation taps on (fresh, zeroed accumulators [n_layers, S, 8]) or off."""
+        if not enable:
+            _check(self.L.pw_observe(self.handle, None, _stream_ptr(stream)), "pw_observe")
+            self.obs = None
+            return None
+        S = self.cfg.n_experts + self.cfg.n_shared
+        self.obs = torch.empty(self.cfg.n_layers, S, PW_OBS_FIELDS, dtype=torch.float32, device=self.device)
+        _check(self.L.pw_observe(self.handle, self.obs.data_ptr(), _stream_ptr(stream)), "pw_observe")
+        return self.obs
+
+    def pw_observation_summary(self, layer: int, stream: Optional[torch.cuda.Stream] = None):
+        """(mass [E], phi [S, 3, 3]) of one layer, computed on the device from the accumulators."""
+        S = self.cfg.n_experts + self.cfg.n_shared
+        mass = torch.empty(self.cfg.n_experts, dtype=torch.float32, device=self.device)
+        phi = torch.empty(S, 3, 3, dtype=torch.float32, device=self.device)
+        _check(self.L.pw_observation_summary(self.handle, layer, mass.data_ptr(), phi.data_ptr(),
+                                             _stream_ptr(stream)), "pw_observation_summary")
+        return mass, phi
 
     def pw_last_device_status(self) -> int:
         return int(self.L.pw_last_device_status(self.handle))

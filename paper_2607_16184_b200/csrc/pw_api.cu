@@ -56,6 +56,7 @@ WsMap make_wsmap(const pw_config& c) {
   m.io_hidden = take((size_t)c.max_tokens * c.hidden * 2);
   m.io_logits = take((size_t)c.max_tokens * c.n_experts * 4);
   m.io_out = take((size_t)c.max_tokens * c.hidden * 4);
+  m.obs_part = take(4 * (size_t)kNormSplit * 2 * m.Rpad);
   m.total = o;
   return m;
 }
@@ -114,6 +115,7 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   ctx->timing_ev = nullptr;
   ctx->timing_cur = 0;
   ctx->timing_calls = 0;
+  ctx->obs_acc = nullptr;
   for (int i = 0; i < pw_ctx::kTimingSlots; ++i) ctx->timing_busy[i] = false;
   for (int i = 0; i < PW_NUM_KERNELS; ++i) ctx->timing_ms[i] = 0.0;
   const size_t nrows = (size_t)cfg->n_layers * m.S * 3;
@@ -287,6 +289,8 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
                             : launch_ffn_tensor(ctx, layer, T, top_k, nt_tile, ksplit, stream);
   if (st != PW_OK) return st;
   st = launch_combine(ctx, T, top_k, ksplit, out, stream);
+  if (st != PW_OK) return st;
+  st = launch_observe(ctx, layer, T, top_k, stream);
   ctx->last_T = T;
   ctx->last_k = top_k;
   return st;

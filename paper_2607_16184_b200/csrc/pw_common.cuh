@@ -13,6 +13,7 @@ namespace pw {
 constexpr int kGroup = 128;      // weights per quantization group
 constexpr int kTileRows = 128;   // rows of one page tile
 constexpr int kPadRows = 256;    // zero rows appended to the token-major operand buffers
+constexpr int kNormSplit = 8;    // observation taps: the squares of an operand row are summed in this many slices
 
 // One row of the device-resident page table (48 bytes).
 struct DevRow {
@@ -58,6 +59,7 @@ struct WsMap {
   size_t io_hidden;   // fp16 [Tmax][H]   device staging of pw_moe_forward_host
   size_t io_logits;   // float [Tmax][E]
   size_t io_out;      // float [Tmax][H]
+  size_t obs_part;    // float [8][2][Rpad]  partial squared norms of the operand rows (observation taps)
   size_t total;
   // derived sizes
   int S;              // segments = E + n_shared
@@ -105,6 +107,7 @@ struct pw_ctx {
   int timing_cur;                 // slot of the forward call being enqueued
   uint64_t timing_calls;
   double timing_ms[PW_NUM_KERNELS];
+  float* obs_acc;                 // observation accumulators of the caller (device), or null: taps off
 };
 
 #define PW_CUDA_OK(expr)                                   \
@@ -119,6 +122,7 @@ namespace pw {
 pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
                        int ksplit, cudaStream_t s);
 pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cudaStream_t s);
+pw_status launch_observe(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
 int tensor_token_tile(const pw_ctx* ctx, int T, int k);

@@ -338,7 +338,6 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
                               reinterpret_cast<const float*>(b + w.gates),
                               reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
                               (size_t)R * H4, reinterpret_cast<float4*>(out)));
-  timing_mark(ctx, PW_NUM_KERNELS, s);
   ctx->launches += 1;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;

@@ -110,7 +110,7 @@ def test_forward_from_imported_oracle_pages(orc):
 def test_router_ties_follow_the_index_rule(orc):
     cfg = synth.CONFIGS["tiny"]
     ctx = make_ctx(cfg, max_tokens=64, n_layers=1)
-    build_layer(ctx, cfg, 0, np.full((8, 3), 4, np.int32))
+    pages, _ = build_layer(ctx, cfg, 0, np.full((8, 3), 4, np.int32))
     x = synth.activations(cfg, device="cuda", tokens=64)
     logits = torch.round(synth.router_logits(cfg, device="cuda", tokens=64) * 2) / 2     # many exact ties
     logits[0] = 0.0
@@ -198,7 +198,7 @@ def test_forward_is_bitwise_reproducible(mode):
     T = 48
     ctx = make_ctx(cfg, max_tokens=T, n_layers=1)
     try:
-        build_layer(ctx, cfg, 0, None)
+        pages, _ = build_layer(ctx, cfg, 0, None)
         x = synth.activations(cfg, device="cuda", tokens=T)
         logits = synth.router_logits(cfg, device="cuda", tokens=T)
         first = ctx.pw_moe_forward(0, x, logits, cfg.top_k, mode=mode).clone()

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 def reference_routing(cfg, logits, T):
     ctx = make_ctx(cfg, max_tokens=T, n_layers=1)
-    build_layer(ctx, cfg, 0, np.full((cfg.n_experts + cfg.n_shared, 3), 16, np.int32))
+    pages, _ = build_layer(ctx, cfg, 0, np.full((cfg.n_experts + cfg.n_shared, 3), 16, np.int32))
     x = synth.activations(cfg, device="cuda", tokens=T)
     ctx.pw_moe_forward(0, x, logits, cfg.top_k)
     r = {k: v.clone() for k, v in ctx.pw_get_routing(T, cfg.top_k).items()}
