@@ -260,6 +260,75 @@ def run_demote(ctx, cfg, layers, device, peaks, decode_fn, decode_ms):
                              "demote_16to4_gbs_side_stream": gbs(b16 + b4, ms_side), "steps": n_steps}}
 
 
+def run_residency(ctx, cfg, layers, device, decode_fn, decode_ms):
+    """pw_offload_page / pw_reload_page of 16-bit blocks (rows whose committed bitwidth is lower): each direction
+    alone, against a plain pinned copy of the same size, and both directions on a side stream under decode."""
+    from paper_2607_16184_b200 import binding as B
+    rows, cols = cfg.block_shape(0)
+    nbytes = B.pw_page_bytes(rows, cols, 16)[0]
+    bits = layers[0]["bits"]
+    targets = [(0, e, u) for e in range(cfg.n_experts) for u in (0, 1) if int(bits[e, u]) != 16][:6]
+    if not targets:
+        return None
+    page = ctx.pw_quantize_block(synth.block_weights(cfg, 200, 0, 0, device=device), 16)
+    hosts = [torch.empty(nbytes, dtype=torch.uint8).pin_memory() for _ in targets]
+    side = torch.cuda.Stream(device=device)
+    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
+
+    def timed_side(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(device)
+        a.record(side)
+        fn()
+        b.record(side)
+        side.synchronize()
+        return a.elapsed_time(b)
+
+    # the link itself: the same bytes with a plain asynchronous copy
+    with torch.cuda.stream(side):
+        ms_d2h = timed_side(lambda: [hosts[i].copy_(page.codes, non_blocking=True) for i in range(len(targets))])
+        ms_h2d = timed_side(lambda: [page.codes.copy_(hosts[i], non_blocking=True) for i in range(len(targets))])
+    ms_off = timed_side(lambda: [ctx.pw_offload_page(*t, page, stream=side, host=hosts[i]) for i, t in enumerate(targets)])
+    assert all(ctx.pw_page_state(*t, 16) == B.PW_STATE_CPU_RESIDENT for t in targets)
+    back = []
+    ms_rel = timed_side(lambda: back.extend(ctx.pw_reload_page(*t, 16, hosts[i], stream=side) for i, t in enumerate(targets)))
+    assert all(ctx.pw_page_state(*t, 16) == B.PW_STATE_GPU_RESIDENT for t in targets)
+    assert torch.equal(back[-1].codes, page.codes)
+    total = nbytes * len(targets)
+    # under decode: every step one page moves (out if it is resident, back in if it is away), on the side stream
+    n_steps, moved = 240, 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(device)
+    e0.record()
+    s0.record(side)
+    for i in range(n_steps):
+        j = i % len(targets)
+        st = ctx.pw_page_state(*targets[j], 16)
+        if st == B.PW_STATE_GPU_RESIDENT:
+            ctx.pw_offload_page(*targets[j], back[j], stream=side, host=hosts[j])
+            moved += nbytes
+        elif st == B.PW_STATE_CPU_RESIDENT:
+            back[j] = ctx.pw_reload_page(*targets[j], 16, hosts[j], stream=side)
+            moved += nbytes
+        decode_fn(i)
+    e1.record()
+    s1.record(side)
+    torch.cuda.synchronize(device)
+    ms_dec = e0.elapsed_time(e1) / n_steps
+    ms_side = s0.elapsed_time(s1)
+    for t in targets:                                  # leave no record behind for the rest of the run
+        if ctx.pw_page_state(*t, 16) != B.PW_STATE_IN_TRANSFER:
+            ctx.pw_drop_page(*t, 16)
+    return {"block": "%dx%d at 16 bits, %d bytes, %d pages per measurement" % (rows, cols, nbytes, len(targets)),
+            "offload_gbs": gbs(total, ms_off), "reload_gbs": gbs(total, ms_rel),
+            "plain_copy_d2h_gbs": gbs(total, ms_d2h), "plain_copy_h2d_gbs": gbs(total, ms_h2d),
+            "under_decode": {"decode_ms_per_step": ms_dec, "decode_ms_alone": decode_ms,
+                             "decode_slowdown": 1.0 - decode_ms / ms_dec if ms_dec > 0 else None,
+                             "moved_gbs_side_stream": gbs(moved, ms_side), "moved_bytes": moved,
+                             "steps": n_steps}}
+
+
 def run_gpu(args):
     from paper_2607_16184_b200 import binding as B
     from paper_2607_16184_b200 import build as pwbuild
@@ -401,6 +470,7 @@ def run_gpu(args):
                            "mass_layer0_sum": float(mass.sum().item())}
         ctx.pw_observe(False)
         line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
+        line["residency"] = run_residency(ctx, cfg, layers, device, step, ms_step)
         del layers
         ctx.close()
         torch.cuda.empty_cache()

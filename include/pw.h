@@ -69,7 +69,12 @@ typedef enum {
 enum { PW_LAYOUT_CANONICAL = 0, PW_LAYOUT_TILED = 1 };
 
 /* Residency state of a page-table row (Sec. 3.1).  Only GPU_RESIDENT rows can be used. */
-enum { PW_STATE_GPU_RESIDENT = 0, PW_STATE_CPU_RESIDENT = 1, PW_STATE_IN_TRANSFER = 2 };
+enum {
+  PW_STATE_GPU_RESIDENT = 0,
+  PW_STATE_CPU_RESIDENT = 1,
+  PW_STATE_IN_TRANSFER = 2,
+  PW_STATE_NONE = 3 /* pw_page_state only: the library knows no page of the row at that bitwidth */
+};
 
 typedef struct CUstream_st* pw_stream; /* a cudaStream_t */
 typedef struct pw_ctx pw_ctx;
@@ -170,7 +175,8 @@ pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst
  * may be released once work enqueued before this call has finished.  entries: host.  epoch_out
  * (optional, host) receives the table epoch after the update; each call increments it by one.
  * Errors: INVALID_ARG, SHAPE (page shape does not match kind and ctx), BITS, ALIGN,
- * STATE (layout not TILED, state not GPU_RESIDENT, shared expert below 16 bits), CUDA. */
+ * STATE (layout not TILED, state not GPU_RESIDENT, the page of the row at that bitwidth is CPU_RESIDENT or
+ * IN_TRANSFER, shared expert below 16 bits), CUDA. */
 pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entries, size_t n, pw_stream stream,
                             uint64_t* epoch_out);
 
@@ -179,6 +185,44 @@ const pw_page_table* pw_get_page_table(pw_ctx* ctx);
 
 /* Host-side query of a committed row (what the last pw_set_page_table published). */
 pw_status pw_query_row(pw_ctx* ctx, int layer, int expert, int kind, pw_table_entry* out);
+
+/* ---- page residency: offload and reload ------------------------------------------------ */
+
+/* The rest of a page's life-cycle (Sec. 3.1; Sec. 3.3, asynchronous page movement).  For every row and
+ * every bitwidth the library keeps the residency state of the row's page at that bitwidth: a page
+ * becomes GPU_RESIDENT when it is published with pw_set_page_table, and the calls below move it.  The
+ * paper's two ordering rules are enforced on the host, before anything is enqueued:
+ *   - offload: the committed bitwidth is lowered first, then the page that is no longer needed moves
+ *     out -- the page a row is committed to cannot be offloaded (STATE);
+ *   - reload: the page moves back first; pw_set_page_table refuses (STATE) a bitwidth whose page is
+ *     CPU_RESIDENT or IN_TRANSFER, and accepts it once pw_page_state reports GPU_RESIDENT.
+ * A TILED page is one buffer, so each direction is one asynchronous copy on `stream` (use a side stream
+ * to overlap it with forward calls); host buffers should be pinned and are owned by the caller.
+ *
+ * pw_offload_page: copies `page` (device, TILED, pw_page_bytes bytes) of row (layer, expert, kind) to
+ * host_dst; the page is IN_TRANSFER until the copy has finished, then CPU_RESIDENT.  The caller may
+ * release the device buffer once pw_page_state reports CPU_RESIDENT and every forward call enqueued
+ * before the commit that moved the row off this page has finished.
+ * Errors: INVALID_ARG, SHAPE, BITS, ALIGN, STATE (not TILED; the row is committed to this page; the page
+ * is already away or on its way), CUDA.
+ *
+ * pw_reload_page: copies the page of the row at `bits` from host_src (the buffer it was offloaded to)
+ * into dst->codes (device, caller-allocated, pw_page_bytes bytes) and fills dst's header; IN_TRANSFER
+ * until the copy has finished, then GPU_RESIDENT and ready for pw_set_page_table.
+ * Errors: INVALID_ARG (also: host_src is not the buffer of the offload), SHAPE, BITS, ALIGN,
+ * STATE (the page is not CPU_RESIDENT), CUDA.
+ *
+ * pw_page_state: the state now (looks at the transfer's event; never blocks); PW_STATE_NONE if the
+ * library knows no page of the row at that bitwidth.
+ *
+ * pw_drop_page: forgets the page of the row at `bits` (its host copy is abandoned, or the caller is about
+ * to build a new page at that bitwidth).  Errors: STATE (the row is committed to it; it is in transfer). */
+pw_status pw_offload_page(pw_ctx* ctx, int layer, int expert, int kind, const pw_page* page, void* host_dst,
+                          pw_stream stream);
+pw_status pw_reload_page(pw_ctx* ctx, int layer, int expert, int kind, int bits, const void* host_src, pw_page* dst,
+                         pw_stream stream);
+pw_status pw_page_state(pw_ctx* ctx, int layer, int expert, int kind, int bits, int* state_out);
+pw_status pw_drop_page(pw_ctx* ctx, int layer, int expert, int kind, int bits);
 
 /* ---- forward ------------------------------------------------------------------------ */
 

@@ -21,12 +21,13 @@ STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_SHAPE", 3: "PW_E
 PW_GATE, PW_UP, PW_DOWN = 0, 1, 2
 PW_MODE_AUTO, PW_MODE_SIMT, PW_MODE_TENSOR = 0, 1, 2
 PW_LAYOUT_CANONICAL, PW_LAYOUT_TILED = 0, 1
-PW_STATE_GPU_RESIDENT, PW_STATE_CPU_RESIDENT, PW_STATE_IN_TRANSFER = 0, 1, 2
+PW_STATE_GPU_RESIDENT, PW_STATE_CPU_RESIDENT, PW_STATE_IN_TRANSFER, PW_STATE_NONE = 0, 1, 2, 3
 GROUP = 128
 
 # every symbol include/pw.h declares
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
+           "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
            "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_last_device_status",
            "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_status_str")
 KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "observe")
@@ -90,6 +91,14 @@ def load():
     L.pw_get_page_table.argtypes = [vp]
     L.pw_query_row.restype = i32
     L.pw_query_row.argtypes = [vp, i32, i32, i32, C.POINTER(pw_table_entry)]
+    L.pw_offload_page.restype = i32
+    L.pw_offload_page.argtypes = [vp, i32, i32, i32, C.POINTER(pw_page), vp, vp]
+    L.pw_reload_page.restype = i32
+    L.pw_reload_page.argtypes = [vp, i32, i32, i32, i32, vp, C.POINTER(pw_page), vp]
+    L.pw_page_state.restype = i32
+    L.pw_page_state.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_int)]
+    L.pw_drop_page.restype = i32
+    L.pw_drop_page.argtypes = [vp, i32, i32, i32, i32]
     L.pw_moe_forward.restype = i32
     L.pw_moe_forward.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp]
     L.pw_moe_forward_host.restype = i32
@@ -270,6 +279,35 @@ class Context:
         out = pw_table_entry()
         _check(self.L.pw_query_row(self.handle, layer, expert, kind, C.byref(out)), "pw_query_row")
         return out
+
+    # ---- residency ----
+    def pw_offload_page(self, layer: int, expert: int, kind: int, page: Page,
+                        stream: Optional[torch.cuda.Stream] = None, host: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Starts the copy of a (not committed) page to pinned host memory; returns the host buffer."""
+        nbytes = pw_page_bytes(page.rows, page.cols, page.bits)[0]
+        if host is None:
+            host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+        assert host.numel() >= nbytes and not host.is_cuda
+        _check(self.L.pw_offload_page(self.handle, layer, expert, kind, C.byref(page.c), host.data_ptr(),
+                                      _stream_ptr(stream)), "pw_offload_page")
+        return host
+
+    def pw_reload_page(self, layer: int, expert: int, kind: int, bits: int, host: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> Page:
+        """Starts the copy of an offloaded page back into a fresh device buffer; returns the page."""
+        rows, cols = (self.cfg.hidden, self.cfg.ffn) if kind == PW_DOWN else (self.cfg.ffn, self.cfg.hidden)
+        dst = Page(rows, cols, bits, self.device)
+        _check(self.L.pw_reload_page(self.handle, layer, expert, kind, bits, host.data_ptr(), C.byref(dst.c),
+                                     _stream_ptr(stream)), "pw_reload_page")
+        return dst
+
+    def pw_page_state(self, layer: int, expert: int, kind: int, bits: int) -> int:
+        st = C.c_int()
+        _check(self.L.pw_page_state(self.handle, layer, expert, kind, bits, C.byref(st)), "pw_page_state")
+        return int(st.value)
+
+    def pw_drop_page(self, layer: int, expert: int, kind: int, bits: int):
+        _check(self.L.pw_drop_page(self.handle, layer, expert, kind, bits), "pw_drop_page")
 
     # ---- forward ----
     def pw_moe_forward(self, layer: int, hidden: torch.Tensor, router_logits: torch.Tensor, top_k: int,

@@ -79,10 +79,6 @@ void timing_mark(pw_ctx* ctx, int i, cudaStream_t s) {
   cudaEventRecord(ctx->timing_ev[(size_t)ctx->timing_cur * (PW_NUM_KERNELS + 1) + i], s);
 }
 
-static size_t row_index(const pw_ctx* ctx, int layer, int expert, int kind) {
-  return ((size_t)layer * ctx->ws.S + expert) * 3 + kind;
-}
-
 }  // namespace pw
 
 using namespace pw;
@@ -122,12 +118,14 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   ctx->stage_rows = nrows;
   ctx->host_rows = new (std::nothrow) pw_table_entry[nrows]();
   ctx->host_valid = new (std::nothrow) uint8_t[nrows]();
+  ctx->records = new (std::nothrow) PageRecord[nrows * kBitLevels]();
+  for (size_t i = 0; ctx->records && i < nrows * kBitLevels; ++i) ctx->records[i].state = PW_STATE_NONE;
   for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
     ctx->stage[i] = nullptr;
     ctx->stage_ev[i] = nullptr;
     ctx->stage_used[i] = false;
   }
-  bool ok = ctx->host_rows && ctx->host_valid;
+  bool ok = ctx->host_rows && ctx->host_valid && ctx->records;
   int dev = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess;
   ok = ok && cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
@@ -159,6 +157,7 @@ extern "C" pw_status pw_destroy(pw_ctx* ctx) {
       if (ctx->timing_ev[i]) cudaEventDestroy(ctx->timing_ev[i]);
     delete[] ctx->timing_ev;
   }
+  residency_teardown(ctx);
   delete[] ctx->host_rows;
   delete[] ctx->host_valid;
   delete ctx;
@@ -184,6 +183,9 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
     if (p.layout != PW_LAYOUT_TILED || e.state != PW_STATE_GPU_RESIDENT) return PW_ERR_STATE;
     if (e.expert >= c.n_experts && p.bits != 16) return PW_ERR_STATE;
     if (e.desired_bits != 0 && !bits_ok(e.desired_bits)) return PW_ERR_BITS;
+    // q_i is only set to a bitwidth whose page is GPU-resident (Sec. 3.1): not while it is away or on its way
+    const pw_status rs = residency_check_commit(ctx, row_index(ctx, e.layer, e.expert, e.kind), p);
+    if (rs != PW_OK) return rs;
   }
   if (n) {
     const int slot = ctx->stage_next;
@@ -204,6 +206,7 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       const size_t idx = row_index(ctx, e.layer, e.expert, e.kind);
       ctx->host_rows[idx] = e;
       ctx->host_valid[idx] = 1;
+      residency_note_commit(ctx, idx, e.page);
       const bool last = i + 1 == n;
       const bool contiguous =
           !last && row_index(ctx, entries[i + 1].layer, entries[i + 1].expert, entries[i + 1].kind) == idx + 1;

@@ -80,6 +80,21 @@ struct pw_page_table {
   pw_ctx* owner;
 };
 
+namespace pw {
+// Residency record of the page of one page-table row at one bitwidth (Sec. 3.1: GPU-resident, CPU-resident
+// or in transfer).  A transfer is a copy enqueued on a stream plus an event behind it; the record moves on
+// to `heading` when a later call finds the event complete.
+constexpr int kBitLevels = 5;                      // 16, 8, 4, 3, 2
+struct PageRecord {
+  uint8_t state;        // PW_STATE_*
+  uint8_t heading;      // state the page reaches when its transfer has finished
+  void* dev;            // device buffer (GPU-resident, or source / target of the transfer)
+  void* host;           // host buffer (CPU-resident, or target / source of the transfer)
+  cudaEvent_t ev;       // created on first use
+};
+inline int bit_level(int bits) { return bits == 16 ? 0 : bits == 8 ? 1 : bits == 4 ? 2 : bits == 3 ? 3 : bits == 2 ? 4 : -1; }
+}  // namespace pw
+
 struct pw_ctx {
   pw_config cfg;
   pw::WsMap ws;
@@ -108,7 +123,14 @@ struct pw_ctx {
   uint64_t timing_calls;
   double timing_ms[PW_NUM_KERNELS];
   float* obs_acc;                 // observation accumulators of the caller (device), or null: taps off
+  pw::PageRecord* records;        // [rows of the table][kBitLevels]
 };
+
+namespace pw {
+inline size_t row_index(const pw_ctx* ctx, int layer, int expert, int kind) {
+  return ((size_t)layer * ctx->ws.S + expert) * 3 + kind;
+}
+}  // namespace pw
 
 #define PW_CUDA_OK(expr)                                   \
   do {                                                     \
@@ -123,6 +145,12 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
                        int ksplit, cudaStream_t s);
 pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cudaStream_t s);
 pw_status launch_observe(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
+// residency records: the state of (row, bits) after looking at its transfer event; registration of a page
+// that is being committed (PW_ERR_STATE if the record says that page is away or on its way)
+int residency_poll(pw_ctx* ctx, size_t row, int bits);
+pw_status residency_check_commit(pw_ctx* ctx, size_t row, const pw_page& page);
+void residency_note_commit(pw_ctx* ctx, size_t row, const pw_page& page);
+void residency_teardown(pw_ctx* ctx);
 pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
 int tensor_token_tile(const pw_ctx* ctx, int T, int k);
