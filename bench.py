@@ -345,7 +345,7 @@ def run_gpu(args):
     if args.uniform_bits:
         import dataclasses
         cfg = dataclasses.replace(cfg, bit_rule="uniform%d" % args.uniform_bits)
-    L = args.layers
+    L = args.layers or (8 if cfg.name in ("latency_b1", "latency_b4", "manyexpert_decode") else 3)
     ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
     layers = build_layers(ctx, cfg, L, device)
     T, k = cfg.tokens, cfg.top_k
@@ -687,8 +687,11 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode", "demote_under_load"])
-    ap.add_argument("--layers", type=int, default=3, help="distinct layer copies the decode loop rotates over")
+    ap.add_argument("--config", default="mixtral_decode", choices=["mixtral_decode", "finegrained_decode", "demote_under_load", "latency_b1", "latency_b4",
+                             "manyexpert_decode"])
+    ap.add_argument("--layers", type=int, default=0,
+                    help="distinct layer copies the decode loop rotates over (default: 3, or 8 for the small-batch "
+                         "configurations, whose calls read less than the L2 holds)")
     ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
     ap.add_argument("--cpu-tokens", type=int, default=64)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="oracle time to spend on the cpu_baseline sample")

@@ -254,40 +254,62 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
 }
 
 // out[t] = sum_j gate[t,j] * (sum_s y[s][inv_perm[t*k+j]]) + sum over shared experts (sum_s y[s][row]).
-__global__ void __launch_bounds__(256) combine_kernel(const float4* __restrict__ y, const float* __restrict__ gates,
-                                                      const int32_t* __restrict__ inv_perm, int T, int k, int n_shared,
-                                                      int H4, int ksplit, size_t split_stride4,
-                                                      float4* __restrict__ out) {
+// A CTA takes 64 float4 columns of one token; its four thread rows each form the term of one expert choice at
+// a time (all split-K partials are loaded before they are added, in split order), and thread row 0 adds the
+// terms in choice order: the arithmetic and its order do not depend on the launch shape, only the latency does
+// (a one-token call has a handful of CTAs, so a serial walk over choices x splits would be all latency).
+constexpr int kCombineCols = 64, kCombineRows = 4, kMaxSplit = 8;
+__global__ void __launch_bounds__(kCombineCols * kCombineRows)
+    combine_kernel(const float4* __restrict__ y, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
+                   int T, int k, int n_shared, int H4, int ksplit, size_t split_stride4, float4* __restrict__ out) {
   grid_dep_sync();
   grid_dep_trigger();
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  __shared__ float4 term[kCombineRows][kCombineCols];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int c = blockIdx.x * kCombineCols + tx;
   const int t = blockIdx.y;
-  if (c >= H4) return;
+  const int J = k + n_shared;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j = 0; j < k + n_shared; ++j) {
-    int row;
-    float g;
-    if (j < k) {
-      row = inv_perm[(size_t)t * k + j];
-      g = gates[(size_t)t * k + j];
-    } else {
-      row = T * k + (j - k) * T + t;
-      g = 1.0f;
+  for (int j0 = 0; j0 < J; j0 += kCombineRows) {
+    const int j = j0 + ty;
+    if (j < J && c < H4) {
+      int row;
+      float g;
+      if (j < k) {
+        row = inv_perm[(size_t)t * k + j];
+        g = gates[(size_t)t * k + j];
+      } else {
+        row = T * k + (j - k) * T + t;
+        g = 1.0f;
+      }
+      float4 v[kMaxSplit];
+#pragma unroll
+      for (int s = 0; s < kMaxSplit; ++s)
+        if (s < ksplit) v[s] = y[s * split_stride4 + (size_t)row * H4 + c];
+      float4 a = v[0];
+#pragma unroll
+      for (int s = 1; s < kMaxSplit; ++s)
+        if (s < ksplit) {
+          a.x = __fadd_rn(a.x, v[s].x);
+          a.y = __fadd_rn(a.y, v[s].y);
+          a.z = __fadd_rn(a.z, v[s].z);
+          a.w = __fadd_rn(a.w, v[s].w);
+        }
+      term[ty][tx] = make_float4(__fmul_rn(g, a.x), __fmul_rn(g, a.y), __fmul_rn(g, a.z), __fmul_rn(g, a.w));
     }
-    float4 a = y[(size_t)row * H4 + c];
-    for (int s = 1; s < ksplit; ++s) {
-      const float4 b = y[s * split_stride4 + (size_t)row * H4 + c];
-      a.x = __fadd_rn(a.x, b.x);
-      a.y = __fadd_rn(a.y, b.y);
-      a.z = __fadd_rn(a.z, b.z);
-      a.w = __fadd_rn(a.w, b.w);
+    __syncthreads();
+    if (ty == 0) {
+      for (int i = 0; i < kCombineRows && j0 + i < J; ++i) {
+        const float4 b = term[i][tx];
+        acc.x = __fadd_rn(acc.x, b.x);
+        acc.y = __fadd_rn(acc.y, b.y);
+        acc.z = __fadd_rn(acc.z, b.z);
+        acc.w = __fadd_rn(acc.w, b.w);
+      }
     }
-    acc.x = __fadd_rn(acc.x, __fmul_rn(g, a.x));
-    acc.y = __fadd_rn(acc.y, __fmul_rn(g, a.y));
-    acc.z = __fadd_rn(acc.z, __fmul_rn(g, a.z));
-    acc.w = __fadd_rn(acc.w, __fmul_rn(g, a.w));
+    __syncthreads();
   }
-  out[(size_t)t * H4 + c] = acc;
+  if (ty == 0 && c < H4) out[(size_t)t * H4 + c] = acc;
 }
 
 pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
@@ -332,9 +354,9 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
   char* b = ctx->base;
   const int H4 = c.hidden / 4;
   const int R = T * k + c.n_shared * T;
-  dim3 grid((H4 + 255) / 256, T);
+  dim3 grid((H4 + kCombineCols - 1) / kCombineCols, T);
   timing_mark(ctx, PW_K_COMBINE, s);
-  PW_CUDA_OK(launch_dependent(combine_kernel, grid, dim3(256), 0, s, reinterpret_cast<const float4*>(b + w.y),
+  PW_CUDA_OK(launch_dependent(combine_kernel, grid, dim3(kCombineCols, kCombineRows), 0, s, reinterpret_cast<const float4*>(b + w.y),
                               reinterpret_cast<const float*>(b + w.gates),
                               reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
                               (size_t)R * H4, reinterpret_cast<float4*>(out)));

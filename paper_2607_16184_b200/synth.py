@@ -61,6 +61,14 @@ CONFIGS: Dict[str, LayerConfig] = {
                                       zipf_a=1.2, bit_rule="int4_10fp16_20int2"),
     # configs[3]: 8-expert top-2 prefill, 4096 tokens, uniform-random routing, bits from {16,8,4}
     "mixtral_prefill": LayerConfig("mixtral_prefill", 8, 2, 4096, 14336, 4096, routing="gumbel", bit_rule="iid3"),
+    # latency decode (Table 3 of the paper: batch 1 and batch 4) on a 60 routed top-4 + 4 shared layer
+    "latency_b1": LayerConfig("latency_b1", 60, 4, 2048, 1408, 1, n_shared=4, routing="normal",
+                              bit_rule="mix_25_25_30_10_10"),
+    "latency_b4": LayerConfig("latency_b4", 60, 4, 2048, 1408, 4, n_shared=4, routing="normal",
+                              bit_rule="mix_25_25_30_10_10"),
+    # many small experts (Table 1: 128 routed + 1 shared, top-8); hidden and FFN sizes are stand-ins
+    "manyexpert_decode": LayerConfig("manyexpert_decode", 128, 8, 2048, 768, 64, n_shared=1, routing="zipf",
+                                     zipf_a=1.2, bit_rule="int4_10fp16_20int2"),
     # configs[4]: 32 stacked layers, all fp16 at start, 1/3 of the blocks demoted 16->4->2 under load
     "demote_under_load": LayerConfig("demote_under_load", 8, 2, 4096, 14336, 64, n_layers=32, routing="zipf",
                                      zipf_a=1.1, bit_rule="all16"),

@@ -60,3 +60,13 @@ def test_finegrained_decode_full_size(orc):
 
 def test_mixtral_prefill_full_size(orc):
     full_case(orc, "mixtral_prefill", 8, [(5, 1)])
+
+
+@pytest.mark.parametrize("name", ["latency_b1", "latency_b4"])
+def test_latency_decode_full_size(orc, name):
+    # batch 1 and batch 4 on the 60 + 4 expert layer: every token is checked
+    full_case(orc, name, 4, [(0, 0), (33, 2), (61, 1)])
+
+
+def test_manyexpert_decode_full_size(orc):
+    full_case(orc, "manyexpert_decode", 24, [(0, 0), (77, 1), (128, 2)])
