@@ -262,20 +262,21 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
     const int R = T * top_k + c.n_shared * T;
     const int active = ctx->ws.S < R ? ctx->ws.S : R;
     const long long tiles = (long long)active * ((R / active + nt_tile - 1) / nt_tile) * (c.hidden / kTileRows);
-    // Pick the split (1..8) whose unit count fills whole rounds of one CTA per SM best; at least three
-    // rounds so that the pipeline of a CTA stays fed, and on ties the smaller split (less partial traffic).
+    // Pick the split (1..8) that finishes soonest under a simple cost model: the CTAs (one per SM) work through
+    // ceil(units / SMs) rounds of units, and a unit costs a fixed part -- claiming it, the accumulator
+    // hand-over, the epilogue: about three tiles' worth of time, measured -- plus one part per 128-wide tile of
+    // its K range.  A finer split fills the last round better but multiplies the fixed parts, so it only pays
+    // when units are long (an 8-expert layer with F = 14336: split 4); layers with short contractions or many
+    // small experts are fastest unsplit.  On ties the smaller split (less partial traffic).
     const int ng = c.ffn / kGroup;
     const long long G = ctx->num_sms;
-    long long want = 1;
-    double best = -1.0;
+    long long want = 1, best = -1;
     for (int ks = 1; ks <= 8 && ks <= ng; ++ks) {
       if ((size_t)ks * R > ctx->ws.y_slots) break;
-      const long long units = tiles * ks;
-      const long long rounds = (units + G - 1) / G;
-      double eff = (double)units / (double)(rounds * G);
-      if (rounds < 3) eff *= 0.5 + 0.15 * (double)rounds;       // too few units per SM: prefer a finer split
-      if (eff > best + 1e-9) {
-        best = eff;
+      const long long rounds = (tiles * ks + G - 1) / G;
+      const long long cost = rounds * (3 + (ng + ks - 1) / ks);
+      if (best < 0 || cost < best) {
+        best = cost;
         want = ks;
       }
     }
