@@ -483,9 +483,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = c->tmem_base;
-  // This CTA may have been placed while the kernel before this one is still finishing on other SMs.  Unit
-  // lists, work counters and page-table rows were written earlier in the chain and are final (see
-  // grid_dep_sync); the token rows are not: the token-tile producer waits for them, everybody else starts.
+  // This CTA may have been placed while the kernel before this one is still finishing on other SMs.  Work
+  // counters, page-table rows and the unit counts were written two or more kernels back and are final (see
+  // grid_dep_sync).  What the kernel directly ahead writes is not: the token rows (both kernels; the
+  // token-tile producer waits for them) and the gate/up unit list (PHASE 0; the weight producers wait).
 
   // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
   // (the weight producer claims, the other roles follow its list).
@@ -503,6 +504,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       uint32_t pass = 0;                           // seq / n_slots
       const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]);
       bool ok = true;
+      // The gate/up kernel's unit list is written by the kernel directly ahead of it (the one that gathers
+      // the token rows), which may still be running: the producers wait for it before they read a unit, and
+      // every other role learns of its first unit from producer 0 only after that.  The down kernel's list is
+      // two kernels back and final (see grid_dep_sync), so its producers stream at once.
+      if (PHASE == 0) grid_dep_sync();
       // the work list: unit blockIdx.x first, then whatever the global counter hands out
       int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
       if (P == 0) {
