@@ -469,6 +469,26 @@ def run_gpu(args):
                            "bytes_read_per_call": 2.0 * R * (cfg.hidden + cfg.ffn),
                            "mass_layer0_sum": float(mass.sum().item())}
         ctx.pw_observe(False)
+        # the same step with each layer's forward call replayed from a CUDA graph (the commit stays eager)
+        graphs = []
+        torch.cuda.synchronize(device)
+        for li, lay in enumerate(layers):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                ctx.pw_moe_forward(li, lay["x"], lay["logits"], k, out=out, mode=mode)
+            graphs.append(g)
+
+        def step_graph(i):
+            lay = layers[i % L]
+            ctx.pw_set_page_table(lay["entries"][(i // L) % len(lay["entries"]):][:1])
+            graphs[i % L].replay()
+
+        for i in range(3):
+            step_graph(i)
+        ms_graph = time_region(step_graph, args.steps, device) / args.steps
+        line["cuda_graph"] = {"ms_per_step": ms_graph, "tokens_per_s": T / (ms_graph * 1e-3),
+                              "ms_per_step_eager": ms_step}
+        del graphs
         line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
         line["residency"] = run_residency(ctx, cfg, layers, device, step, ms_step)
         del layers

@@ -243,3 +243,30 @@ def test_wide_and_narrow_token_tiles_together(orc, tokens):
     """Enough tokens per expert for 128-token tiles (the kernel variant whose issuer warps share the epilogue),
     with remainders that make narrow, double-buffered units in the same launch."""
     run_case(orc, synth.CONFIGS["tiny_cover"], B.PW_MODE_TENSOR, tokens=tokens)
+
+
+def test_forward_call_replays_from_a_cuda_graph(orc):
+    """A layer call is six dependent launches; captured once into a CUDA graph it replays on new contents of
+    the same buffers (what a launch-bound decode loop does) and returns the bits of the eager call."""
+    cfg = synth.CONFIGS["tiny_cover"]
+    ctx = make_ctx(cfg, n_layers=1)
+    try:
+        pages, _ = build_layer(ctx, cfg, 0, None)
+        xs = [synth.activations(cfg, step=s, device="cuda") for s in range(3)]
+        lgs = [synth.router_logits(cfg, step=s, device="cuda") for s in range(3)]
+        eager = [ctx.pw_moe_forward(0, xs[s], lgs[s], cfg.top_k).clone() for s in range(3)]   # also sets the kernels up
+        x, lg = xs[0].clone(), lgs[0].clone()
+        out = torch.empty(cfg.tokens, cfg.hidden, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            ctx.pw_moe_forward(0, x, lg, cfg.top_k, out=out)
+        for s in (1, 2, 0, 2):
+            x.copy_(xs[s])
+            lg.copy_(lgs[s])
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, eager[s]), s
+        assert ctx.pw_last_device_status() == 0
+    finally:
+        ctx.close()
