@@ -85,6 +85,9 @@ static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 #endif
 __device__ long long g_trace[16][512];
 __device__ unsigned long long g_spins[32];      // polling-loop iterations per warp index, all CTAs
+__device__ unsigned long long g_sleeps[4][32];  // sleep-and-look iterations per site and warp index, all CTAs
+#define SLEEP_COUNT(site) \
+  if ((threadIdx.x & 31) == 0) atomicAdd(&g_sleeps[site][threadIdx.x >> 5], 1ull)
 #define TRACE(ev, n) \
   if (PHASE == PW_TRACE_PHASE && blockIdx.x == 0 && lane == 0 && (uint32_t)(n) < 512u) g_trace[ev][(n)] = clock64()
 #define TRACEV(ev, n, v) \
@@ -92,6 +95,7 @@ __device__ unsigned long long g_spins[32];      // polling-loop iterations per w
 #else
 #define TRACE(ev, n)
 #define TRACEV(ev, n, v)
+#define SLEEP_COUNT(site)
 #endif
 
 struct TmapSet {                               // token-tile copies: one map per tile height 16, 32, .. 128
@@ -137,6 +141,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_s, uint32_t parity, uin
   uint32_t spins = 0;
   while (true) {
     if (sleep_ns > 0) __nanosleep(sleep_ns);       // leave the issue slots to the warps doing arithmetic
+    SLEEP_COUNT(3);
 #ifdef PW_TC_PROFILE
     if ((threadIdx.x & 31) == 0) atomicAdd(&g_spins[threadIdx.x >> 5], 1ull);
 #endif
@@ -185,6 +190,31 @@ __device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, Ctr
 #endif
   if (ok) return true;
   return mbar_wait_slow(bar_s, parity, SLEEP_NS, c, status);
+}
+// The same bound without an out-of-line path: for waits that sit between producing a long register vector and
+// consuming it (a call there makes the compiler park the vector in call-preserved registers and copy it back).
+// 100000 polls of up to kSuspendHintNs each are the 2 s limit.
+__device__ __forceinline__ bool mbar_wait_nocall(uint32_t bar_s, uint32_t parity, Ctrl* c, int32_t* status) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n"
+      "PW_WAITN:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra PW_DONEN;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "setp.lt.u32 q, n, 100000;\n\t"
+      "@q bra PW_WAITN;\n"
+      "PW_DONEN:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs)
+      : "memory");
+  if (!ok) {
+    c->abort_flag = 1;
+    atomicMax(status, (int)PW_ERR_TIMEOUT);
+  }
+  return ok != 0;
 }
 template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
@@ -363,6 +393,7 @@ __device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* stat
   uint32_t spins = 0;
   while (true) {
     __nanosleep(32);
+    SLEEP_COUNT(0);
     if (c->issued[n & 1] > n) return true;
     if (c->abort_flag) return false;
     if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
@@ -383,6 +414,7 @@ __device__ __noinline__ int next_unit_slow(uint32_t i, Ctrl* c, int32_t* status)
   uint32_t spins = 0;
   while (true) {
     __nanosleep(64);
+    SLEEP_COUNT(1);
     if (c->sched_n > i) return c->sched_unit[i & 31];
     if (c->abort_flag) return -2;
     if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
@@ -667,6 +699,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const unsigned long long t0 = globaltimer();
             while (c->b_issued <= bt && !c->abort_flag) {
               __nanosleep(32);
+              SLEEP_COUNT(2);
               if (globaltimer() - t0 > kWaitLimitNs) {
                 c->abort_flag = 1;
                 atomicMax(status, (int)PW_ERR_TIMEOUT);
@@ -813,6 +846,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const unsigned long long t0 = globaltimer();
             while (c->b_issued <= bt && !c->abort_flag) {
               __nanosleep(32);
+              SLEEP_COUNT(2);
               if (globaltimer() - t0 > kWaitLimitNs) {
                 c->abort_flag = 1;
                 atomicMax(status, (int)PW_ERR_TIMEOUT);
@@ -1009,7 +1043,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             }
             publish();                               // the previous half's store, overlapped with the decode above
             const int hs = 2 * grp + h;
-            ok = mbar_wait<20>(&c->a_empty[hs], use_par ^ 1, c, status);
+            ok = mbar_wait_nocall(smem_u32(&c->a_empty[hs]), use_par ^ 1, c, status);
             if (!ok) break;
             tc_fence_after();
             tmem_st32(lane_addr + h * 32, w);
@@ -1123,8 +1157,10 @@ extern "C" int pw_debug_read_trace(long long* host_out) {
   cudaDeviceSynchronize();
   cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace));
   cudaMemcpyFromSymbol(host_out + 16 * 512, g_spins, sizeof(g_spins));
-  static unsigned long long zeros[32];
-  cudaMemcpyToSymbol(g_spins, zeros, sizeof(zeros));
+  cudaMemcpyFromSymbol(host_out + 16 * 512 + 32, g_sleeps, sizeof(g_sleeps));
+  static unsigned long long zeros[4 * 32];
+  cudaMemcpyToSymbol(g_spins, zeros, sizeof(g_spins));
+  cudaMemcpyToSymbol(g_sleeps, zeros, sizeof(g_sleeps));
   return 0;
 }
 #endif
