@@ -710,7 +710,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               break;
             }
           }
-          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
+          ok = mbar_wait_nocall(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
@@ -743,14 +743,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
-            ok = mbar_wait_s(f0, use_par, c, status);
+            ok = mbar_wait_nocall(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_s(f0 + 8, use_par, c, status);
+            ok = mbar_wait_nocall(f0 + 8, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
@@ -857,7 +857,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               break;
             }
           }
-          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
+          ok = mbar_wait_nocall(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
@@ -890,14 +890,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
-            ok = mbar_wait_s(f0, use_par, c, status);
+            ok = mbar_wait_nocall(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_s(f0 + 8, use_par, c, status);
+            ok = mbar_wait_nocall(f0 + 8, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
