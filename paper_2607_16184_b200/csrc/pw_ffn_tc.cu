@@ -133,68 +133,16 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Returns false when the CTA is aborting or the limit ran out (and then raises the abort).
-// The polling loop is kept out of line so that the hot loops of every role stay short.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_s, uint32_t parity, uint32_t sleep_ns, Ctrl* c,
-                                            int32_t* status) {
-  const unsigned long long t0 = globaltimer();
-  uint32_t spins = 0;
-  while (true) {
-    if (sleep_ns > 0) __nanosleep(sleep_ns);       // leave the issue slots to the warps doing arithmetic
-    SLEEP_COUNT(3);
-#ifdef PW_TC_PROFILE
-    if ((threadIdx.x & 31) == 0) atomicAdd(&g_spins[threadIdx.x >> 5], 1ull);
-#endif
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar_s), "r"(parity)
-        : "memory");
-    if (ok) return true;
-    if (c->abort_flag) return false;
-    if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
-      c->abort_flag = 1;
-      atomicMax(status, (int)PW_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-// Fast path: a short loop around try_wait with a suspend-time hint, so that a waiting thread sleeps inside the
-// barrier unit instead of spending issue slots (an arrival that does not complete the phase still wakes it, hence
-// the loop).  After kFastPolls wake-ups it falls into the bounded out-of-line loop above.
-constexpr uint32_t kFastPolls = 64;
+// Bounded wait.  Returns false when the limit ran out (and then raises the abort: the other roles run into
+// their own limits or find the flag at their next sleep-and-look wait).  Each poll is a try_wait with a
+// suspend-time hint, so a waiting thread sleeps inside the barrier unit instead of spending issue slots (an
+// arrival that does not complete the phase still wakes it, hence the loop); 100000 polls of up to kSuspendHintNs
+// each are the 2 s limit.  The loop is inline and written in PTX on purpose: with an out-of-line slow path the
+// call made the compiler keep each role's loop state -- for the dequantizers a vector of 32 results between
+// decode and store -- in call-preserved registers and copy it around, which cost 2 % of the decode step.
 constexpr uint32_t kSuspendHintNs = 20000;
 // (the barrier is given by its shared-memory address: the control loops keep those in registers)
-template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, Ctrl* c, int32_t* status) {
-  uint32_t ok, polls;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "mov.u32 %1, 0;\n"
-      "PW_WAIT:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%2], %3, %4;\n\t"
-      "@p bra PW_DONE;\n\t"
-      "add.u32 %1, %1, 1;\n\t"
-      "setp.lt.u32 q, %1, %5;\n\t"
-      "@q bra PW_WAIT;\n"
-      "PW_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok), "=&r"(polls)
-      : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "r"(kFastPolls)
-      : "memory");
-#ifdef PW_TC_PROFILE
-  if ((threadIdx.x & 31) == 0 && polls) atomicAdd(&g_spins[threadIdx.x >> 5], (unsigned long long)polls);
-#endif
-  if (ok) return true;
-  return mbar_wait_slow(bar_s, parity, SLEEP_NS, c, status);
-}
-// The same bound without an out-of-line path: for waits that sit between producing a long register vector and
-// consuming it (a call there makes the compiler park the vector in call-preserved registers and copy it back).
-// 100000 polls of up to kSuspendHintNs each are the 2 s limit.
-__device__ __forceinline__ bool mbar_wait_nocall(uint32_t bar_s, uint32_t parity, Ctrl* c, int32_t* status) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
@@ -215,10 +163,6 @@ __device__ __forceinline__ bool mbar_wait_nocall(uint32_t bar_s, uint32_t parity
     atomicMax(status, (int)PW_ERR_TIMEOUT);
   }
   return ok != 0;
-}
-template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(unsigned long long* b, uint32_t parity, Ctrl* c, int32_t* status) {
-  return mbar_wait_s<SLEEP_NS>(smem_u32(b), parity, c, status);
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -388,45 +332,57 @@ __device__ __forceinline__ void ring_advance(RingPos& p, uint32_t step, uint32_t
 __device__ __forceinline__ uint32_t slot_items(uint32_t bits) { return bits == 16 ? 2u : 1u; }
 // Bounded wait until the weight producer has armed slot item n.  A consumer looks at a slot item's full barrier
 // only after this, so it can never mistake an older phase of the slot's barrier for the item's.
-__device__ __noinline__ bool wait_issued_slow(uint32_t n, Ctrl* c, int32_t* status) {
-  const unsigned long long t0 = globaltimer();
-  uint32_t spins = 0;
-  while (true) {
-    __nanosleep(32);
-    SLEEP_COUNT(0);
-    if (c->issued[n & 1] > n) return true;
-    if (c->abort_flag) return false;
-    if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
-      c->abort_flag = 1;
-      atomicMax(status, (int)PW_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
+// Sleep-and-look, at least 32 ns per look, 2^25 looks (inline for the reason given at mbar_wait_s).
 __device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
-  if (c->issued[n & 1] > n) return true;
-  return wait_issued_slow(n, c, status);
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
+      "mov.u32 k, 0;\n"
+      "PW_WI:\n\t"
+      "ld.volatile.shared.u32 v, [%1];\n\t"
+      "setp.gt.u32 p, v, %2;\n\t"
+      "@p bra PW_WID;\n\t"
+      "nanosleep.u32 32;\n\t"
+      "add.u32 k, k, 1;\n\t"
+      "setp.lt.u32 q, k, 33554432;\n\t"
+      "@q bra PW_WI;\n"
+      "PW_WID:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(const_cast<uint32_t*>(&c->issued[n & 1]))), "r"(n)
+      : "memory");
+  if (!ok) {
+    c->abort_flag = 1;
+    atomicMax(status, (int)PW_ERR_TIMEOUT);
+  }
+  return ok != 0;
 }
 // Unit i of this CTA's work list (bounded wait until the weight producer has posted it); -1 = no more work,
 // -2 = the CTA is aborting.
-__device__ __noinline__ int next_unit_slow(uint32_t i, Ctrl* c, int32_t* status) {
-  const unsigned long long t0 = globaltimer();
-  uint32_t spins = 0;
-  while (true) {
-    __nanosleep(64);
-    SLEEP_COUNT(1);
-    if (c->sched_n > i) return c->sched_unit[i & 31];
-    if (c->abort_flag) return -2;
-    if ((++spins & 1023u) == 0 && globaltimer() - t0 > kWaitLimitNs) {
-      c->abort_flag = 1;
-      atomicMax(status, (int)PW_ERR_TIMEOUT);
-      return -2;
-    }
-  }
-}
 __device__ __forceinline__ int next_unit(uint32_t i, Ctrl* c, int32_t* status) {
   if (c->sched_n > i) return c->sched_unit[i & 31];
-  return next_unit_slow(i, c, status);
+  // sleep-and-look, at least 64 ns per look, 2^24 looks (inline for the reason given at mbar_wait_s)
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
+      "mov.u32 k, 0;\n"
+      "PW_NU:\n\t"
+      "nanosleep.u32 64;\n\t"
+      "ld.volatile.shared.u32 v, [%1];\n\t"
+      "setp.gt.u32 p, v, %2;\n\t"
+      "@p bra PW_NUD;\n\t"
+      "add.u32 k, k, 1;\n\t"
+      "setp.lt.u32 q, k, 16777216;\n\t"
+      "@q bra PW_NU;\n"
+      "PW_NUD:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(const_cast<uint32_t*>(&c->sched_n))), "r"(i)
+      : "memory");
+  if (ok) return c->sched_unit[i & 31];
+  c->abort_flag = 1;
+  atomicMax(status, (int)PW_ERR_TIMEOUT);
+  return -2;
 }
 
 // Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
@@ -577,7 +533,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             ms[m].src += ms[m].tb;
             for (int sub = 0; sub < nsub; ++sub, src += 16384) {
               if ((seq & 1u) == P) {
-                if (pass) ok = mbar_wait<32>(&c->empty[s], (pass - 1) & 1, c, status);
+                if (pass) ok = mbar_wait_s(smem_u32(&c->empty[s]), (pass - 1) & 1, c, status);
                 if (!ok) break;
                 const uint32_t bar_s = full_s + 8 * s;
                 if (P == 0) { TRACE(0, seq); }
@@ -620,7 +576,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         for (int g = un.g0; ok && g < un.g1; ++g) {
           // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
           const int bs = bcount % n_bslots;
-          ok = mbar_wait<64>(&c->b_empty[bs], ((bcount / n_bslots) & 1) ^ 1, c, status);
+          ok = mbar_wait_s(smem_u32(&c->b_empty[bs]), ((bcount / n_bslots) & 1) ^ 1, c, status);
           if (!ok) break;
           mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
           tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
@@ -685,8 +641,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
         // the epilogue has drained the buffer(s) this unit accumulates into
-        if (wide || dbuf == 0) ok = mbar_wait<32>(&c->d_empty[0], (duse0 & 1) ^ 1, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait<32>(&c->d_empty[1], (duse1 & 1) ^ 1, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
         tc_fence_after();
@@ -710,7 +666,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               break;
             }
           }
-          ok = mbar_wait_nocall(bf_s + 8 * bp.s, bp.par, c, status);
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
@@ -720,7 +676,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
               if (my_j == 0) { TRACE(12, sq + hh); }
-              ok = wait_issued(sq + hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
+              ok = wait_issued(sq + hh, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
               if (my_j == 0) { TRACE(8, sq + hh); }
@@ -743,14 +699,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
-            ok = mbar_wait_nocall(f0, use_par, c, status);
+            ok = mbar_wait_s(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_nocall(f0 + 8, use_par, c, status);
+            ok = mbar_wait_s(f0 + 8, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
@@ -832,8 +788,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           do {
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 16); }
         // the epilogue has drained the buffer(s) this unit accumulates into
-        if (wide || dbuf == 0) ok = mbar_wait<32>(&c->d_empty[0], (duse0 & 1) ^ 1, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait<32>(&c->d_empty[1], (duse1 & 1) ^ 1, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         if (my_m == 0 && my_j == 0) { TRACE(15, ucount + 32); }
         tc_fence_after();
@@ -857,7 +813,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               break;
             }
           }
-          ok = mbar_wait_nocall(bf_s + 8 * bp.s, bp.par, c, status);
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           if (my_m == 0 && my_j == 0) { TRACE(11, bt); }
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
@@ -867,7 +823,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
               if (my_j == 0) { TRACE(12, sq + hh); }
-              ok = wait_issued(sq + hh, c, status) && mbar_wait(&c->full[hp.s], hp.par, c, status);
+              ok = wait_issued(sq + hh, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
               if (my_j == 0) { TRACE(8, sq + hh); }
@@ -890,14 +846,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
-            ok = mbar_wait_nocall(f0, use_par, c, status);
+            ok = mbar_wait_s(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_nocall(f0 + 8, use_par, c, status);
+            ok = mbar_wait_s(f0 + 8, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
@@ -921,8 +877,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
         if (wide || dbuf == 1) ++duse1;
         // every issuer warp sees every phase of the accumulator barriers, also of the narrow units it has no
         // part in: it must not run ahead of the epilogue by more than the phase parity can tell apart
-        if (wide || dbuf == 0) ok = mbar_wait<200>(&c->d_full[0], par0, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait<200>(&c->d_full[1], par1, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), par0, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), par1, c, status);
         if (!ok) break;
         if (wide) {
           tc_fence_after();
@@ -1022,7 +978,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           ++uses;
           if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
             publish();                               // do not sit on a finished half while waiting for HBM
-            ok = wait_issued(sq, c, status) && mbar_wait<20>(&c->full[rp.s], rp.par, c, status);
+            ok = wait_issued(sq, c, status) && mbar_wait_s(smem_u32(&c->full[rp.s]), rp.par, c, status);
             if (!ok) break;
           }
           if (q == 0) { TRACE(1, sq); }
@@ -1043,7 +999,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             }
             publish();                               // the previous half's store, overlapped with the decode above
             const int hs = 2 * grp + h;
-            ok = mbar_wait_nocall(smem_u32(&c->a_empty[hs]), use_par ^ 1, c, status);
+            ok = mbar_wait_s(smem_u32(&c->a_empty[hs]), use_par ^ 1, c, status);
             if (!ok) break;
             tc_fence_after();
             tmem_st32(lane_addr + h * 32, w);
@@ -1079,8 +1035,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       const bool wide = NMAT * npart * nb_rows > acol / 2;
       const uint32_t dbuf = wide ? 0u : dtoggle;
       if (!wide) dtoggle ^= 1u;
-      if (wide || dbuf == 0) ok = mbar_wait<200>(&c->d_full[0], duse0 & 1, c, status);
-      if (ok && (wide || dbuf == 1)) ok = mbar_wait<200>(&c->d_full[1], duse1 & 1, c, status);
+      if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), duse0 & 1, c, status);
+      if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), duse1 & 1, c, status);
       if (!ok) break;
       if (q == 0) { TRACE(13, ucount); }
       if (q == 0) { TRACEV(7, ucount, rows[un.seg * 3].bits * 100 + rows[un.seg * 3 + 1].bits + 10000 * un.ntok); }
