@@ -234,21 +234,29 @@ def run_demote(ctx, cfg, layers, device, peaks, decode_fn, decode_ms):
     ms42 = time_region(lambda i: ctx.pw_demote_block(dst4[i % n_src], 2, dst=dst2[i % n_src]), reps, device) / reps
     # overlapped: decode on the current stream, one 16->4 demote per decode step on a side stream (never committed)
     side = torch.cuda.Stream(device=device)
-    n_steps = 60
-    torch.cuda.synchronize(device)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    side.wait_stream(torch.cuda.current_stream(device))
-    e0.record()
-    s0.record(side)
-    for i in range(n_steps):
-        ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src], stream=side)
-        decode_fn(i)
-    e1.record()
-    s1.record(side)
-    torch.cuda.synchronize(device)
-    ms_dec = e0.elapsed_time(e1) / n_steps
-    ms_side = s0.elapsed_time(s1) / n_steps
+    # Blocks of decode steps alone and with the demotes alternate, so that both see the same clocks (a short
+    # burst after an idle moment runs at boost clocks, a long loop under the power cap does not).
+    n_steps, rounds = 60, 4
+    alone_ms = over_ms = side_ms = 0.0
+    for _ in range(rounds):
+        alone_ms += time_region(decode_fn, n_steps, device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        side.wait_stream(torch.cuda.current_stream(device))
+        e0.record()
+        s0.record(side)
+        for i in range(n_steps):
+            ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src], stream=side)
+            decode_fn(i)
+        e1.record()
+        s1.record(side)
+        torch.cuda.synchronize(device)
+        over_ms += e0.elapsed_time(e1)
+        side_ms += s0.elapsed_time(s1)
+    decode_ms = alone_ms / (rounds * n_steps)
+    ms_dec = over_ms / (rounds * n_steps)
+    ms_side = side_ms / (rounds * n_steps)
+    n_steps *= rounds
     gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
     return {"block": "%dx%d" % (rows, cols),
             "16to4": {"ms": ms164, "gbs": gbs(b16 + b4, ms164), "frac_of_measured_hbm": gbs(b16 + b4, ms164) / peaks["hbm_gbs"],
@@ -296,27 +304,33 @@ def run_residency(ctx, cfg, layers, device, decode_fn, decode_ms):
     assert torch.equal(back[-1].codes, page.codes)
     total = nbytes * len(targets)
     # under decode: every step one page moves (out if it is resident, back in if it is away), on the side stream
-    n_steps, moved = 240, 0
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize(device)
-    e0.record()
-    s0.record(side)
-    for i in range(n_steps):
-        j = i % len(targets)
-        st = ctx.pw_page_state(*targets[j], 16)
-        if st == B.PW_STATE_GPU_RESIDENT:
-            ctx.pw_offload_page(*targets[j], back[j], stream=side, host=hosts[j])
-            moved += nbytes
-        elif st == B.PW_STATE_CPU_RESIDENT:
-            back[j] = ctx.pw_reload_page(*targets[j], 16, hosts[j], stream=side)
-            moved += nbytes
-        decode_fn(i)
-    e1.record()
-    s1.record(side)
-    torch.cuda.synchronize(device)
-    ms_dec = e0.elapsed_time(e1) / n_steps
-    ms_side = s0.elapsed_time(s1)
+    # (blocks alone and with page movement alternate, so that both see the same clocks)
+    n_steps, rounds, moved = 60, 4, 0
+    alone_ms = over_ms = ms_side = 0.0
+    for _ in range(rounds):
+        alone_ms += time_region(decode_fn, n_steps, device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        s0.record(side)
+        for i in range(n_steps):
+            j = i % len(targets)
+            st = ctx.pw_page_state(*targets[j], 16)
+            if st == B.PW_STATE_GPU_RESIDENT:
+                ctx.pw_offload_page(*targets[j], back[j], stream=side, host=hosts[j])
+                moved += nbytes
+            elif st == B.PW_STATE_CPU_RESIDENT:
+                back[j] = ctx.pw_reload_page(*targets[j], 16, hosts[j], stream=side)
+                moved += nbytes
+            decode_fn(i)
+        e1.record()
+        s1.record(side)
+        torch.cuda.synchronize(device)
+        over_ms += e0.elapsed_time(e1)
+        ms_side += s0.elapsed_time(s1)
+    decode_ms = alone_ms / (rounds * n_steps)
+    ms_dec = over_ms / (rounds * n_steps)
+    n_steps *= rounds
     for t in targets:                                  # leave no record behind for the rest of the run
         if ctx.pw_page_state(*t, 16) != B.PW_STATE_IN_TRANSFER:
             ctx.pw_drop_page(*t, 16)
@@ -434,24 +448,6 @@ def run_gpu(args):
                         "kernel_ms": kavg, "kernel_timed_ms_per_step": ms_timed / args.steps,
                         "ffn_down_gbs": dn_gbs}}
 
-    if rank == 0 and world == 1 and not args.skip_cpu:
-        # the oracle as it stands, on the same steps the GPU loop rotates over: one call per layer copy, until
-        # about --cpu-seconds of CPU time have been spent (at least one call)
-        n_tok, dt_all, cores, calls = 0, 0.0, 0, 0
-        while dt_all < args.cpu_seconds and calls < 4 * L:
-            lay = layers[calls % L]
-            host_pages = export_layer_to_host(ctx, lay, cfg)
-            v, dt, cores = cpu_oracle_sample(cfg, host_pages, lay["x"].cpu().numpy(), lay["logits"].cpu().numpy(),
-                                             min(args.cpu_tokens, T))
-            del host_pages
-            n_tok += min(args.cpu_tokens, T)
-            dt_all += dt
-            calls += 1
-        line["cpu_baseline"] = {"value": n_tok / dt_all, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                                "sample": "%d layer calls of %d of the %d tokens each, %.1f s of oracle time"
-                                          % (calls, min(args.cpu_tokens, T), T, dt_all)}
-    else:
-        line["cpu_baseline"] = None
     if rank == 0 and world == 1 and not args.skip_extra:
         # observation taps (routing mass, routed-input features): the same timed loop with the taps on
         ctx.pw_observe(True)
@@ -472,7 +468,7 @@ def run_gpu(args):
         # the same step with each layer's forward call replayed from a CUDA graph (the commit stays eager)
         graphs = []
         torch.cuda.synchronize(device)
-        for li, lay in enumerate(layers):
+        for li, lay in enumerate(layers if not args.skip_graph else []):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
                 ctx.pw_moe_forward(li, lay["x"], lay["logits"], k, out=out, mode=mode)
@@ -483,18 +479,36 @@ def run_gpu(args):
             ctx.pw_set_page_table(lay["entries"][(i // L) % len(lay["entries"]):][:1])
             graphs[i % L].replay()
 
-        for i in range(3):
-            step_graph(i)
-        ms_graph = time_region(step_graph, args.steps, device) / args.steps
-        line["cuda_graph"] = {"ms_per_step": ms_graph, "tokens_per_s": T / (ms_graph * 1e-3),
-                              "ms_per_step_eager": ms_step}
+        if graphs:
+            for i in range(3):
+                step_graph(i)
+            ms_graph = time_region(step_graph, args.steps, device) / args.steps
+            line["cuda_graph"] = {"ms_per_step": ms_graph, "tokens_per_s": T / (ms_graph * 1e-3),
+                                  "ms_per_step_eager": ms_step}
         del graphs
         line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
         line["residency"] = run_residency(ctx, cfg, layers, device, step, ms_step)
-        del layers
-        ctx.close()
-        torch.cuda.empty_cache()
-        line["prefill"] = run_prefill(device, peaks)
+        line["prefill"] = run_prefill(device, peaks)     # its own context and pages (about 2 GB more)
+    # (the CPU oracle runs after the GPU extras: its OpenMP threads keep the host cores busy for a while
+    # afterwards, and the extras' launch loops must not compete with them)
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        # the oracle as it stands, on the same steps the GPU loop rotates over: one call per layer copy, until
+        # about --cpu-seconds of CPU time have been spent (at least one call)
+        n_tok, dt_all, cores, calls = 0, 0.0, 0, 0
+        while dt_all < args.cpu_seconds and calls < 4 * L:
+            lay = layers[calls % L]
+            host_pages = export_layer_to_host(ctx, lay, cfg)
+            v, dt, cores = cpu_oracle_sample(cfg, host_pages, lay["x"].cpu().numpy(), lay["logits"].cpu().numpy(),
+                                             min(args.cpu_tokens, T))
+            del host_pages
+            n_tok += min(args.cpu_tokens, T)
+            dt_all += dt
+            calls += 1
+        line["cpu_baseline"] = {"value": n_tok / dt_all, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                "sample": "%d layer calls of %d of the %d tokens each, %.1f s of oracle time"
+                                          % (calls, min(args.cpu_tokens, T), T, dt_all)}
+    else:
+        line["cpu_baseline"] = None
     if rank == 0:
         print(json.dumps(line))
     replicas.shutdown()
@@ -720,6 +734,7 @@ def main():
                     help="diagnostic: give every routed block this bitwidth instead of the configured mix")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-extra", action="store_true")
+    ap.add_argument("--skip-graph", action="store_true", help="leave out the CUDA-graph replay of the step")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps

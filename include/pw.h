@@ -16,7 +16,7 @@
  *   - "device" pointers are CUDA global memory of the current device, "host"
  *     pointers are ordinary host memory.  All device buffers are owned and
  *     allocated by the caller; the library never allocates device memory.
- *     pw_create allocates only a small host object and a pinned host staging area.
+ *     pw_create allocates only a small host object.
  *   - Work is enqueued on the caller's stream and returns immediately.  Argument
  *     errors are detected on the host before anything is enqueued.  Problems met
  *     on the device (a bounded wait that ran out, a failed self check) are written
@@ -169,7 +169,9 @@ pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst
 
 /* Publishes n rows of the weight page table (Sec. 3.1): for each entry the row
  * (layer, expert, kind) now maps to entry.page with committed bitwidth page.bits.  Rows not
- * named keep their value.  The update is ordered on `stream`: forward calls enqueued on the same
+ * named keep their value (a row named twice takes its last entry).  The rows are carried to the device in
+ * the parameters of a small kernel, so the update is ordered on `stream` like any kernel and does not wait
+ * behind copies that other streams have queued on a DMA engine: forward calls enqueued on the same
  * stream before this call read the old rows, calls enqueued after it read the new rows -- the
  * "safe boundary" of Sec. 3.3 is the gap between two forward calls.  The previous page of a row
  * may be released once work enqueued before this call has finished.  entries: host.  epoch_out

@@ -61,6 +61,20 @@ WsMap make_wsmap(const pw_config& c) {
   return m;
 }
 
+// Rows of one page-table update, passed by value to the kernel that writes them (3.3 KB of the 4 KB a kernel's
+// parameters may take).
+constexpr int kCommitBatch = 64;
+struct CommitBatch {
+  int n;
+  uint32_t index[kCommitBatch];
+  DevRow row[kCommitBatch];
+};
+__global__ void __launch_bounds__(kCommitBatch) commit_rows_kernel(const __grid_constant__ CommitBatch batch,
+                                                                  DevRow* __restrict__ table) {
+  const int j = threadIdx.x;
+  if (j < batch.n) table[batch.index[j]] = batch.row[j];
+}
+
 static void timing_drain_slot(pw_ctx* ctx, int slot) {
   if (!ctx->timing_busy[slot]) return;
   cudaEvent_t* ev = ctx->timing_ev + (size_t)slot * (PW_NUM_KERNELS + 1);
@@ -106,7 +120,6 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   ctx->launches = 0;
   ctx->last_T = ctx->last_k = 0;
   ctx->tc_state = nullptr;
-  ctx->stage_next = 0;
   ctx->timing_on = false;
   ctx->timing_ev = nullptr;
   ctx->timing_cur = 0;
@@ -115,24 +128,15 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   for (int i = 0; i < pw_ctx::kTimingSlots; ++i) ctx->timing_busy[i] = false;
   for (int i = 0; i < PW_NUM_KERNELS; ++i) ctx->timing_ms[i] = 0.0;
   const size_t nrows = (size_t)cfg->n_layers * m.S * 3;
-  ctx->stage_rows = nrows;
+  ctx->n_rows = nrows;
   ctx->host_rows = new (std::nothrow) pw_table_entry[nrows]();
   ctx->host_valid = new (std::nothrow) uint8_t[nrows]();
   ctx->records = new (std::nothrow) PageRecord[nrows * kBitLevels]();
   for (size_t i = 0; ctx->records && i < nrows * kBitLevels; ++i) ctx->records[i].state = PW_STATE_NONE;
-  for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
-    ctx->stage[i] = nullptr;
-    ctx->stage_ev[i] = nullptr;
-    ctx->stage_used[i] = false;
-  }
   bool ok = ctx->host_rows && ctx->host_valid && ctx->records;
   int dev = 0;
   ok = ok && cudaGetDevice(&dev) == cudaSuccess;
   ok = ok && cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
-  for (int i = 0; ok && i < pw_ctx::kStageSlots; ++i) {
-    ok = cudaMallocHost(reinterpret_cast<void**>(&ctx->stage[i]), sizeof(DevRow) * nrows) == cudaSuccess &&
-         cudaEventCreateWithFlags(&ctx->stage_ev[i], cudaEventDisableTiming) == cudaSuccess;
-  }
   // the table (valid = 0), status word, counters and operand padding start out as zeros
   ok = ok && cudaMemset(ctx->base, 0, m.total) == cudaSuccess;
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -147,10 +151,6 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
 extern "C" pw_status pw_destroy(pw_ctx* ctx) {
   if (!ctx) return PW_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
-  for (int i = 0; i < pw_ctx::kStageSlots; ++i) {
-    if (ctx->stage[i]) cudaFreeHost(ctx->stage[i]);
-    if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
-  }
   tc_teardown(ctx);
   if (ctx->timing_ev) {
     for (int i = 0; i < pw_ctx::kTimingSlots * (PW_NUM_KERNELS + 1); ++i)
@@ -168,7 +168,7 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
                                        uint64_t* epoch_out) {
   if (!ctx || (!entries && n)) return PW_ERR_INVALID_ARG;
   const pw_config& c = ctx->cfg;
-  if (n > ctx->stage_rows) return PW_ERR_INVALID_ARG;
+  if (n > ctx->n_rows) return PW_ERR_INVALID_ARG;
   // validate everything before anything is enqueued
   for (size_t i = 0; i < n; ++i) {
     const pw_table_entry& e = entries[i];
@@ -187,14 +187,15 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
     const pw_status rs = residency_check_commit(ctx, row_index(ctx, e.layer, e.expert, e.kind), p);
     if (rs != PW_OK) return rs;
   }
-  if (n) {
-    const int slot = ctx->stage_next;
-    ctx->stage_next = (slot + 1) % pw_ctx::kStageSlots;
-    if (ctx->stage_used[slot]) PW_CUDA_OK(cudaEventSynchronize(ctx->stage_ev[slot]));
-    DevRow* st = ctx->stage[slot];
-    DevRow* dtab = reinterpret_cast<DevRow*>(ctx->base + ctx->ws.table);
-    size_t run_begin = 0;  // entries [run_begin, i) map to consecutive device rows
-    for (size_t i = 0; i < n; ++i) {
+  // The rows travel in the parameter space of a small kernel, 64 at a time: the update is ordered on the
+  // stream like any kernel and never queues behind a large copy on a DMA engine (a page being reloaded on a
+  // side stream would otherwise hold up the commits of the stream that runs the forward calls).
+  DevRow* dtab = reinterpret_cast<DevRow*>(ctx->base + ctx->ws.table);
+  size_t i = 0;
+  while (i < n) {
+    CommitBatch batch;
+    batch.n = 0;
+    for (; i < n && batch.n < kCommitBatch; ++i) {
       const pw_table_entry& e = entries[i];
       DevRow r{};
       r.codes = e.page.codes;
@@ -202,23 +203,19 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       r.cols = e.page.cols;
       r.bits = e.page.bits;
       r.valid = 1;
-      st[i] = r;
       const size_t idx = row_index(ctx, e.layer, e.expert, e.kind);
+      int j = 0;                                   // a row named twice keeps its last entry
+      while (j < batch.n && batch.index[j] != (uint32_t)idx) ++j;
+      batch.row[j] = r;
+      batch.index[j] = (uint32_t)idx;
+      if (j == batch.n) ++batch.n;
       ctx->host_rows[idx] = e;
       ctx->host_valid[idx] = 1;
       residency_note_commit(ctx, idx, e.page);
-      const bool last = i + 1 == n;
-      const bool contiguous =
-          !last && row_index(ctx, entries[i + 1].layer, entries[i + 1].expert, entries[i + 1].kind) == idx + 1;
-      if (!contiguous) {
-        const size_t first = idx - (i - run_begin);
-        PW_CUDA_OK(cudaMemcpyAsync(dtab + first, st + run_begin, sizeof(DevRow) * (i + 1 - run_begin),
-                                   cudaMemcpyHostToDevice, stream));
-        run_begin = i + 1;
-      }
     }
-    PW_CUDA_OK(cudaEventRecord(ctx->stage_ev[slot], stream));
-    ctx->stage_used[slot] = true;
+    commit_rows_kernel<<<1, kCommitBatch, 0, stream>>>(batch, dtab);
+    ctx->launches++;
+    PW_CUDA_OK(cudaGetLastError());
   }
   ctx->epoch++;
   if (epoch_out) *epoch_out = ctx->epoch;

@@ -103,13 +103,7 @@ struct pw_ctx {
   pw_table_entry* host_rows;      // mirror of the committed table
   uint8_t* host_valid;
   uint64_t epoch;
-  // pinned staging ring for table updates
-  static constexpr int kStageSlots = 8;
-  pw::DevRow* stage[kStageSlots];
-  size_t stage_rows;
-  cudaEvent_t stage_ev[kStageSlots];
-  bool stage_used[kStageSlots];
-  int stage_next;
+  size_t n_rows;                  // rows of the table = n_layers * (n_experts + n_shared) * 3
   uint64_t launches;
   int last_T, last_k;
   int num_sms;

@@ -38,7 +38,7 @@ void residency_note_commit(pw_ctx* ctx, size_t row, const pw_page& page) {
 
 void residency_teardown(pw_ctx* ctx) {
   if (!ctx->records) return;
-  for (size_t i = 0; i < ctx->stage_rows * kBitLevels; ++i)
+  for (size_t i = 0; i < ctx->n_rows * kBitLevels; ++i)
     if (ctx->records[i].ev) cudaEventDestroy(ctx->records[i].ev);
   delete[] ctx->records;
   ctx->records = nullptr;
