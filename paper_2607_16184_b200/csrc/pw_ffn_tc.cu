@@ -16,7 +16,8 @@
 // instruction of theirs waits its turn, so each of them does as little per item as possible.
 //   warps 0-15   dequantize: four groups of four warps; tile k of a matrix goes to that matrix's group
 //                k mod (groups per matrix); warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
-//                a group has two operand half-slots in tensor memory (K 0..63 / 64..127 of its tile);
+//                a group has one operand slot of 64 columns in tensor memory (a whole tile, K 0..127) and hands
+//                it to its issuer once per tile, while it decodes the first half of its next tile in registers;
 //   warps 16,18  weight producers: producer P arms the slot items with number = P mod 2 (which sit in the
 //                slots = P mod 2) and issues their copies, as far ahead as the ring allows; producer 0 also
 //                claims the CTA's units from a global counter and posts them on the CTA's work list;
@@ -44,7 +45,7 @@ namespace pw {
 
 constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item (16 KB codes + 512 B) fits
 constexpr int kMaxSlots = 16;
-constexpr int kMaxASlots = 8;                  // operand half-slots in tensor memory (32 columns = 64 K each)
+constexpr int kMaxASlots = 4;                  // operand slots in tensor memory, one per group (64 columns = a 128 x 128 tile)
 constexpr int kMaxBSlots = 5;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
@@ -432,9 +433,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
   constexpr int IPM = kIssuers / NMAT;           // issuers per matrix = dequantizer groups per matrix
   int npart = IPM;
-  while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 32 > kTmemCols) npart >>= 1;
+  while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 64 > kTmemCols) npart >>= 1;
   const int n_issuers = NMAT * npart;            // active issuers
-  const int acol = NMAT * npart * nt_tile;       // operand half-slot hs = 2 * group + K-half sits at acol + 32 * hs
+  const int acol = NMAT * npart * nt_tile;       // the operand slot of group g sits at acol + 64 * g
   const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
@@ -447,7 +448,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       mbar_init(&c->b_empty[i], NMAT);             // one issuer per matrix multiplies a token tile
     }
     for (int i = 0; i < kMaxASlots; ++i) {
-      mbar_init(&c->a_full[i], 4);                // the four warps of the group that owns the half-slot
+      mbar_init(&c->a_full[i], 4);                // the four warps of the group that owns the slot
       mbar_init(&c->a_empty[i], 1);                // the issuer that serves the group
     }
     for (int i = 0; i < 2; ++i) {
@@ -598,7 +599,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     if (lane == 0 && my_j < npart) {
       uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
-      uint32_t upar = 0;                            // per group: parity of the next use of its operand half-slots
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
       uint32_t ucount = 0;
       // Accumulators: partial (m, j) of a unit sits at buffer base + (m * npart + j) * nb_rows.  A unit whose
       // accumulators fit half of the accumulator columns takes one of two buffers in turn, so that its MMAs
@@ -691,26 +692,23 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             sq += (uint32_t)npart * W;
             ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
           } else {
-            // the group that dequantizes this tile, and the parity of this use of its half-slots
+            // the group that dequantizes this tile, and the parity of this use of its operand slot
             const uint32_t k = base + j;
             const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
             const uint32_t use_par = (upar >> grp) & 1u;
             upar ^= 1u << grp;
-            const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
+            const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
             ok = mbar_wait_s(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
+            // all eight k-steps of the tile, then one commit hands the group's operand slot back
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_s(f0 + 8, use_par, c, status);
-            if (!ok) break;
-            tc_fence_after();
-            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
-            tc_commit_s(e0 + 8);
           }
           tc_commit_s(be_s + 8 * bp.s);
           later = 1;
@@ -746,7 +744,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     {
       uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
-      uint32_t upar = 0;                            // per group: parity of the next use of its operand half-slots
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
       uint32_t ucount = 0;
       uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
       const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
@@ -838,26 +836,23 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
             sq += (uint32_t)npart * W;
             ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
           } else {
-            // the group that dequantizes this tile, and the parity of this use of its half-slots
+            // the group that dequantizes this tile, and the parity of this use of its operand slot
             const uint32_t k = base + j;
             const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
             const uint32_t use_par = (upar >> grp) & 1u;
             upar ^= 1u << grp;
-            const uint32_t f0 = af_s + 16 * grp, e0 = ae_s + 16 * grp;     // barriers of half-slot 2 * grp
+            const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
             if (my_j == 0) { TRACE(12, k); }
             ok = mbar_wait_s(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             if (my_j == 0) { TRACE(8, k); }
+            // all eight k-steps of the tile, then one commit hands the group's operand slot back
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
             tc_commit_s(e0);
             if (my_j == 0) { TRACE(9, k); }
-            ok = mbar_wait_s(f0 + 8, use_par, c, status);
-            if (!ok) break;
-            tc_fence_after();
-            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
-            tc_commit_s(e0 + 8);
           }
           tc_commit_s(be_s + 8 * bp.s);
           later = 1;
@@ -933,8 +928,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
   } else if (warp < kDqWarps) {    // ---------------- dequantize ----------------
     // Four groups of four warps, each taking every other quantized item of one matrix (every fourth when
     // the unit has a single matrix; an item = one group of one matrix).  Warp q of a group owns rows (= TMEM lanes) 32q .. 32q+31 of the item, one row per
-    // thread.  Each group has two operand half-slots (K 0..63 and K 64..127 of its item): while the
-    // issuers consume one half the group decodes the other.
+    // thread.  Each group has one operand slot (64 columns: both K-halves of an item): it stores the two halves
+    // as it decodes them and hands the slot over once per item; while the issuer's eight MMAs read it, the group
+    // decodes the first half of its next item in registers.
     const int grp = warp >> 2, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + grp * 64;
@@ -943,18 +939,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
     constexpr uint32_t kStride = NMAT == 2 ? 2 : 4;  // groups per matrix = distance between my tiles
     uint32_t seq_unit = 0;                           // slot items before the current unit
     uint32_t base = 0;                               // tiles of one matrix before the current unit
-    uint32_t uses = 0;                               // tiles I have taken so far (parity of my half-slots' use)
-    int pending = -1;                                // operand half-slot whose store has not been published yet
+    uint32_t uses = 0;                               // tiles I have taken so far (parity of my slot's use)
     bool ok = true;
-    auto publish = [&]() {
-      if (pending >= 0) {
-        tmem_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&c->a_full[pending]);
-        pending = -1;
-      }
-    };
     for (int i = 0; ok; ++i) {
       const int u = next_unit((uint32_t)i, c, status);
       if (u < 0) break;
@@ -977,7 +963,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
           const uint32_t use_par = uses & 1u;
           ++uses;
           if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
-            publish();                               // do not sit on a finished half while waiting for HBM
             ok = wait_issued(sq, c, status) && mbar_wait_s(smem_u32(&c->full[rp.s]), rp.par, c, status);
             if (!ok) break;
           }
@@ -993,24 +978,25 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
               default: decode_item_half<2>(item, r, h, w); break;
             }
             if (q == 0) { TRACE(2 + 3 * h, sq); }
-            if (h == 1) {
+            if (h == 0) {
+              // The slot is free once the MMAs of the group's previous tile have read it; they ran while the
+              // half above was being decoded.
+              ok = mbar_wait_s(smem_u32(&c->a_empty[grp]), use_par ^ 1, c, status);
+              if (!ok) break;
+              tc_fence_after();
+            } else {
               __syncwarp();
               if (lane == 0) mbar_arrive(&c->empty[rp.s]);   // this warp has read its rows of the tile
             }
-            publish();                               // the previous half's store, overlapped with the decode above
-            const int hs = 2 * grp + h;
-            ok = mbar_wait_s(smem_u32(&c->a_empty[hs]), use_par ^ 1, c, status);
-            if (!ok) break;
-            tc_fence_after();
             tmem_st32(lane_addr + h * 32, w);
             if (q == 0) { TRACE(3 + 3 * h, sq); }
-            pending = hs;
           }
           if (!ok) break;
-          // The second half goes out at once: its half-slot is the one this group needs back soonest (for the
-          // second half of its next tile), and holding it over the next tile's first decode would delay that.
-          // The first half's store stays overlapped with the decode of the second.
-          publish();
+          // hand the tile over: both stores have landed, then one arrival per warp
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&c->a_full[grp]);
           sq += step;
           ring_advance(rp, step, (uint32_t)n_slots);
         }
@@ -1018,7 +1004,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* __restrict__ units, c
       base += ng;
       seq_unit += ng * W;
     }
-    publish();
   } else if (warp >= kWarpEpi) {
     // ---------------- epilogue ----------------
     const int q = warp & 3;
@@ -1201,7 +1186,7 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   for (int phase = 0; phase < 2; ++phase) {
     const int nmat = phase == 0 ? 2 : 1;
     int npart = kIssuers / nmat;
-    while (npart > 1 && nmat * npart * nt_tile + kMaxASlots * 32 > kTmemCols) npart >>= 1;
+    while (npart > 1 && nmat * npart * nt_tile + kMaxASlots * 64 > kTmemCols) npart >>= 1;
     n_bslots[phase] = npart + 1 > kMaxBSlots ? kMaxBSlots : npart + 1;
     int ns = (kMaxDynSmem - kCtrlBytes - n_bslots[phase] * bslot_bytes) / kSlotBytes;
     if (ns > kMaxSlots) ns = kMaxSlots;
