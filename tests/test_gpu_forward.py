@@ -270,3 +270,13 @@ def test_forward_call_replays_from_a_cuda_graph(orc):
         assert ctx.pw_last_device_status() == 0
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("shape", [(256, 32, 16, 128, 128, 40),     # the most experts, choices and shared experts a context takes
+                                   (4, 4, 0, 128, 256, 19),          # every expert chosen by every token
+                                   (1, 1, 0, 256, 128, 5)])          # a single expert
+def test_limits_of_the_configuration(orc, shape, mode):
+    E, k, n_shared, H, F, T = shape
+    cfg = synth.LayerConfig("limits_%d_%d" % (E, k), E, k, H, F, T, n_shared=n_shared, routing="normal", bit_rule="iid5")
+    run_case(orc, cfg, mode)
