@@ -5,15 +5,12 @@
 namespace pw {
 
 constexpr int kMaxExpertsPerLane = 8;  // E <= 256
+constexpr int kFusedRouteWork = 256;   // (token, choice) pairs x 32-expert strides up to which the grouping kernel routes itself
 
-// One warp per token.  Slot j holds the j-th largest logit; equal logits: lower expert index first.
-__global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ logits, int T, int E, int k,
-                                                     int32_t* __restrict__ topk_ids, float* __restrict__ gates) {
-  grid_dep_sync();   // the gates of the call before this one may still be read by its combine kernel
-  grid_dep_trigger();
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= T) return;
-  const float* l = logits + (size_t)warp * E;
+// Routing of one token by one warp.  Slot j holds the j-th largest logit; equal logits: lower expert index first.
+__device__ __forceinline__ void route_token(const float* __restrict__ logits, int token, int E, int k,
+                                            int32_t* __restrict__ topk_ids, float* __restrict__ gates, int lane) {
+  const float* l = logits + (size_t)token * E;
   float v[kMaxExpertsPerLane];
 #pragma unroll
   for (int i = 0; i < kMaxExpertsPerLane; ++i) {
@@ -55,9 +52,19 @@ __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ l
   }
   // k <= 32: lane j owns slot j
   if (lane < k) {
-    topk_ids[(size_t)warp * k + lane] = myid;
-    gates[(size_t)warp * k + lane] = __fdiv_rn(myp, S);
+    topk_ids[(size_t)token * k + lane] = myid;
+    gates[(size_t)token * k + lane] = __fdiv_rn(myp, S);
   }
+}
+
+// One warp per token.
+__global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ logits, int T, int E, int k,
+                                                     int32_t* __restrict__ topk_ids, float* __restrict__ gates) {
+  grid_dep_sync();   // the gates of the call before this one may still be read by its combine kernel
+  grid_dep_trigger();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= T) return;
+  route_token(logits, warp, E, k, topk_ids, gates, lane);
 }
 
 #ifdef PW_TC_PROFILE
@@ -69,8 +76,10 @@ __device__ long long g_ptrace[32];
 
 // Single CTA.  Stable counting sort of the P = T*k pairs by expert (positions come from ordered
 // prefix counts, never from atomics), segment table including the shared experts, operand-row ->
-// token map, and the unit lists of the tensor-core kernels.
-__global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict__ topk_ids, int T, int k, int E,
+// token map, and the unit lists of the tensor-core kernels.  With `logits` given the CTA routes the tokens
+// itself first (a warp per token, 32 at a time): for a decode batch that is cheaper than a launch of its own.
+__global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__ logits, float* __restrict__ gates,
+                                                       int32_t* topk_ids, int T, int k, int E,
                                                        int n_shared, int32_t* __restrict__ counts,
                                                        int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
                                                        int32_t* __restrict__ inv_perm,
@@ -92,6 +101,10 @@ __global__ void __launch_bounds__(1024) permute_kernel(const int32_t* __restrict
   int32_t* order = ubase + S + 1;    // [S]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = T * k;
+  if (logits) {
+    for (int t = warp; t < T; t += (int)(blockDim.x >> 5)) route_token(logits, t, E, k, topk_ids, gates, lane);
+    __syncthreads();                                 // the pairs below are read back from global memory
+  }
 
   PSTAMP(0);
   for (int e = tid; e < S; e += blockDim.x) cnt[e] = e < E ? 0 : T;
@@ -319,14 +332,20 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
   char* b = ctx->base;
   const int E = c.n_experts, S = w.S;
   int32_t* ids = reinterpret_cast<int32_t*>(b + w.topk_ids);
+  // a decode batch is routed by the grouping kernel's own CTA; a long prompt gets a grid of its own
+  const bool fused = (long long)T * k * ((E + 31) / 32) <= kFusedRouteWork;
   timing_mark(ctx, PW_K_ROUTER, s);
-  PW_CUDA_OK(launch_dependent(router_kernel, dim3((T * 32 + 255) / 256), dim3(256), 0, s, logits, T, E, k, ids,
-                              reinterpret_cast<float*>(b + w.gates)));
+  if (!fused) {
+    PW_CUDA_OK(launch_dependent(router_kernel, dim3((T * 32 + 255) / 256), dim3(256), 0, s, logits, T, E, k, ids,
+                                reinterpret_cast<float*>(b + w.gates)));
+    ctx->launches += 1;
+  }
   timing_mark(ctx, PW_K_PERMUTE, s);
   const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + E + 32 * (size_t)E + (S + 1) + S);
   const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * S * 3;
   PW_CUDA_OK(launch_dependent(
-      permute_kernel, dim3(1), dim3(1024), smem, s, ids, T, k, E, c.n_shared, reinterpret_cast<int32_t*>(b + w.counts),
+      permute_kernel, dim3(1), dim3(1024), smem, s, fused ? logits : static_cast<const float*>(nullptr),
+      reinterpret_cast<float*>(b + w.gates), ids, T, k, E, c.n_shared, reinterpret_cast<int32_t*>(b + w.counts),
       reinterpret_cast<int32_t*>(b + w.offsets), reinterpret_cast<int32_t*>(b + w.perm),
       reinterpret_cast<int32_t*>(b + w.inv_perm), reinterpret_cast<int32_t*>(b + w.row_token),
       reinterpret_cast<int32_t*>(b + w.counter), rows, c.hidden, c.ffn, nt_tile, ksplit,
@@ -343,7 +362,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
                               reinterpret_cast<const int32_t*>(b + w.n_units), nt_tile, ksplit, c.hidden / kGroup,
                               c.ffn / kGroup, reinterpret_cast<Unit*>(b + w.units_gu),
                               reinterpret_cast<Unit*>(b + w.units_dn)));
-  ctx->launches += 3;
+  ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;
 }
@@ -409,7 +428,7 @@ extern "C" pw_status pw_route_tokens_static(const float* router_logits, int T, i
   const int S = n_experts;
   const size_t smem = sizeof(int32_t) * ((size_t)S + (S + 1) + n_experts + 32 * (size_t)n_experts + (S + 1) + S);
   // the grouping kernel clears the counters it uses; everything else in the scratch is overwritten before it is read
-  permute_kernel<<<1, 1024, smem, stream>>>(topk_ids, T, top_k, n_experts, 0, counts, offsets, perm,
+  permute_kernel<<<1, 1024, smem, stream>>>(nullptr, nullptr, topk_ids, T, top_k, n_experts, 0, counts, offsets, perm,
                                             reinterpret_cast<int32_t*>(sc + kStaticInvPerm),
                                             reinterpret_cast<int32_t*>(sc + kStaticRowToken),
                                             reinterpret_cast<int32_t*>(sc + kStaticCounter), nullptr, 0, 0, 0, 1, nullptr,
