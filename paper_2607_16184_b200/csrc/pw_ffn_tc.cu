@@ -134,8 +134,9 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Returns false when the limit ran out (and then raises the abort: the other roles run into
-// their own limits or find the flag at their next sleep-and-look wait).  Each poll is a try_wait with a
+// Bounded wait.  Returns false when the limit ran out (and then raises the abort; the other roles of the CTA,
+// starved by the one that gave up, run into their own limits within the same second or two, and since every
+// role has then been idle for at least a second no copy of the CTA is still in flight when it leaves).  Each poll is a try_wait with a
 // suspend-time hint, so a waiting thread sleeps inside the barrier unit instead of spending issue slots (an
 // arrival that does not complete the phase still wakes it, hence the loop); 100000 polls of up to kSuspendHintNs
 // each are the 2 s limit.  The loop is inline and written in PTX on purpose: with an out-of-line slow path the
