@@ -297,7 +297,7 @@ pw_status pw_route_tokens_static(const float* router_logits, int T, int n_expert
  * pw_observe(ctx, accumulators, stream): accumulators is a device array of
  * n_layers * (n_experts + n_shared) * PW_OBS_FIELDS floats owned by the caller; the call zeroes it on
  * `stream` and from then on every forward call of the context adds its tokens to the rows of its layer
- * (two small kernels at the end of the call, ordered on the call's stream; sums in a fixed order).
+ * (one small kernel at the end of the call, ordered on the call's stream; sums in a fixed order).
  * NULL switches the taps off.  The array must stay valid while the taps are on.
  * Errors: INVALID_ARG, ALIGN, CUDA. */
 enum {
@@ -340,7 +340,7 @@ enum {
   PW_K_FFN_GATE_UP = 3,
   PW_K_FFN_DOWN = 4,
   PW_K_COMBINE = 5,
-  PW_K_OBSERVE = 6, /* the two kernels of the observation taps; ~0 while the taps are off */
+  PW_K_OBSERVE = 6, /* the kernel of the observation taps; ~0 while the taps are off */
   PW_NUM_KERNELS = 7
 };
 pw_status pw_kernel_timing(pw_ctx* ctx, int enable);

@@ -59,7 +59,7 @@ struct WsMap {
   size_t io_hidden;   // fp16 [Tmax][H]   device staging of pw_moe_forward_host
   size_t io_logits;   // float [Tmax][E]
   size_t io_out;      // float [Tmax][H]
-  size_t obs_part;    // float [8][2][Rpad]  partial squared norms of the operand rows (observation taps)
+  size_t obs_part;    // float [kNormSplit][2][Rpad]  partial squared norms of the operand rows (observation taps)
   size_t total;
   // derived sizes
   int S;              // segments = E + n_shared

@@ -1,7 +1,7 @@
 // Observation taps of a layer call: the sums behind the routing mass of every expert (Eq. 1) and behind the
 // routed-input features of every linear-block (Sec. 3.2: routing-weighted mean and RMS input norm, maximum
 // input norm).  They are by-products of buffers the forward call has just filled -- the gathered token rows,
-// the SwiGLU rows, the gates and the grouping -- so two small kernels at the end of the call's chain read
+// the SwiGLU rows, the gates and the grouping -- so one small kernel at the end of the call's chain reads
 // them while they are still in L2.  All sums are taken in a fixed order: the same calls give the same bits.
 #include "pw_common.cuh"
 
@@ -10,12 +10,23 @@ namespace pw {
 // part[(z * 2 + which) * Rpad + n] = sum of squares of slice z of operand row n; which = 0: token rows
 // ([H/8][Rpad][8] fp16), which = 1: SwiGLU rows ([F/8][Rpad][8] fp16).  A CTA takes 32 rows; its eight warps
 // stride over the slice's k-chunks, so every load instruction of a warp reads 512 contiguous bytes.
+__device__ __forceinline__ float warp_sum(float v);
+__device__ __forceinline__ float warp_max(float v);
+__device__ void accumulate_segment(const float* part, int Rpad, const int32_t* __restrict__ offsets,
+                                   const int32_t* __restrict__ perm, const float* __restrict__ gates, int E, int s,
+                                   int lane, float* __restrict__ acc);
+
 __global__ void __launch_bounds__(256) row_norm_kernel(const uint4* __restrict__ xt, int chunks_x,
                                                        const uint4* __restrict__ ht, int chunks_h, int Rpad, int R,
-                                                       float* __restrict__ part) {
+                                                       float* part, int32_t* __restrict__ done_counter,
+                                                       const int32_t* __restrict__ offsets,
+                                                       const int32_t* __restrict__ perm,
+                                                       const float* __restrict__ gates, int E, int S,
+                                                       float* __restrict__ acc) {
   grid_dep_sync();
   grid_dep_trigger();
   __shared__ float sm[8][32];
+  __shared__ int is_last;
   const int which = blockIdx.y, z = blockIdx.z;
   const uint4* buf = which ? ht : xt;
   const int chunks = which ? chunks_h : chunks_x;
@@ -24,7 +35,8 @@ __global__ void __launch_bounds__(256) row_norm_kernel(const uint4* __restrict__
   const int n = blockIdx.x * 32 + r;
   float a = 0.f;
   if (n < R) {
-    for (int c = c0 + cl; c < c1; c += 8) {
+#pragma unroll 8
+    for (int c = c0 + cl; c < c1; c += 8) {        // independent loads: the unrolled loop keeps eight in flight
       const uint4 v = buf[(size_t)c * Rpad + n];
       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -43,6 +55,18 @@ __global__ void __launch_bounds__(256) row_norm_kernel(const uint4* __restrict__
     for (int i = 0; i < 8; ++i) s += sm[i][r];
     part[(size_t)(z * 2 + which) * Rpad + n] = s;
   }
+  // The CTA that finishes last adds the call to the accumulators (a warp per segment, fixed order): one
+  // launch instead of two, and still a single writer per accumulator row.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int total = (int)(gridDim.x * gridDim.y * gridDim.z);
+    is_last = atomicAdd(done_counter, 1) == total - 1;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int s = cl; s < S; s += 8) accumulate_segment(part, Rpad, offsets, perm, gates, E, s, r, acc);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -58,16 +82,10 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // One warp per expert segment: adds this call's pairs to the segment's eight accumulators (PW_OBS_*).  The
 // routing weight of operand row n of a routed expert is the gate of the pair perm[n]; a shared expert takes
-// every token with weight 1.
-__global__ void __launch_bounds__(128) observe_accumulate_kernel(const float* __restrict__ part, int Rpad,
-                                                                 const int32_t* __restrict__ offsets,
-                                                                 const int32_t* __restrict__ perm,
-                                                                 const float* __restrict__ gates, int E, int S,
-                                                                 float* __restrict__ acc) {
-  grid_dep_sync();
-  grid_dep_trigger();
-  const int s = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (s >= S) return;
+// every token with weight 1.  (`part` was written by other CTAs of this launch: read it past the L1.)
+__device__ void accumulate_segment(const float* part, int Rpad, const int32_t* __restrict__ offsets,
+                                   const int32_t* __restrict__ perm, const float* __restrict__ gates, int E, int s,
+                                   int lane, float* __restrict__ acc) {
   const int n0 = offsets[s], n1 = offsets[s + 1];
   if (n1 <= n0) return;
   float sr = 0.f, srx = 0.f, srx2 = 0.f, mx = 0.f, srh = 0.f, srh2 = 0.f, mh = 0.f;
@@ -76,8 +94,8 @@ __global__ void __launch_bounds__(128) observe_accumulate_kernel(const float* __
     float x2 = 0.f, h2 = 0.f;
 #pragma unroll
     for (int z = 0; z < kNormSplit; ++z) {
-      x2 += part[(size_t)(z * 2 + 0) * Rpad + n];
-      h2 += part[(size_t)(z * 2 + 1) * Rpad + n];
+      x2 += __ldcg(part + (size_t)(z * 2 + 0) * Rpad + n);
+      h2 += __ldcg(part + (size_t)(z * 2 + 1) * Rpad + n);
     }
     const float nx = sqrtf(x2), nh = sqrtf(h2);
     sr += r;
@@ -152,14 +170,13 @@ pw_status launch_observe(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s) {
     float* part = reinterpret_cast<float*>(b + w.obs_part);
     PW_CUDA_OK(launch_dependent(row_norm_kernel, dim3((R + 31) / 32, 2, kNormSplit), dim3(256), 0, s,
                                 reinterpret_cast<const uint4*>(b + w.xt), c.hidden / 8,
-                                reinterpret_cast<const uint4*>(b + w.ht), c.ffn / 8, w.Rpad, R, part));
-    PW_CUDA_OK(launch_dependent(observe_accumulate_kernel, dim3((w.S + 3) / 4), dim3(128), 0, s,
-                                static_cast<const float*>(part), w.Rpad,
+                                reinterpret_cast<const uint4*>(b + w.ht), c.ffn / 8, w.Rpad, R, part,
+                                reinterpret_cast<int32_t*>(b + w.counter) + 2,   // zeroed by the grouping kernel
                                 reinterpret_cast<const int32_t*>(b + w.offsets),
                                 reinterpret_cast<const int32_t*>(b + w.perm),
                                 reinterpret_cast<const float*>(b + w.gates), c.n_experts, w.S,
                                 ctx->obs_acc + (size_t)layer * w.S * PW_OBS_FIELDS));
-    ctx->launches += 2;
+    ctx->launches += 1;
     PW_CUDA_OK(cudaGetLastError());
   }
   timing_mark(ctx, PW_NUM_KERNELS, s);
