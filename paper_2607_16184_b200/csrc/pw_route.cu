@@ -226,8 +226,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
                                                      uint4* __restrict__ xt, const int32_t* __restrict__ counts,
                                                      const int2* __restrict__ tile_tab, int max_tiles,
                                                      const int32_t* __restrict__ n_units, int nt_tile, int ksplit,
-                                                     int ng_gu, int ng_dn, Unit* __restrict__ units_gu,
-                                                     Unit* __restrict__ units_dn) {
+                                                     int ng_gu, int ng_dn, int dn_token_tile_outer,
+                                                     Unit* __restrict__ units_gu, Unit* __restrict__ units_dn) {
   grid_dep_sync();
   grid_dep_trigger();
   if (nt_tile > 0) {
@@ -239,8 +239,22 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
       const int ng = phase == 0 ? ng_gu : ng_dn;
       const int2* tab = tile_tab + (size_t)phase * max_tiles;
       Unit* out = phase == 0 ? units_gu : units_dn;
+      // Row tile outermost by default: weight pages stream once, the token rows they multiply stay in L2.  When
+      // the operand rows of the down projection do not fit in L2 (a long prompt: 235 MB at 4096 tokens of a
+      // 14336-wide FFN) every row tile would pull them from HBM again; that list is laid out token tile
+      // outermost instead -- a token tile's rows are read once, and the pages of its expert (the tables keep an
+      // expert's token tiles together) are what stays in L2.
+      const bool tt_outer = phase == 1 && dn_token_tile_outer;
+      const int RS = TT > 0 ? total / TT : 0;
       for (int u = gt; u < total; u += n_threads) {
-        const int rs = u / TT, j = u - rs * TT;
+        int rs, j;
+        if (tt_outer) {
+          j = u / RS;
+          rs = u - j * RS;
+        } else {
+          rs = u / TT;
+          j = u - rs * TT;
+        }
         const int rt = rs / splits, sp = rs - rt * splits;
         const int2 t = tab[j];
         const int n = counts[t.x];
@@ -272,20 +286,25 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
 // terms in choice order: the arithmetic and its order do not depend on the launch shape, only the latency does
 // (a one-token call has a handful of CTAs, so a serial walk over choices x splits would be all latency).
 constexpr int kCombineCols = 64, kCombineRows = 4, kMaxSplit = 8;
+// kCombineChunks columns per thread, 64 apart: that many independent load chains in flight.  Four for a long
+// prompt (thousands of tokens: fewer, fatter CTAs), one for a decode batch (more CTAs for the few tokens).
+template <int kCombineChunks>
 __global__ void __launch_bounds__(kCombineCols * kCombineRows)
     combine_kernel(const float4* __restrict__ y, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
                    int T, int k, int n_shared, int H4, int ksplit, size_t split_stride4, float4* __restrict__ out) {
   grid_dep_sync();
   grid_dep_trigger();
-  __shared__ float4 term[kCombineRows][kCombineCols];
+  __shared__ float4 term[kCombineRows][kCombineChunks][kCombineCols];
   const int tx = threadIdx.x, ty = threadIdx.y;
-  const int c = blockIdx.x * kCombineCols + tx;
+  const int c_first = blockIdx.x * (kCombineCols * kCombineChunks) + tx;
   const int t = blockIdx.y;
   const int J = k + n_shared;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 acc[kCombineChunks];
+#pragma unroll
+  for (int cc = 0; cc < kCombineChunks; ++cc) acc[cc] = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int j0 = 0; j0 < J; j0 += kCombineRows) {
     const int j = j0 + ty;
-    if (j < J && c < H4) {
+    if (j < J) {
       int row;
       float g;
       if (j < k) {
@@ -295,34 +314,47 @@ __global__ void __launch_bounds__(kCombineCols * kCombineRows)
         row = T * k + (j - k) * T + t;
         g = 1.0f;
       }
-      float4 v[kMaxSplit];
 #pragma unroll
-      for (int s = 0; s < kMaxSplit; ++s)
-        if (s < ksplit) v[s] = y[s * split_stride4 + (size_t)row * H4 + c];
-      float4 a = v[0];
+      for (int cc = 0; cc < kCombineChunks; ++cc) {
+        const int c = c_first + cc * kCombineCols;
+        if (c >= H4) continue;
+        float4 v[kMaxSplit];
 #pragma unroll
-      for (int s = 1; s < kMaxSplit; ++s)
-        if (s < ksplit) {
-          a.x = __fadd_rn(a.x, v[s].x);
-          a.y = __fadd_rn(a.y, v[s].y);
-          a.z = __fadd_rn(a.z, v[s].z);
-          a.w = __fadd_rn(a.w, v[s].w);
-        }
-      term[ty][tx] = make_float4(__fmul_rn(g, a.x), __fmul_rn(g, a.y), __fmul_rn(g, a.z), __fmul_rn(g, a.w));
-    }
-    __syncthreads();
-    if (ty == 0) {
-      for (int i = 0; i < kCombineRows && j0 + i < J; ++i) {
-        const float4 b = term[i][tx];
-        acc.x = __fadd_rn(acc.x, b.x);
-        acc.y = __fadd_rn(acc.y, b.y);
-        acc.z = __fadd_rn(acc.z, b.z);
-        acc.w = __fadd_rn(acc.w, b.w);
+        for (int s = 0; s < kMaxSplit; ++s)
+          if (s < ksplit) v[s] = y[s * split_stride4 + (size_t)row * H4 + c];
+        float4 a = v[0];
+#pragma unroll
+        for (int s = 1; s < kMaxSplit; ++s)
+          if (s < ksplit) {
+            a.x = __fadd_rn(a.x, v[s].x);
+            a.y = __fadd_rn(a.y, v[s].y);
+            a.z = __fadd_rn(a.z, v[s].z);
+            a.w = __fadd_rn(a.w, v[s].w);
+          }
+        term[ty][cc][tx] = make_float4(__fmul_rn(g, a.x), __fmul_rn(g, a.y), __fmul_rn(g, a.z), __fmul_rn(g, a.w));
       }
     }
     __syncthreads();
+    if (ty == 0) {
+#pragma unroll
+      for (int cc = 0; cc < kCombineChunks; ++cc)
+        for (int i = 0; i < kCombineRows && j0 + i < J; ++i) {
+          const float4 b = term[i][cc][tx];
+          acc[cc].x = __fadd_rn(acc[cc].x, b.x);
+          acc[cc].y = __fadd_rn(acc[cc].y, b.y);
+          acc[cc].z = __fadd_rn(acc[cc].z, b.z);
+          acc[cc].w = __fadd_rn(acc[cc].w, b.w);
+        }
+    }
+    __syncthreads();
   }
-  if (ty == 0 && c < H4) out[(size_t)t * H4 + c] = acc;
+  if (ty == 0) {
+#pragma unroll
+    for (int cc = 0; cc < kCombineChunks; ++cc) {
+      const int c = c_first + cc * kCombineCols;
+      if (c < H4) out[(size_t)t * H4 + c] = acc[cc];
+    }
+  }
 }
 
 pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
@@ -352,6 +384,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
       reinterpret_cast<int2*>(b + w.tile_tab), w.max_tiles, reinterpret_cast<int32_t*>(b + w.n_units),
       reinterpret_cast<int32_t*>(b + w.seg_order), w.max_units, reinterpret_cast<int32_t*>(b + w.status)));
   const int R = T * k + c.n_shared * T;
+  const int dn_tt_outer = (size_t)R * c.ffn * 2 > ((size_t)64 << 20) ? 1 : 0;   // SwiGLU rows beyond half of the L2
   timing_mark(ctx, PW_K_GATHER, s);
   dim3 grid((R + 255) / 256, c.hidden / 8);
   PW_CUDA_OK(launch_dependent(gather_kernel, grid, dim3(256), 0, s, reinterpret_cast<const uint4*>(hidden),
@@ -360,7 +393,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
                               reinterpret_cast<uint4*>(b + w.xt), reinterpret_cast<const int32_t*>(b + w.counts),
                               reinterpret_cast<const int2*>(b + w.tile_tab), w.max_tiles,
                               reinterpret_cast<const int32_t*>(b + w.n_units), nt_tile, ksplit, c.hidden / kGroup,
-                              c.ffn / kGroup, reinterpret_cast<Unit*>(b + w.units_gu),
+                              c.ffn / kGroup, dn_tt_outer, reinterpret_cast<Unit*>(b + w.units_gu),
                               reinterpret_cast<Unit*>(b + w.units_dn)));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
@@ -373,9 +406,10 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
   char* b = ctx->base;
   const int H4 = c.hidden / 4;
   const int R = T * k + c.n_shared * T;
-  dim3 grid((H4 + kCombineCols - 1) / kCombineCols, T);
+  const int chunks = T >= 256 ? 4 : 1;
+  dim3 grid((H4 + kCombineCols * chunks - 1) / (kCombineCols * chunks), T);
   timing_mark(ctx, PW_K_COMBINE, s);
-  PW_CUDA_OK(launch_dependent(combine_kernel, grid, dim3(kCombineCols, kCombineRows), 0, s, reinterpret_cast<const float4*>(b + w.y),
+  PW_CUDA_OK(launch_dependent(chunks == 4 ? combine_kernel<4> : combine_kernel<1>, grid, dim3(kCombineCols, kCombineRows), 0, s, reinterpret_cast<const float4*>(b + w.y),
                               reinterpret_cast<const float*>(b + w.gates),
                               reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
                               (size_t)R * H4, reinterpret_cast<float4*>(out)));
