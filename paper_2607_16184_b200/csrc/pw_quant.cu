@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
   const size_t tile = (size_t)rt * ng + g;
 
   float v[32];
+  __half2 h16[SRC_BITS == 16 ? 16 : 1];             // the packed halves of a 16-bit source
   if constexpr (SRC_KIND == SRC_RAW) {
     const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(src_codes) +
                                                     ((size_t)rt * kTileRows + r) * cols + (size_t)g * kGroup + 32 * q);
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float2 f = __half22float2(h[j]);
+        h16[4 * i + j] = h[j];
         v[8 * i + 2 * j] = f.x;
         v[8 * i + 2 * j + 1] = f.y;
       }
@@ -68,7 +70,8 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
     if constexpr (SRC_BITS == 16) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float2 f = __half22float2(u32_as_h2(w[i]));
+        h16[i] = u32_as_h2(w[i]);
+        float2 f = __half22float2(h16[i]);
         v[2 * i] = f.x;
         v[2 * i + 1] = f.y;
       }
@@ -95,11 +98,27 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
     return;
   }
 
-  float lo = v[0], hi = v[0];
+  // minimum and maximum of my 32 values (of fp16 sources taken on the packed halves: half as many operations,
+  // and exact like the fp32 ones)
+  float lo, hi;
+  if constexpr (SRC_BITS == 16) {
+    __half2 lo2 = h16[0], hi2 = h16[0];
 #pragma unroll
-  for (int i = 1; i < 32; ++i) {
-    lo = fminf(lo, v[i]);
-    hi = fmaxf(hi, v[i]);
+    for (int i = 1; i < 16; ++i) {
+      lo2 = __hmin2(lo2, h16[i]);
+      hi2 = __hmax2(hi2, h16[i]);
+    }
+    const float2 lf = __half22float2(lo2), hf = __half22float2(hi2);
+    lo = fminf(lf.x, lf.y);
+    hi = fmaxf(hf.x, hf.y);
+  } else {
+    lo = v[0];
+    hi = v[0];
+#pragma unroll
+    for (int i = 1; i < 32; ++i) {
+      lo = fminf(lo, v[i]);
+      hi = fmaxf(hi, v[i]);
+    }
   }
 #pragma unroll
   for (int d = 1; d <= 2; d <<= 1) {
@@ -120,9 +139,10 @@ __global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict_
   int code[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) {
-    float c = rintf(__fmul_rn(__fsub_rn(v[i], lo), rinv));
-    c = fminf(fmaxf(c, 0.0f), (float)L);
-    code[i] = (int)c;
+    // round half to even and convert in one step (the product is never negative; a huge one saturates), then
+    // clamp: the same code as clamp(rint(x), 0, L)
+    const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v[i], lo), rinv));
+    code[i] = (int)(c < (uint32_t)L ? c : (uint32_t)L);
   }
   constexpr int NW = SliceWords<DST_BITS>::kWords;
   uint32_t w[NW];
