@@ -322,6 +322,58 @@ pw_status pw_observe(pw_ctx* ctx, float* accumulators, pw_stream stream);
  * Errors: INVALID_ARG, ALIGN, STATE (taps are off), CUDA. */
 pw_status pw_observation_summary(pw_ctx* ctx, int layer, float* mass, float* phi, pw_stream stream);
 
+/* ---- planner ------------------------------------------------------------------------- */
+
+/* One scoring + selection step of the runtime planner (Sec. 3.2, Alg. 1).  Host code, no context and no GPU
+ * needed; every pointer below is host memory.  A step lowers one linear-block from its current bitwidth to
+ * the next lower bitwidth it supports; its predicted damage is
+ *     d = max(epsilon, mu_bucket * g * eta)                                   (Eq. 8)
+ *     g = max(s^{b'} - s^{b}, 0)                                              (Eq. 4)
+ *     eta = exp(alpha * c * clip(w . phi + a, rho_min, rho_max))              (Eqs. 5-6; 1 without heads or
+ *                                                                              for an expert that saw no token)
+ * and the steps are taken cheapest damage per released byte first (ties: lower row index; a block's next step
+ * becomes available when the one before has been taken) until `target` bytes are released.  The experts of a
+ * layer are ranked by routing mass, hottest first, and bucket j holds the ranks below bucket_share[j] *
+ * n_experts; a bucket has a damage multiplier and, per stage, a bitwidth floor.  Stages are tried in order:
+ * the plan of the first stage that reaches the target is returned, otherwise the plan of the last stage (the
+ * largest reduction the floors allow).  Shared experts are never touched.  The paper does not print its
+ * calibrated constants (sensitivities, heads, buckets): they are the caller's.
+ * Row index i = (layer * (n_experts + n_shared) + expert) * 3 + kind; bitwidth levels in the order 16, 8, 4, 3, 2. */
+typedef struct {
+  int32_t n_layers, n_experts, n_shared;
+  const uint8_t* committed;     /* [rows] committed bitwidth q_i                                        */
+  const uint8_t* supported;     /* [rows][5] non-zero where the block has a page at that level (B_i)    */
+  const float* sensitivity;     /* [rows][5] offline sensitivity s_i^b                                  */
+  const uint64_t* page_bytes;   /* [rows][5] size table M_i^b (Eq. 3), e.g. from pw_page_bytes          */
+  const float* mass;            /* [n_layers][n_experts] routing mass (Eq. 1), e.g. pw_observation_summary */
+  const float* phi;             /* [rows][3] routed-input features, or NULL                            */
+  const float* head_w;          /* [3 kinds][5 from][5 to][3], or NULL: no prompt residual             */
+  const float* head_a;          /* [3][5][5]                                                            */
+  const float* head_c;          /* [3][5][5] confidence                                                 */
+  float alpha, rho_min, rho_max, epsilon;
+  int32_t n_buckets, n_stages;
+  const float* bucket_share;    /* [n_buckets] ascending, the last one 1                                */
+  const float* bucket_mu;       /* [n_buckets] damage multiplier, hottest bucket first                  */
+  const uint8_t* stage_floor;   /* [n_stages][n_buckets] lowest bitwidth a bucket may reach in a stage  */
+} pw_plan_tables;
+
+typedef struct {
+  int32_t layer, expert, kind;
+  uint8_t from_bits, to_bits;
+  uint64_t released_bytes;      /* M^{from} - M^{to}                                                    */
+  double damage;                /* d of Eq. 8                                                           */
+} pw_plan_item;
+
+/* steps: array of max_steps items (may be NULL with max_steps 0 to ask for the count); n_steps_out
+ * receives the number of steps of the plan, released_out (optional) their bytes, stage_out (optional) the
+ * stage used.  Errors: INVALID_ARG, BITS (a committed bitwidth or floor outside the levels), NOMEM (the plan
+ * has more than max_steps steps: nothing is written but the counts). */
+pw_status pw_plan_step(const pw_plan_tables* tables, uint64_t target, pw_plan_item* steps, size_t max_steps,
+                       size_t* n_steps_out, uint64_t* released_out, int32_t* stage_out);
+
+/* Eq. 7: bytes to release = max(0, free_block_threshold + 1 - free_blocks) * kv_block_bytes. */
+uint64_t pw_kv_pressure_bytes(int64_t free_block_threshold, int64_t free_blocks, uint64_t kv_block_bytes);
+
 /* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
  * then clears it. */
 pw_status pw_last_device_status(pw_ctx* ctx);

@@ -28,7 +28,8 @@ GROUP = 128
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
            "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
-           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_last_device_status",
+           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_kv_pressure_bytes",
+           "pw_last_device_status",
            "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_status_str")
 KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "observe")
 PW_OBS_FIELDS = 8
@@ -55,6 +56,20 @@ class pw_page(C.Structure):
 class pw_table_entry(C.Structure):
     _fields_ = [("layer", C.c_int32), ("expert", C.c_int32), ("kind", C.c_int32), ("page", pw_page),
                 ("desired_bits", C.c_uint8), ("state", C.c_uint8)]
+
+
+class pw_plan_tables(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_experts", C.c_int32), ("n_shared", C.c_int32),
+                ("committed", C.c_void_p), ("supported", C.c_void_p), ("sensitivity", C.c_void_p),
+                ("page_bytes", C.c_void_p), ("mass", C.c_void_p), ("phi", C.c_void_p), ("head_w", C.c_void_p),
+                ("head_a", C.c_void_p), ("head_c", C.c_void_p), ("alpha", C.c_float), ("rho_min", C.c_float),
+                ("rho_max", C.c_float), ("epsilon", C.c_float), ("n_buckets", C.c_int32), ("n_stages", C.c_int32),
+                ("bucket_share", C.c_void_p), ("bucket_mu", C.c_void_p), ("stage_floor", C.c_void_p)]
+
+
+class pw_plan_item(C.Structure):
+    _fields_ = [("layer", C.c_int32), ("expert", C.c_int32), ("kind", C.c_int32), ("from_bits", C.c_uint8),
+                ("to_bits", C.c_uint8), ("released_bytes", C.c_uint64), ("damage", C.c_double)]
 
 
 _lib = None
@@ -111,6 +126,11 @@ def load():
     L.pw_observe.argtypes = [vp, vp, vp]
     L.pw_observation_summary.restype = i32
     L.pw_observation_summary.argtypes = [vp, i32, vp, vp, vp]
+    L.pw_plan_step.restype = i32
+    L.pw_plan_step.argtypes = [C.POINTER(pw_plan_tables), C.c_uint64, C.POINTER(pw_plan_item), sz, C.POINTER(sz),
+                               C.POINTER(C.c_uint64), C.POINTER(C.c_int32)]
+    L.pw_kv_pressure_bytes.restype = C.c_uint64
+    L.pw_kv_pressure_bytes.argtypes = [C.c_int64, C.c_int64, C.c_uint64]
     L.pw_last_device_status.restype = i32
     L.pw_last_device_status.argtypes = [vp]
     L.pw_kernel_timing.restype = i32
@@ -141,6 +161,46 @@ def pw_page_bytes(rows: int, cols: int, bits: int, group: int = GROUP) -> Tuple[
     a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
     tot = load().pw_page_bytes(rows, cols, bits, group, C.byref(a), C.byref(b), C.byref(c))
     return int(tot), int(a.value), int(b.value), int(c.value)
+
+
+def pw_kv_pressure_bytes(free_block_threshold: int, free_blocks: int, kv_block_bytes: int) -> int:
+    """Eq. 7: bytes the planner has to release."""
+    return int(load().pw_kv_pressure_bytes(free_block_threshold, free_blocks, kv_block_bytes))
+
+
+def pw_plan_step(n_layers: int, n_experts: int, n_shared: int, committed, supported, sensitivity, page_bytes, mass,
+                 bucket_share, bucket_mu, stage_floor, target: int, phi=None, heads=None, alpha: float = 1.0,
+                 rho_min: float = -1.0, rho_max: float = 1.0, epsilon: float = 1e-9):
+    """One planner step on host arrays (numpy; shapes as in include/pw.h).  Returns (steps, released bytes,
+    stage) with steps as tuples (layer, expert, kind, from_bits, to_bits, damage)."""
+    import numpy as np
+    keep = []
+
+    def ptr(a, dt):
+        if a is None:
+            return None
+        a = np.ascontiguousarray(a, dt)
+        keep.append(a)
+        return a.ctypes.data
+
+    floors = np.ascontiguousarray(stage_floor, np.uint8)
+    t = pw_plan_tables()
+    t.n_layers, t.n_experts, t.n_shared = n_layers, n_experts, n_shared
+    t.committed, t.supported = ptr(committed, np.uint8), ptr(supported, np.uint8)
+    t.sensitivity, t.page_bytes = ptr(sensitivity, np.float32), ptr(page_bytes, np.uint64)
+    t.mass, t.phi = ptr(mass, np.float32), ptr(phi, np.float32)
+    if heads is not None:
+        t.head_w, t.head_a, t.head_c = ptr(heads["w"], np.float32), ptr(heads["a"], np.float32), ptr(heads["c"], np.float32)
+    t.alpha, t.rho_min, t.rho_max, t.epsilon = alpha, rho_min, rho_max, epsilon
+    t.n_buckets, t.n_stages = floors.shape[1], floors.shape[0]
+    t.bucket_share, t.bucket_mu, t.stage_floor = ptr(bucket_share, np.float32), ptr(bucket_mu, np.float32), ptr(floors, np.uint8)
+    n_rows = n_layers * (n_experts + n_shared) * 3
+    cap = n_rows * 4
+    items = (pw_plan_item * cap)()
+    n, rel, stage = C.c_size_t(), C.c_uint64(), C.c_int32()
+    _check(load().pw_plan_step(C.byref(t), target, items, cap, C.byref(n), C.byref(rel), C.byref(stage)), "pw_plan_step")
+    steps = [(it.layer, it.expert, it.kind, it.from_bits, it.to_bits, it.damage) for it in items[: n.value]]
+    return steps, int(rel.value), int(stage.value)
 
 
 def pw_route_tokens_static(router_logits: torch.Tensor, top_k: int,
