@@ -8,12 +8,13 @@ constexpr int kMaxExpertsPerLane = 8;  // E <= 256
 constexpr int kFusedRouteWork = 256;   // (token, choice) pairs x 32-expert strides up to which the grouping kernel routes itself
 
 // Routing of one token by one warp.  Slot j holds the j-th largest logit; equal logits: lower expert index first.
-__device__ __forceinline__ void route_token(const float* __restrict__ logits, int token, int E, int k,
-                                            int32_t* __restrict__ topk_ids, float* __restrict__ gates, int lane) {
+template <int NS>   // NS = 32-expert strides a lane holds (1, 2, 4 or 8): the loops below cost in proportion
+__device__ __forceinline__ void route_token_n(const float* __restrict__ logits, int token, int E, int k,
+                                              int32_t* __restrict__ topk_ids, float* __restrict__ gates, int lane) {
   const float* l = logits + (size_t)token * E;
-  float v[kMaxExpertsPerLane];
+  float v[NS];
 #pragma unroll
-  for (int i = 0; i < kMaxExpertsPerLane; ++i) {
+  for (int i = 0; i < NS; ++i) {
     const int e = lane + 32 * i;
     v[i] = e < E ? l[e] : -INFINITY;
   }
@@ -24,7 +25,7 @@ __device__ __forceinline__ void route_token(const float* __restrict__ logits, in
     float bv = -INFINITY;
     int bi = 0x7fffffff;
 #pragma unroll
-    for (int i = 0; i < kMaxExpertsPerLane; ++i) {
+    for (int i = 0; i < NS; ++i) {
       const int e = lane + 32 * i;
       const bool ok = e < E && !((taken >> i) & 1u);
       if (ok && (v[i] > bv || (v[i] == bv && e < bi))) {
@@ -57,6 +58,14 @@ __device__ __forceinline__ void route_token(const float* __restrict__ logits, in
   }
 }
 
+__device__ __forceinline__ void route_token(const float* __restrict__ logits, int token, int E, int k,
+                                            int32_t* __restrict__ topk_ids, float* __restrict__ gates, int lane) {
+  if (E <= 32) route_token_n<1>(logits, token, E, k, topk_ids, gates, lane);
+  else if (E <= 64) route_token_n<2>(logits, token, E, k, topk_ids, gates, lane);
+  else if (E <= 128) route_token_n<4>(logits, token, E, k, topk_ids, gates, lane);
+  else route_token_n<kMaxExpertsPerLane>(logits, token, E, k, topk_ids, gates, lane);
+}
+
 // One warp per token.
 __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ logits, int T, int E, int k,
                                                      int32_t* __restrict__ topk_ids, float* __restrict__ gates) {
@@ -68,11 +77,35 @@ __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ l
 }
 
 #ifdef PW_TC_PROFILE
+// Diagnostic build only: clock stamps of the grouping kernel's phases.
 __device__ long long g_ptrace[32];
 #define PSTAMP(i) if (threadIdx.x == 0) g_ptrace[i] = clock64()
+extern "C" int pw_debug_read_ptrace(long long* host_out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host_out, g_ptrace, sizeof(g_ptrace));
+  return 0;
+}
 #else
 #define PSTAMP(i)
 #endif
+
+// out[i] = in[0] + .. + in[i - 1] for i = 0 .. n (n + 1 results), by one warp, 32 values per step.
+__device__ __forceinline__ void warp_exclusive_scan(const int32_t* in, int32_t* out, int n, int lane) {
+  int carry = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int i = base + lane;
+    const int x = i < n ? in[i] : 0;
+    int incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (i < n) out[i] = carry + incl - x;
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) out[n] = carry;
+}
 
 // Single CTA.  Stable counting sort of the P = T*k pairs by expert (positions come from ordered
 // prefix counts, never from atomics), segment table including the shared experts, operand-row ->
@@ -101,6 +134,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
   int32_t* order = ubase + S + 1;    // [S]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = T * k;
+  PSTAMP(12);
   if (logits) {
     for (int t = warp; t < T; t += (int)(blockDim.x >> 5)) route_token(logits, t, E, k, topk_ids, gates, lane);
     __syncthreads();                                 // the pairs below are read back from global memory
@@ -114,14 +148,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
   for (int p = tid; p < P; p += blockDim.x) atomicAdd(&cnt[topk_ids[p]], 1);
   __syncthreads();
   PSTAMP(1);
-  if (tid == 0) {
-    int a = 0;
-    for (int e = 0; e < S; ++e) {
-      off[e] = a;
-      a += cnt[e];
-    }
-    off[S] = a;
-  }
+  if (warp == 0) warp_exclusive_scan(cnt, off, S, lane);
   __syncthreads();
   for (int e = tid; e < S; e += blockDim.x) counts[e] = cnt[e];
   for (int e = tid; e <= S; e += blockDim.x) offsets[e] = off[e];
@@ -188,17 +215,12 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
     PSTAMP(5 + 4 * phase);
     const int row_tiles = (phase == 0 ? F : H) / kTileRows;
     const int splits = phase == 0 ? 1 : ksplit;
-    // token tiles per segment in rank order (in parallel), then their prefix (S additions by one thread)
+    // token tiles per segment in rank order (in parallel), then their prefix (one warp)
     for (int i = tid; i < S; i += blockDim.x) ubase[i + 1] = (cnt[order[i]] + nt_tile - 1) / nt_tile;
     __syncthreads();
+    if (warp == 0) warp_exclusive_scan(ubase + 1, ubase, S, lane);   // in place: a value is read before its slot is written
     if (tid == 0) {
-      int a = 0;
-      for (int i = 0; i < S; ++i) {
-        const int tt = ubase[i + 1];
-        ubase[i] = a;
-        a += tt;
-      }
-      ubase[S] = a;
+      const int a = ubase[S];
       const long long total = (long long)a * row_tiles * splits;
       const bool fits = total <= max_units && a <= max_tiles;
       n_units[phase] = fits ? (int)total : 0;
