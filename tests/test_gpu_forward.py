@@ -280,3 +280,31 @@ def test_limits_of_the_configuration(orc, shape, mode):
     E, k, n_shared, H, F, T = shape
     cfg = synth.LayerConfig("limits_%d_%d" % (E, k), E, k, H, F, T, n_shared=n_shared, routing="normal", bit_rule="iid5")
     run_case(orc, cfg, mode)
+
+
+def test_host_buffer_entry_point_matches_the_device_one(orc):
+    """pw_moe_forward_host stages the inputs, runs the same kernels and copies the result back, ordered on the
+    stream: same bits as the device call, with pinned and with pageable host buffers, several calls in a row."""
+    cfg = synth.CONFIGS["tiny_cover"]
+    ctx = make_ctx(cfg, n_layers=1)
+    try:
+        pages, _ = build_layer(ctx, cfg, 0, None)
+        for step, pinned in ((0, True), (1, False), (2, True)):
+            x = synth.activations(cfg, step=step, device="cuda")
+            lg = synth.router_logits(cfg, step=step, device="cuda")
+            want = ctx.pw_moe_forward(0, x, lg, cfg.top_k).clone()
+            xh, lh = x.cpu(), lg.cpu()
+            oh = torch.empty(cfg.tokens, cfg.hidden, dtype=torch.float32)
+            if pinned:
+                xh, lh, oh = xh.pin_memory(), lh.pin_memory(), oh.pin_memory()
+            ctx.pw_moe_forward_host(0, xh, lh, cfg.top_k, oh)
+            torch.cuda.synchronize()
+            assert torch.equal(oh, want.cpu()), (step, pinned)
+        with pytest.raises(B.PwError) as e:
+            big = torch.zeros(cfg.tokens + 1, cfg.hidden, dtype=torch.float16)
+            ctx.pw_moe_forward_host(0, big, torch.zeros(cfg.tokens + 1, cfg.n_experts), cfg.top_k,
+                                    torch.empty(cfg.tokens + 1, cfg.hidden))
+        assert e.value.status == 1
+        assert ctx.pw_last_device_status() == 0
+    finally:
+        ctx.close()
