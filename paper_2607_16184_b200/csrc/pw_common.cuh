@@ -160,8 +160,9 @@ void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 // are visible; a thread calls it before it reads anything that kernel wrote.  grid_dep_trigger() lets the
 // kernel after this one be placed as soon as SMs free up; a kernel calls it only after its own
 // grid_dep_sync(), so "my CTA has been placed" implies that every kernel two or more steps back in the chain
-// has completed.  That is what allows the FFN kernels to start streaming weight pages at once (unit lists
-// and page-table rows are written two steps back or earlier) and to wait only before their first token tile.
+// has completed.  That is what allows the down kernel to start streaming weight pages at once (its unit list
+// and the page-table rows are written two steps back or earlier) and to wait only before its first token
+// tile; the gate/up kernel's unit list is written one step back, so its weight producers wait as well.
 // With the timing events between the kernels the attribute has no effect.
 __device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
