@@ -1,6 +1,7 @@
 """pw_route_tokens_static: the routing entry point for callers that cannot allocate device memory
 (no context, no workspace; scratch lives in a fixed array inside the library).  Checked against the
-routing that pw_moe_forward performs, on two calls in a row, since every call reuses the same scratch."""
+routing that pw_moe_forward performs and against the CPU oracle's router and stable permutation, on two
+calls in a row, since every call reuses the same scratch."""
 import numpy as np
 import pytest
 import torch
@@ -24,7 +25,19 @@ def reference_routing(cfg, logits, T):
     return r
 
 
-def test_static_routing_matches_forward_routing_twice_in_a_row():
+def check_against_oracle(orc, got, logits, top_k):
+    """Indices bit for bit, gates to 1e-6 relative (expf differs by ulps between libm and the device)."""
+    lg = logits.cpu().numpy()
+    ids, gates = orc.router(lg, top_k)
+    counts, offsets, perm, _ = orc.permute(ids, lg.shape[1])
+    assert np.array_equal(got["topk_ids"].cpu().numpy(), ids)
+    assert np.array_equal(got["counts"].cpu().numpy(), counts)
+    assert np.array_equal(got["offsets"].cpu().numpy(), offsets)
+    assert np.array_equal(got["perm"].cpu().numpy(), perm)
+    np.testing.assert_allclose(got["gates"].cpu().numpy(), gates, rtol=1e-6, atol=1e-9)
+
+
+def test_static_routing_matches_forward_routing_twice_in_a_row(orc):
     cfg = synth.LayerConfig("route_small", 64, 6, 256, 384, 200, routing="zipf", zipf_a=1.2, bit_rule="all16")
     T = cfg.tokens
     first = synth.router_logits(cfg, 0, 0, device="cuda")
@@ -36,10 +49,12 @@ def test_static_routing_matches_forward_routing_twice_in_a_row():
         for name in ("topk_ids", "counts", "offsets", "perm"):
             assert torch.equal(got[name], ref[name]), name
         assert torch.equal(got["gates"].view(torch.int32), ref["gates"].view(torch.int32))
+        check_against_oracle(orc, got, logits, cfg.top_k)
     # and again the first input: same answer as before
     again = B.pw_route_tokens_static(first.contiguous(), cfg.top_k)
     ref = reference_routing(cfg, first.contiguous(), T)
     assert torch.equal(again["perm"], ref["perm"]) and torch.equal(again["counts"], ref["counts"])
+    check_against_oracle(orc, again, first, cfg.top_k)
 
 
 def test_static_routing_rejects_what_does_not_fit():
