@@ -50,12 +50,16 @@ def measured_peaks():
 
 
 def profiled_traffic(name: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None."""
+    """(DRAM bytes per launch of the dominant kernel, algorithmic bytes of the same captured launches) from the
+    committed ncu summary, or (None, None).  The capture covers one launch per layer the bench rotates over, so
+    the two averages are like for like with `algorithmic_bytes_per_launch`."""
     p = os.path.join(ROOT, "profiles", name)
     if not os.path.exists(p):
-        return None
-    m = re.search(r"dram_bytes_per_launch_full_size:\s*([0-9.eE+]+)", open(p).read())
-    return float(m.group(1)) if m else None
+        return None, None
+    txt = open(p).read()
+    m = re.search(r"dram_bytes_per_launch_full_size:\s*([0-9.eE+]+)", txt)
+    a = re.search(r"algorithmic_bytes_per_launch_of_capture:\s*([0-9.eE+]+)", txt)
+    return (float(m.group(1)) if m else None), (float(a.group(1)) if a else None)
 
 
 class ClockSampler:
@@ -195,7 +199,7 @@ def export_layer_to_host(ctx, layer, cfg):
     return out
 
 
-def run_prefill(device, peaks, steps=3, warmup=1):
+def run_prefill(device, peaks, steps=20, warmup=3):
     """Prefill configuration (4096 tokens, bits from {16,8,4}): useful TFLOP/s of one layer call."""
     from paper_2607_16184_b200 import binding as B
     cfg = synth.CONFIGS["mixtral_prefill"]
@@ -343,6 +347,76 @@ def run_residency(ctx, cfg, layers, device, decode_fn, decode_ms):
                              "steps": n_steps}}
 
 
+def algorithmic_bytes(ctx, cfg, layers, out, mode):
+    """(gate+up page bytes, down page bytes) of the experts that hold tokens, averaged over the layers."""
+    T, k, L = cfg.tokens, cfg.top_k, len(layers)
+    gu_bytes = dn_bytes = 0.0
+    for li, lay in enumerate(layers):
+        ctx.pw_moe_forward(li, lay["x"], lay["logits"], k, out=out, mode=mode)
+        counts = ctx.pw_get_routing(T, k)["counts"].cpu().numpy()
+        active = np.concatenate([counts > 0, np.ones(cfg.n_shared, bool)])
+        gu, dn = page_bytes_total(lay["bits"], cfg, active)
+        gu_bytes += gu / L
+        dn_bytes += dn / L
+    return gu_bytes, dn_bytes
+
+
+def kernel_pass(ctx, step, steps, device):
+    """Per-kernel device times of the same loop: events recorded around every kernel of the call."""
+    ctx.pw_kernel_timing(True)
+    ms = time_region(step, steps, device)
+    ktimes, kcalls = ctx.pw_get_kernel_times()
+    ctx.pw_kernel_timing(False)
+    return {n: v / max(kcalls, 1) for n, v in ktimes.items()}, ms / steps
+
+
+def decode_workload(device, peaks, cfg, L, mode, steps, warmup, min_seconds=0.6):
+    """One decode configuration in a context of its own: step time, per-kernel times and roofline fractions of a
+    region of at least `min_seconds` of back-to-back steps (sampled clocks), rotating over L distinct layers."""
+    from paper_2607_16184_b200 import binding as B
+    ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
+    layers = build_layers(ctx, cfg, L, device)
+    T, k = cfg.tokens, cfg.top_k
+    out = torch.empty(T, cfg.hidden, dtype=torch.float32, device=device)
+
+    def step(i):
+        lay = layers[i % L]
+        ctx.pw_set_page_table(lay["entries"][(i // L) % len(lay["entries"]):][:1])
+        ctx.pw_moe_forward(i % L, lay["x"], lay["logits"], k, out=out, mode=mode)
+
+    for i in range(max(warmup, 3)):
+        step(i)
+    ms_probe = time_region(step, max(steps, 20), device) / max(steps, 20)
+    n = max(steps, int(np.ceil(min_seconds / (ms_probe * 1e-3))))
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    ms_step = time_region(step, n, device) / n
+    clocks = sampler.stop()
+    kavg, _ = kernel_pass(ctx, step, n, device)
+    status = ctx.pw_last_device_status()
+    gu_bytes, dn_bytes = algorithmic_bytes(ctx, cfg, layers, out, mode)
+    R = T * k + cfg.n_shared * T
+    io_bytes = 2 * T * cfg.hidden + 4 * T * cfg.n_experts + 4 * T * cfg.hidden
+    call_bytes = gu_bytes + dn_bytes + io_bytes
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    gu_gbs = gbs(gu_bytes + 2.0 * R * cfg.hidden, kavg["ffn_gate_up"])
+    dn_gbs = gbs(dn_bytes + 2.0 * R * cfg.ffn, kavg["ffn_down"])
+    res = {"workload": "%s: E=%d+%d top-%d H=%d F=%d T=%d, %s routing, bit rule %s, %d layers of %.3f GB of pages"
+                       % (cfg.name, cfg.n_experts, cfg.n_shared, k, cfg.hidden, cfg.ffn, T, cfg.routing, cfg.bit_rule, L,
+                          (gu_bytes + dn_bytes) / 1e9),
+           "steps": n, "ms_per_step": ms_step, "tokens_per_s": T / (ms_step * 1e-3), "sm_mhz": clocks["sm_mhz"],
+           "reasons": clocks["reasons"], "algorithmic_bytes_per_call": call_bytes,
+           "forward_gbs": gbs(call_bytes, ms_step), "forward_frac": gbs(call_bytes, ms_step) / peaks["hbm_gbs"],
+           "gate_up_ms": kavg["ffn_gate_up"], "gate_up_gbs": gu_gbs, "gate_up_frac": gu_gbs / peaks["hbm_gbs"],
+           "down_ms": kavg["ffn_down"], "down_gbs": dn_gbs, "down_frac": dn_gbs / peaks["hbm_gbs"],
+           "small_kernels_ms": sum(v for n_, v in kavg.items() if not n_.startswith("ffn")),
+           "device_status": status}
+    ctx.close()
+    del layers, ctx
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_gpu(args):
     from paper_2607_16184_b200 import binding as B
     from paper_2607_16184_b200 import build as pwbuild
@@ -385,34 +459,42 @@ def run_gpu(args):
     value = tokens_all / (ms_max * 1e-3)
 
     # per-kernel device times, same loop, events recorded around every kernel of the call
-    ctx.pw_kernel_timing(True)
-    ms_timed = time_region(step, args.steps, device)
-    ktimes, kcalls = ctx.pw_get_kernel_times()
-    ctx.pw_kernel_timing(False)
-    kavg = {n: v / max(kcalls, 1) for n, v in ktimes.items()}
+    kavg, ms_timed_step = kernel_pass(ctx, step, args.steps, device)
 
     # algorithmic bytes of a layer call: pages of experts that hold tokens + activations in/out
-    gu_bytes = dn_bytes = 0.0
-    for li, lay in enumerate(layers):
-        ctx.pw_moe_forward(li, lay["x"], lay["logits"], k, out=out, mode=mode)
-        counts = ctx.pw_get_routing(T, k)["counts"].cpu().numpy()
-        active = np.concatenate([counts > 0, np.ones(cfg.n_shared, bool)])
-        gu, dn = page_bytes_total(lay["bits"], cfg, active)
-        gu_bytes += gu / L
-        dn_bytes += dn / L
+    gu_bytes, dn_bytes = algorithmic_bytes(ctx, cfg, layers, out, mode)
     R = T * k + cfg.n_shared * T
     io_bytes = 2 * T * cfg.hidden + 4 * T * cfg.n_experts + 4 * T * cfg.hidden
     call_bytes = gu_bytes + dn_bytes + io_bytes
     ms_step = ms_max / args.steps
     gu_kernel_bytes = gu_bytes + 2.0 * R * cfg.hidden           # pages + the gathered fp16 token rows it reads
-    gu_gbs = gu_kernel_bytes / (kavg["ffn_gate_up"] * 1e-3) / 1e9 if kavg["ffn_gate_up"] > 0 else 0.0
-    dn_gbs = (dn_bytes + 2.0 * R * cfg.ffn) / (kavg["ffn_down"] * 1e-3) / 1e9 if kavg["ffn_down"] > 0 else 0.0
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    gu_gbs = gbs(gu_kernel_bytes, kavg["ffn_gate_up"])
+    dn_gbs = gbs(dn_bytes + 2.0 * R * cfg.ffn, kavg["ffn_down"])
+    traffic, traffic_alg = (profiled_traffic("ffn_gate_up_mixtral_decode.md")
+                            if cfg.name == "mixtral_decode" and not args.uniform_bits else (None, None))
     roofline = {"bound": "hbm", "kernel": "ffn_tc_kernel<0> (gate/up + SwiGLU)", "achieved": gu_gbs,
                 "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": gu_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gu_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": gu_kernel_bytes, "avg_launch_ms": kavg["ffn_gate_up"],
-                "traffic": profiled_traffic("ffn_gate_up_mixtral_decode.md")
-                if cfg.name == "mixtral_decode" and not args.uniform_bits else None}
+                "traffic": traffic, "traffic_capture_algorithmic_bytes": traffic_alg}
+
+    # Steady state: whatever --steps was, at least 0.6 s of back-to-back steps with the clocks sampled (a short
+    # region right after an idle moment runs at boost clocks; a serving loop runs under the power cap), then the
+    # per-kernel pass of the same length.
+    n_steady = max(args.steps, int(np.ceil(args.steady_seconds / (ms_step * 1e-3))))
+    sampler2 = ClockSampler(device.index or 0)
+    sampler2.start()
+    ms_steady = time_region(step, n_steady, device) / n_steady
+    clocks2 = sampler2.stop()
+    kavg2, _ = kernel_pass(ctx, step, n_steady, device)
+    steady = {"steps": n_steady, "ms_per_step": ms_steady, "tokens_per_s": T / (ms_steady * 1e-3),
+              "sm_mhz": clocks2["sm_mhz"], "reasons": clocks2["reasons"],
+              "roofline_frac": gbs(gu_kernel_bytes, kavg2["ffn_gate_up"]) / peaks["hbm_gbs"],
+              "gate_up_ms": kavg2["ffn_gate_up"], "down_ms": kavg2["ffn_down"],
+              "down_frac": gbs(dn_bytes + 2.0 * R * cfg.ffn, kavg2["ffn_down"]) / peaks["hbm_gbs"],
+              "forward_frac": gbs(call_bytes, ms_steady) / peaks["hbm_gbs"],
+              "forward_frac_of_nominal_8000": gbs(call_bytes, ms_steady) / NOMINAL_HBM_GBS}
 
     # end to end: host buffers in, host buffer out, through the host-buffer entry point
     xh = [lay["x"].cpu().pin_memory() for lay in layers]
@@ -441,11 +523,11 @@ def run_gpu(args):
                        "mode": args.mode, "l2": "inputs larger than L2", "replicas": world,
                        "bits_realised": {str(b): int((np.stack([l["bits"] for l in layers]) == b).sum()) for b in synth.BITS}},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": status,
-            "roofline": roofline,
-            "forward": {"algorithmic_bytes_per_call": call_bytes, "hbm_gbs": call_bytes / (ms_step * 1e-3) / 1e9,
-                        "frac_of_measured_hbm": call_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                        "frac_of_nominal_8000": call_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                        "kernel_ms": kavg, "kernel_timed_ms_per_step": ms_timed / args.steps,
+            "roofline": roofline, "steady": steady,
+            "forward": {"algorithmic_bytes_per_call": call_bytes, "hbm_gbs": gbs(call_bytes, ms_step),
+                        "frac_of_measured_hbm": gbs(call_bytes, ms_step) / peaks["hbm_gbs"],
+                        "frac_of_nominal_8000": gbs(call_bytes, ms_step) / NOMINAL_HBM_GBS,
+                        "kernel_ms": kavg, "kernel_timed_ms_per_step": ms_timed_step,
                         "ffn_down_gbs": dn_gbs}}
 
     if rank == 0 and world == 1 and not args.skip_extra:
@@ -489,6 +571,22 @@ def run_gpu(args):
         line["demote"] = run_demote(ctx, cfg, layers, device, peaks, step, ms_step)
         line["residency"] = run_residency(ctx, cfg, layers, device, step, ms_step)
         line["prefill"] = run_prefill(device, peaks)     # its own context and pages (about 2 GB more)
+        if cfg.name == "mixtral_decode" and not args.uniform_bits:
+            # does a demote buy time?  the gate/up and down kernels on tables of one bitwidth each
+            import dataclasses
+            per_bits = {}
+            for b in synth.BITS:
+                r = decode_workload(device, peaks, dataclasses.replace(cfg, bit_rule="uniform%d" % b), 1, mode, 100, 3,
+                                    min_seconds=0.15)
+                per_bits[str(b)] = {key: r[key] for key in ("ms_per_step", "gate_up_ms", "gate_up_gbs", "gate_up_frac",
+                                                             "down_ms", "down_gbs", "down_frac", "forward_frac",
+                                                             "sm_mhz")}
+                per_bits[str(b)]["gate_up_tiles_per_s"] = (2.0 * cfg.n_experts * (cfg.ffn // 128) * (cfg.hidden // 128)
+                                                           / (r["gate_up_ms"] * 1e-3))
+            line["per_bits"] = per_bits
+            # the other decode configuration (64 routed top-6 + 2 shared experts, batch 256)
+            line["finegrained_decode"] = decode_workload(device, peaks, synth.CONFIGS["finegrained_decode"], 6, mode,
+                                                         200, 5)
     # (the CPU oracle runs after the GPU extras: its OpenMP threads keep the host cores busy for a while
     # afterwards, and the extras' launch loops must not compete with them)
     if rank == 0 and world == 1 and not args.skip_cpu:
@@ -509,25 +607,55 @@ def run_gpu(args):
                                           % (calls, min(args.cpu_tokens, T), T, dt_all)}
     else:
         line["cpu_baseline"] = None
+    if rank == 0 and world == 1 and not args.skip_extra and cfg.name == "mixtral_decode" and not args.uniform_bits:
+        # the fifth configuration at full size, when the device has the memory for it (90 GB of pages)
+        ctx.close()
+        del layers, ctx, xh, lh
+        torch.cuda.empty_cache()
+        free, _ = torch.cuda.mem_get_info(device)
+        if free >= 110e9:
+            d5 = measure_d5(device, peaks, parity_pages=2)
+            line["demote_under_load"] = {"workload": d5["config"]["workload"], "tokens_per_s": d5["value"],
+                                         "ms_per_step": d5["ms_per_step"], "roofline_frac_all_16bit": d5["roofline"]["frac"],
+                                         "d5": d5["d5"], "device_status": d5["device_status"], "clocks": d5["clocks"]}
+        else:
+            line["demote_under_load"] = {"skipped": "%.0f GB of device memory free, 110 GB needed" % (free / 1e9)}
     if rank == 0:
         print(json.dumps(line))
     replicas.shutdown()
 
 
-def run_d5(args):
+def check_pages_against_oracle(ctx, cfg, pages, keys, chain):
+    """A checking leg, not part of the timed path: the committed pages `keys` compared bit for bit with the CPU
+    oracle's quantize / demote chain on the regenerated weights.  Returns the number of pages that matched."""
+    from oracle import oracle
+    oracle.build()
+    ok = 0
+    for key in keys:
+        w = synth.block_weights(cfg, *key, device=ctx.device).cpu().numpy()   # the same draw as the page's
+        op = oracle.quantize_block(w, 16)
+        for b in chain:
+            op = oracle.demote_block(op, b)
+        ex = ctx.pw_export_page(pages[key])
+        torch.cuda.synchronize()
+        ng = pages[key].cols // 128
+        same = ex.bits == op.bits and np.array_equal(ex.codes.cpu().numpy(), op.codes)
+        if same and op.bits < 16:
+            same = (np.array_equal(ex.scales.view(torch.int16).cpu().numpy().view(np.uint16).reshape(-1, ng), op.scales)
+                    and np.array_equal(ex.zps.view(torch.int16).cpu().numpy().view(np.uint16).reshape(-1, ng), op.zps))
+        ok += int(bool(same))
+        del ex, op
+    return ok
+
+
+def measure_d5(device, peaks, parity_pages=4):
     """The demotion-under-load configuration at full size: 32 stacked Mixtral-shaped layers, all 16-bit at the
     start (90 GB of pages), a seeded third of the blocks demoted 16->4 and then 4->2 on a side stream while
     batch-64 decode steps (one call per layer) keep running.  Three runs: decode alone; "shadow" (demotes run
     but are never committed: pure interference); "committed" (every finished demote is published at the next
-    call boundary and the page it replaces is released)."""
+    call boundary and the page it replaces is released).  Afterwards a seeded sample of the committed pages is
+    compared with the oracle's chain."""
     from paper_2607_16184_b200 import binding as B
-    from paper_2607_16184_b200 import build as pwbuild
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    device = torch.device("cuda", 0)
-    torch.cuda.set_device(device)
-    pwbuild.build()
-    peaks = measured_peaks()
     cfg = synth.CONFIGS["demote_under_load"]
     T, k = cfg.tokens, cfg.top_k
     per_layer = sum(B.pw_page_bytes(*cfg.block_shape(u), 16)[0] for u in range(3)) * cfg.n_experts
@@ -670,18 +798,35 @@ def run_d5(args):
                               "slowdown": 1.0 - ms_base / ms_shadow, "demotes_per_step": per_step,
                               "demote_gbs_side_stream": shadow_gbs},
                    "committed": phases, "page_bytes_start": bytes_start}}
-    print(json.dumps(line), flush=True)
+    picks = [sched[i] for i in np.random.default_rng(11).choice(len(sched), size=min(parity_pages, len(sched)),
+                                                                replace=False)] if parity_pages else []
+    matched = check_pages_against_oracle(ctx, cfg, pages, picks, (4, 2))
+    line["d5"]["parity_checked_pages"] = len(picks)
+    line["d5"]["parity_matched_pages"] = matched
+    ctx.close()
+    return line
+
+
+def run_d5(args):
+    from paper_2607_16184_b200 import build as pwbuild
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    pwbuild.build()
+    print(json.dumps(measure_d5(device, measured_peaks())), flush=True)
 
 
 def run_reference(args):
-    """The CPU oracle as the reference arm: same config and metric, each step a bounded sample of the batch."""
+    """The CPU oracle as the reference arm: the same configuration and metric, each step one whole layer call
+    (all tokens of the batch) of the oracle as it stands, on the host cores."""
     rank, _, world = replicas.env_world()
     if rank != 0:
         return
     from oracle import oracle
     oracle.build()
     cfg = synth.CONFIGS[args.config]
-    n_tok = args.ref_tokens
+    n_tok = cfg.tokens if args.ref_tokens <= 0 else min(args.ref_tokens, cfg.tokens)
     x = synth.activations(cfg, 0).numpy()
     logits = synth.router_logits(cfg, 0).numpy()
     bits = synth.assign_bits(cfg, 0)
@@ -693,7 +838,7 @@ def run_reference(args):
             rows, cols = cfg.block_shape(u)
             if e in need:
                 pages.append(oracle.quantize_block(synth.block_weights(cfg, 0, e, u).numpy(), int(bits[e, u])))
-            else:   # never read: the sampled tokens are not routed here
+            else:   # never read: no token of the step is routed here
                 pages.append(oracle.Page(np.zeros(16, np.uint8), None, None, rows, cols, 16))
     toks = list(range(n_tok))
     run = lambda: oracle.moe_forward(x, logits, cfg.top_k, pages, n_shared=cfg.n_shared, tokens=toks)
@@ -705,11 +850,14 @@ def run_reference(args):
     dt = time.time() - t0
     v = n_tok * args.steps / dt
     cores = oracle.num_threads()
-    sample = "first %d of %d tokens of layer 0 per step" % (n_tok, cfg.tokens)
+    same = n_tok == cfg.tokens
+    sample = ("whole layer calls of layer 0, all %d tokens per step" % cfg.tokens) if same else \
+             ("first %d of %d tokens of layer 0 per step" % (n_tok, cfg.tokens))
     print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": world,
                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
                       "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-                      "data": "synthetic", "config": {"workload": "%s (CPU oracle, %s)" % (cfg.name, sample)},
+                      "data": "synthetic", "same_config": same,
+                      "config": {"workload": "%s (CPU oracle, %s)" % (cfg.name, sample)},
                       "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
                       "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                       "gpu_launches": 0}))
@@ -729,16 +877,20 @@ def main():
     ap.add_argument("--mode", default="auto", choices=["auto", "tensor", "simt"])
     ap.add_argument("--cpu-tokens", type=int, default=64)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="oracle time to spend on the cpu_baseline sample")
-    ap.add_argument("--ref-tokens", type=int, default=2)
+    ap.add_argument("--ref-tokens", type=int, default=0,
+                    help="reference arm: tokens of the batch per step (0 = the whole batch, the configuration itself)")
     ap.add_argument("--uniform-bits", type=int, default=0, choices=[0, 16, 8, 4, 3, 2],
                     help="diagnostic: give every routed block this bitwidth instead of the configured mix")
+    ap.add_argument("--steady-seconds", type=float, default=0.6,
+                    help="least duration of the steady-state region (0: just --steps steps, for profiler captures)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-extra", action="store_true")
     ap.add_argument("--skip-graph", action="store_true", help="leave out the CUDA-graph replay of the step")
     args = ap.parse_args()
     if args.impl == "reference":
-        args.steps = 3 if args.steps is None else args.steps
-        args.warmup = 1 if args.warmup is None else args.warmup
+        # a whole layer call of the oracle takes about 2 s on 16 cores: bound the run to about two minutes
+        args.steps = 3 if args.steps is None else min(args.steps, 40)
+        args.warmup = 1 if args.warmup is None else min(args.warmup, 5)
         run_reference(args)
     else:
         args.steps = 2000 if args.steps is None else args.steps

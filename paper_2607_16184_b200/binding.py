@@ -30,7 +30,7 @@ EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw
            "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
            "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_kv_pressure_bytes",
            "pw_last_device_status",
-           "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_status_str")
+           "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_debug_set_wait", "pw_status_str")
 KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "observe")
 PW_OBS_FIELDS = 8
 OBS_FIELD_NAMES = ("sum_r", "pairs", "sum_r_nx", "sum_r_nx2", "max_nx", "sum_r_nh", "sum_r_nh2", "max_nh")
@@ -139,6 +139,8 @@ def load():
     L.pw_get_kernel_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     L.pw_launch_count.restype = C.c_uint64
     L.pw_launch_count.argtypes = [vp]
+    L.pw_debug_set_wait.restype = C.c_int
+    L.pw_debug_set_wait.argtypes = [vp, C.c_uint32, C.c_uint32]
     L.pw_status_str.restype = C.c_char_p
     L.pw_status_str.argtypes = [i32]
     _lib = L
@@ -444,3 +446,7 @@ class Context:
 
     def pw_launch_count(self) -> int:
         return int(self.L.pw_launch_count(self.handle))
+
+    def pw_debug_set_wait(self, polls: int = 0, hook: int = 0) -> None:
+        """Limit of the device-side waits (polls of up to 20 us; 0 = default) and test hooks of the FFN kernels."""
+        _check(self.L.pw_debug_set_wait(self.handle, polls, hook), "pw_debug_set_wait")

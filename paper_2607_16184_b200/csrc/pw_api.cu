@@ -120,6 +120,8 @@ extern "C" pw_status pw_create(pw_ctx** out, const pw_config* cfg) {
   ctx->launches = 0;
   ctx->last_T = ctx->last_k = 0;
   ctx->tc_state = nullptr;
+  ctx->wait_polls = 0;
+  ctx->test_hook = 0;
   ctx->timing_on = false;
   ctx->timing_ev = nullptr;
   ctx->timing_cur = 0;
@@ -364,6 +366,13 @@ extern "C" pw_status pw_get_kernel_times(pw_ctx* ctx, double* ms_out, uint64_t* 
     for (int i = 0; i < pw_ctx::kTimingSlots; ++i) timing_drain_slot(ctx, i);
   for (int i = 0; i < PW_NUM_KERNELS; ++i) ms_out[i] = ctx->timing_ms[i];
   if (calls_out) *calls_out = ctx->timing_calls;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_debug_set_wait(pw_ctx* ctx, uint32_t polls, uint32_t hook) {
+  if (!ctx) return PW_ERR_INVALID_ARG;
+  ctx->wait_polls = polls;
+  ctx->test_hook = hook;
   return PW_OK;
 }
 

@@ -108,6 +108,8 @@ struct pw_ctx {
   int last_T, last_k;
   int num_sms;
   void* tc_state;                 // tensor-core path state (set up lazily)
+  uint32_t wait_polls;            // limit of the device-side waits in polls of 20 us (0 = the default, 2 s)
+  uint32_t test_hook;             // device-side test hooks (pw_debug_set_wait)
   // optional per-kernel timing: a ring of call slots, PW_NUM_KERNELS + 1 events each
   static constexpr int kTimingSlots = 256;
   bool timing_on;
