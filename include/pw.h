@@ -405,7 +405,7 @@ uint64_t pw_launch_count(pw_ctx* ctx);
  * wait of those kernels is bounded: `polls` polls of up to 20 us each (0 restores the default, 100000 = 2 s).
  * When a wait runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
  * memory and returns; the call's output is then undefined and pw_last_device_status reports the timeout.
- * hook: 0 = none; bit 0 = the token-tile producer of the gate/up kernel stops before its third tile, so that
+ * hook: 0 = none; bit 0 = the token-tile producer of the gate/up kernel stops before its second tile, so that
  * the waits on that tile run out -- the one safe way to exercise the path (nothing faults, traps or spins
  * without a limit).  Applies to forward calls enqueued after it.  Errors: INVALID_ARG. */
 pw_status pw_debug_set_wait(pw_ctx* ctx, uint32_t polls, uint32_t hook);

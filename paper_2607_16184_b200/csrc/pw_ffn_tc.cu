@@ -331,7 +331,7 @@ struct KArgs {
   int32_t* work_counter;
   int32_t* status;
   uint32_t wait_polls;                           // limit of every wait, in polls of kSuspendHintNs
-  uint32_t hook;                                 // test hook: bit 0 = the token-tile producer stops before its third tile
+  uint32_t hook;                                 // test hook: bit 0 = the token-tile producer stops before its second tile
 };
 
 // ---- dequantizers: the tiles of one unit that belong to one group -------------------------------------------
@@ -581,7 +581,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
 #pragma unroll 1
         for (int g = d.g0; ok && g < d.g0 + d.ng; ++g) {
-          if ((ka.hook & 1u) && bcount == 2) {     // test hook: leave the tile unarmed, so that the waits on it run out
+          if ((ka.hook & 1u) && bcount == 1) {     // test hook: leave the tile unarmed, so that the waits on it run out
             ok = false;
             break;
           }

@@ -76,18 +76,6 @@ __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ l
   route_token(logits, warp, E, k, topk_ids, gates, lane);
 }
 
-#ifdef PW_TC_PROFILE
-// Diagnostic build only: clock stamps of the grouping kernel's phases.
-__device__ long long g_ptrace[32];
-#define PSTAMP(i) if (threadIdx.x == 0) g_ptrace[i] = clock64()
-extern "C" int pw_debug_read_ptrace(long long* host_out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, g_ptrace, sizeof(g_ptrace));
-  return 0;
-}
-#else
-#define PSTAMP(i)
-#endif
 
 // out[i] = in[0] + .. + in[i - 1] for i = 0 .. n (n + 1 results), by one warp, 32 values per step.
 __device__ __forceinline__ void warp_exclusive_scan(const int32_t* in, int32_t* out, int n, int lane) {
@@ -134,25 +122,20 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
   int32_t* order = ubase + S + 1;    // [S]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = T * k;
-  PSTAMP(12);
   if (logits) {
     for (int t = warp; t < T; t += (int)(blockDim.x >> 5)) route_token(logits, t, E, k, topk_ids, gates, lane);
     __syncthreads();                                 // the pairs below are read back from global memory
   }
-
-  PSTAMP(0);
   for (int e = tid; e < S; e += blockDim.x) cnt[e] = e < E ? 0 : T;
   for (int e = tid; e < E; e += blockDim.x) run[e] = 0;
   if (tid < 64) counter[tid] = 0;
   __syncthreads();
   for (int p = tid; p < P; p += blockDim.x) atomicAdd(&cnt[topk_ids[p]], 1);
   __syncthreads();
-  PSTAMP(1);
   if (warp == 0) warp_exclusive_scan(cnt, off, S, lane);
   __syncthreads();
   for (int e = tid; e < S; e += blockDim.x) counts[e] = cnt[e];
   for (int e = tid; e <= S; e += blockDim.x) offsets[e] = off[e];
-  PSTAMP(2);
 
   for (int base = 0; base < P; base += blockDim.x) {
     for (int i = tid; i < 32 * E; i += blockDim.x) wcnt[i] = 0;
@@ -181,13 +164,11 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
     }
     __syncthreads();
   }
-  PSTAMP(3);
   const int R = off[S];
   for (int i = tid; i < n_shared * T; i += blockDim.x) row_token[P + i] = i % T;
   for (int i = tid; i < kPadRows; i += blockDim.x) row_token[R + i] = -1;
 
   if (nt_tile <= 0) return;  // SIMT path: no unit lists
-  PSTAMP(4);
 
   // Tables of the unit lists (the lists themselves are written by the gather kernel, which has the threads
   // for it).  The CTAs of the FFN kernels claim units in list order, so the lists are laid out for that: row
@@ -212,7 +193,6 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
       order[rk] = s;
     }
     __syncthreads();
-    PSTAMP(5 + 4 * phase);
     const int row_tiles = (phase == 0 ? F : H) / kTileRows;
     const int splits = phase == 0 ? 1 : ksplit;
     // token tiles per segment in rank order (in parallel), then their prefix (one warp)
@@ -228,14 +208,12 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
       if (!fits) atomicMax(status, (int)PW_ERR_NOMEM);
     }
     __syncthreads();
-    PSTAMP(6 + 4 * phase);
     if (ubase[S] > max_tiles) continue;
     if (phase == 0)
       for (int i = tid; i < S; i += blockDim.x) seg_order[i] = order[i];
     int2* tab = tile_tab + (size_t)phase * max_tiles;
     for (int i = tid; i < S; i += blockDim.x)
       for (int j = ubase[i]; j < ubase[i + 1]; ++j) tab[j] = make_int2(order[i], j - ubase[i]);
-    PSTAMP(7 + 4 * phase);
   }
 }
 
