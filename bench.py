@@ -236,40 +236,50 @@ def run_demote(ctx, cfg, layers, device, peaks, decode_fn, decode_ms):
     reps = 18
     ms164 = time_region(lambda i: ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src]), reps, device) / reps
     ms42 = time_region(lambda i: ctx.pw_demote_block(dst4[i % n_src], 2, dst=dst2[i % n_src]), reps, device) / reps
-    # overlapped: decode on the current stream, one 16->4 demote per decode step on a side stream (never committed)
-    side = torch.cuda.Stream(device=device)
+    # overlapped: one 16->4 demote per decode step on a side stream (never committed).  Two arrangements: both
+    # streams at the default priority, and the decode on a stream of higher priority than the demote's, which is
+    # how a server keeps page movement in the gaps of the forward pass (the block scheduler then places a waiting
+    # CTA of the forward call before any further CTA of the demote).
     # Blocks of decode steps alone and with the demotes alternate, so that both see the same clocks (a short
     # burst after an idle moment runs at boost clocks, a long loop under the power cap does not).
-    n_steps, rounds = 60, 4
-    alone_ms = over_ms = side_ms = 0.0
-    for _ in range(rounds):
-        alone_ms += time_region(decode_fn, n_steps, device)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        side.wait_stream(torch.cuda.current_stream(device))
-        e0.record()
-        s0.record(side)
-        for i in range(n_steps):
-            ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src], stream=side)
-            decode_fn(i)
-        e1.record()
-        s1.record(side)
-        torch.cuda.synchronize(device)
-        over_ms += e0.elapsed_time(e1)
-        side_ms += s0.elapsed_time(s1)
-    decode_ms = alone_ms / (rounds * n_steps)
-    ms_dec = over_ms / (rounds * n_steps)
-    ms_side = side_ms / (rounds * n_steps)
-    n_steps *= rounds
+    def overlapped(main, side):
+        n_steps, rounds = 60, 4
+        alone_ms = over_ms = side_ms = 0.0
+        with torch.cuda.stream(main):
+            for _ in range(rounds):
+                alone_ms += time_region(decode_fn, n_steps, device)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                side.wait_stream(main)
+                e0.record()
+                s0.record(side)
+                for i in range(n_steps):
+                    ctx.pw_demote_block(srcs[i % n_src], 4, dst=dst4[i % n_src], stream=side)
+                    decode_fn(i)
+                e1.record()
+                s1.record(side)
+                torch.cuda.synchronize(device)
+                over_ms += e0.elapsed_time(e1)
+                side_ms += s0.elapsed_time(s1)
+        n = rounds * n_steps
+        return {"decode_ms_per_step": over_ms / n, "decode_ms_alone": alone_ms / n,
+                "decode_slowdown": 1.0 - alone_ms / over_ms if over_ms > 0 else None,
+                "demote_16to4_gbs_side_stream": (b16 + b4) / (side_ms / n * 1e-3) / 1e9, "steps": n}
+
+    cur = torch.cuda.current_stream(device)
+    cur.synchronize()
+    under_default = overlapped(cur, torch.cuda.Stream(device=device))
+    hp = torch.cuda.Stream(device=device, priority=-1)
+    hp.wait_stream(cur)
+    under_prio = overlapped(hp, torch.cuda.Stream(device=device, priority=0))
+    cur.wait_stream(hp)
     gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
     return {"block": "%dx%d" % (rows, cols),
             "16to4": {"ms": ms164, "gbs": gbs(b16 + b4, ms164), "frac_of_measured_hbm": gbs(b16 + b4, ms164) / peaks["hbm_gbs"],
                       "frac_of_nominal_8000": gbs(b16 + b4, ms164) / NOMINAL_HBM_GBS, "bytes": b16 + b4},
             "4to2": {"ms": ms42, "gbs": gbs(b4 + b2, ms42), "frac_of_measured_hbm": gbs(b4 + b2, ms42) / peaks["hbm_gbs"],
                      "frac_of_nominal_8000": gbs(b4 + b2, ms42) / NOMINAL_HBM_GBS, "bytes": b4 + b2},
-            "under_decode": {"decode_ms_per_step": ms_dec, "decode_ms_alone": decode_ms,
-                             "decode_slowdown": 1.0 - decode_ms / ms_dec if ms_dec > 0 else None,
-                             "demote_16to4_gbs_side_stream": gbs(b16 + b4, ms_side), "steps": n_steps}}
+            "under_decode": under_prio, "under_decode_equal_priorities": under_default}
 
 
 def run_residency(ctx, cfg, layers, device, decode_fn, decode_ms):
@@ -679,8 +689,12 @@ def measure_d5(device, peaks, parity_pages=4):
     torch.cuda.synchronize(device)
     sched = [key for key in synth.demote_schedule(cfg) if key[0] < L]
     out = torch.empty(T, cfg.hidden, dtype=torch.float32, device=device)
-    main = torch.cuda.current_stream(device)
-    side = torch.cuda.Stream(device=device)
+    # forward calls on a stream of higher priority than the demotes' (page movement takes the gaps)
+    boot = torch.cuda.current_stream(device)
+    main = torch.cuda.Stream(device=device, priority=-1)
+    main.wait_stream(boot)
+    torch.cuda.set_stream(main)
+    side = torch.cuda.Stream(device=device, priority=0)
 
     def decode_step():
         for layer in range(L):
@@ -803,6 +817,8 @@ def measure_d5(device, peaks, parity_pages=4):
     matched = check_pages_against_oracle(ctx, cfg, pages, picks, (4, 2))
     line["d5"]["parity_checked_pages"] = len(picks)
     line["d5"]["parity_matched_pages"] = matched
+    torch.cuda.synchronize(device)
+    torch.cuda.set_stream(boot)
     ctx.close()
     return line
 
