@@ -37,7 +37,7 @@ __device__ __forceinline__ void load_slice_words(const char* tb, int r, int q, u
 }
 
 template <int SRC_KIND, int SRC_BITS, int DST_BITS>
-__global__ void __launch_bounds__(512) quant_tile_kernel(const void* __restrict__ src_codes, uint32_t cols,
+__global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restrict__ src_codes, uint32_t cols,
                                                          void* __restrict__ dst_codes) {
   const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
   const int r = threadIdx.x >> 2, q = threadIdx.x & 3;

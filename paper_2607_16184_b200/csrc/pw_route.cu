@@ -221,6 +221,7 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
 // accumulator columns that nobody reads, so they keep whatever they hold.
 // The same grid first writes the two unit lists from the tables of the permute kernel: unit u of a list is
 // (row tile, K split) pair u / TT and token tile u mod TT.
+constexpr int kGatherChunks = 4;
 __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
                                                      const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
                                                      uint4* __restrict__ xt, const int32_t* __restrict__ counts,
@@ -271,13 +272,21 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
       }
     }
   }
+  // kGatherChunks consecutive 16-byte chunks of one operand row per thread: the loads of a thread are in flight
+  // together (64 contiguous bytes of the token's row), the stores of a warp are contiguous per chunk
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  const int c = blockIdx.y;
+  const int c0 = blockIdx.y * kGatherChunks;
   if (n >= offsets[S]) return;
   const int t = row_token[n];
-  uint4 v = make_uint4(0, 0, 0, 0);
-  if (t >= 0) v = __ldg(hidden + (size_t)t * H8 + c);
-  xt[(size_t)c * Rpad + n] = v;
+  uint4 v[kGatherChunks];
+#pragma unroll
+  for (int i = 0; i < kGatherChunks; ++i) {
+    v[i] = make_uint4(0, 0, 0, 0);
+    if (t >= 0 && c0 + i < H8) v[i] = __ldg(hidden + (size_t)t * H8 + c0 + i);
+  }
+#pragma unroll
+  for (int i = 0; i < kGatherChunks; ++i)
+    if (c0 + i < H8) xt[(size_t)(c0 + i) * Rpad + n] = v[i];
 }
 
 // out[t] = sum_j gate[t,j] * (sum_s y[s][inv_perm[t*k+j]]) + sum over shared experts (sum_s y[s][row]).
@@ -357,6 +366,64 @@ __global__ void __launch_bounds__(kCombineCols * kCombineRows)
   }
 }
 
+// The same sum for batches with enough tokens to fill the machine by themselves: one thread per (token, float4
+// column), U expert choices in flight at a time, no shared memory and no barrier.  The arithmetic and its order
+// are those of combine_kernel (splits added in split order, times the gate, terms added in choice order).
+template <int U>
+__global__ void __launch_bounds__(128)
+    combine_stream_kernel(const float4* __restrict__ y, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
+                          int T, int k, int n_shared, int H4, int ksplit, size_t split_stride4, float4* __restrict__ out) {
+  grid_dep_sync();
+  grid_dep_trigger();
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = blockIdx.y;
+  if (c >= H4) return;
+  const int J = k + n_shared;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j0 = 0; j0 < J; j0 += U) {
+    size_t row[U];
+    float g[U];
+    float4 a[U];
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      const int j = j0 + i;
+      if (j < k) {
+        row[i] = (size_t)inv_perm[(size_t)t * k + j];
+        g[i] = gates[(size_t)t * k + j];
+      } else {
+        row[i] = (size_t)T * k + (size_t)(j - k) * T + t;
+        g[i] = 1.0f;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < U; ++i)
+      if (j0 + i < J) a[i] = y[row[i] * H4 + c];
+    for (int sp = 1; sp < ksplit; ++sp) {
+      float4 v[U];
+#pragma unroll
+      for (int i = 0; i < U; ++i)
+        if (j0 + i < J) v[i] = y[sp * split_stride4 + row[i] * H4 + c];
+#pragma unroll
+      for (int i = 0; i < U; ++i)
+        if (j0 + i < J) {
+          a[i].x = __fadd_rn(a[i].x, v[i].x);
+          a[i].y = __fadd_rn(a[i].y, v[i].y);
+          a[i].z = __fadd_rn(a[i].z, v[i].z);
+          a[i].w = __fadd_rn(a[i].w, v[i].w);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < U; ++i)
+      if (j0 + i < J) {
+        acc.x = __fadd_rn(acc.x, __fmul_rn(g[i], a[i].x));
+        acc.y = __fadd_rn(acc.y, __fmul_rn(g[i], a[i].y));
+        acc.z = __fadd_rn(acc.z, __fmul_rn(g[i], a[i].z));
+        acc.w = __fadd_rn(acc.w, __fmul_rn(g[i], a[i].w));
+      }
+  }
+  out[(size_t)t * H4 + c] = acc;
+}
+
 pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int k, int nt_tile,
                        int ksplit, cudaStream_t s) {
   const pw_config& c = ctx->cfg;
@@ -386,7 +453,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
   const int R = T * k + c.n_shared * T;
   const int dn_tt_outer = (size_t)R * c.ffn * 2 > ((size_t)64 << 20) ? 1 : 0;   // SwiGLU rows beyond half of the L2
   timing_mark(ctx, PW_K_GATHER, s);
-  dim3 grid((R + 255) / 256, c.hidden / 8);
+  dim3 grid((R + 255) / 256, (c.hidden / 8 + kGatherChunks - 1) / kGatherChunks);
   PW_CUDA_OK(launch_dependent(gather_kernel, grid, dim3(256), 0, s, reinterpret_cast<const uint4*>(hidden),
                               reinterpret_cast<const int32_t*>(b + w.row_token),
                               reinterpret_cast<const int32_t*>(b + w.offsets), S, c.hidden / 8, w.Rpad,
@@ -409,6 +476,15 @@ pw_status launch_combine(pw_ctx* ctx, int T, int k, int ksplit, float* out, cuda
   const int chunks = T >= 256 ? 4 : 1;
   dim3 grid((H4 + kCombineCols * chunks - 1) / (kCombineCols * chunks), T);
   timing_mark(ctx, PW_K_COMBINE, s);
+  if ((long long)T * ((H4 + 127) / 128) >= 2 * ctx->num_sms) {   // enough (token, column) CTAs to fill the machine
+    PW_CUDA_OK(launch_dependent(combine_stream_kernel<4>, dim3((H4 + 127) / 128, T), dim3(128), 0, s,
+                                reinterpret_cast<const float4*>(b + w.y), reinterpret_cast<const float*>(b + w.gates),
+                                reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
+                                (size_t)R * H4, reinterpret_cast<float4*>(out)));
+    ctx->launches += 1;
+    PW_CUDA_OK(cudaGetLastError());
+    return PW_OK;
+  }
   PW_CUDA_OK(launch_dependent(chunks == 4 ? combine_kernel<4> : combine_kernel<1>, grid, dim3(kCombineCols, kCombineRows), 0, s, reinterpret_cast<const float4*>(b + w.y),
                               reinterpret_cast<const float*>(b + w.gates),
                               reinterpret_cast<const int32_t*>(b + w.inv_perm), T, k, c.n_shared, H4, ksplit,
