@@ -66,7 +66,7 @@ typedef enum {
  * the 128 scales and the 128 zero-points of its rows, so a tile travels in a single copy;
  * `scales` and `zps` of a TILED page are ignored (may be NULL).  Both layouts have the same
  * total size. */
-enum { PW_LAYOUT_CANONICAL = 0, PW_LAYOUT_TILED = 1 };
+enum { PW_LAYOUT_CANONICAL = 0, PW_LAYOUT_TILED = 1, PW_LAYOUT_PLANES = 2 /* overlaid bit-planes, see below */ };
 
 /* Residency state of a page-table row (Sec. 3.1).  Only GPU_RESIDENT rows can be used. */
 enum {
@@ -165,6 +165,36 @@ pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bits, pw_page
 pw_status pw_export_page(pw_ctx* ctx, const pw_page* src_tiled, pw_page* dst_canonical, pw_stream stream);
 pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst_tiled, pw_stream stream);
 
+/* ---- overlaid bit-plane pages --------------------------------------------------------- */
+
+/* The paper's own page representation (Sec. 2.2 "Any-Precision"; Sec. 3.1: one bit-plane with its lookup-table
+ * state is one weight page; Eq. 3: size table with the lookup-table metadata): a block is stored once as
+ * overlaid bit-planes, a subset of the planes is a lower-precision version of the same block, and lowering the
+ * precision computes nothing -- the planes above the committed bitwidth simply stop being read and may move to
+ * host memory or be freed.  The paper does not say how its codes and centroids are fit; here the code is nested
+ * on the group quantizer: master code c4 = the 4-bit code of pw_quantize_block, code at q bits = c4 >> (4 - q),
+ * lookup table of q bits affine with scale_q = scale_4 * 2^(4-q) and zero-point_q = fp16(zero-point_4 +
+ * scale_4 * (2^(4-q) - 1) / 2), the middle of the levels that the shorter code merges.  Supported q: 4, 3, 2.
+ *
+ * A PLANES block is three device buffers, carried by a pw_page with layout PW_LAYOUT_PLANES:
+ *   codes  -> TOP   the two leading bits of every code, and the lookup-table state of all three bitwidths
+ *   scales -> BIT1  the third bit   (needed for bits >= 3; may be NULL in a page published at 2 bits)
+ *   zps    -> BIT0  the fourth bit  (needed for bits == 4; may be NULL below that)
+ * and `bits` = the bitwidth it is read at.  pw_plane_bytes gives the buffer sizes (TOP, then each bit plane).
+ * At q bits a forward call reads q/8 bytes per weight plus one lookup-table state per group: the bytes of
+ * pw_page_bytes(rows, cols, q).
+ *
+ * pw_quantize_planes builds the three buffers from an fp16 block (device, [rows, cols] row-major) and fills the
+ * header with bits = 4.  To lower or raise the precision the caller copies the header, sets `bits` (and may
+ * clear the pointers of detached planes) and publishes it with pw_set_page_table: no kernel runs.
+ * pw_export_planes writes the block's view at src->bits as a CANONICAL page (dst as for pw_export_page).
+ * Errors: INVALID_ARG, SHAPE, BITS (bits outside 2..4), ALIGN, STATE (not a PLANES page; a needed plane is
+ * detached). */
+size_t pw_plane_bytes(uint32_t rows, uint32_t cols, size_t* top_bytes, size_t* bit_plane_bytes);
+pw_status pw_quantize_planes(pw_ctx* ctx, const void* w_fp16, uint32_t rows, uint32_t cols, pw_page* dst,
+                             pw_stream stream);
+pw_status pw_export_planes(pw_ctx* ctx, const pw_page* src_planes, pw_page* dst_canonical, pw_stream stream);
+
 /* ---- page table --------------------------------------------------------------------- */
 
 /* Publishes n rows of the weight page table (Sec. 3.1): for each entry the row
@@ -177,7 +207,7 @@ pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst
  * may be released once work enqueued before this call has finished.  entries: host.  epoch_out
  * (optional, host) receives the table epoch after the update; each call increments it by one.
  * Errors: INVALID_ARG, SHAPE (page shape does not match kind and ctx), BITS, ALIGN,
- * STATE (layout not TILED, state not GPU_RESIDENT, the page of the row at that bitwidth is CPU_RESIDENT or
+ * STATE (layout neither TILED nor PLANES, a plane the bitwidth needs is missing, state not GPU_RESIDENT, the page of the row at that bitwidth is CPU_RESIDENT or
  * IN_TRANSFER, shared expert below 16 bits), CUDA. */
 pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entries, size_t n, pw_stream stream,
                             uint64_t* epoch_out);

@@ -20,13 +20,13 @@ STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_SHAPE", 3: "PW_E
                 5: "PW_ERR_STATE", 6: "PW_ERR_NOMEM", 7: "PW_ERR_CUDA", 8: "PW_ERR_TIMEOUT"}
 PW_GATE, PW_UP, PW_DOWN = 0, 1, 2
 PW_MODE_AUTO, PW_MODE_SIMT, PW_MODE_TENSOR = 0, 1, 2
-PW_LAYOUT_CANONICAL, PW_LAYOUT_TILED = 0, 1
+PW_LAYOUT_CANONICAL, PW_LAYOUT_TILED, PW_LAYOUT_PLANES = 0, 1, 2
 PW_STATE_GPU_RESIDENT, PW_STATE_CPU_RESIDENT, PW_STATE_IN_TRANSFER, PW_STATE_NONE = 0, 1, 2, 3
 GROUP = 128
 
 # every symbol include/pw.h declares
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
-           "pw_export_page", "pw_import_page", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
+           "pw_export_page", "pw_import_page", "pw_plane_bytes", "pw_quantize_planes", "pw_export_planes", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
            "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
            "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_kv_pressure_bytes",
            "pw_last_device_status",
@@ -137,6 +137,12 @@ def load():
     L.pw_kernel_timing.argtypes = [vp, i32]
     L.pw_get_kernel_times.restype = i32
     L.pw_get_kernel_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+    L.pw_plane_bytes.restype = C.c_size_t
+    L.pw_plane_bytes.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.pw_quantize_planes.restype = C.c_int
+    L.pw_quantize_planes.argtypes = [vp, vp, C.c_uint32, C.c_uint32, C.POINTER(pw_page), vp]
+    L.pw_export_planes.restype = C.c_int
+    L.pw_export_planes.argtypes = [vp, C.POINTER(pw_page), C.POINTER(pw_page), vp]
     L.pw_launch_count.restype = C.c_uint64
     L.pw_launch_count.argtypes = [vp]
     L.pw_debug_set_wait.restype = C.c_int
@@ -254,6 +260,39 @@ class Page:
     layout = property(lambda self: self.c.layout)
 
 
+def pw_plane_bytes(rows: int, cols: int) -> Tuple[int, int, int]:
+    """(total, TOP buffer, one bit-plane buffer) bytes of a bit-plane block."""
+    t, b = C.c_size_t(), C.c_size_t()
+    tot = load().pw_plane_bytes(rows, cols, C.byref(t), C.byref(b))
+    return int(tot), int(t.value), int(b.value)
+
+
+class PlanePage:
+    """A bit-plane block (three device buffers) read at ``bits`` in {2, 3, 4}: the ``pw_page`` header of layout
+    PW_LAYOUT_PLANES.  ``at(q)`` gives the same buffers at another bitwidth -- lowering or raising the precision
+    is a new header, nothing else; with ``detach=True`` the header no longer names the planes q does not need."""
+
+    def __init__(self, rows: int, cols: int, device="cuda", _buffers=None, bits: int = 4, detach: bool = False):
+        if _buffers is None:
+            _, tb, bb = pw_plane_bytes(rows, cols)
+            _buffers = (torch.empty(tb, dtype=torch.uint8, device=device), torch.empty(bb, dtype=torch.uint8, device=device),
+                        torch.empty(bb, dtype=torch.uint8, device=device))
+        self.top, self.bit1, self.bit0 = _buffers
+        self.codes = self.top
+        p1 = self.bit1.data_ptr() if (bits >= 3 or not detach) else None
+        p0 = self.bit0.data_ptr() if (bits == 4 or not detach) else None
+        self.c = pw_page(self.top.data_ptr(), p1, p0, rows, cols, GROUP, bits, PW_LAYOUT_PLANES)
+        self.nbytes = pw_page_bytes(rows, cols, bits)[0] if bits in (2, 3, 4) else 0
+
+    rows = property(lambda self: self.c.rows)
+    cols = property(lambda self: self.c.cols)
+    bits = property(lambda self: self.c.bits)
+    layout = property(lambda self: self.c.layout)
+
+    def at(self, bits: int, detach: bool = False) -> "PlanePage":
+        return PlanePage(self.rows, self.cols, _buffers=(self.top, self.bit1, self.bit0), bits=bits, detach=detach)
+
+
 class Context:
     """Owns the workspace tensor and the ``pw_ctx``; methods carry the names of the C calls."""
 
@@ -310,6 +349,20 @@ class Context:
         dst = Page(src.rows, src.cols, src.bits, self.device, PW_LAYOUT_CANONICAL)
         _check(self.L.pw_export_page(self.handle, C.byref(src.c), C.byref(dst.c), _stream_ptr(stream)),
                "pw_export_page")
+        return dst
+
+    def pw_quantize_planes(self, w_fp16: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> PlanePage:
+        assert w_fp16.dtype == torch.float16 and w_fp16.is_contiguous() and w_fp16.is_cuda
+        rows, cols = w_fp16.shape
+        dst = PlanePage(rows, cols, self.device)
+        _check(self.L.pw_quantize_planes(self.handle, w_fp16.data_ptr(), rows, cols, C.byref(dst.c), _stream_ptr(stream)),
+               "pw_quantize_planes")
+        return dst
+
+    def pw_export_planes(self, src: PlanePage, stream: Optional[torch.cuda.Stream] = None) -> Page:
+        dst = Page(src.rows, src.cols, src.bits, self.device, PW_LAYOUT_CANONICAL)
+        _check(self.L.pw_export_planes(self.handle, C.byref(src.c), C.byref(dst.c), _stream_ptr(stream)),
+               "pw_export_planes")
         return dst
 
     def pw_import_page(self, src: Page, stream: Optional[torch.cuda.Stream] = None) -> Page:

@@ -177,17 +177,25 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
     const pw_page& p = e.page;
     if (e.layer < 0 || e.layer >= c.n_layers || e.expert < 0 || e.expert >= ctx->ws.S || e.kind < 0 || e.kind > 2)
       return PW_ERR_INVALID_ARG;
-    if (!bits_ok(p.bits)) return PW_ERR_BITS;
+    const bool planes = p.layout == PW_LAYOUT_PLANES;
+    if (planes ? (p.bits < 2 || p.bits > 4) : !bits_ok(p.bits)) return PW_ERR_BITS;
     const uint32_t er = e.kind == PW_DOWN ? c.hidden : c.ffn, ec = e.kind == PW_DOWN ? c.ffn : c.hidden;
     if (p.rows != er || p.cols != ec || p.group != kGroup) return PW_ERR_SHAPE;
     if (!p.codes) return PW_ERR_INVALID_ARG;   // a TILED page is one buffer: scales and zero-points sit inside it
     if (!aligned16(p.codes)) return PW_ERR_ALIGN;
-    if (p.layout != PW_LAYOUT_TILED || e.state != PW_STATE_GPU_RESIDENT) return PW_ERR_STATE;
-    if (e.expert >= c.n_experts && p.bits != 16) return PW_ERR_STATE;
+    if ((p.layout != PW_LAYOUT_TILED && !planes) || e.state != PW_STATE_GPU_RESIDENT) return PW_ERR_STATE;
+    if (planes) {
+      // the bitwidth is only set to what the attached planes can give (Sec. 3.1)
+      if ((p.bits >= 3 && !p.scales) || (p.bits == 4 && !p.zps)) return PW_ERR_STATE;
+      if (!aligned16(p.scales) || !aligned16(p.zps)) return PW_ERR_ALIGN;
+    }
+    if (e.expert >= c.n_experts && (p.bits != 16 || planes)) return PW_ERR_STATE;
     if (e.desired_bits != 0 && !bits_ok(e.desired_bits)) return PW_ERR_BITS;
     // q_i is only set to a bitwidth whose page is GPU-resident (Sec. 3.1): not while it is away or on its way
-    const pw_status rs = residency_check_commit(ctx, row_index(ctx, e.layer, e.expert, e.kind), p);
-    if (rs != PW_OK) return rs;
+    if (!planes) {
+      const pw_status rs = residency_check_commit(ctx, row_index(ctx, e.layer, e.expert, e.kind), p);
+      if (rs != PW_OK) return rs;
+    }
   }
   // The rows travel in the parameter space of a small kernel, 64 at a time: the update is ordered on the
   // stream like any kernel and never queues behind a large copy on a DMA engine (a page being reloaded on a
@@ -204,7 +212,9 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       r.rows = e.page.rows;
       r.cols = e.page.cols;
       r.bits = e.page.bits;
-      r.valid = 1;
+      r.valid = e.page.layout == PW_LAYOUT_PLANES ? 2 : 1;
+      r.bit1 = r.valid == 2 ? e.page.scales : nullptr;
+      r.bit0 = r.valid == 2 ? e.page.zps : nullptr;
       const size_t idx = row_index(ctx, e.layer, e.expert, e.kind);
       int j = 0;                                   // a row named twice keeps its last entry
       while (j < batch.n && batch.index[j] != (uint32_t)idx) ++j;
@@ -213,7 +223,7 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       if (j == batch.n) ++batch.n;
       ctx->host_rows[idx] = e;
       ctx->host_valid[idx] = 1;
-      residency_note_commit(ctx, idx, e.page);
+      if (e.page.layout != PW_LAYOUT_PLANES) residency_note_commit(ctx, idx, e.page);
     }
     commit_rows_kernel<<<1, kCommitBatch, 0, stream>>>(batch, dtab);
     ctx->launches++;
@@ -254,6 +264,10 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
   // against 1.96 ms for the CUDA-core kernel), so AUTO means TENSOR; the CUDA-core kernel stays selectable as
   // an independent second implementation.
   if (mode == PW_MODE_AUTO) mode = PW_MODE_TENSOR;
+  if (mode == PW_MODE_SIMT)                      // the CUDA-core kernel reads TILED pages only
+    for (int e = 0; e < ctx->ws.S; ++e)
+      for (int u = 0; u < 3; ++u)
+        if (ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES) return PW_ERR_STATE;
   int nt_tile = 0, ksplit = 1;
   if (mode == PW_MODE_TENSOR) {
     nt_tile = tensor_token_tile(ctx, T, top_k);

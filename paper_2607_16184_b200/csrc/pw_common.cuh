@@ -20,8 +20,10 @@ struct DevRow {
   const void* codes;             // the TILED page buffer (tile images: codes, scales, zero-points)
   uint32_t rows, cols;
   uint32_t bits;
-  uint32_t valid;
-  uint64_t reserved[3];
+  uint32_t valid;                // 0 = unpublished, 1 = TILED page, 2 = overlaid bit-planes (codes = TOP buffer)
+  const void* bit1;              // bit-plane buffers of a PLANES block (null where detached)
+  const void* bit0;
+  uint64_t reserved;
 };
 static_assert(sizeof(DevRow) == 48, "DevRow layout");
 

@@ -284,7 +284,9 @@ __device__ __forceinline__ bool get_desc(uint32_t i, uint32_t polls, Ctrl* c, in
 }
 
 // Chunks: tiles per chunk = 1 << chunk_log(bits).
-__device__ __forceinline__ uint32_t chunk_log(uint32_t bits) { return bits == 16 ? 0u : bits == 8 ? 1u : 2u; }
+// (a bit-plane tile, flagged by kPlanesFlag in the unit's bitwidth byte, is gathered from up to four places and travels alone)
+constexpr uint32_t kPlanesFlag = 0x40;
+__device__ __forceinline__ uint32_t chunk_log(uint32_t bits) { return (bits == 16 || (bits & kPlanesFlag)) ? 0u : bits == 8 ? 1u : 2u; }
 // Chunk number inside a unit.  The producer walks the unit's groups in order and, at every group that starts a
 // chunk of a matrix, issues that chunk (matrix 0 first): chunk i of matrix 0 is preceded by its own earlier
 // chunks and by the chunks of matrix 1 that start before its first group, and the other way round.
@@ -337,12 +339,13 @@ struct KArgs {
 // ---- dequantizers: the tiles of one unit that belong to one group -------------------------------------------
 // Tile j of the unit sits in chunk j >> L of its matrix; a warp looks at a chunk's barrier once, decodes its
 // tiles of the chunk and makes one arrival on the slot per tile.
-template <int BITS, int NMAT>
+template <int BITS, int NMAT, bool PLANES>
 __device__ __forceinline__ bool dq_unit(Ctrl* c, const KArgs& ka, char* wring, uint32_t m, uint32_t j0, uint32_t stride,
                                         uint32_t ng, uint32_t seq_unit, uint32_t l0, uint32_t l1, Cursor& cu,
                                         uint32_t& uses, int r, int lane, uint32_t lane_addr, uint32_t af_s, uint32_t ae_s) {
-  constexpr uint32_t L = BITS == 8 ? 1u : 2u;
+  constexpr uint32_t L = PLANES ? 0u : BITS == 8 ? 1u : 2u;
   constexpr uint32_t TB = BITS * 2048 + 512;
+  constexpr uint32_t META = PLANES ? (uint32_t)kPlaneSlotLut : BITS * 2048u;   // scales, then zero-points, of the tile's rows
   const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
   uint32_t cur = 0xffffffffu;
   const char* chunk = nullptr;
@@ -363,17 +366,19 @@ __device__ __forceinline__ bool dq_unit(Ctrl* c, const KArgs& ka, char* wring, u
     }
     const char* tile = chunk + (j & ((1u << L) - 1u)) * TB;
     const uint4* row_units = reinterpret_cast<const uint4*>(tile) + r;
-    const __half2 s2 = __half2half2(*reinterpret_cast<const __half*>(tile + BITS * 2048 + 2 * r));
-    const __half2 z2 = __half2half2(*reinterpret_cast<const __half*>(tile + BITS * 2048 + 256 + 2 * r));
+    const __half2 s2 = __half2half2(*reinterpret_cast<const __half*>(tile + META + 2 * r));
+    const __half2 z2 = __half2half2(*reinterpret_cast<const __half*>(tile + META + 256 + 2 * r));
     __half2 w[32];
-    decode_half<BITS>(row_units, 0, s2, z2, w);
+    if constexpr (PLANES) decode_half_planes<BITS>(tile, r, 0, s2, z2, w);
+    else decode_half<BITS>(row_units, 0, s2, z2, w);
     // The operand slot is free once the MMAs of the group's previous tile have read it; they ran while the
     // half above was being decoded.
     if (!wait_bar(ae_s, (uses & 1u) ^ 1u, ka.wait_polls, c, ka.status)) return false;
     ++uses;
     tc_fence_after();
     tmem_st32(lane_addr, w);
-    decode_half<BITS>(row_units, 1, s2, z2, w);
+    if constexpr (PLANES) decode_half_planes<BITS>(tile, r, 1, s2, z2, w);
+    else decode_half<BITS>(row_units, 1, s2, z2, w);
     __syncwarp();
     mbar_arrive_if_s(slot_empty_s, lane == 0);     // this warp has read its rows of the tile
     tmem_st32(lane_addr + 32, w);
@@ -508,7 +513,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         d.row_tile = d.tok0 = d.ntok = d.g0 = d.ng = d.split = 0;
         d.bits = 0;
         const char* src[NMAT];
-        uint32_t tb[NMAT], lg[NMAT];
+        const char* pb1[NMAT];                      // bit-plane blocks: the BIT1 and BIT0 buffers
+        const char* pb0[NMAT];
+        uint32_t tb[NMAT], lg[NMAT], pq[NMAT];      // pq: bitwidth a bit-plane block is read at, 0 = an ordinary page
         if (u >= 0) {
           // (the unit list may have been written by the kernel directly ahead: read around the non-coherent path)
           const int4* up = reinterpret_cast<const int4*>(ka.units + u);
@@ -522,12 +529,17 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
             const DevRow row = ka.rows[u0.x * 3 + (PHASE == 0 ? m : 2)];
-            d.bits |= row.bits << (8 * m);
-            tb[m] = (uint32_t)tile_bytes((int)row.bits);
-            lg[m] = chunk_log(row.bits);
+            const bool planes = row.valid == 2;
+            const uint32_t ubits = row.bits | (planes ? kPlanesFlag : 0u);
+            d.bits |= ubits << (8 * m);
+            pq[m] = planes ? row.bits : 0u;
+            tb[m] = planes ? (uint32_t)kPlaneTopTile : (uint32_t)tile_bytes((int)row.bits);
+            lg[m] = chunk_log(ubits);
             // consecutive groups of a row tile are consecutive tiles of the page
             const size_t tile = (size_t)d.row_tile * (row.cols / kGroup) + d.g0;
             src[m] = reinterpret_cast<const char*>(row.codes) + tile * tb[m];
+            pb1[m] = reinterpret_cast<const char*>(row.bit1) + tile * kPlaneBitTile;
+            pb0[m] = reinterpret_cast<const char*>(row.bit0) + tile * kPlaneBitTile;
           }
         }
         UDesc* slot = &c->sched[i & (kSched - 1)];
@@ -547,14 +559,28 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             if (g & ((1u << lg[m]) - 1u)) continue;
             const uint32_t left = ng - g, full_n = 1u << lg[m];
             const uint32_t nt = left < full_n ? left : full_n;
-            const uint32_t bytes = nt * tb[m];
+            const uint32_t q = pq[m];
+            const uint32_t bytes = q ? (uint32_t)kPlaneTopCodes + 512u + (q - 2u) * (uint32_t)kPlaneBitTile : nt * tb[m];
             const uint32_t es = empty_s + 8 * s, fs = full_s + 8 * s;
             if (pass) ok = wait_bar(es, (pass - 1) & 1, polls, c, status);
             if (!ok) break;
             if (nt < 4) mbar_arrive_n_s(es, (4 - nt) * 4);   // a short chunk: the arrivals its missing tiles would make
             mbar_expect_tx_s(fs, bytes);
-            bulk_g2s_s(wring_s + s * kSlotBytes, src[m], bytes, fs);
-            src[m] += bytes;
+            const uint32_t slot_s = wring_s + s * kSlotBytes;
+            if (q) {
+              // a bit-plane tile read at q bits: the top codes, the planes below them that q needs, and the
+              // lookup-table state of q -- only the first q bits of every weight leave HBM
+              bulk_g2s_s(slot_s, src[m], kPlaneTopCodes, fs);
+              bulk_g2s_s(slot_s + kPlaneSlotLut, src[m] + plane_lut_offset((int)q), 512, fs);
+              if (q >= 3) bulk_g2s_s(slot_s + kPlaneSlotBit1, pb1[m], kPlaneBitTile, fs);
+              if (q == 4) bulk_g2s_s(slot_s + kPlaneSlotBit0, pb0[m], kPlaneBitTile, fs);
+              src[m] += kPlaneTopTile;
+              pb1[m] += kPlaneBitTile;
+              pb0[m] += kPlaneBitTile;
+            } else {
+              bulk_g2s_s(slot_s, src[m], bytes, fs);
+              src[m] += bytes;
+            }
             c->issued = ++seq;
             if (++s == (uint32_t)n_slots) {
               s = 0;
@@ -760,10 +786,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // in this unit is tile j0, then every kStride-th.  (The MMA reads 16-bit tiles straight from shared memory.)
       const uint32_t j0 = (gsub - base) & (kStride - 1);
       switch (bits) {
-        case 8: ok = dq_unit<8, NMAT>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 4: ok = dq_unit<4, NMAT>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 3: ok = dq_unit<3, NMAT>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 2: ok = dq_unit<2, NMAT>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case 8: ok = dq_unit<8, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case 4: ok = dq_unit<4, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case 3: ok = dq_unit<3, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case 2: ok = dq_unit<2, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case kPlanesFlag | 4: ok = dq_unit<4, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case kPlanesFlag | 3: ok = dq_unit<3, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        case kPlanesFlag | 2: ok = dq_unit<2, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
         default: break;
       }
       base += ng;

@@ -214,4 +214,60 @@ __device__ __forceinline__ void decode_half(const uint4* row_units, int h, __hal
   decode_quarter<BITS>(row_units, 2 * h + 1, s2, z2, out + 16);
 }
 
+// ---- overlaid bit-plane pages (PW_LAYOUT_PLANES) -----------------------------------------------
+// A block quantized once to a 4-bit master code c4 is stored as three plane buffers, each cut into the same
+// (128-row, one-group) tiles as a TILED page: tile (rt, g) of a plane is one contiguous image at
+// (rt * n_groups + g) * tile size.
+//   TOP   5632 B per tile: the two leading bits of every code in the 2-bit arrangement above (4096 B), then the
+//         lookup-table state of each bitwidth the planes can be read at: 128 scales + 128 zero-points (fp16) for
+//         2 bits, the same for 3 bits, the same for 4 bits.  The table is affine, entry c = zero-point + c * scale.
+//   BIT1  2048 B per tile: the third bit.  Row r owns 16 bytes at r * 16; word w of them covers k = 32w .. 32w+31:
+//         bit m (m < 16) belongs to k = 32w + 2m, bit 16 + m to k = 32w + 2m + 1.
+//   BIT0  the fourth bit, same arrangement.
+// Read at q bits the code of a weight is its first q bits, c4 >> (4 - q): q = 2 needs TOP alone, q = 3 TOP and
+// BIT1, q = 4 all three.  Lowering the precision moves and computes nothing.
+constexpr int kPlaneTopCodes = 4096;
+constexpr int kPlaneTopTile = kPlaneTopCodes + 3 * 512;
+constexpr int kPlaneBitTile = 2048;
+__host__ __device__ inline int plane_lut_offset(int q) { return kPlaneTopCodes + 512 * (q - 2); }
+// image of one tile inside a ring slot of the FFN kernels: top codes, BIT1, BIT0, then the table state of the
+// committed bitwidth (fixed offsets whatever the bitwidth)
+constexpr int kPlaneSlotBit1 = 4096, kPlaneSlotBit0 = 6144, kPlaneSlotLut = 8192;
+constexpr int kPlaneSlotBytes = kPlaneSlotLut + 512;
+
+// Quarter t of a row-group read from such an image at Q = 3 or 4 bits (Q = 2 is the plain 2-bit decoder on the
+// top codes): out[p] = weights (32t + 2p, 32t + 2p + 1).
+template <int Q>
+__device__ __forceinline__ void decode_quarter_planes(const char* image, int r, int t, __half2 s2, __half2 z2, __half2* out) {
+  const uint4* row_units = reinterpret_cast<const uint4*>(image) + r;
+  const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + (t >> 1) * kUnitStride) +
+                                                   2 * (t & 1));
+  const uint32_t w[2] = {u.x, u.y};
+  const uint32_t h1 = reinterpret_cast<const uint32_t*>(image + kPlaneSlotBit1 + r * 16)[t];
+  uint32_t h0 = 0;
+  if constexpr (Q == 4) h0 = reinterpret_cast<const uint32_t*>(image + kPlaneSlotBit0 + r * 16)[t];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int p = 8 * i + m;
+      constexpr int up = Q - 2;                    // the top two bits sit `up` places above bit 0 of the code
+      const uint32_t top = 2 * m >= up ? (w[i] >> (2 * m - up)) : (w[i] << (up - 2 * m));
+      uint32_t v = (top & (0x00030003u << up)) | 0x64006400u;
+      const uint32_t b1 = p >= up - 1 ? (h1 >> (p - (up - 1))) : (h1 << ((up - 1) - p));
+      v |= b1 & (0x00010001u << (up - 1));
+      if constexpr (Q == 4) v |= (h0 >> p) & 0x00010001u;
+      out[p] = dq_pair(v, s2, z2);
+    }
+}
+template <int Q>
+__device__ __forceinline__ void decode_half_planes(const char* image, int r, int h, __half2 s2, __half2 z2, __half2* out) {
+  if constexpr (Q == 2) {
+    decode_half<2>(reinterpret_cast<const uint4*>(image) + r, h, s2, z2, out);
+  } else {
+    decode_quarter_planes<Q>(image, r, 2 * h, s2, z2, out);
+    decode_quarter_planes<Q>(image, r, 2 * h + 1, s2, z2, out + 16);
+  }
+}
+
 }  // namespace pw

@@ -3,6 +3,7 @@
 // 32-weight slice; HBM-bound: reads the source once, writes the page once.
 #include "pw_common.cuh"
 #include "pw_layout.cuh"
+#include "pw_quant_core.cuh"
 
 namespace pw {
 
@@ -98,52 +99,10 @@ __global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restri
     return;
   }
 
-  // minimum and maximum of my 32 values (of fp16 sources taken on the packed halves: half as many operations,
-  // and exact like the fp32 ones)
-  float lo, hi;
-  if constexpr (SRC_BITS == 16) {
-    __half2 lo2 = h16[0], hi2 = h16[0];
-#pragma unroll
-    for (int i = 1; i < 16; ++i) {
-      lo2 = __hmin2(lo2, h16[i]);
-      hi2 = __hmax2(hi2, h16[i]);
-    }
-    const float2 lf = __half22float2(lo2), hf = __half22float2(hi2);
-    lo = fminf(lf.x, lf.y);
-    hi = fmaxf(hf.x, hf.y);
-  } else {
-    lo = v[0];
-    hi = v[0];
-#pragma unroll
-    for (int i = 1; i < 32; ++i) {
-      lo = fminf(lo, v[i]);
-      hi = fmaxf(hi, v[i]);
-    }
-  }
-#pragma unroll
-  for (int d = 1; d <= 2; d <<= 1) {
-    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
-    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
-  }
-  if (lo == 0.0f) lo = 0.0f;  // store -0 as +0
-  constexpr int L = (1 << DST_BITS) - 1;
-  const float rng = __fsub_rn(hi, lo);
-  __half sh;
-  if (rng == 0.0f) {
-    sh = __ushort_as_half((unsigned short)0x3c00);
-  } else {
-    sh = __float2half_rn(__fdiv_rn(rng, (float)L));
-    if ((__half_as_ushort(sh) & 0x7fff) == 0) sh = __ushort_as_half((unsigned short)0x0001);
-  }
-  const float rinv = __fdiv_rn(1.0f, __half2float(sh));
   int code[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    // round half to even and convert in one step (the product is never negative; a huge one saturates), then
-    // clamp: the same code as clamp(rint(x), 0, L)
-    const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v[i], lo), rinv));
-    code[i] = (int)(c < (uint32_t)L ? c : (uint32_t)L);
-  }
+  __half sh;
+  float lo;
+  group_quantize<SRC_BITS == 16>(v, h16, (1 << DST_BITS) - 1, code, sh, lo);
   constexpr int NW = SliceWords<DST_BITS>::kWords;
   uint32_t w[NW];
   pack_slice<DST_BITS>(code, w);
