@@ -139,15 +139,22 @@ def page_bytes_total(bits_table, cfg, active_mask=None):
     return gu, dn
 
 
-def build_layers(ctx, cfg, n_layers, device):
+def build_layers(ctx, cfg, n_layers, device, planes_q=0):
+    """planes_q: 0 = ordinary pages at the configured bitwidths; 2, 3 or 4 = every routed block is a bit-plane
+    block read at that many bits."""
     layers = []
     for layer in range(n_layers):
         bits = synth.assign_bits(cfg, layer)
+        if planes_q:
+            bits[:cfg.n_experts] = planes_q
         pages, entries = [], []
         for e in range(cfg.n_experts + cfg.n_shared):
             for u in range(3):
                 w = synth.block_weights(cfg, layer, e, u, device=device)
-                pg = ctx.pw_quantize_block(w, int(bits[e, u]))
+                if planes_q and e < cfg.n_experts:
+                    pg = ctx.pw_quantize_planes(w).at(planes_q, detach=True)
+                else:
+                    pg = ctx.pw_quantize_block(w, int(bits[e, u]))
                 pages.append(pg)
                 entries.append((layer, e, u, pg))
                 del w
@@ -380,12 +387,12 @@ def kernel_pass(ctx, step, steps, device):
     return {n: v / max(kcalls, 1) for n, v in ktimes.items()}, ms / steps
 
 
-def decode_workload(device, peaks, cfg, L, mode, steps, warmup, min_seconds=0.6):
+def decode_workload(device, peaks, cfg, L, mode, steps, warmup, min_seconds=0.6, planes_q=0):
     """One decode configuration in a context of its own: step time, per-kernel times and roofline fractions of a
     region of at least `min_seconds` of back-to-back steps (sampled clocks), rotating over L distinct layers."""
     from paper_2607_16184_b200 import binding as B
     ctx = B.Context(L, cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.ffn, cfg.tokens, cfg.top_k, device=device)
-    layers = build_layers(ctx, cfg, L, device)
+    layers = build_layers(ctx, cfg, L, device, planes_q)
     T, k = cfg.tokens, cfg.top_k
     out = torch.empty(T, cfg.hidden, dtype=torch.float32, device=device)
 
@@ -594,6 +601,15 @@ def run_gpu(args):
                 per_bits[str(b)]["gate_up_tiles_per_s"] = (2.0 * cfg.n_experts * (cfg.ffn // 128) * (cfg.hidden // 128)
                                                            / (r["gate_up_ms"] * 1e-3))
             line["per_bits"] = per_bits
+            # the same layer with every routed block held as overlaid bit-planes and read at 4, 3 and 2 bits
+            planes = {}
+            keys = ("ms_per_step", "gate_up_ms", "gate_up_gbs", "gate_up_frac", "down_ms", "down_gbs", "down_frac",
+                    "forward_frac", "sm_mhz")
+            for q in (4, 3, 2):
+                r = decode_workload(device, peaks, dataclasses.replace(cfg, bit_rule="all16"), 1, mode, 100, 3,
+                                    min_seconds=0.15, planes_q=q)
+                planes[str(q)] = {key: r[key] for key in keys}
+            line["bit_planes"] = planes
             # the other decode configuration (64 routed top-6 + 2 shared experts, batch 256)
             line["finegrained_decode"] = decode_workload(device, peaks, synth.CONFIGS["finegrained_decode"], 6, mode,
                                                          200, 5)

@@ -432,7 +432,9 @@ __device__ __forceinline__ void epilogue_cols(const KArgs& ka, const UDesc& d, u
 
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
-template <int PHASE, bool HELP>
+// PLANES: the instantiation that also reads overlaid bit-plane blocks; launched only for a layer that has one (the
+// extra code paths cost the ordinary ones instruction-cache room).
+template <int PHASE, bool HELP, bool PLANES>
 __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ KArgs ka, const __grid_constant__ TmapSet tmaps) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
@@ -529,7 +531,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
             const DevRow row = ka.rows[u0.x * 3 + (PHASE == 0 ? m : 2)];
-            const bool planes = row.valid == 2;
+            const bool planes = PLANES && row.valid == 2;
             const uint32_t ubits = row.bits | (planes ? kPlanesFlag : 0u);
             d.bits |= ubits << (8 * m);
             pq[m] = planes ? row.bits : 0u;
@@ -559,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             if (g & ((1u << lg[m]) - 1u)) continue;
             const uint32_t left = ng - g, full_n = 1u << lg[m];
             const uint32_t nt = left < full_n ? left : full_n;
-            const uint32_t q = pq[m];
+            const uint32_t q = PLANES ? pq[m] : 0u;
             const uint32_t bytes = q ? (uint32_t)kPlaneTopCodes + 512u + (q - 2u) * (uint32_t)kPlaneBitTile : nt * tb[m];
             const uint32_t es = empty_s + 8 * s, fs = full_s + 8 * s;
             if (pass) ok = wait_bar(es, (pass - 1) & 1, polls, c, status);
@@ -790,9 +792,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         case 4: ok = dq_unit<4, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
         case 3: ok = dq_unit<3, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
         case 2: ok = dq_unit<2, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case kPlanesFlag | 4: ok = dq_unit<4, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case kPlanesFlag | 3: ok = dq_unit<3, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case kPlanesFlag | 2: ok = dq_unit<2, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+#define PW_PLANE_CASE(Q) case kPlanesFlag | Q: if constexpr (PLANES) ok = dq_unit<Q, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
+        PW_PLANE_CASE(4)
+        PW_PLANE_CASE(3)
+        PW_PLANE_CASE(2)
+#undef PW_PLANE_CASE
         default: break;
       }
       base += ng;
@@ -875,6 +879,14 @@ static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, Tma
   return true;
 }
 
+typedef void (*FfnKernel)(const KArgs, const TmapSet);
+static FfnKernel ffn_kernel_of(int phase, int help, int planes) {
+  static const FfnKernel tab[8] = {ffn_tc_kernel<0, false, false>, ffn_tc_kernel<1, false, false>, ffn_tc_kernel<0, true, false>,
+                                   ffn_tc_kernel<1, true, false>,  ffn_tc_kernel<0, false, true>,  ffn_tc_kernel<1, false, true>,
+                                   ffn_tc_kernel<0, true, true>,   ffn_tc_kernel<1, true, true>};
+  return tab[phase + 2 * help + 4 * planes];
+}
+
 static pw_status tc_setup(pw_ctx* ctx) {
   if (ctx->tc_state) return PW_OK;
   void* fn = nullptr;
@@ -890,10 +902,9 @@ static pw_status tc_setup(pw_ctx* ctx) {
     delete st;
     return PW_ERR_CUDA;
   }
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
-  PW_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+  for (int i = 0; i < 8; ++i)
+    PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_of(i & 1, (i >> 1) & 1, (i >> 2) & 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxDynSmem));
   ctx->tc_state = st;
   return PW_OK;
 }
@@ -952,6 +963,9 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   // token tiles of 128 leave no second accumulator buffer: the variant whose issuer warps share the epilogue
   const bool help = nt_tile > 64;
+  bool planes = false;                           // does the layer hold a bit-plane block?
+  for (int e = 0; e < w.S && !planes; ++e)
+    for (int u = 0; u < 3; ++u) planes |= ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES;
   ka.units = reinterpret_cast<const Unit*>(b + w.units_gu);
   ka.n_bslots = n_bslots[0];
   ka.n_slots = n_slots[0];
@@ -959,7 +973,7 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   ka.y = nullptr;
   ka.y_split_stride = 0;
   ka.work_counter = work_counter;
-  PW_CUDA_OK(launch_dependent(help ? ffn_tc_kernel<0, true> : ffn_tc_kernel<0, false>, dim3(ctx->num_sms), dim3(kThreads),
+  PW_CUDA_OK(launch_dependent(ffn_kernel_of(0, help, planes), dim3(ctx->num_sms), dim3(kThreads),
                               (size_t)smem[0], s, ka, st->xt));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   ka.units = reinterpret_cast<const Unit*>(b + w.units_dn);
@@ -970,7 +984,7 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   ka.y_split_stride = (size_t)R * c.hidden;
   ka.work_counter = work_counter + 1;
   ka.hook = 0;
-  PW_CUDA_OK(launch_dependent(help ? ffn_tc_kernel<1, true> : ffn_tc_kernel<1, false>, dim3(ctx->num_sms), dim3(kThreads),
+  PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads),
                               (size_t)smem[1], s, ka, st->ht));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
