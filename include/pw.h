@@ -401,6 +401,27 @@ typedef struct {
 pw_status pw_plan_step(const pw_plan_tables* tables, uint64_t target, pw_plan_item* steps, size_t max_steps,
                        size_t* n_steps_out, uint64_t* released_out, int32_t* stage_out);
 
+/* The plan queue of Alg. 1.  The runtime calls the planner step again and again while requests run: every call
+ * converts the KV-cache pressure into the byte target D_t (Eq. 7), builds one candidate plan per bitwidth-floor
+ * stage (ScoreActions + GreedySelect) and keeps the candidates in the queue (RefreshPlanQueue), so that newer
+ * observations replace older plans; only when the pressure is there (D_t > 0) does it hand out a plan
+ * (SelectBestPlan: the candidate of the first stage that meets D_t, else the last stage's, the largest reduction
+ * the floors allow).  Without pressure the candidates are prepared for `lookahead_bytes`, what the caller expects
+ * to need next, and the call returns no steps (triggered_out = 0).  steps / max_steps / n_steps_out /
+ * released_out / stage_out as for pw_plan_step.  pw_plan_queue_peek reports a stage's queued candidate (target
+ * it was built for, bytes it releases, number of steps, the planner step that refreshed it).  Host code, no GPU.
+ * Errors: INVALID_ARG (also: tables with another number of stages than the queue), BITS, NOMEM, STATE (peek of a
+ * stage that has never been refreshed). */
+typedef struct pw_plan_queue pw_plan_queue;
+pw_status pw_plan_queue_create(pw_plan_queue** queue, int32_t n_stages);
+pw_status pw_plan_queue_destroy(pw_plan_queue* queue);
+pw_status pw_plan_queue_step(pw_plan_queue* queue, const pw_plan_tables* tables, int64_t free_block_threshold,
+                             int64_t free_blocks, uint64_t kv_block_bytes, uint64_t lookahead_bytes, pw_plan_item* steps,
+                             size_t max_steps, size_t* n_steps_out, uint64_t* released_out, int32_t* stage_out,
+                             int32_t* triggered_out);
+pw_status pw_plan_queue_peek(const pw_plan_queue* queue, int32_t stage, uint64_t* target_out, uint64_t* released_out,
+                             size_t* n_steps_out, uint64_t* refreshed_at_out);
+
 /* Eq. 7: bytes to release = max(0, free_block_threshold + 1 - free_blocks) * kv_block_bytes. */
 uint64_t pw_kv_pressure_bytes(int64_t free_block_threshold, int64_t free_blocks, uint64_t kv_block_bytes);
 

@@ -120,3 +120,31 @@ def plan(committed: np.ndarray, supported: np.ndarray, sensitivity: np.ndarray, 
         if released >= target:
             break
     return result
+
+
+def plan_queue_step(queue: dict, steps_taken: int, tables: dict, free_block_threshold: int, free_blocks: int,
+                    kv_block_bytes: int, lookahead_bytes: int):
+    """One PlanStep of Alg. 1 with its plan queue.  ``queue`` maps stage -> (target, steps, released bytes,
+    refreshed at); ``tables`` are the keyword arguments of plan() without ``target``.  The byte target is Eq. 7;
+    every stage's candidate plan is rebuilt for it (for ``lookahead_bytes`` while there is no pressure) and replaces
+    the stage's entry; under pressure the candidate of the first stage that meets the target is returned, else the
+    last stage's.  Returns (queue, steps taken, triggered, plan or None)."""
+    D = target_bytes(free_block_threshold, free_blocks, kv_block_bytes)
+    triggered = D > 0
+    target = D if triggered else lookahead_bytes
+    floors = tables["floors"]
+    queue = dict(queue)
+    steps_taken += 1
+    for s in range(floors.shape[0]):
+        one = dict(tables, floors=floors[s:s + 1])                  # GreedySelect under the floors of stage s alone
+        st, released, _ = plan(target=target, **one)
+        queue[s] = (target, st, released, steps_taken)
+    best = None
+    if triggered:
+        best = floors.shape[0] - 1
+        for s in range(floors.shape[0]):
+            if queue[s][2] >= D:
+                best = s
+                break
+        best = (queue[best][1], queue[best][2], best)
+    return queue, steps_taken, triggered, best

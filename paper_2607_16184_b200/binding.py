@@ -28,7 +28,7 @@ GROUP = 128
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_plane_bytes", "pw_quantize_planes", "pw_export_planes", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
            "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
-           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_kv_pressure_bytes",
+           "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_plan_queue_create", "pw_plan_queue_destroy", "pw_plan_queue_step", "pw_plan_queue_peek", "pw_kv_pressure_bytes",
            "pw_last_device_status",
            "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_debug_set_wait", "pw_status_str")
 KERNEL_NAMES = ("router", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "observe")
@@ -143,6 +143,17 @@ def load():
     L.pw_quantize_planes.argtypes = [vp, vp, C.c_uint32, C.c_uint32, C.POINTER(pw_page), vp]
     L.pw_export_planes.restype = C.c_int
     L.pw_export_planes.argtypes = [vp, C.POINTER(pw_page), C.POINTER(pw_page), vp]
+    L.pw_plan_queue_create.restype = C.c_int
+    L.pw_plan_queue_create.argtypes = [C.POINTER(C.c_void_p), C.c_int32]
+    L.pw_plan_queue_destroy.restype = C.c_int
+    L.pw_plan_queue_destroy.argtypes = [vp]
+    L.pw_plan_queue_step.restype = C.c_int
+    L.pw_plan_queue_step.argtypes = [vp, C.POINTER(pw_plan_tables), C.c_int64, C.c_int64, C.c_uint64, C.c_uint64,
+                                     C.POINTER(pw_plan_item), C.c_size_t, C.POINTER(C.c_size_t), C.POINTER(C.c_uint64),
+                                     C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    L.pw_plan_queue_peek.restype = C.c_int
+    L.pw_plan_queue_peek.argtypes = [vp, C.c_int32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_size_t),
+                                     C.POINTER(C.c_uint64)]
     L.pw_launch_count.restype = C.c_uint64
     L.pw_launch_count.argtypes = [vp]
     L.pw_debug_set_wait.restype = C.c_int
@@ -176,11 +187,9 @@ def pw_kv_pressure_bytes(free_block_threshold: int, free_blocks: int, kv_block_b
     return int(load().pw_kv_pressure_bytes(free_block_threshold, free_blocks, kv_block_bytes))
 
 
-def pw_plan_step(n_layers: int, n_experts: int, n_shared: int, committed, supported, sensitivity, page_bytes, mass,
-                 bucket_share, bucket_mu, stage_floor, target: int, phi=None, heads=None, alpha: float = 1.0,
-                 rho_min: float = -1.0, rho_max: float = 1.0, epsilon: float = 1e-9):
-    """One planner step on host arrays (numpy; shapes as in include/pw.h).  Returns (steps, released bytes,
-    stage) with steps as tuples (layer, expert, kind, from_bits, to_bits, damage)."""
+def _plan_tables(n_layers, n_experts, n_shared, committed, supported, sensitivity, page_bytes, mass, bucket_share,
+                 bucket_mu, stage_floor, phi, heads, alpha, rho_min, rho_max, epsilon):
+    """pw_plan_tables over host arrays (numpy; shapes as in include/pw.h) + the arrays it points into."""
     import numpy as np
     keep = []
 
@@ -202,13 +211,67 @@ def pw_plan_step(n_layers: int, n_experts: int, n_shared: int, committed, suppor
     t.alpha, t.rho_min, t.rho_max, t.epsilon = alpha, rho_min, rho_max, epsilon
     t.n_buckets, t.n_stages = floors.shape[1], floors.shape[0]
     t.bucket_share, t.bucket_mu, t.stage_floor = ptr(bucket_share, np.float32), ptr(bucket_mu, np.float32), ptr(floors, np.uint8)
-    n_rows = n_layers * (n_experts + n_shared) * 3
-    cap = n_rows * 4
+    return t, keep
+
+
+def _plan_items(items, n):
+    return [(it.layer, it.expert, it.kind, it.from_bits, it.to_bits, it.damage) for it in items[:n]]
+
+
+def pw_plan_step(n_layers: int, n_experts: int, n_shared: int, committed, supported, sensitivity, page_bytes, mass,
+                 bucket_share, bucket_mu, stage_floor, target: int, phi=None, heads=None, alpha: float = 1.0,
+                 rho_min: float = -1.0, rho_max: float = 1.0, epsilon: float = 1e-9):
+    """One planner step on host arrays (numpy; shapes as in include/pw.h).  Returns (steps, released bytes,
+    stage) with steps as tuples (layer, expert, kind, from_bits, to_bits, damage)."""
+    t, keep = _plan_tables(n_layers, n_experts, n_shared, committed, supported, sensitivity, page_bytes, mass, bucket_share,
+                           bucket_mu, stage_floor, phi, heads, alpha, rho_min, rho_max, epsilon)
+    cap = n_layers * (n_experts + n_shared) * 3 * 4
     items = (pw_plan_item * cap)()
     n, rel, stage = C.c_size_t(), C.c_uint64(), C.c_int32()
     _check(load().pw_plan_step(C.byref(t), target, items, cap, C.byref(n), C.byref(rel), C.byref(stage)), "pw_plan_step")
-    steps = [(it.layer, it.expert, it.kind, it.from_bits, it.to_bits, it.damage) for it in items[: n.value]]
-    return steps, int(rel.value), int(stage.value)
+    return _plan_items(items, n.value), int(rel.value), int(stage.value)
+
+
+class PlanQueue:
+    """The plan queue of Alg. 1 (host code): ``step`` is one PlanStep -- refresh every stage's candidate plan from
+    the tables, hand out a plan only under KV-cache pressure."""
+
+    def __init__(self, n_stages: int):
+        self.handle = C.c_void_p()
+        _check(load().pw_plan_queue_create(C.byref(self.handle), n_stages), "pw_plan_queue_create")
+
+    def close(self):
+        if self.handle:
+            load().pw_plan_queue_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def step(self, n_layers, n_experts, n_shared, committed, supported, sensitivity, page_bytes, mass, bucket_share,
+             bucket_mu, stage_floor, free_block_threshold: int, free_blocks: int, kv_block_bytes: int,
+             lookahead_bytes: int, phi=None, heads=None, alpha: float = 1.0, rho_min: float = -1.0, rho_max: float = 1.0,
+             epsilon: float = 1e-9):
+        """Returns (triggered, steps, released bytes, stage); without pressure: (False, [], 0, -1)."""
+        t, keep = _plan_tables(n_layers, n_experts, n_shared, committed, supported, sensitivity, page_bytes, mass,
+                               bucket_share, bucket_mu, stage_floor, phi, heads, alpha, rho_min, rho_max, epsilon)
+        cap = n_layers * (n_experts + n_shared) * 3 * 4
+        items = (pw_plan_item * cap)()
+        n, rel, stage, trig = C.c_size_t(), C.c_uint64(), C.c_int32(), C.c_int32()
+        _check(load().pw_plan_queue_step(self.handle, C.byref(t), free_block_threshold, free_blocks, kv_block_bytes,
+                                         lookahead_bytes, items, cap, C.byref(n), C.byref(rel), C.byref(stage),
+                                         C.byref(trig)), "pw_plan_queue_step")
+        return bool(trig.value), _plan_items(items, n.value), int(rel.value), int(stage.value)
+
+    def peek(self, stage: int):
+        """(target, released bytes, number of steps, refreshed at planner step) of a stage's queued candidate."""
+        tg, rel, n, at = C.c_uint64(), C.c_uint64(), C.c_size_t(), C.c_uint64()
+        _check(load().pw_plan_queue_peek(self.handle, stage, C.byref(tg), C.byref(rel), C.byref(n), C.byref(at)),
+               "pw_plan_queue_peek")
+        return int(tg.value), int(rel.value), int(n.value), int(at.value)
 
 
 def pw_route_tokens_static(router_logits: torch.Tensor, top_k: int,

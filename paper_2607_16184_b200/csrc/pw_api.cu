@@ -246,8 +246,9 @@ extern "C" pw_status pw_query_row(pw_ctx* ctx, int layer, int expert, int kind, 
   return PW_OK;
 }
 
-extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int top_k,
-                                    const pw_page_table* table, float* out, pw_mode mode, pw_stream stream) {
+// Argument checks of a forward call: everything that can be refused is refused here, before anything is enqueued.
+static pw_status check_forward_args(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int top_k,
+                                    const pw_page_table* table, const float* out, pw_mode mode) {
   if (!ctx || !hidden || !logits || !out) return PW_ERR_INVALID_ARG;
   const pw_config& c = ctx->cfg;
   if (table && table->owner != ctx) return PW_ERR_INVALID_ARG;
@@ -259,15 +260,23 @@ extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, 
   for (int e = 0; e < ctx->ws.S; ++e)
     for (int u = 0; u < 3; ++u)
       if (!ctx->host_valid[row_index(ctx, layer, e, u)]) return PW_ERR_STATE;
+  if (mode == PW_MODE_SIMT)                      // the CUDA-core kernel reads TILED pages only
+    for (int e = 0; e < ctx->ws.S; ++e)
+      for (int u = 0; u < 3; ++u)
+        if (ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES) return PW_ERR_STATE;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden, const float* logits, int T, int top_k,
+                                    const pw_page_table* table, float* out, pw_mode mode, pw_stream stream) {
+  const pw_status as = check_forward_args(ctx, layer, hidden, logits, T, top_k, table, out, mode);
+  if (as != PW_OK) return as;
+  const pw_config& c = ctx->cfg;
 
   // The tensor-core kernels win at every batch size measured (one token of a Mixtral-shaped layer: 0.12 ms
   // against 1.96 ms for the CUDA-core kernel), so AUTO means TENSOR; the CUDA-core kernel stays selectable as
   // an independent second implementation.
   if (mode == PW_MODE_AUTO) mode = PW_MODE_TENSOR;
-  if (mode == PW_MODE_SIMT)                      // the CUDA-core kernel reads TILED pages only
-    for (int e = 0; e < ctx->ws.S; ++e)
-      for (int u = 0; u < 3; ++u)
-        if (ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES) return PW_ERR_STATE;
   int nt_tile = 0, ksplit = 1;
   if (mode == PW_MODE_TENSOR) {
     nt_tile = tensor_token_tile(ctx, T, top_k);
@@ -320,6 +329,10 @@ extern "C" pw_status pw_moe_forward_host(pw_ctx* ctx, int layer, const void* hid
   if (T < 1 || T > c.max_tokens) return PW_ERR_INVALID_ARG;
   char* b = ctx->base;
   const WsMap& w = ctx->ws;
+  // refuse what the forward call would refuse before the first copy is enqueued (the staging buffers stay untouched)
+  const pw_status as = check_forward_args(ctx, layer, b + w.io_hidden, reinterpret_cast<const float*>(b + w.io_logits), T,
+                                          top_k, nullptr, reinterpret_cast<const float*>(b + w.io_out), mode);
+  if (as != PW_OK) return as;
   PW_CUDA_OK(cudaMemcpyAsync(b + w.io_hidden, hidden_host, (size_t)T * c.hidden * 2, cudaMemcpyHostToDevice, stream));
   PW_CUDA_OK(cudaMemcpyAsync(b + w.io_logits, logits_host, (size_t)T * c.n_experts * 4, cudaMemcpyHostToDevice, stream));
   pw_status st = pw_moe_forward(ctx, layer, b + w.io_hidden, reinterpret_cast<const float*>(b + w.io_logits), T, top_k,

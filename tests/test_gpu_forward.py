@@ -305,6 +305,17 @@ def test_host_buffer_entry_point_matches_the_device_one(orc):
             ctx.pw_moe_forward_host(0, big, torch.zeros(cfg.tokens + 1, cfg.n_experts), cfg.top_k,
                                     torch.empty(cfg.tokens + 1, cfg.hidden))
         assert e.value.status == 1
+        # an argument error is found before any copy is enqueued: nothing is launched, the staging buffers keep
+        # the previous call's inputs (the next device-side call on them gives the previous result)
+        n0 = ctx.pw_launch_count()
+        junk = torch.full((cfg.tokens, cfg.hidden), 7.0, dtype=torch.float16)
+        with pytest.raises(B.PwError) as e:
+            ctx.pw_moe_forward_host(0, junk, lh, cfg.n_experts + 1, oh)       # top_k out of range
+        assert e.value.status == 1 and ctx.pw_launch_count() == n0
+        torch.cuda.synchronize()
+        ctx.pw_moe_forward_host(0, xh, lh, cfg.top_k, oh)
+        torch.cuda.synchronize()
+        assert torch.equal(oh, want.cpu())
         assert ctx.pw_last_device_status() == 0
     finally:
         ctx.close()

@@ -127,3 +127,31 @@ def test_properties_on_random_tables(pl):
     bigger, _, stage2 = pl.plan(*args, 2500, E, n_shared)
     if stage2 == 0:
         assert bigger[: len(small)] == small
+
+
+def test_plan_queue_step_refreshes_and_selects(pl):
+    """Alg. 1: without pressure the queue is refreshed and no plan leaves it; under pressure the selected plan is
+    the one a fresh planner step returns for the target of Eq. 7; a later step replaces older candidates."""
+    L, E = 1, 4
+    committed = np.full((L, E, 3), 16, np.int32)
+    supported = np.ones((L, E, 3, 5), bool)
+    sens = np.tile(np.array([0.0, 1.0, 2.0, 4.0, 8.0], np.float32), (L, E, 3, 1))
+    sens[0, 0] *= 0.1                                           # expert 0 is the cheapest to lower
+    nbytes = np.tile(np.array([1000, 600, 400, 300, 200], np.int64), (L, E, 3, 1))
+    mass = np.array([[0.1, 0.2, 0.3, 0.4]], np.float32)
+    tables = dict(committed=committed, supported=supported, sensitivity=sens, page_bytes=nbytes, mass=mass, phi=None,
+                  heads=None, shares=[0.5, 1.0], mu=[2.0, 1.0], floors=np.array([[8, 4], [4, 2]], np.int32), alpha=1.0,
+                  rho_min=-1.0, rho_max=1.0, eps=1e-9, n_experts=E, n_shared=0)
+    q, n, trig, best = pl.plan_queue_step({}, 0, tables, free_block_threshold=4, free_blocks=9, kv_block_bytes=500,
+                                          lookahead_bytes=900)
+    assert not trig and best is None and n == 1
+    assert q[0][0] == 900 and q[0][3] == 1 and q[0][2] >= 900   # candidates built for the look-ahead bytes
+    # pressure: 4 + 1 - 1 = 4 blocks of 500 bytes
+    q, n, trig, best = pl.plan_queue_step(q, n, tables, 4, 1, 500, 900)
+    assert trig and n == 2 and q[0][0] == 2000 and q[1][3] == 2
+    fresh = pl.plan(target=2000, **tables)
+    assert best[0] == fresh[0] and best[1] == fresh[1] and best[2] == fresh[2]
+    # a target the first stage cannot meet (its floors allow 12 blocks x 400 + ... ): falls to the later stage
+    big = sum(1000 - 400 for _ in range(6)) + sum(1000 - 600 for _ in range(6)) + 1
+    q, n, trig, best = pl.plan_queue_step(q, n, tables, big // 500 + 1, 0, 500, 0)
+    assert trig and best[2] == 1 and best[1] >= pl.target_bytes(big // 500 + 1, 0, 500)

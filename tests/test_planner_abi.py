@@ -67,3 +67,39 @@ def test_pressure_bytes_and_argument_errors():
     with pytest.raises(B.PwError) as e:
         B.pw_plan_step(0, 2, 0, np.full((1, 2, 3), 16, np.uint8), ones, ones, ones, np.ones((1, 2)), [1.0], [1.0], [[2]], 10)
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_library_plan_queue_matches_the_oracle(pl, seed):
+    """The plan queue of Alg. 1 behind the C ABI replayed against the oracle's: a run of planner steps with changing
+    KV-cache pressure and routing mass; queued candidates, the trigger and the selected plans agree."""
+    rng = np.random.default_rng(seed)
+    L, E, n_shared = 2, 8, 1
+    committed, supported, sens, nbytes, mass, phi, heads = random_tables(rng, L, E, n_shared, True)
+    shares, mu = np.array([0.25, 0.5, 1.0], np.float32), np.array([4.0, 2.0, 1.0], np.float32)
+    floors = np.array([[8, 4, 3], [4, 3, 2], [2, 2, 2]], np.uint8)
+    q = B.PlanQueue(3)
+    oq, on = {}, 0
+    kv = 64 << 20
+    for step, free_blocks in enumerate([40, 12, 3, 30, 0]):                  # threshold 8: pressure at steps 2 and 4
+        mass = rng.dirichlet(np.ones(E), size=L).astype(np.float32)          # newer observations every step
+        trig, got, released, stage = q.step(L, E, n_shared, committed, supported, sens, nbytes, mass, shares, mu, floors,
+                                            8, free_blocks, kv, 5 * kv, phi=phi, heads=heads, alpha=0.7, rho_min=-1.5,
+                                            rho_max=1.5, epsilon=1e-6)
+        tables = dict(committed=committed.astype(np.int32), supported=supported, sensitivity=sens,
+                      page_bytes=nbytes.astype(np.int64), mass=mass, phi=phi, heads=heads, shares=shares.tolist(),
+                      mu=mu.tolist(), floors=floors.astype(np.int32), alpha=float(np.float32(0.7)), rho_min=-1.5,
+                      rho_max=1.5, eps=float(np.float32(1e-6)), n_experts=E, n_shared=n_shared)
+        oq, on, otrig, best = pl.plan_queue_step(oq, on, tables, 8, free_blocks, kv, 5 * kv)
+        assert trig == otrig == (free_blocks <= 8)
+        for s in range(3):
+            target, rel, n, at = q.peek(s)
+            assert (target, rel, n, at) == (oq[s][0], oq[s][2], len(oq[s][1]), oq[s][3])
+        if trig:
+            assert [x[:5] for x in got] == [x[:5] for x in best[0]]
+            assert released == best[1] and stage == best[2]
+        else:
+            assert got == [] and released == 0 and stage == -1
+    q.close()
+    with pytest.raises(B.PwError):
+        B.PlanQueue(0)
