@@ -2,35 +2,32 @@
 //
 //   D[128 weight rows, N tokens] += W[128, 16] * X[N, 16]^T      (tcgen05.mma, kind::f16, fp32 in TMEM)
 //
-// Weight pages stream HBM -> shared memory with bulk async copies into a ring of 34 KB slots.  What travels
-// in one copy is a "chunk": up to four consecutive tile images of one row tile of a quantized page (a tile
-// image = 128 rows x one group: codes, scales, zero-points; consecutive groups of a row tile are contiguous
-// in the page), two for 8-bit pages, or one whole 16-bit tile (32 KB).  Chunks are numbered in issue order;
-// number `seq` lives in slot seq mod n_slots, so every role finds its own chunks from their numbers alone.
-// A 16-bit tile is already in the tensor core's K-major core-matrix layout: the MMA reads it from shared
-// memory as the A operand without any thread touching it.  A quantized tile is unpacked and dequantized in
-// registers (one weight row per thread) and written to tensor memory, which the MMA then reads as its A
-// operand.  The token tile (B operand) comes from the k-chunk-major operand buffers with one 2-D TMA copy
-// per group.
+// Weight pages stream HBM -> shared memory with bulk async copies into a ring of 17 KB slots.  A "slot item"
+// is one tile image of a quantized page (128 rows x one group: codes, scales, zero-points, 4.5 .. 16.5 KB,
+// one copy) or one K-half (16 KB) of a 16-bit tile; slot item number seq lives in slot seq mod n_slots, so
+// every role finds its own items from their numbers alone.  A 16-bit half is already in the tensor core's
+// K-major core-matrix layout: the MMA reads it from shared memory as the A operand without any thread
+// touching it.  A quantized tile is unpacked and dequantized in registers (one weight row per thread) and
+// written to tensor memory, which the MMA then reads as its A operand.  The token tile (B operand) comes
+// from the k-chunk-major operand buffers with one 2-D TMA copy per group.
 //
-// One persistent CTA per SM, 26 warps.  The arithmetic pipes that the dequantizers use run at half rate and
-// are shared with every control instruction, so each role does as little per tile as it can: a unit's
-// description is read from global memory once (by the weight producer) and handed to the other roles through
-// shared memory, barrier traffic of the ring is per chunk, and the dequantizer loop is compiled once per
-// bitwidth with nothing but the decode between its waits.
+// One persistent CTA per SM, 27 warps.  The control roles are single threads with short dependent
+// instruction chains: they share the schedulers with the arithmetic-heavy dequantizers, and every
+// instruction of theirs waits its turn, so each of them does as little per item as possible.
 //   warps 0-15   dequantize: four groups of four warps; tile k of a matrix goes to that matrix's group
 //                k mod (groups per matrix); warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
 //                a group has one operand slot of 64 columns in tensor memory (a whole tile, K 0..127) and hands
 //                it to its issuer once per tile, while it decodes the first half of its next tile in registers;
-//   warp 16      weight producer: claims the CTA's units from a global counter, posts their descriptions on the
-//                CTA's work list and issues the chunk copies as far ahead as the ring allows;
+//   warps 16,18  weight producers: producer P arms the slot items with number = P mod 2 (which sit in the
+//                slots = P mod 2) and issues their copies, as far ahead as the ring allows; producer 0 also
+//                claims the CTA's units from a global counter and posts them on the CTA's work list;
 //   warp 17      token-tile producer (its own few slots, never holds back the weight stream);
-//   warps 18-21  MMA issuers (warp 18 also allocates tensor memory).  Dependent MMAs into one accumulator
-//                follow each other ~100 cycles apart whatever their size, so the issuers work in parallel:
-//                issuer j of a matrix issues all eight k-steps of the tiles k = j mod (issuers per matrix) into
-//                its own partial accumulator -- with as many issuers as groups, each dequantizer group has an
+//   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  A tcgen05.mma holds its issuing
+//                thread for ~100 cycles whatever its size, so the issuers work in parallel: issuer j of a
+//                matrix issues all eight k-steps of the tiles k = j mod (issuers per matrix) into its own
+//                partial accumulator -- with as many issuers as groups, each dequantizer group has an
 //                issuer of its own -- and no two threads ever accumulate into the same columns;
-//   warps 22-25  epilogue: adds the partials; SwiGLU -> fp16 operand of the down projection (PHASE 0), or the
+//   warps 23-26  epilogue: adds the partials; SwiGLU -> fp16 operand of the down projection (PHASE 0), or the
 //                fp32 split-K partial of the down projection (PHASE 1).  Narrow token tiles alternate
 //                between two accumulator buffers, so the next unit's MMAs overlap the epilogue.
 //                Token tiles wider than 64 leave no second buffer: the HELP instantiation, launched for
@@ -46,52 +43,45 @@
 
 namespace pw {
 
-constexpr int kSlotBytes = 34816;              // one ring slot: four 4-bit tile images (4 x 8704), two 8-bit, one 16-bit tile
-constexpr int kMaxSlots = 6;
-constexpr int kChunkArrivals = 16;             // arrivals that hand a slot back: four tiles x four warps
+constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item (16 KB codes + 512 B) fits
+constexpr int kMaxSlots = 16;
 constexpr int kMaxASlots = 4;                  // operand slots in tensor memory, one per group (64 columns = a 128 x 128 tile)
 constexpr int kMaxBSlots = 5;
-constexpr int kSched = 32;                     // entries of the CTA's work list
-constexpr int kCtrlBytes = 2048;
+constexpr int kCtrlBytes = 1024;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
 constexpr int kDqWarps = 16;
-constexpr int kWarpW = 16, kWarpB = 17, kWarpMma = 18, kIssuers = 4, kWarpEpi = 22;
-constexpr int kThreads = 832;
+constexpr int kWarpCodes = 16, kWarpTokens = 17, kWarpCodes2 = 18, kWarpMma = 19, kIssuers = 4, kWarpEpi = 23;
+constexpr int kThreads = 864;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kSuspendHintNs = 20000;     // a blocked barrier wait sleeps up to this long per poll
-constexpr uint32_t kDefaultWaitPolls = 100000; // x kSuspendHintNs = 2 s
-
-// What the other roles need to know of a unit; posted by the weight producer.
-struct UDesc {
-  int32_t unit;                                // index in the unit list, -1 = no more work
-  int32_t row_tile, tok0, ntok, g0, ng, split;
-  uint32_t bits;                               // bitwidth of matrix 0 | bitwidth of matrix 1 << 8
-};
-static_assert(sizeof(UDesc) == 32, "UDesc layout");
+constexpr uint32_t kSuspendHintNs = 20000;                   // a blocked barrier wait sleeps up to this long per poll
+constexpr uint32_t kDefaultWaitPolls = 100000;               // x kSuspendHintNs = 2 s
 
 struct Ctrl {                                  // lives at the start of dynamic shared memory
-  // One full barrier per ring slot (armed by the weight producer).  A slot is handed back by sixteen arrivals:
-  // four per tile of the chunk, from the warps of the dequantizer group that read the tile, or from the MMA
-  // issuer that read a 16-bit tile (one tcgen05.commit plus three plain arrivals); for a chunk of fewer than
-  // four tiles the producer itself makes up the difference when it arms the slot.
+  // One full barrier per ring slot (armed by the weight producer).  A slot is handed back either by the
+  // four warps of the dequantizer group that read it, or by the MMA issuer that read a 16-bit half from it
+  // (one tcgen05.commit plus three plain arrivals, so that both kinds complete the same four-arrival phase
+  // and the weight producers need not remember who holds a slot).
   unsigned long long full[kMaxSlots], empty[kMaxSlots];
   unsigned long long b_full[kMaxBSlots], b_empty[kMaxBSlots];
   unsigned long long a_full[kMaxASlots], a_empty[kMaxASlots];
   unsigned long long d_full[2], d_empty[2];     // two accumulator buffers (a wide token tile takes both)
   uint32_t tmem_base;
   volatile int abort_flag;
-  volatile uint32_t issued;                    // chunks armed so far
-  volatile uint32_t b_issued;                  // token tiles armed so far
+  // Slot items with an even number are armed by weight producer 0, odd ones by producer 1 (the number of
+  // slots is even, so each producer also owns every other slot).  issued[p]: producer p has armed all of
+  // its slot items below this number.
+  volatile uint32_t issued[2];
+  volatile uint32_t b_issued;                  // token tiles armed so far (same purpose, for the token-tile slots)
   // Work list of this CTA: the weight producer claims units from a global counter and posts them here;
-  // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others).
+  // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
+  volatile int32_t sched_unit[32];
   // Set once the kernel ahead of this one in the stream has completed.  Until then a wait that runs out is not a
-  // fault (the CTA may have been placed long before its inputs exist) and simply starts over.
+  // fault and simply starts over.
   volatile uint32_t dep_ready;
-  uint32_t pad_[2];
-  UDesc sched[kSched];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
+
 
 struct TmapSet {                               // token-tile copies: one map per tile height 16, 32, .. 128
   CUtensorMap m[8];
@@ -103,89 +93,146 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(unsigned long long* b, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
 }
-__device__ __forceinline__ void mbar_arrive_s(uint32_t bar_s) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_s) : "memory");
+__device__ __forceinline__ void mbar_arrive(unsigned long long* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
-// one arrival by the threads for which `pred` holds (no branch around it)
-__device__ __forceinline__ void mbar_arrive_if_s(uint32_t bar_s, bool pred) {
+__device__ __forceinline__ void mbar_arrive_n(unsigned long long* b, uint32_t n) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(n) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(unsigned long long* b, uint32_t parity) {
+  uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %1, 0;\n\t"
-      "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(bar_s),
-      "r"((uint32_t)pred)
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(b)), "r"(parity)
       : "memory");
+  return ok != 0;
 }
-__device__ __forceinline__ void mbar_arrive_n_s(uint32_t bar_s, uint32_t n) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(n) : "memory");
+// Bounded wait.  Returns false when the limit ran out (and then raises the abort; the other roles of the CTA,
+// starved by the one that gave up, run into their own limits within the same second or two, and since every
+// role has then been idle for at least a second no copy of the CTA is still in flight when it leaves).  Each poll is a try_wait with a
+// suspend-time hint, so a waiting thread sleeps inside the barrier unit instead of spending issue slots (an
+// arrival that does not complete the phase still wakes it, hence the loop); 100000 polls of up to kSuspendHintNs
+// each are the 2 s limit.  The loop is inline and written in PTX on purpose: with an out-of-line slow path the
+// call made the compiler keep each role's loop state -- for the dequantizers a vector of 32 results between
+// decode and store -- in call-preserved registers and copy it around, which cost 2 % of the decode step.
+// (the barrier is given by its shared-memory address: the control loops keep those in registers)
+// A wait ran out: not a fault while the kernel ahead in the stream is still running (the CTA may have been placed
+// long before its inputs exist), otherwise the CTA gives up.
+__device__ __forceinline__ bool wait_failed(Ctrl* c, int32_t* status) {
+  if (!c->dep_ready) return false;               // start over
+  c->abort_flag = 1;
+  atomicMax(status, (int)PW_ERR_TIMEOUT);
+  return true;
 }
+__device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, uint32_t polls, Ctrl* c, int32_t* status) {
+  for (;;) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+        "mov.u32 n, 0;\n"
+        "PW_WAITN:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "@p bra PW_DONEN;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "setp.lt.u32 q, n, %4;\n\t"
+        "@q bra PW_WAITN;\n"
+        "PW_DONEN:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "r"(polls)
+        : "memory");
+    if (ok) return true;
+    if (wait_failed(c, status)) return false;
+  }
+}
+// Sleep-and-look until the shared-memory word at `addr_s` exceeds `value`: at least 64 ns per look, polls * 256 looks.
+__device__ __forceinline__ bool flag_wait(uint32_t addr_s, uint32_t value, uint32_t polls, Ctrl* c, int32_t* status) {
+  const uint32_t looks = polls < (1u << 24) ? polls << 8 : 0xffffffffu;
+  for (;;) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
+        "mov.u32 k, 0;\n"
+        "PW_FL:\n\t"
+        "ld.volatile.shared.u32 v, [%1];\n\t"
+        "setp.gt.u32 p, v, %2;\n\t"
+        "@p bra PW_FLD;\n\t"
+        "nanosleep.u32 64;\n\t"
+        "add.u32 k, k, 1;\n\t"
+        "setp.lt.u32 q, k, %3;\n\t"
+        "@q bra PW_FL;\n"
+        "PW_FLD:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr_s), "r"(value), "r"(looks)
+        : "memory");
+    if (ok) return true;
+    if (wait_failed(c, status)) return false;
+  }
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// the same with shared-memory addresses already in hand (saves the address conversions in a hot control loop)
 __device__ __forceinline__ void mbar_expect_tx_s(uint32_t bar_s, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(bytes) : "memory");
-}
-// One bounded wait: up to `polls` try_waits, each of which sleeps inside the barrier unit for up to
-// kSuspendHintNs (an arrival that does not complete the phase still wakes it, hence the loop).  The loop is
-// inline PTX on purpose: an out-of-line slow path in a hot loop makes the compiler keep the loop's state in
-// call-preserved registers.
-__device__ __forceinline__ bool mbar_poll(uint32_t bar_s, uint32_t parity, uint32_t polls) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
-      "mov.u32 n, 0;\n"
-      "PW_WAITN:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "@p bra PW_DONEN;\n\t"
-      "add.u32 n, n, 1;\n\t"
-      "setp.lt.u32 q, n, %4;\n\t"
-      "@q bra PW_WAITN;\n"
-      "PW_DONEN:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "r"(polls)
-      : "memory");
-  return ok != 0;
-}
-// Sleep-and-look until the shared-memory word at `addr_s` exceeds `value`: at least 64 ns per look, `looks` looks.
-__device__ __forceinline__ bool flag_poll(uint32_t addr_s, uint32_t value, uint32_t looks) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
-      "mov.u32 k, 0;\n"
-      "PW_FL:\n\t"
-      "ld.volatile.shared.u32 v, [%1];\n\t"
-      "setp.gt.u32 p, v, %2;\n\t"
-      "@p bra PW_FLD;\n\t"
-      "nanosleep.u32 64;\n\t"
-      "add.u32 k, k, 1;\n\t"
-      "setp.lt.u32 q, k, %3;\n\t"
-      "@q bra PW_FL;\n"
-      "PW_FLD:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(addr_s), "r"(value), "r"(looks)
-      : "memory");
-  return ok != 0;
 }
 __device__ __forceinline__ void bulk_g2s_s(uint32_t dst_s, const void* src, uint32_t bytes, uint32_t bar_s) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_s),
                "l"(src), "r"(bytes), "r"(bar_s)
                : "memory");
 }
-__device__ __forceinline__ void tma_2d_g2s_s(uint32_t dst_s, const CUtensorMap* map, int x, int y, uint32_t bar_s) {
+__device__ __forceinline__ void tma_2d_g2s(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          dst_s),
-      "l"(map), "r"(x), "r"(y), "r"(bar_s)
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(unsigned long long* b) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(b))
+               : "memory");
+}
 __device__ __forceinline__ void tc_commit_s(uint32_t bar_s) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_s) : "memory");
 }
-// Four consecutive k-steps issued from one asm block (the issuing thread gets few issue slots, so every
-// instruction around an MMA counts).  Descriptors are passed as (lo, hi) words; only lo moves.
+// A operand in tensor memory
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// A operand in shared memory
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// NK consecutive k-steps of one item issued from one asm block (the issuing thread gets few issue slots,
+// so every instruction around an MMA counts).  Descriptors are passed as (lo, hi) words; only lo moves.
 // TS: A in tensor memory at a_tmem (+a_step per k-step).  `acc0`: accumulate flag of the first k-step.
-__device__ __forceinline__ void tc_mma_ts_burst4(uint32_t d_tmem, uint32_t a_tmem, uint32_t a_step, uint32_t b_lo,
-                                                 uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t acc0) {
+template <int NK>
+__device__ __forceinline__ void tc_mma_ts_burst(uint32_t d_tmem, uint32_t a_tmem, uint32_t a_step, uint32_t b_lo,
+                                                uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t acc0) {
   asm volatile(
       "{\n\t.reg .pred p, t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
       "setp.ne.b32 p, %7, 0;\n\t"
@@ -194,18 +241,27 @@ __device__ __forceinline__ void tc_mma_ts_burst4(uint32_t d_tmem, uint32_t a_tme
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %6, p;\n\t"
       "add.u32 lo, %3, %5;\n\tadd.u32 a, %1, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
-      "add.u32 lo, lo, %5;\n\tadd.u32 a, a, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
-      "add.u32 lo, lo, %5;\n\tadd.u32 a, a, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
       "}" ::"r"(d_tmem),
       "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
       : "memory");
+  if (NK == 4) {
+    asm volatile(
+        "{\n\t.reg .pred t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "mad.lo.u32 lo, %5, 2, %3;\n\tmad.lo.u32 a, %2, 2, %1;\n\tmov.b64 bd, {lo, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "add.u32 lo, lo, %5;\n\tadd.u32 a, a, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        : "memory");
+  }
 }
 // SS: A in shared memory, descriptor (a_lo, a_hi), +a_step per k-step.
-__device__ __forceinline__ void tc_mma_ss_burst4(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step,
-                                                 uint32_t b_lo, uint32_t b_hi, uint32_t b_step, uint32_t idesc,
-                                                 uint32_t acc0) {
+template <int NK>
+__device__ __forceinline__ void tc_mma_ss_burst(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step,
+                                                uint32_t b_lo, uint32_t b_hi, uint32_t b_step, uint32_t idesc,
+                                                uint32_t acc0) {
   asm volatile(
       "{\n\t.reg .pred p, t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
       "setp.ne.b32 p, %8, 0;\n\t"
@@ -214,13 +270,21 @@ __device__ __forceinline__ void tc_mma_ss_burst4(uint32_t d_tmem, uint32_t a_lo,
       "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, p;\n\t"
       "add.u32 la, %1, %3;\n\tadd.u32 lb, %4, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
-      "add.u32 la, la, %3;\n\tadd.u32 lb, lb, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
-      "add.u32 la, la, %3;\n\tadd.u32 lb, lb, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
       "}" ::"r"(d_tmem),
       "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
       : "memory");
+  if (NK == 4) {
+    asm volatile(
+        "{\n\t.reg .pred t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "mad.lo.u32 la, %3, 2, %1;\n\tmad.lo.u32 lb, %6, 2, %4;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "add.u32 la, la, %3;\n\tadd.u32 lb, lb, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        : "memory");
+  }
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const __half2* v) {
   const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
@@ -231,6 +295,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const __half2* v) {
       "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
       "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const __half2* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
@@ -246,67 +319,66 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// ---- the pieces every role shares -------------------------------------------------------------------
-// A wait ran out: not a fault while the kernel ahead is still running, otherwise the CTA gives up.
-__device__ __forceinline__ bool wait_failed(Ctrl* c, int32_t* status) {
-  if (!c->dep_ready) return false;               // start over
-  c->abort_flag = 1;
-  atomicMax(status, (int)PW_ERR_TIMEOUT);
-  return true;
-}
-__device__ __forceinline__ bool wait_bar(uint32_t bar_s, uint32_t parity, uint32_t polls, Ctrl* c, int32_t* status) {
-  while (!mbar_poll(bar_s, parity, polls))
-    if (wait_failed(c, status)) return false;
-  return true;
-}
-__device__ __forceinline__ bool wait_flag(const volatile uint32_t* flag, uint32_t value, uint32_t polls, Ctrl* c,
-                                          int32_t* status) {
-  if (*flag > value) return true;
-  const uint32_t looks = polls < (1u << 24) ? polls << 8 : 0xffffffffu;
-  while (!flag_poll(smem_u32(const_cast<uint32_t*>(flag)), value, looks))
-    if (wait_failed(c, status)) return false;
-  return true;
-}
-// Entry i of this CTA's work list (bounded wait until the weight producer has posted it).
-__device__ __forceinline__ bool get_desc(uint32_t i, uint32_t polls, Ctrl* c, int32_t* status, UDesc& d) {
-  if (!wait_flag(&c->sched_n, i, polls, c, status)) return false;
-  const uint4* p = reinterpret_cast<const uint4*>(&c->sched[i & (kSched - 1)]);
-  const uint4 a = p[0], b = p[1];
-  d.unit = (int32_t)a.x;
-  d.row_tile = (int32_t)a.y;
-  d.tok0 = (int32_t)a.z;
-  d.ntok = (int32_t)a.w;
-  d.g0 = (int32_t)b.x;
-  d.ng = (int32_t)b.y;
-  d.split = (int32_t)b.z;
-  d.bits = b.w;
-  return true;
-}
-
-// Chunks: tiles per chunk = 1 << chunk_log(bits).
-// (a bit-plane tile, flagged by kPlanesFlag in the unit's bitwidth byte, is gathered from up to four places and travels alone)
-constexpr uint32_t kPlanesFlag = 0x40;
-__device__ __forceinline__ uint32_t chunk_log(uint32_t bits) { return (bits == 16 || (bits & kPlanesFlag)) ? 0u : bits == 8 ? 1u : 2u; }
-// Chunk number inside a unit.  The producer walks the unit's groups in order and, at every group that starts a
-// chunk of a matrix, issues that chunk (matrix 0 first): chunk i of matrix 0 is preceded by its own earlier
-// chunks and by the chunks of matrix 1 that start before its first group, and the other way round.
-template <int NMAT>
-__device__ __forceinline__ uint32_t chunk_seq(uint32_t m, uint32_t i, uint32_t l0, uint32_t l1) {
-  if (NMAT == 1) return i;
-  if (m == 0) return i + (((i << l0) + (1u << l1) - 1u) >> l1);
-  return i + ((i << l1) >> l0) + 1u;
-}
-// Position of a chunk in the ring, advanced incrementally.
-struct Cursor {
-  uint32_t seq, s, par;
+// The slot ring.  Everything that travels through it is one "slot item" of at most kSlotBytes: a quantized
+// tile image (codes, scales, zero-points), or one K-half (64 columns, 16 KB) of a 16-bit tile -- the two halves
+// of a 16-bit tile are consecutive slot items.  Slot items are numbered in issue order; number `seq` sits in
+// slot seq % n_slots and uses phase seq / n_slots of that slot's barriers, so every role finds its own slot
+// items without replaying anybody else's.
+struct RingPos {
+  uint32_t s, par;                               // slot, parity of the full-barrier phase
 };
-__device__ __forceinline__ void cursor_to(Cursor& cu, uint32_t seq, uint32_t n_slots) {
-  cu.s += seq - cu.seq;
-  cu.seq = seq;
-  while (cu.s >= n_slots) {
-    cu.s -= n_slots;
-    cu.par ^= 1u;
+__device__ __forceinline__ RingPos ring_pos(uint32_t seq, uint32_t n_slots) {
+  const uint32_t q = seq / n_slots;
+  RingPos p;
+  p.s = seq - q * n_slots;
+  p.par = q & 1u;
+  return p;
+}
+__device__ __forceinline__ void ring_advance(RingPos& p, uint32_t step, uint32_t n_slots) {
+  p.s += step;
+  while (p.s >= n_slots) {
+    p.s -= n_slots;
+    p.par ^= 1u;
   }
+}
+__device__ __forceinline__ uint32_t slot_items(uint32_t bits) { return bits == 16 ? 2u : 1u; }
+// Bounded wait until the weight producer has armed slot item n.  A consumer looks at a slot item's full barrier
+// only after this, so it can never mistake an older phase of the slot's barrier for the item's.
+__device__ __forceinline__ bool wait_issued(uint32_t n, uint32_t polls, Ctrl* c, int32_t* status) {
+  if (c->issued[n & 1] > n) return true;
+  return flag_wait(smem_u32(const_cast<uint32_t*>(&c->issued[n & 1])), n, polls, c, status);
+}
+// Unit i of this CTA's work list (bounded wait until the weight producer has posted it); -1 = no more work,
+// -2 = the CTA is aborting.
+__device__ __forceinline__ int next_unit(uint32_t i, uint32_t polls, Ctrl* c, int32_t* status) {
+  if (c->sched_n > i) return c->sched_unit[i & 31];
+  if (flag_wait(smem_u32(const_cast<uint32_t*>(&c->sched_n)), i, polls, c, status)) return c->sched_unit[i & 31];
+  return -2;
+}
+// A unit of the list.  The gate/up list is written by the kernel directly ahead of this one in the stream, possibly
+// while this grid is already resident; no role reads it before producer 0 has waited for that kernel and posted the
+// unit, so an ordinary cached load sees final data -- what it must not be is a load through the non-coherent path,
+// which the compiler may choose for a `const __restrict__` pointer: hence the explicit cache operator.
+__device__ __forceinline__ Unit load_unit(const Unit* units, int u) {
+  const int4* p = reinterpret_cast<const int4*>(units + u);
+  const int4 a = __ldca(p), b = __ldca(p + 1);
+  Unit un;
+  un.seg = a.x;
+  un.row_tile = a.y;
+  un.tok0 = a.z;
+  un.ntok = a.w;
+  un.g0 = b.x;
+  un.g1 = b.y;
+  un.split = b.z;
+  un.pad_ = b.w;
+  return un;
+}
+// Bitwidth of a page-table row as the kernel's roles pass it around: the bitwidth, with kPlanesFlag for a block of
+// overlaid bit-planes (whose tiles are gathered from up to four places and decoded by their own routines).
+constexpr uint32_t kPlanesFlag = 0x40;
+template <bool PLANES>
+__device__ __forceinline__ uint32_t row_ubits(const DevRow& r) {
+  return r.bits | (PLANES && r.valid == 2 ? kPlanesFlag : 0u);
 }
 
 // Shared-memory matrix descriptor, K-major, no swizzle.  A core matrix is 8 rows x 16 bytes (8 fp16
@@ -321,143 +393,58 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t saddr, uint32_t lb
   return d;
 }
 
-struct KArgs {
-  const DevRow* rows;                            // page-table rows of the layer (final before the call's first kernel)
-  const Unit* units;
-  const int32_t* n_units_ptr;
-  int Rpad, nt_tile, n_bslots, n_slots;
-  __half* ht;
-  float* y;
-  int H;
-  size_t y_split_stride;
-  int32_t* work_counter;
-  int32_t* status;
-  uint32_t wait_polls;                           // limit of every wait, in polls of kSuspendHintNs
-  uint32_t hook;                                 // test hook: bit 0 = the token-tile producer stops before its second tile
+// Source of the next item of one matrix of a unit (weight producer).
+struct MatSrc {
+  uint32_t bits, tb;                              // bitwidth; bytes of a tile image (of a TOP tile for a bit-plane block)
+  uint32_t q;                                     // bitwidth a bit-plane block is read at, 0 = an ordinary page
+  const char* src;
+  const char* b1;                                 // bit-plane blocks: the BIT1 and BIT0 buffers
+  const char* b0;
 };
 
-// ---- dequantizers: the tiles of one unit that belong to one group -------------------------------------------
-// Tile j of the unit sits in chunk j >> L of its matrix; a warp looks at a chunk's barrier once, decodes its
-// tiles of the chunk and makes one arrival on the slot per tile.
-template <int BITS, int NMAT, bool PLANES>
-__device__ __forceinline__ bool dq_unit(Ctrl* c, const KArgs& ka, char* wring, uint32_t m, uint32_t j0, uint32_t stride,
-                                        uint32_t ng, uint32_t seq_unit, uint32_t l0, uint32_t l1, Cursor& cu,
-                                        uint32_t& uses, int r, int lane, uint32_t lane_addr, uint32_t af_s, uint32_t ae_s) {
-  constexpr uint32_t L = PLANES ? 0u : BITS == 8 ? 1u : 2u;
-  constexpr uint32_t TB = BITS * 2048 + 512;
-  constexpr uint32_t META = PLANES ? (uint32_t)kPlaneSlotLut : BITS * 2048u;   // scales, then zero-points, of the tile's rows
-  const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
-  uint32_t cur = 0xffffffffu;
-  const char* chunk = nullptr;
-  uint32_t slot_empty_s = 0;
-#pragma unroll 1
-  for (uint32_t j = j0; j < ng; j += stride) {
-    const uint32_t ci = j >> L;
-    if (ci != cur) {
-      cur = ci;
-      const uint32_t seq = seq_unit + chunk_seq<NMAT>(m, ci, l0, l1);
-      cursor_to(cu, seq, (uint32_t)ka.n_slots);
-      // a chunk's barrier is looked at only once the producer is known to have armed it: the phase parity
-      // cannot tell an old phase of the slot from the chunk's own
-      if (!wait_flag(&c->issued, seq, ka.wait_polls, c, ka.status)) return false;
-      if (!wait_bar(full_s + 8 * cu.s, cu.par, ka.wait_polls, c, ka.status)) return false;
-      chunk = wring + cu.s * kSlotBytes;
-      slot_empty_s = empty_s + 8 * cu.s;
-    }
-    const char* tile = chunk + (j & ((1u << L) - 1u)) * TB;
-    const uint4* row_units = reinterpret_cast<const uint4*>(tile) + r;
-    const __half2 s2 = __half2half2(*reinterpret_cast<const __half*>(tile + META + 2 * r));
-    const __half2 z2 = __half2half2(*reinterpret_cast<const __half*>(tile + META + 256 + 2 * r));
-    __half2 w[32];
-    if constexpr (PLANES) decode_half_planes<BITS>(tile, r, 0, s2, z2, w);
-    else decode_half<BITS>(row_units, 0, s2, z2, w);
-    // The operand slot is free once the MMAs of the group's previous tile have read it; they ran while the
-    // half above was being decoded.
-    if (!wait_bar(ae_s, (uses & 1u) ^ 1u, ka.wait_polls, c, ka.status)) return false;
-    ++uses;
-    tc_fence_after();
-    tmem_st32(lane_addr, w);
-    if constexpr (PLANES) decode_half_planes<BITS>(tile, r, 1, s2, z2, w);
-    else decode_half<BITS>(row_units, 1, s2, z2, w);
-    __syncwarp();
-    mbar_arrive_if_s(slot_empty_s, lane == 0);     // this warp has read its rows of the tile
-    tmem_st32(lane_addr + 32, w);
-    // hand the tile over: both stores have landed, then one arrival per warp
-    tmem_wait_st();
-    tc_fence_before();
-    __syncwarp();
-    mbar_arrive_if_s(af_s, lane == 0);
-  }
-  return true;
-}
-
-// ---- epilogue of token columns [c_begin, c_end) of one unit, one accumulator row per thread ------------------
-template <int PHASE>
-__device__ __forceinline__ void epilogue_cols(const KArgs& ka, const UDesc& d, uint32_t dbase, int npart, uint32_t written,
-                                              int nb_rows, int row, int c_begin, int c_end) {
-  for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-    float a[16], b[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
-    for (int p = 0; p < npart; ++p) {              // add the issuers' partial sums, in order
-      if (!((written >> p) & 1u)) continue;
-      float t[16];
-      tmem_ld16(dbase + p * nb_rows + c0, t);
-      tmem_wait_ld();
-#pragma unroll
-      for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
-      if (PHASE == 0) {
-        tmem_ld16(dbase + (npart + p) * nb_rows + c0, t);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const int nn = c0 + j;
-      if (nn < d.ntok) {
-        if (PHASE == 0) {
-          // SwiGLU: silu(gate) * up; the result is rounded to fp16, so the fast exponential and
-          // division (relative error ~1e-6) change nothing that survives the rounding
-          const float hval = __fmul_rn(__fdividef(a[j], __fadd_rn(1.0f, __expf(-a[j]))), b[j]);
-          ka.ht[((size_t)(row >> 3) * ka.Rpad + d.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
-        } else {
-          ka.y[(size_t)d.split * ka.y_split_stride + (size_t)(d.tok0 + nn) * ka.H + row] = a[j];
-        }
-      }
-    }
-  }
+// K-half `h` of one row of an item: shared memory -> 32 registers (half2 pairs in K order).
+template <int BITS>
+__device__ __forceinline__ void decode_item_half(const char* item, int r, int h, __half2* w) {
+  const uint4* row_units = reinterpret_cast<const uint4*>(item) + r;
+  const __half2 s2 = __half2half2(reinterpret_cast<const __half*>(item + BITS * 2048)[r]);
+  const __half2 z2 = __half2half2(reinterpret_cast<const __half*>(item + BITS * 2048 + 256)[r]);
+  decode_half<BITS>(row_units, h, s2, z2, w);
 }
 
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
-// PLANES: the instantiation that also reads overlaid bit-plane blocks; launched only for a layer that has one (the
-// extra code paths cost the ordinary ones instruction-cache room).
+// PLANES: the instantiation that also reads blocks of overlaid bit-planes; launched only for a layer that holds one
+// (the extra code paths cost the ordinary ones instruction-cache room).
+// wait_polls: limit of every wait, in polls of kSuspendHintNs.  hook: test hook, bit 0 = the token-tile producer
+// stops before its second tile (so that the waits on it run out).
 template <int PHASE, bool HELP, bool PLANES>
-__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ KArgs ka, const __grid_constant__ TmapSet tmaps) {
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t* __restrict__ n_units_ptr,
+              const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
+              __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
+              int32_t* __restrict__ work_counter, int32_t* __restrict__ status, uint32_t wait_polls, uint32_t hook) {
+  const uint32_t polls = wait_polls;
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   char* wring = smem + kCtrlBytes;
-  const int n_slots = ka.n_slots, n_bslots = ka.n_bslots, nt_tile = ka.nt_tile;
   char* bslots = wring + n_slots * kSlotBytes;
   const int bslot_bytes = nt_tile * 256;
   constexpr int NMAT = PHASE == 0 ? 2 : 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int32_t* status = ka.status;
-  const uint32_t polls = ka.wait_polls;
+  const int n_units = n_units_ptr[PHASE];
   // tensor-memory columns: partial accumulators first ([matrix][partial][nt_tile]), dequantized-operand
-  // slots after them.  Partials per matrix: as many as issuers per matrix, while the operand slots still fit.
+  // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
   constexpr int IPM = kIssuers / NMAT;           // issuers per matrix = dequantizer groups per matrix
   int npart = IPM;
   while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 64 > kTmemCols) npart >>= 1;
   const int n_issuers = NMAT * npart;            // active issuers
   const int acol = NMAT * npart * nt_tile;       // the operand slot of group g sits at acol + 64 * g
+  const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(&c->full[i], 1);
-      mbar_init(&c->empty[i], kChunkArrivals);
+      mbar_init(&c->empty[i], 4);                 // four dequantizer warps, or an issuer's commit + 3 arrivals
     }
     for (int i = 0; i < kMaxBSlots; ++i) {
       mbar_init(&c->b_full[i], 1);
@@ -472,7 +459,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       mbar_init(&c->d_empty[i], HELP ? 8 : 4);    // epilogue warps (+ the issuer warps when they share the epilogue)
     }
     c->abort_flag = 0;
-    c->issued = 0;
+    c->issued[0] = c->issued[1] = 0;
     c->b_issued = 0;
     c->sched_n = 0;
     c->dep_ready = 0;
@@ -492,156 +479,158 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   // This CTA may have been placed while the kernel before this one is still finishing on other SMs.  Work
   // counters, page-table rows and the unit counts were written two or more kernels back and are final (see
   // grid_dep_sync).  What the kernel directly ahead writes is not: the token rows (both kernels; the
-  // token-tile producer waits for them) and the gate/up unit list (PHASE 0; the weight producer waits).
-  // Nothing else reads global memory that a kernel of this call writes: the other roles learn of their units
-  // from the weight producer, through shared memory.
+  // token-tile producer waits for them) and the gate/up unit list (PHASE 0; the weight producers wait).
 
-  if (warp == kWarpW) {
-    // ---------------- weight producer ----------------
+  // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
+  // (the weight producer claims, the other roles follow its list).
+
+  if (warp == kWarpCodes || warp == kWarpCodes2) {
+    // ---------------- weight producers ----------------
+    // Two single-thread producers share the stream: producer P arms the slot items with number = P mod 2,
+    // which (even slot count) always land in the slots = P mod 2, so each keeps the state of its own slots.
+    // Producer 0 also claims the units.
     if (lane == 0) {
+      const uint32_t P = warp == kWarpCodes ? 0u : 1u;
+      uint32_t seq = 0, s = 0;                     // number and slot of the next slot item of the stream
+      // A slot is free for slot item seq once the phase seq / n_slots - 1 of its empty barrier has completed
+      // (nothing to wait for during the first pass over the ring).
+      uint32_t pass = 0;                           // seq / n_slots
+      const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]);
+      bool ok = true;
+      // The gate/up kernel's unit list is written by the kernel directly ahead of it (the one that gathers
+      // the token rows), which may still be running: the producers wait for it before they read a unit, and
+      // every other role learns of its first unit from producer 0 only after that.  The down kernel's list is
+      // two kernels back and final (see grid_dep_sync), so its producers stream at once.
       if (PHASE == 0) {
         grid_dep_sync();
         c->dep_ready = 1;
       }
-      const int n_units = ka.n_units_ptr[PHASE];
-      const int G = gridDim.x;
-      const uint32_t wring_s = smem_u32(wring), full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
-      uint32_t seq = 0, s = 0, pass = 0;           // number and slot of the next chunk, laps around the ring
-      int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;   // unit blockIdx.x first, then whatever the counter hands out
-      bool ok = true;
-      for (uint32_t i = 0; ok; ++i) {
-        UDesc d;
-        d.unit = u;
-        d.row_tile = d.tok0 = d.ntok = d.g0 = d.ng = d.split = 0;
-        d.bits = 0;
-        const char* src[NMAT];
-        const char* pb1[NMAT];                      // bit-plane blocks: the BIT1 and BIT0 buffers
-        const char* pb0[NMAT];
-        uint32_t tb[NMAT], lg[NMAT], pq[NMAT];      // pq: bitwidth a bit-plane block is read at, 0 = an ordinary page
-        if (u >= 0) {
-          // (the unit list may have been written by the kernel directly ahead: read around the non-coherent path)
-          const int4* up = reinterpret_cast<const int4*>(ka.units + u);
-          const int4 u0 = __ldcg(up), u1 = __ldcg(up + 1);
-          d.row_tile = u0.y;
-          d.tok0 = u0.z;
-          d.ntok = u0.w;
-          d.g0 = u1.x;
-          d.ng = u1.y - u1.x;
-          d.split = u1.z;
-#pragma unroll
-          for (int m = 0; m < NMAT; ++m) {
-            const DevRow row = ka.rows[u0.x * 3 + (PHASE == 0 ? m : 2)];
-            const bool planes = PLANES && row.valid == 2;
-            const uint32_t ubits = row.bits | (planes ? kPlanesFlag : 0u);
-            d.bits |= ubits << (8 * m);
-            pq[m] = planes ? row.bits : 0u;
-            tb[m] = planes ? (uint32_t)kPlaneTopTile : (uint32_t)tile_bytes((int)row.bits);
-            lg[m] = chunk_log(ubits);
-            // consecutive groups of a row tile are consecutive tiles of the page
-            const size_t tile = (size_t)d.row_tile * (row.cols / kGroup) + d.g0;
-            src[m] = reinterpret_cast<const char*>(row.codes) + tile * tb[m];
-            pb1[m] = reinterpret_cast<const char*>(row.bit1) + tile * kPlaneBitTile;
-            pb0[m] = reinterpret_cast<const char*>(row.bit0) + tile * kPlaneBitTile;
-          }
-        }
-        UDesc* slot = &c->sched[i & (kSched - 1)];
-        *slot = d;
+      // the work list: unit blockIdx.x first, then whatever the global counter hands out
+      int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
+      if (P == 0) {
+        c->sched_unit[0] = u;
         __threadfence_block();
-        c->sched_n = i + 1;
-        if (u < 0) break;
-        const uint32_t ng = (uint32_t)d.ng;
-        const uint32_t claim_at = ng >> 1;
+        c->sched_n = 1;
+      }
+      for (int i = 0; ok && u >= 0; ++i) {
+        const Unit un = load_unit(units, u);
         int claimed = 0;
+        // per matrix of the unit: bitwidth, bytes of a tile image, address of the unit's first tile;
+        // consecutive groups of a row tile are consecutive tiles of the page
+        MatSrc ms[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) {
+          const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+          const bool planes = PLANES && row.valid == 2;
+          ms[m].bits = row.bits;
+          ms[m].q = planes ? row.bits : 0u;
+          ms[m].tb = planes ? (uint32_t)kPlaneTopTile : (uint32_t)tile_bytes((int)row.bits);
+          const size_t tile = (size_t)un.row_tile * (row.cols / kGroup) + un.g0;
+          ms[m].src = reinterpret_cast<const char*>(row.codes) + tile * ms[m].tb;
+          ms[m].b1 = reinterpret_cast<const char*>(row.bit1) + tile * kPlaneBitTile;
+          ms[m].b0 = reinterpret_cast<const char*>(row.bit0) + tile * kPlaneBitTile;
+        }
+        const int ng = un.g1 - un.g0;
+        const int claim_at = ng >> 1;
 #pragma unroll 1
-        for (uint32_t g = 0; ok && g < ng; ++g) {
+        for (int g = 0; ok && g < ng; ++g) {
           // claim the next unit half-way through this one: the answer is back long before it is needed
-          if (g == claim_at) claimed = atomicAdd(ka.work_counter, 1) + G;
+          if (P == 0 && g == claim_at) claimed = atomicAdd(work_counter, 1) + G;
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
-            if (g & ((1u << lg[m]) - 1u)) continue;
-            const uint32_t left = ng - g, full_n = 1u << lg[m];
-            const uint32_t nt = left < full_n ? left : full_n;
-            const uint32_t q = PLANES ? pq[m] : 0u;
-            const uint32_t bytes = q ? (uint32_t)kPlaneTopCodes + 512u + (q - 2u) * (uint32_t)kPlaneBitTile : nt * tb[m];
-            const uint32_t es = empty_s + 8 * s, fs = full_s + 8 * s;
-            if (pass) ok = wait_bar(es, (pass - 1) & 1, polls, c, status);
+            const bool f16 = ms[m].bits == 16;
+            const uint32_t q = PLANES ? ms[m].q : 0u;
+            // a 16-bit tile goes as two K-halves; of a bit-plane tile read at q bits only the first q bits of every
+            // weight leave HBM: the top codes, the planes below them that q needs, the lookup-table state of q
+            const uint32_t bytes = f16 ? 16384u : q ? (uint32_t)kPlaneTopCodes + 512u + (q - 2u) * (uint32_t)kPlaneBitTile : ms[m].tb;
+            const int nsub = f16 ? 2 : 1;
+            const char* src = ms[m].src;
+            const char* b1 = ms[m].b1;
+            const char* b0 = ms[m].b0;
+            ms[m].src += ms[m].tb;
+            ms[m].b1 += kPlaneBitTile;
+            ms[m].b0 += kPlaneBitTile;
+            for (int sub = 0; sub < nsub; ++sub, src += 16384) {
+              if ((seq & 1u) == P) {
+                if (pass) ok = mbar_wait_s(smem_u32(&c->empty[s]), (pass - 1) & 1, polls, c, status);
+                if (!ok) break;
+                const uint32_t bar_s = full_s + 8 * s;
+                mbar_expect_tx_s(bar_s, bytes);
+                const uint32_t slot_s = wring_s + s * kSlotBytes;
+                if (q) {
+                  bulk_g2s_s(slot_s, src, kPlaneTopCodes, bar_s);
+                  bulk_g2s_s(slot_s + kPlaneSlotLut, src + plane_lut_offset((int)q), 512, bar_s);
+                  if (q >= 3) bulk_g2s_s(slot_s + kPlaneSlotBit1, b1, kPlaneBitTile, bar_s);
+                  if (q == 4) bulk_g2s_s(slot_s + kPlaneSlotBit0, b0, kPlaneBitTile, bar_s);
+                } else {
+                  bulk_g2s_s(slot_s, src, bytes, bar_s);
+                }
+                c->issued[P] = seq + 2;                // my next slot item is seq + 2
+              }
+              ++seq;
+              if (++s == (uint32_t)n_slots) {
+                s = 0;
+                ++pass;
+              }
+            }
             if (!ok) break;
-            if (nt < 4) mbar_arrive_n_s(es, (4 - nt) * 4);   // a short chunk: the arrivals its missing tiles would make
-            mbar_expect_tx_s(fs, bytes);
-            const uint32_t slot_s = wring_s + s * kSlotBytes;
-            if (q) {
-              // a bit-plane tile read at q bits: the top codes, the planes below them that q needs, and the
-              // lookup-table state of q -- only the first q bits of every weight leave HBM
-              bulk_g2s_s(slot_s, src[m], kPlaneTopCodes, fs);
-              bulk_g2s_s(slot_s + kPlaneSlotLut, src[m] + plane_lut_offset((int)q), 512, fs);
-              if (q >= 3) bulk_g2s_s(slot_s + kPlaneSlotBit1, pb1[m], kPlaneBitTile, fs);
-              if (q == 4) bulk_g2s_s(slot_s + kPlaneSlotBit0, pb0[m], kPlaneBitTile, fs);
-              src[m] += kPlaneTopTile;
-              pb1[m] += kPlaneBitTile;
-              pb0[m] += kPlaneBitTile;
-            } else {
-              bulk_g2s_s(slot_s, src[m], bytes, fs);
-              src[m] += bytes;
-            }
-            c->issued = ++seq;
-            if (++s == (uint32_t)n_slots) {
-              s = 0;
-              ++pass;
-            }
           }
         }
-        u = claimed < n_units ? claimed : -1;
+        if (P == 0) {
+          u = claimed < n_units ? claimed : -1;
+          c->sched_unit[(i + 1) & 31] = u;
+          __threadfence_block();
+          c->sched_n = (uint32_t)i + 2;
+        } else {
+          u = next_unit((uint32_t)i + 1, polls, c, status);
+        }
       }
     }
-  } else if (warp == kWarpB) {
+  } else if (warp == kWarpTokens) {
     // ---------------- token-tile producer ----------------
     if (lane == 0) {
       grid_dep_sync();
       grid_dep_trigger();
       if (PHASE == 1) c->dep_ready = 1;
-      const uint32_t bslots_s = smem_u32(bslots), bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
-      uint32_t bcount = 0, bs = 0, bpass = 0;
+      uint32_t bcount = 0;
       bool ok = true;
-      for (uint32_t i = 0; ok; ++i) {
-        UDesc d;
-        if (!get_desc(i, polls, c, status, d) || d.unit < 0) break;
-        const int nb_rows = (d.ntok + 15) & ~15;
+      for (int i = 0; ok; ++i) {
+        const int u = next_unit((uint32_t)i, polls, c, status);
+        if (u < 0) break;
+        const Unit un = load_unit(units, u);
+        const int nb_rows = (un.ntok + 15) & ~15;
         const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
-#pragma unroll 1
-        for (int g = d.g0; ok && g < d.g0 + d.ng; ++g) {
-          if ((ka.hook & 1u) && bcount == 1) {     // test hook: leave the tile unarmed, so that the waits on it run out
+        for (int g = un.g0; ok && g < un.g1; ++g) {
+          if ((hook & 1u) && bcount == 1) {        // test hook: leave the tile unarmed, so that the waits on it run out
             ok = false;
             break;
           }
           // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
-          if (bpass) ok = wait_bar(be_s + 8 * bs, (bpass - 1) & 1, polls, c, status);
+          const int bs = bcount % n_bslots;
+          ok = mbar_wait_s(smem_u32(&c->b_empty[bs]), ((bcount / n_bslots) & 1) ^ 1, polls, c, status);
           if (!ok) break;
-          mbar_expect_tx_s(bf_s + 8 * bs, nb_rows * 256);
-          tma_2d_g2s_s(bslots_s + bs * (uint32_t)bslot_bytes, map, d.tok0 * 2, g * 16, bf_s + 8 * bs);
-          c->b_issued = ++bcount;
-          if (++bs == (uint32_t)n_bslots) {
-            bs = 0;
-            ++bpass;
-          }
+          mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
+          tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
+          ++bcount;
+          c->b_issued = bcount;
         }
       }
     }
-  } else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
+  }
+  else if (warp >= kWarpMma && warp < kWarpMma + kIssuers) {
     // ---------------- MMA issuers ----------------
     // Tile k of a matrix (counted over all units) belongs to issuer k mod npart of that matrix, which issues
     // all eight k-steps of it into its own partial accumulator; a quantized tile k is dequantized by the
     // matrix's group k mod IPM, so with npart == IPM every dequantizer group has an issuer of its own.
-    // The epilogue adds the partials.  With HELP every lane follows the units (the warp shares the epilogue of
-    // wide units, taking the upper half of the token columns of its lane quarter); lane 0 issues.
+    // The epilogue adds the partials.
+    if constexpr (!HELP) {
     const int iss = warp - kWarpMma;
     const int my_m = iss / IPM, my_j = iss % IPM;
-    const bool issuing = my_j < npart;
-    if ((HELP || (lane == 0 && issuing))) {
-      const int hq = warp & 3;
-      const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
-      uint32_t seq_unit = 0;                        // chunks before the current unit
+    if (lane == 0 && my_j < npart) {
+      uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
       uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
+      uint32_t ucount = 0;
       // Accumulators: partial (m, j) of a unit sits at buffer base + (m * npart + j) * nb_rows.  A unit whose
       // accumulators fit half of the accumulator columns takes one of two buffers in turn, so that its MMAs
       // overlap the epilogue of the unit before it; a wider unit takes both.
@@ -651,194 +640,434 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const uint32_t w_lo_base = smem_u32(wring) >> 4;
       const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
       const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
-      const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
-      const uint32_t df_s = smem_u32(&c->d_full[0]), de_s = smem_u32(&c->d_empty[0]);
       const uint32_t a_base = tmem + acol;
-      Cursor cu = {0, 0, 0};
-      Cursor bp = {0, 0, 0};
       bool ok = true;
-      for (uint32_t i = 0; ok; ++i) {
-        UDesc d;
-        if (!get_desc(i, polls, c, status, d) || d.unit < 0) break;
-        const uint32_t bits0 = d.bits & 0xffu, bits1 = NMAT == 2 ? (d.bits >> 8) & 0xffu : bits0;
-        const uint32_t my_bits = my_m ? bits1 : bits0;
-        const uint32_t l0 = chunk_log(bits0), l1 = chunk_log(bits1);
-        const uint32_t ng = (uint32_t)d.ng;
-        const uint32_t nch = ((ng + (1u << l0) - 1u) >> l0) + (NMAT == 2 ? ((ng + (1u << l1) - 1u) >> l1) : 0u);
-        const int nb_rows = (d.ntok + 15) & ~15;
+      for (int i = 0; ok; ++i, ++ucount) {
+        const int u = next_unit((uint32_t)i, polls, c, status);
+        if (u < 0) break;
+        const Unit un = load_unit(units, u);
+        uint32_t ubits[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
+        // slot items per group of the unit (W) and the offset of my matrix's inside a group
+        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
+        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+        const int nb_rows = (un.ntok + 15) & ~15;
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
+        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
+        const uint32_t b_step = (uint32_t)(2 * nb_rows);
+        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        uint32_t bt = base + j0;                     // token-tile number
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
         const bool wide = NMAT * npart * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
-        if (lane == 0 && issuing) {
-          const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-          // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
-          const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
-          const uint32_t b_step = (uint32_t)(2 * nb_rows);
-          const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
-          const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
-          // the epilogue has drained the buffer(s) this unit accumulates into
-          if (wide || dbuf == 0) ok = wait_bar(de_s, (duse0 & 1) ^ 1, polls, c, status);
-          if (ok && (wide || dbuf == 1)) ok = wait_bar(de_s + 8, (duse1 & 1) ^ 1, polls, c, status);
-          if (ok) {
-            tc_fence_after();
-            uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
-            // my first tile of the unit, then every npart-th
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        // the epilogue has drained the buffer(s) this unit accumulates into
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, polls, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, polls, c, status);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
 #pragma unroll 1
-            for (uint32_t j = ((uint32_t)my_j - base) & (uint32_t)(npart - 1); j < ng; j += (uint32_t)npart) {
-              // the token tile of this group (a tile is looked at only once it is known to have been armed)
-              const uint32_t bt = base + j;
-              cursor_to(bp, bt, (uint32_t)n_bslots);
-              ok = wait_flag(&c->b_issued, bt, polls, c, status) && wait_bar(bf_s + 8 * bp.s, bp.par, polls, c, status);
+        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
+          // the token tile of this group (a tile is looked at only once it is known to have been armed)
+          if (c->b_issued <= bt) {
+            ok = flag_wait(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, polls, c, status);
+            if (!ok) break;
+          }
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, polls, c, status);
+          if (!ok) break;
+          const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
+          if (my_bits == 16) {
+            // each K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3, 4 KB apart)
+            RingPos hp = rp;
+#pragma unroll 1
+            for (uint32_t hh = 0; hh < 2; ++hh) {
+              ok = wait_issued(sq + hh, polls, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, polls, c, status);
               if (!ok) break;
-              const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
-              if (my_bits == 16) {
-                // the whole tile lies in one slot as a K-major core-matrix image (k-steps 4 KB apart)
-                const uint32_t seq = seq_unit + chunk_seq<NMAT>((uint32_t)my_m, j, l0, l1);
-                cursor_to(cu, seq, (uint32_t)n_slots);
-                ok = wait_flag(&c->issued, seq, polls, c, status) && wait_bar(full_s + 8 * cu.s, cu.par, polls, c, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_lo = (w_lo_base + cu.s * (kSlotBytes >> 4)) | a_lo_lbo;
-                tc_mma_ss_burst4(d_t, a_lo, desc_hi, 256, b_lo, desc_hi, b_step, idesc, later);
-                tc_mma_ss_burst4(d_t, a_lo + 4 * 256, desc_hi, 256, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
-                mbar_arrive_n_s(empty_s + 8 * cu.s, 3);  // with the commit: the four arrivals of the tile
-                tc_commit_s(empty_s + 8 * cu.s);
-              } else {
-                // the group that dequantizes this tile, and the parity of this use of its operand slot
-                const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (bt & 1u) : (bt & 3u);
-                const uint32_t use_par = (upar >> grp) & 1u;
-                upar ^= 1u << grp;
-                const uint32_t a_t = a_base + grp * 64;
-                ok = wait_bar(af_s + 8 * grp, use_par, polls, c, status);
-                if (!ok) break;
-                tc_fence_after();
-                // all eight k-steps of the tile, then one commit hands the group's operand slot back
-                tc_mma_ts_burst4(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
-                tc_mma_ts_burst4(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
-                tc_commit_s(ae_s + 8 * grp);
-              }
-              tc_commit_s(be_s + 8 * bp.s);
-              later = 1;
+              tc_fence_after();
+              const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
+              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
+              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
+              tc_commit(&c->empty[hp.s]);
+              ring_advance(hp, 1, (uint32_t)n_slots);
             }
-          }
-          if (ok) {
-            if (wide || dbuf == 0) tc_commit_s(df_s);
-            if (wide || dbuf == 1) tc_commit_s(df_s + 8);
-          }
-        }
-        const uint32_t par0 = duse0 & 1u, par1 = duse1 & 1u;     // phases of d_full this unit completes
-        if (wide || dbuf == 0) ++duse0;
-        if (wide || dbuf == 1) ++duse1;
-        if (HELP) {
-          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-          if (!ok) break;
-          // every issuer warp sees every phase of the accumulator barriers, also of the narrow units it has no
-          // part in: it must not run ahead of the epilogue by more than the phase parity can tell apart
-          if (wide || dbuf == 0) ok = wait_bar(df_s, par0, polls, c, status);
-          if (ok && (wide || dbuf == 1)) ok = wait_bar(df_s + 8, par1, polls, c, status);
-          if (!ok) break;
-          if (wide) {
+            if (!ok) break;
+            sq += (uint32_t)npart * W;
+            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
+          } else {
+            // the group that dequantizes this tile, and the parity of this use of its operand slot
+            const uint32_t k = base + j;
+            const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
+            const uint32_t use_par = (upar >> grp) & 1u;
+            upar ^= 1u << grp;
+            const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
+            const uint32_t a_t = a_base + grp * 64;
+            ok = mbar_wait_s(f0, use_par, polls, c, status);
+            if (!ok) break;
             tc_fence_after();
-            uint32_t written = 0;
-            for (int p = 0; p < npart; ++p)
-              if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
-            const int half = ((nb_rows / 16 + 1) / 2) * 16;         // the epilogue warps take [0, half)
-            epilogue_cols<PHASE>(ka, d, hlane_addr, npart, written, nb_rows, d.row_tile * kTileRows + hq * 32 + lane, half,
-                                 nb_rows);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-              mbar_arrive_s(de_s);
-              mbar_arrive_s(de_s + 8);
-            }
+            // all eight k-steps of the tile, then one commit hands the group's operand slot back
+            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            tc_commit_s(e0);
+          }
+          tc_commit_s(be_s + 8 * bp.s);
+          later = 1;
+          bt += (uint32_t)npart;
+          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
+        }
+        if (ok) {
+          if (wide || dbuf == 0) {
+            tc_commit(&c->d_full[0]);
+            ++duse0;
+          }
+          if (wide || dbuf == 1) {
+            tc_commit(&c->d_full[1]);
+            ++duse1;
           }
         }
         base += ng;
-        seq_unit += nch;
+        seq_unit += ng * W;
       }
     }
-  } else if (warp < kDqWarps) {
-    // ---------------- dequantize ----------------
-    // Four groups of four warps, each taking every other quantized tile of one matrix (every fourth when
-    // the unit has a single matrix).  Warp q of a group owns rows (= TMEM lanes) 32q .. 32q+31 of the tile,
-    // one row per thread.  Each group has one operand slot (64 columns: both K-halves of a tile): it stores the
-    // two halves as it decodes them and hands the slot over once per tile; while the issuer's eight MMAs read
-    // it, the group decodes the first half of its next tile in registers.
+    } else {
+    const int iss = warp - kWarpMma;
+    const int my_m = iss / IPM, my_j = iss % IPM;
+    // Wide token tiles leave no room for a second accumulator buffer, so the epilogue of a unit is not
+    // overlapped: here the four issuer warps share it with the four epilogue warps (they take the upper
+    // half of the token columns of their lane quarter), lane 0 of the warps with an accumulator of their own
+    // issuing the unit's MMAs first.  Every lane tracks the per-unit state; only lane 0 uses the issuing part.
+    const bool issuing = my_j < npart;
+    const int hq = warp & 3;
+    const int hr = hq * 32 + lane;
+    const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
+    {
+      uint32_t seq_unit = 0;                        // slot items before the current unit
+      uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
+      uint32_t ucount = 0;
+      uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
+      const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
+      const uint32_t b_lo_base = smem_u32(bslots) >> 4;
+      const uint32_t w_lo_base = smem_u32(wring) >> 4;
+      const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
+      const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
+      const uint32_t a_base = tmem + acol;
+      bool ok = true;
+      for (int i = 0; ok; ++i, ++ucount) {
+        const int u = next_unit((uint32_t)i, polls, c, status);
+        if (u < 0) break;
+        const Unit un = load_unit(units, u);
+        uint32_t ubits[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
+        // slot items per group of the unit (W) and the offset of my matrix's inside a group
+        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
+        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+        const int nb_rows = (un.ntok + 15) & ~15;
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
+        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
+        const uint32_t b_step = (uint32_t)(2 * nb_rows);
+        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        uint32_t bt = base + j0;                     // token-tile number
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const uint32_t dbuf = wide ? 0u : dtoggle;
+        if (!wide) dtoggle ^= 1u;
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        if (lane == 0 && issuing) {
+          do {
+        // the epilogue has drained the buffer(s) this unit accumulates into
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, polls, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, polls, c, status);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
+#pragma unroll 1
+        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
+          // the token tile of this group (a tile is looked at only once it is known to have been armed)
+          if (c->b_issued <= bt) {
+            ok = flag_wait(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, polls, c, status);
+            if (!ok) break;
+          }
+          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, polls, c, status);
+          if (!ok) break;
+          const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
+          if (my_bits == 16) {
+            // each K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3, 4 KB apart)
+            RingPos hp = rp;
+#pragma unroll 1
+            for (uint32_t hh = 0; hh < 2; ++hh) {
+              ok = wait_issued(sq + hh, polls, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, polls, c, status);
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
+              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
+              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
+              tc_commit(&c->empty[hp.s]);
+              ring_advance(hp, 1, (uint32_t)n_slots);
+            }
+            if (!ok) break;
+            sq += (uint32_t)npart * W;
+            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
+          } else {
+            // the group that dequantizes this tile, and the parity of this use of its operand slot
+            const uint32_t k = base + j;
+            const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
+            const uint32_t use_par = (upar >> grp) & 1u;
+            upar ^= 1u << grp;
+            const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
+            const uint32_t a_t = a_base + grp * 64;
+            ok = mbar_wait_s(f0, use_par, polls, c, status);
+            if (!ok) break;
+            tc_fence_after();
+            // all eight k-steps of the tile, then one commit hands the group's operand slot back
+            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            tc_commit_s(e0);
+          }
+          tc_commit_s(be_s + 8 * bp.s);
+          later = 1;
+          bt += (uint32_t)npart;
+          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
+        }
+            if (ok) {
+              if (wide || dbuf == 0) tc_commit(&c->d_full[0]);
+              if (wide || dbuf == 1) tc_commit(&c->d_full[1]);
+            }
+          } while (false);
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        const uint32_t par0 = duse0 & 1u, par1 = duse1 & 1u;     // phases of d_full this unit completes
+        if (wide || dbuf == 0) ++duse0;
+        if (wide || dbuf == 1) ++duse1;
+        // every issuer warp sees every phase of the accumulator barriers, also of the narrow units it has no
+        // part in: it must not run ahead of the epilogue by more than the phase parity can tell apart
+        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), par0, polls, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), par1, polls, c, status);
+        if (!ok) break;
+        if (wide) {
+          tc_fence_after();
+          uint32_t written = 0;
+          for (int p = 0; p < npart; ++p)
+            if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
+          const int row = un.row_tile * kTileRows + hr;
+          const int half = ((nb_rows / 16 + 1) / 2) * 16;         // the epilogue warps take [0, half)
+          for (int c0 = half; c0 < nb_rows; c0 += 16) {
+            float a[16], b[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
+            for (int p = 0; p < npart; ++p) {
+              if (!((written >> p) & 1u)) continue;
+              float t[16];
+              tmem_ld16(hlane_addr + p * nb_rows + c0, t);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
+              if (PHASE == 0) {
+                tmem_ld16(hlane_addr + (npart + p) * nb_rows + c0, t);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int nn = c0 + j;
+              if (nn < un.ntok) {
+                if (PHASE == 0) {
+                  const float hval = __fmul_rn(__fdividef(a[j], __fadd_rn(1.0f, __expf(-a[j]))), b[j]);
+                  ht[((size_t)(row >> 3) * Rpad + un.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
+                } else {
+                  y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + nn) * H + row] = a[j];
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&c->d_empty[0]);
+            mbar_arrive(&c->d_empty[1]);
+          }
+        }
+        base += ng;
+        seq_unit += ng * W;
+      }
+    }
+    }
+  } else if (warp < kDqWarps) {    // ---------------- dequantize ----------------
+    // Four groups of four warps, each taking every other quantized item of one matrix (every fourth when
+    // the unit has a single matrix; an item = one group of one matrix).  Warp q of a group owns rows (= TMEM lanes) 32q .. 32q+31 of the item, one row per
+    // thread.  Each group has one operand slot (64 columns: both K-halves of an item): it stores the two halves
+    // as it decodes them and hands the slot over once per item; while the issuer's eight MMAs read it, the group
+    // decodes the first half of its next item in registers.
     const int grp = warp >> 2, q = warp & 3;
     const int r = q * 32 + lane;                     // weight row inside the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + acol + grp * 64;
-    const uint32_t qm = NMAT == 2 ? (uint32_t)(grp >> 1) : 0u;         // the matrix this group serves
+    const int qm = NMAT == 2 ? grp >> 1 : 0;         // the matrix this group serves
     const uint32_t gsub = NMAT == 2 ? (uint32_t)(grp & 1) : (uint32_t)grp;   // which of that matrix's groups
     constexpr uint32_t kStride = NMAT == 2 ? 2 : 4;  // groups per matrix = distance between my tiles
-    const uint32_t af_s = smem_u32(&c->a_full[grp]), ae_s = smem_u32(&c->a_empty[grp]);
-    uint32_t seq_unit = 0;                           // chunks before the current unit
+    uint32_t seq_unit = 0;                           // slot items before the current unit
     uint32_t base = 0;                               // tiles of one matrix before the current unit
     uint32_t uses = 0;                               // tiles I have taken so far (parity of my slot's use)
-    Cursor cu = {0, 0, 0};
     bool ok = true;
-    for (uint32_t i = 0; ok; ++i) {
-      UDesc d;
-      if (!get_desc(i, polls, c, status, d) || d.unit < 0) break;
-      const uint32_t bits0 = d.bits & 0xffu, bits1 = NMAT == 2 ? (d.bits >> 8) & 0xffu : bits0;
-      const uint32_t bits = qm ? bits1 : bits0;
-      const uint32_t l0 = chunk_log(bits0), l1 = chunk_log(bits1);
-      const uint32_t ng = (uint32_t)d.ng;
-      const uint32_t nch = ((ng + (1u << l0) - 1u) >> l0) + (NMAT == 2 ? ((ng + (1u << l1) - 1u) >> l1) : 0u);
-      // Tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my first one
-      // in this unit is tile j0, then every kStride-th.  (The MMA reads 16-bit tiles straight from shared memory.)
-      const uint32_t j0 = (gsub - base) & (kStride - 1);
-      switch (bits) {
-        case 8: ok = dq_unit<8, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 4: ok = dq_unit<4, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 3: ok = dq_unit<3, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        case 2: ok = dq_unit<2, NMAT, false>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-#define PW_PLANE_CASE(Q) case kPlanesFlag | Q: if constexpr (PLANES) ok = dq_unit<Q, NMAT, true>(c, ka, wring, qm, j0, kStride, ng, seq_unit, l0, l1, cu, uses, r, lane, lane_addr, af_s, ae_s); break;
-        PW_PLANE_CASE(4)
-        PW_PLANE_CASE(3)
-        PW_PLANE_CASE(2)
-#undef PW_PLANE_CASE
-        default: break;
+    for (int i = 0; ok; ++i) {
+      const int u = next_unit((uint32_t)i, polls, c, status);
+      if (u < 0) break;
+      const Unit un = load_unit(units, u);
+      uint32_t ubits[NMAT];
+#pragma unroll
+      for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+      const uint32_t bits = qm ? ubits[NMAT - 1] : ubits[0];
+      const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+      const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+      if (bits != 16) {                              // the MMA reads 16-bit tiles straight from shared memory
+        // Tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my first one
+        // in this unit is group j0, then every kStride-th.
+        const uint32_t j0 = (gsub - base) & (kStride - 1);
+        const uint32_t step = kStride * W;
+        uint32_t sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+#pragma unroll 1
+        for (uint32_t j = j0; ok && j < ng; j += kStride) {
+          const uint32_t use_par = uses & 1u;
+          ++uses;
+          if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
+            ok = wait_issued(sq, polls, c, status) && mbar_wait_s(smem_u32(&c->full[rp.s]), rp.par, polls, c, status);
+            if (!ok) break;
+          }
+          const char* item = wring + rp.s * kSlotBytes;
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h) {
+            __half2 w[32];
+            switch (bits) {
+              case 8: decode_item_half<8>(item, r, h, w); break;
+              case 4: decode_item_half<4>(item, r, h, w); break;
+              case 3: decode_item_half<3>(item, r, h, w); break;
+              case 2: decode_item_half<2>(item, r, h, w); break;
+              default:
+                if constexpr (PLANES) {          // a bit-plane tile: table state of the committed bitwidth at a fixed place
+                  const __half2 s2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut)[r]);
+                  const __half2 z2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut + 256)[r]);
+                  if (bits == (kPlanesFlag | 4)) decode_half_planes<4>(item, r, h, s2, z2, w);
+                  else if (bits == (kPlanesFlag | 3)) decode_half_planes<3>(item, r, h, s2, z2, w);
+                  else decode_half_planes<2>(item, r, h, s2, z2, w);
+                }
+                break;
+            }
+            if (h == 0) {
+              // The slot is free once the MMAs of the group's previous tile have read it; they ran while the
+              // half above was being decoded.
+              ok = mbar_wait_s(smem_u32(&c->a_empty[grp]), use_par ^ 1, polls, c, status);
+              if (!ok) break;
+              tc_fence_after();
+            } else {
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&c->empty[rp.s]);   // this warp has read its rows of the tile
+            }
+            tmem_st32(lane_addr + h * 32, w);
+          }
+          if (!ok) break;
+          // hand the tile over: both stores have landed, then one arrival per warp
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&c->a_full[grp]);
+          sq += step;
+          ring_advance(rp, step, (uint32_t)n_slots);
+        }
       }
       base += ng;
-      seq_unit += nch;
+      seq_unit += ng * W;
     }
   } else if (warp >= kWarpEpi) {
     // ---------------- epilogue ----------------
     const int q = warp & 3;
+    const int r = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const uint32_t df_s = smem_u32(&c->d_full[0]), de_s = smem_u32(&c->d_empty[0]);
-    uint32_t base = 0;                               // tiles of one matrix before the current unit
+    uint32_t ucount = 0, base = 0;                   // base: tiles of one matrix before the current unit
     uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;      // accumulator buffers: the issuers' rule, replayed
     bool ok = true;
-    for (uint32_t i = 0; ok; ++i) {
-      UDesc d;
-      if (!get_desc(i, polls, c, status, d) || d.unit < 0) break;
-      const int nb_rows = (d.ntok + 15) & ~15;
+    for (int i = 0; ok; ++i, ++ucount) {
+      const int u = next_unit((uint32_t)i, polls, c, status);
+      if (u < 0) break;
+      const Unit un = load_unit(units, u);
+      const int nb_rows = (un.ntok + 15) & ~15;
       const bool wide = NMAT * npart * nb_rows > acol / 2;
       const uint32_t dbuf = wide ? 0u : dtoggle;
       if (!wide) dtoggle ^= 1u;
-      if (wide || dbuf == 0) ok = wait_bar(df_s, duse0 & 1, polls, c, status);
-      if (ok && (wide || dbuf == 1)) ok = wait_bar(df_s + 8, duse1 & 1, polls, c, status);
+      if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), duse0 & 1, polls, c, status);
+      if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), duse1 & 1, polls, c, status);
       if (!ok) break;
       tc_fence_after();
+      const int row = un.row_tile * kTileRows + r;
+      const uint32_t dbase = lane_addr + dbuf * (uint32_t)(acol / 2);
       // partial accumulator p holds the tiles base + j with (base + j) mod npart == p: it has been written in
       // this unit only if there is such a j below the unit's group count
-      const uint32_t ng = (uint32_t)d.ng;
+      const uint32_t ng = (uint32_t)(un.g1 - un.g0);
       uint32_t written = 0;
       for (int p = 0; p < npart; ++p)
         if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
       base += ng;
       // with helpers, the issuer warps take the upper half of the token columns of a wide unit
       const int c_end = HELP && wide ? ((nb_rows / 16 + 1) / 2) * 16 : nb_rows;
-      epilogue_cols<PHASE>(ka, d, lane_addr + dbuf * (uint32_t)(acol / 2), npart, written, nb_rows,
-                           d.row_tile * kTileRows + q * 32 + lane, 0, c_end);
+      for (int c0 = 0; c0 < c_end; c0 += 16) {
+        float a[16], b[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
+        for (int p = 0; p < npart; ++p) {              // add the issuers' partial sums, in order
+          if (!((written >> p) & 1u)) continue;
+          float t[16];
+          tmem_ld16(dbase + p * nb_rows + c0, t);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
+          if (PHASE == 0) {
+            tmem_ld16(dbase + (npart + p) * nb_rows + c0, t);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int nn = c0 + j;
+          if (nn < un.ntok) {
+            if (PHASE == 0) {
+              // SwiGLU: silu(gate) * up; the result is rounded to fp16, so the fast exponential and
+              // division (relative error ~1e-6) change nothing that survives the rounding
+              const float hval = __fmul_rn(__fdividef(a[j], __fadd_rn(1.0f, __expf(-a[j]))), b[j]);
+              ht[((size_t)(row >> 3) * Rpad + un.tok0 + nn) * 8 + (row & 7)] = __float2half_rn(hval);
+            } else {
+              y[(size_t)un.split * y_split_stride + (size_t)(un.tok0 + nn) * H + row] = a[j];
+            }
+          }
+        }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         // (a narrow unit has no helpers: this warp arrives for the issuer warp of its lane quarter as well)
         const uint32_t n_arr = HELP && !wide ? 2u : 1u;
-        if (wide || dbuf == 0) mbar_arrive_n_s(de_s, n_arr);
-        if (wide || dbuf == 1) mbar_arrive_n_s(de_s + 8, n_arr);
+        if (wide || dbuf == 0) mbar_arrive_n(&c->d_empty[0], n_arr);
+        if (wide || dbuf == 1) mbar_arrive_n(&c->d_empty[1], n_arr);
       }
       if (wide || dbuf == 0) ++duse0;
       if (wide || dbuf == 1) ++duse1;
@@ -879,7 +1108,8 @@ static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, Tma
   return true;
 }
 
-typedef void (*FfnKernel)(const KArgs, const TmapSet);
+typedef void (*FfnKernel)(const DevRow*, const Unit*, const int32_t*, const TmapSet, int, int, int, int, __half*, float*, int, size_t,
+                          int32_t*, int32_t*, uint32_t, uint32_t);
 static FfnKernel ffn_kernel_of(int phase, int help, int planes) {
   static const FfnKernel tab[8] = {ffn_tc_kernel<0, false, false>, ffn_tc_kernel<1, false, false>, ffn_tc_kernel<0, true, false>,
                                    ffn_tc_kernel<1, true, false>,  ffn_tc_kernel<0, false, true>,  ffn_tc_kernel<1, false, true>,
@@ -945,47 +1175,32 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
     n_bslots[phase] = npart + 1 > kMaxBSlots ? kMaxBSlots : npart + 1;
     int ns = (kMaxDynSmem - kCtrlBytes - n_bslots[phase] * bslot_bytes) / kSlotBytes;
     if (ns > kMaxSlots) ns = kMaxSlots;
-    if (ns < 3) return PW_ERR_NOMEM;
+    ns &= ~1;                                    // an even number of slots: one set per producer
+    if (ns < 4) return PW_ERR_NOMEM;
     n_slots[phase] = ns;
     smem[phase] = kCtrlBytes + ns * kSlotBytes + n_bslots[phase] * bslot_bytes;
   }
   const int R = T * k + c.n_shared * T;
-  KArgs ka;
-  ka.rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
-  ka.n_units_ptr = reinterpret_cast<const int32_t*>(b + w.n_units);
-  ka.Rpad = w.Rpad;
-  ka.nt_tile = nt_tile;
-  ka.H = c.hidden;
-  ka.status = reinterpret_cast<int32_t*>(b + w.status);
-  ka.wait_polls = ctx->wait_polls ? ctx->wait_polls : kDefaultWaitPolls;
-  ka.hook = ctx->test_hook;
+  const DevRow* rows = reinterpret_cast<const DevRow*>(b + w.table) + (size_t)layer * w.S * 3;
+  int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
+  const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
+  const uint32_t wait_polls = ctx->wait_polls ? ctx->wait_polls : kDefaultWaitPolls;
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   // token tiles of 128 leave no second accumulator buffer: the variant whose issuer warps share the epilogue
   const bool help = nt_tile > 64;
   bool planes = false;                           // does the layer hold a bit-plane block?
   for (int e = 0; e < w.S && !planes; ++e)
     for (int u = 0; u < 3; ++u) planes |= ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES;
-  ka.units = reinterpret_cast<const Unit*>(b + w.units_gu);
-  ka.n_bslots = n_bslots[0];
-  ka.n_slots = n_slots[0];
-  ka.ht = reinterpret_cast<__half*>(b + w.ht);
-  ka.y = nullptr;
-  ka.y_split_stride = 0;
-  ka.work_counter = work_counter;
-  PW_CUDA_OK(launch_dependent(ffn_kernel_of(0, help, planes), dim3(ctx->num_sms), dim3(kThreads),
-                              (size_t)smem[0], s, ka, st->xt));
+  PW_CUDA_OK(launch_dependent(ffn_kernel_of(0, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[0], s, rows,
+                              reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
+                              n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
+                              work_counter, status, wait_polls, ctx->test_hook));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
-  ka.units = reinterpret_cast<const Unit*>(b + w.units_dn);
-  ka.n_bslots = n_bslots[1];
-  ka.n_slots = n_slots[1];
-  ka.ht = nullptr;
-  ka.y = reinterpret_cast<float*>(b + w.y);
-  ka.y_split_stride = (size_t)R * c.hidden;
-  ka.work_counter = work_counter + 1;
-  ka.hook = 0;
-  PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads),
-                              (size_t)smem[1], s, ka, st->ht));
+  PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
+                              reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
+                              n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
+                              (size_t)R * c.hidden, work_counter + 1, status, wait_polls, 0u));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   (void)ksplit;
