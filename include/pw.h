@@ -453,7 +453,10 @@ pw_status pw_get_kernel_times(pw_ctx* ctx, double* ms_out, uint64_t* calls_out);
 uint64_t pw_launch_count(pw_ctx* ctx);
 
 /* Test aid for the failure path of the expert-FFN kernels (the paper has no counterpart).  Every device-side
- * wait of those kernels is bounded: `polls` polls of up to 20 us each (0 restores the default, 100000 = 2 s).
+ * wait of those kernels is bounded, by 100000 polls of up to 20 us each (2 s).  The limit is compiled into the
+ * kernels (carried in a register it cost the decode step 5 %), so `polls` only chooses: 0 = that default;
+ * any other value = the gate/up kernel (narrow token tiles, ordinary pages) runs an instantiation whose limit
+ * is 200 polls (4 ms).
  * When a wait runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
  * memory and returns; the call's output is then undefined and pw_last_device_status reports the timeout.
  * hook: 0 = none; bit 0 = the token-tile producer of the gate/up kernel stops before its second tile, so that

@@ -564,5 +564,5 @@ class Context:
         return int(self.L.pw_launch_count(self.handle))
 
     def pw_debug_set_wait(self, polls: int = 0, hook: int = 0) -> None:
-        """Limit of the device-side waits (polls of up to 20 us; 0 = default) and test hooks of the FFN kernels."""
+        """Wait limit of the gate/up FFN kernel (0 = the default 2 s, else the 4 ms test build) and test hooks."""
         _check(self.L.pw_debug_set_wait(self.handle, polls, hook), "pw_debug_set_wait")

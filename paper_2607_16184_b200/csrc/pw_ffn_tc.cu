@@ -34,6 +34,10 @@
 //                those, has the four issuer warps share the epilogue of every wide unit.
 // Every wait is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing
 // work, frees its tensor memory and returns.
+// A block in the overlaid bit-plane format (Sec. 2.2, Sec. 3.1) is a slot item like any quantized tile: its
+// producer copies the leading two planes, the lookup-table state of the bitwidth the page table names, and only
+// as many further planes as that bitwidth reads.  Layers that hold such a block run the PLANES instantiation, so
+// that the ordinary one keeps its decode switch and its registers.
 #include <cuda.h>
 
 #include <new>
@@ -55,6 +59,7 @@ constexpr int kThreads = 864;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSuspendHintNs = 20000;                   // a blocked barrier wait sleeps up to this long per poll
 constexpr uint32_t kDefaultWaitPolls = 100000;               // x kSuspendHintNs = 2 s
+constexpr uint32_t kTestWaitPolls = 200;                     // 4 ms: the limit of the instantiation that the failure-path test runs
 
 struct Ctrl {                                  // lives at the start of dynamic shared memory
   // One full barrier per ring slot (armed by the weight producer).  A slot is handed back either by the
@@ -76,9 +81,6 @@ struct Ctrl {                                  // lives at the start of dynamic 
   // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
   volatile int32_t sched_unit[32];
-  // Set once the kernel ahead of this one in the stream has completed.  Until then a wait that runs out is not a
-  // fault and simply starts over.
-  volatile uint32_t dep_ready;
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
@@ -115,66 +117,65 @@ __device__ __forceinline__ bool mbar_try(unsigned long long* b, uint32_t parity)
 }
 // Bounded wait.  Returns false when the limit ran out (and then raises the abort; the other roles of the CTA,
 // starved by the one that gave up, run into their own limits within the same second or two, and since every
-// role has then been idle for at least a second no copy of the CTA is still in flight when it leaves).  Each poll is a try_wait with a
+// role has then been idle for at least a second no copy of
+// the CTA is still in flight when it leaves).  Each poll is a try_wait with a
 // suspend-time hint, so a waiting thread sleeps inside the barrier unit instead of spending issue slots (an
 // arrival that does not complete the phase still wakes it, hence the loop); 100000 polls of up to kSuspendHintNs
 // each are the 2 s limit.  The loop is inline and written in PTX on purpose: with an out-of-line slow path the
 // call made the compiler keep each role's loop state -- for the dequantizers a vector of 32 results between
 // decode and store -- in call-preserved registers and copy it around, which cost 2 % of the decode step.
 // (the barrier is given by its shared-memory address: the control loops keep those in registers)
-// A wait ran out: not a fault while the kernel ahead in the stream is still running (the CTA may have been placed
-// long before its inputs exist), otherwise the CTA gives up.
-__device__ __forceinline__ bool wait_failed(Ctrl* c, int32_t* status) {
-  if (!c->dep_ready) return false;               // start over
-  c->abort_flag = 1;
-  atomicMax(status, (int)PW_ERR_TIMEOUT);
-  return true;
-}
-__device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, uint32_t polls, Ctrl* c, int32_t* status) {
-  for (;;) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
-        "mov.u32 n, 0;\n"
-        "PW_WAITN:\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "@p bra PW_DONEN;\n\t"
-        "add.u32 n, n, 1;\n\t"
-        "setp.lt.u32 q, n, %4;\n\t"
-        "@q bra PW_WAITN;\n"
-        "PW_DONEN:\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "r"(polls)
-        : "memory");
-    if (ok) return true;
-    if (wait_failed(c, status)) return false;
+// LIM: polls before the wait gives up.  It is an immediate, and the failure path is two stores, on purpose: the
+// limit carried in a register, or a retry loop around the wait, cost the dequantizers 5 % of the decode step.
+template <uint32_t LIM>
+__device__ __forceinline__ bool mbar_wait_s(uint32_t bar_s, uint32_t parity, Ctrl* c, int32_t* status) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n"
+      "PW_WAITN:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra PW_DONEN;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "setp.lt.u32 q, n, %4;\n\t"
+      "@q bra PW_WAITN;\n"
+      "PW_DONEN:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_s), "r"(parity), "r"(kSuspendHintNs), "n"(LIM)
+      : "memory");
+  if (!ok) {
+    c->abort_flag = 1;
+    atomicMax(status, (int)PW_ERR_TIMEOUT);
   }
+  return ok != 0;
 }
-// Sleep-and-look until the shared-memory word at `addr_s` exceeds `value`: at least 64 ns per look, polls * 256 looks.
-__device__ __forceinline__ bool flag_wait(uint32_t addr_s, uint32_t value, uint32_t polls, Ctrl* c, int32_t* status) {
-  const uint32_t looks = polls < (1u << 24) ? polls << 8 : 0xffffffffu;
-  for (;;) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
-        "mov.u32 k, 0;\n"
-        "PW_FL:\n\t"
-        "ld.volatile.shared.u32 v, [%1];\n\t"
-        "setp.gt.u32 p, v, %2;\n\t"
-        "@p bra PW_FLD;\n\t"
-        "nanosleep.u32 64;\n\t"
-        "add.u32 k, k, 1;\n\t"
-        "setp.lt.u32 q, k, %3;\n\t"
-        "@q bra PW_FL;\n"
-        "PW_FLD:\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(addr_s), "r"(value), "r"(looks)
-        : "memory");
-    if (ok) return true;
-    if (wait_failed(c, status)) return false;
+// Sleep-and-look until the shared-memory word at `addr_s` exceeds `value`: at least 64 ns per look, 256 looks per
+// poll of the barrier limit.
+template <uint32_t LIM>
+__device__ __forceinline__ bool flag_wait(uint32_t addr_s, uint32_t value, Ctrl* c, int32_t* status) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 v, k;\n\t"
+      "mov.u32 k, 0;\n"
+      "PW_FL:\n\t"
+      "ld.volatile.shared.u32 v, [%1];\n\t"
+      "setp.gt.u32 p, v, %2;\n\t"
+      "@p bra PW_FLD;\n\t"
+      "nanosleep.u32 64;\n\t"
+      "add.u32 k, k, 1;\n\t"
+      "setp.lt.u32 q, k, %3;\n\t"
+      "@q bra PW_FL;\n"
+      "PW_FLD:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(addr_s), "r"(value), "n"(LIM * 256u)
+      : "memory");
+  if (!ok) {
+    c->abort_flag = 1;
+    atomicMax(status, (int)PW_ERR_TIMEOUT);
   }
+  return ok != 0;
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -344,15 +345,17 @@ __device__ __forceinline__ void ring_advance(RingPos& p, uint32_t step, uint32_t
 __device__ __forceinline__ uint32_t slot_items(uint32_t bits) { return bits == 16 ? 2u : 1u; }
 // Bounded wait until the weight producer has armed slot item n.  A consumer looks at a slot item's full barrier
 // only after this, so it can never mistake an older phase of the slot's barrier for the item's.
-__device__ __forceinline__ bool wait_issued(uint32_t n, uint32_t polls, Ctrl* c, int32_t* status) {
+template <uint32_t LIM>
+__device__ __forceinline__ bool wait_issued(uint32_t n, Ctrl* c, int32_t* status) {
   if (c->issued[n & 1] > n) return true;
-  return flag_wait(smem_u32(const_cast<uint32_t*>(&c->issued[n & 1])), n, polls, c, status);
+  return flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->issued[n & 1])), n, c, status);
 }
 // Unit i of this CTA's work list (bounded wait until the weight producer has posted it); -1 = no more work,
 // -2 = the CTA is aborting.
-__device__ __forceinline__ int next_unit(uint32_t i, uint32_t polls, Ctrl* c, int32_t* status) {
+template <uint32_t LIM>
+__device__ __forceinline__ int next_unit(uint32_t i, Ctrl* c, int32_t* status) {
   if (c->sched_n > i) return c->sched_unit[i & 31];
-  if (flag_wait(smem_u32(const_cast<uint32_t*>(&c->sched_n)), i, polls, c, status)) return c->sched_unit[i & 31];
+  if (flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->sched_n)), i, c, status)) return c->sched_unit[i & 31];
   return -2;
 }
 // A unit of the list.  The gate/up list is written by the kernel directly ahead of this one in the stream, possibly
@@ -415,15 +418,16 @@ __device__ __forceinline__ void decode_item_half(const char* item, int r, int h,
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
 // PLANES: the instantiation that also reads blocks of overlaid bit-planes; launched only for a layer that holds one
 // (the extra code paths cost the ordinary ones instruction-cache room).
-// wait_polls: limit of every wait, in polls of kSuspendHintNs.  hook: test hook, bit 0 = the token-tile producer
-// stops before its second tile (so that the waits on it run out).
-template <int PHASE, bool HELP, bool PLANES>
+// SHORT: the instantiation with the short wait limit (kTestWaitPolls instead of kDefaultWaitPolls), for the test of
+// the failure path.  hook: test hook, bit 0 = the token-tile producer stops before its second tile (so that the
+// waits on it run out).
+template <int PHASE, bool HELP, bool PLANES, bool SHORT>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t* __restrict__ n_units_ptr,
               const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
               __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
-              int32_t* __restrict__ work_counter, int32_t* __restrict__ status, uint32_t wait_polls, uint32_t hook) {
-  const uint32_t polls = wait_polls;
+              int32_t* __restrict__ work_counter, int32_t* __restrict__ status, uint32_t hook) {
+  constexpr uint32_t LIM = SHORT ? kTestWaitPolls : kDefaultWaitPolls;
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   char* wring = smem + kCtrlBytes;
@@ -462,7 +466,6 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     c->issued[0] = c->issued[1] = 0;
     c->b_issued = 0;
     c->sched_n = 0;
-    c->dep_ready = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -501,10 +504,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       // the token rows), which may still be running: the producers wait for it before they read a unit, and
       // every other role learns of its first unit from producer 0 only after that.  The down kernel's list is
       // two kernels back and final (see grid_dep_sync), so its producers stream at once.
-      if (PHASE == 0) {
-        grid_dep_sync();
-        c->dep_ready = 1;
-      }
+      if (PHASE == 0) grid_dep_sync();
       // the work list: unit blockIdx.x first, then whatever the global counter hands out
       int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
       if (P == 0) {
@@ -552,7 +552,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             ms[m].b0 += kPlaneBitTile;
             for (int sub = 0; sub < nsub; ++sub, src += 16384) {
               if ((seq & 1u) == P) {
-                if (pass) ok = mbar_wait_s(smem_u32(&c->empty[s]), (pass - 1) & 1, polls, c, status);
+                if (pass) ok = mbar_wait_s<LIM>(smem_u32(&c->empty[s]), (pass - 1) & 1, c, status);
                 if (!ok) break;
                 const uint32_t bar_s = full_s + 8 * s;
                 mbar_expect_tx_s(bar_s, bytes);
@@ -582,7 +582,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           __threadfence_block();
           c->sched_n = (uint32_t)i + 2;
         } else {
-          u = next_unit((uint32_t)i + 1, polls, c, status);
+          u = next_unit<LIM>((uint32_t)i + 1, c, status);
         }
       }
     }
@@ -591,11 +591,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     if (lane == 0) {
       grid_dep_sync();
       grid_dep_trigger();
-      if (PHASE == 1) c->dep_ready = 1;
       uint32_t bcount = 0;
       bool ok = true;
       for (int i = 0; ok; ++i) {
-        const int u = next_unit((uint32_t)i, polls, c, status);
+        const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
         const Unit un = load_unit(units, u);
         const int nb_rows = (un.ntok + 15) & ~15;
@@ -607,7 +606,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           }
           // token tile of this group: 16 K-chunks x nb_rows rows x 16 bytes, one 2-D copy
           const int bs = bcount % n_bslots;
-          ok = mbar_wait_s(smem_u32(&c->b_empty[bs]), ((bcount / n_bslots) & 1) ^ 1, polls, c, status);
+          ok = mbar_wait_s<LIM>(smem_u32(&c->b_empty[bs]), ((bcount / n_bslots) & 1) ^ 1, c, status);
           if (!ok) break;
           mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
           tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
@@ -643,7 +642,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       const uint32_t a_base = tmem + acol;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
-        const int u = next_unit((uint32_t)i, polls, c, status);
+        const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
         const Unit un = load_unit(units, u);
         uint32_t ubits[NMAT];
@@ -671,8 +670,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (!wide) dtoggle ^= 1u;
         const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
         // the epilogue has drained the buffer(s) this unit accumulates into
-        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, polls, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, polls, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         tc_fence_after();
         uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
@@ -680,10 +679,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
           // the token tile of this group (a tile is looked at only once it is known to have been armed)
           if (c->b_issued <= bt) {
-            ok = flag_wait(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, polls, c, status);
+            ok = flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, c, status);
             if (!ok) break;
           }
-          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, polls, c, status);
+          ok = mbar_wait_s<LIM>(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
           if (my_bits == 16) {
@@ -691,7 +690,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             RingPos hp = rp;
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
-              ok = wait_issued(sq + hh, polls, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, polls, c, status);
+              ok = wait_issued<LIM>(sq + hh, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[hp.s]), hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
@@ -711,7 +710,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             upar ^= 1u << grp;
             const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
-            ok = mbar_wait_s(f0, use_par, polls, c, status);
+            ok = mbar_wait_s<LIM>(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             // all eight k-steps of the tile, then one commit hands the group's operand slot back
@@ -763,7 +762,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       const uint32_t a_base = tmem + acol;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
-        const int u = next_unit((uint32_t)i, polls, c, status);
+        const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
         const Unit un = load_unit(units, u);
         uint32_t ubits[NMAT];
@@ -793,8 +792,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (lane == 0 && issuing) {
           do {
         // the epilogue has drained the buffer(s) this unit accumulates into
-        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, polls, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, polls, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         tc_fence_after();
         uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
@@ -802,10 +801,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
           // the token tile of this group (a tile is looked at only once it is known to have been armed)
           if (c->b_issued <= bt) {
-            ok = flag_wait(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, polls, c, status);
+            ok = flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, c, status);
             if (!ok) break;
           }
-          ok = mbar_wait_s(bf_s + 8 * bp.s, bp.par, polls, c, status);
+          ok = mbar_wait_s<LIM>(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
           const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
           if (my_bits == 16) {
@@ -813,7 +812,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             RingPos hp = rp;
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
-              ok = wait_issued(sq + hh, polls, c, status) && mbar_wait_s(smem_u32(&c->full[hp.s]), hp.par, polls, c, status);
+              ok = wait_issued<LIM>(sq + hh, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[hp.s]), hp.par, c, status);
               if (!ok) break;
               tc_fence_after();
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
@@ -833,7 +832,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             upar ^= 1u << grp;
             const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
-            ok = mbar_wait_s(f0, use_par, polls, c, status);
+            ok = mbar_wait_s<LIM>(f0, use_par, c, status);
             if (!ok) break;
             tc_fence_after();
             // all eight k-steps of the tile, then one commit hands the group's operand slot back
@@ -859,8 +858,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (wide || dbuf == 1) ++duse1;
         // every issuer warp sees every phase of the accumulator barriers, also of the narrow units it has no
         // part in: it must not run ahead of the epilogue by more than the phase parity can tell apart
-        if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), par0, polls, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), par1, polls, c, status);
+        if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_full[0]), par0, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_full[1]), par1, c, status);
         if (!ok) break;
         if (wide) {
           tc_fence_after();
@@ -929,7 +928,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     uint32_t uses = 0;                               // tiles I have taken so far (parity of my slot's use)
     bool ok = true;
     for (int i = 0; ok; ++i) {
-      const int u = next_unit((uint32_t)i, polls, c, status);
+      const int u = next_unit<LIM>((uint32_t)i, c, status);
       if (u < 0) break;
       const Unit un = load_unit(units, u);
       uint32_t ubits[NMAT];
@@ -950,7 +949,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           const uint32_t use_par = uses & 1u;
           ++uses;
           if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
-            ok = wait_issued(sq, polls, c, status) && mbar_wait_s(smem_u32(&c->full[rp.s]), rp.par, polls, c, status);
+            ok = wait_issued<LIM>(sq, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[rp.s]), rp.par, c, status);
             if (!ok) break;
           }
           const char* item = wring + rp.s * kSlotBytes;
@@ -975,7 +974,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             if (h == 0) {
               // The slot is free once the MMAs of the group's previous tile have read it; they ran while the
               // half above was being decoded.
-              ok = mbar_wait_s(smem_u32(&c->a_empty[grp]), use_par ^ 1, polls, c, status);
+              ok = mbar_wait_s<LIM>(smem_u32(&c->a_empty[grp]), use_par ^ 1, c, status);
               if (!ok) break;
               tc_fence_after();
             } else {
@@ -1006,15 +1005,15 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;      // accumulator buffers: the issuers' rule, replayed
     bool ok = true;
     for (int i = 0; ok; ++i, ++ucount) {
-      const int u = next_unit((uint32_t)i, polls, c, status);
+      const int u = next_unit<LIM>((uint32_t)i, c, status);
       if (u < 0) break;
       const Unit un = load_unit(units, u);
       const int nb_rows = (un.ntok + 15) & ~15;
       const bool wide = NMAT * npart * nb_rows > acol / 2;
       const uint32_t dbuf = wide ? 0u : dtoggle;
       if (!wide) dtoggle ^= 1u;
-      if (wide || dbuf == 0) ok = mbar_wait_s(smem_u32(&c->d_full[0]), duse0 & 1, polls, c, status);
-      if (ok && (wide || dbuf == 1)) ok = mbar_wait_s(smem_u32(&c->d_full[1]), duse1 & 1, polls, c, status);
+      if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_full[0]), duse0 & 1, c, status);
+      if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_full[1]), duse1 & 1, c, status);
       if (!ok) break;
       tc_fence_after();
       const int row = un.row_tile * kTileRows + r;
@@ -1109,13 +1108,16 @@ static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, Tma
 }
 
 typedef void (*FfnKernel)(const DevRow*, const Unit*, const int32_t*, const TmapSet, int, int, int, int, __half*, float*, int, size_t,
-                          int32_t*, int32_t*, uint32_t, uint32_t);
+                          int32_t*, int32_t*, uint32_t);
 static FfnKernel ffn_kernel_of(int phase, int help, int planes) {
-  static const FfnKernel tab[8] = {ffn_tc_kernel<0, false, false>, ffn_tc_kernel<1, false, false>, ffn_tc_kernel<0, true, false>,
-                                   ffn_tc_kernel<1, true, false>,  ffn_tc_kernel<0, false, true>,  ffn_tc_kernel<1, false, true>,
-                                   ffn_tc_kernel<0, true, true>,   ffn_tc_kernel<1, true, true>};
+  static const FfnKernel tab[8] = {
+      ffn_tc_kernel<0, false, false, false>, ffn_tc_kernel<1, false, false, false>, ffn_tc_kernel<0, true, false, false>,
+      ffn_tc_kernel<1, true, false, false>,  ffn_tc_kernel<0, false, true, false>,  ffn_tc_kernel<1, false, true, false>,
+      ffn_tc_kernel<0, true, true, false>,   ffn_tc_kernel<1, true, true, false>};
   return tab[phase + 2 * help + 4 * planes];
 }
+// the gate/up kernel with the short wait limit (narrow token tiles, ordinary pages): what the failure-path test runs
+static FfnKernel ffn_kernel_short() { return ffn_tc_kernel<0, false, false, true>; }
 
 static pw_status tc_setup(pw_ctx* ctx) {
   if (ctx->tc_state) return PW_OK;
@@ -1135,6 +1137,7 @@ static pw_status tc_setup(pw_ctx* ctx) {
   for (int i = 0; i < 8; ++i)
     PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_of(i & 1, (i >> 1) & 1, (i >> 2) & 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     kMaxDynSmem));
+  PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_short(), cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
   ctx->tc_state = st;
   return PW_OK;
 }
@@ -1154,6 +1157,13 @@ int tensor_token_tile(const pw_ctx* ctx, int T, int k) {
   const int cap = avg > 64 ? 128 : 64;
   if (nt > cap) nt = cap;
   return nt;
+}
+
+static bool planes_layer(const pw_ctx* ctx, int layer) {     // does the layer hold a bit-plane block?
+  for (int e = 0; e < ctx->ws.S; ++e)
+    for (int u = 0; u < 3; ++u)
+      if (ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES) return true;
+  return false;
 }
 
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s) {
@@ -1185,22 +1195,22 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   int32_t* status = reinterpret_cast<int32_t*>(b + w.status);
   const int32_t* n_units = reinterpret_cast<const int32_t*>(b + w.n_units);
   int32_t* work_counter = reinterpret_cast<int32_t*>(b + w.counter);   // [0] gate/up, [1] down; zeroed by the permute kernel
-  const uint32_t wait_polls = ctx->wait_polls ? ctx->wait_polls : kDefaultWaitPolls;
   timing_mark(ctx, PW_K_FFN_GATE_UP, s);
   // token tiles of 128 leave no second accumulator buffer: the variant whose issuer warps share the epilogue
   const bool help = nt_tile > 64;
-  bool planes = false;                           // does the layer hold a bit-plane block?
-  for (int e = 0; e < w.S && !planes; ++e)
-    for (int u = 0; u < 3; ++u) planes |= ctx->host_rows[row_index(ctx, layer, e, u)].page.layout == PW_LAYOUT_PLANES;
-  PW_CUDA_OK(launch_dependent(ffn_kernel_of(0, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[0], s, rows,
+  const bool planes = planes_layer(ctx, layer);
+  // a context with a lowered wait limit (pw_debug_set_wait) runs the gate/up kernel's short-limit instantiation
+  const bool short_wait = ctx->wait_polls != 0 && !help && !planes;
+  PW_CUDA_OK(launch_dependent(short_wait ? ffn_kernel_short() : ffn_kernel_of(0, help, planes), dim3(ctx->num_sms),
+                              dim3(kThreads), (size_t)smem[0], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
                               n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
-                              work_counter, status, wait_polls, ctx->test_hook));
+                              work_counter, status, ctx->test_hook));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
                               n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
-                              (size_t)R * c.hidden, work_counter + 1, status, wait_polls, 0u));
+                              (size_t)R * c.hidden, work_counter + 1, status, 0u));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   (void)ksplit;

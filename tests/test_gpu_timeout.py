@@ -26,7 +26,7 @@ def test_wait_runs_out_then_context_recovers(orc):
         ref = orc.moe_forward(x.cpu().numpy(), logits.cpu().numpy(), cfg.top_k, opages)
         good = ctx.pw_moe_forward(0, x, logits, cfg.top_k).clone()
         assert ctx.pw_last_device_status() == 0
-        ctx.pw_debug_set_wait(polls=200, hook=1)             # 200 polls of up to 20 us; the second token tile never comes
+        ctx.pw_debug_set_wait(polls=200, hook=1)             # the 4 ms build; the second token tile never comes
         ctx.pw_moe_forward(0, x, logits, cfg.top_k)
         torch.cuda.synchronize()                              # the call returns: every wait is bounded
         assert ctx.pw_last_device_status() == 8               # PW_ERR_TIMEOUT, and reading it clears it
