@@ -414,6 +414,39 @@ __device__ __forceinline__ void decode_item_half(const char* item, int r, int h,
   decode_half<BITS>(row_units, h, s2, z2, w);
 }
 
+// One slot item, dequantized by one warp of its group: row r of the tile, both K-halves, into the group's operand
+// slot in tensor memory.  The slot is free once the MMAs of the group's previous tile have read it; they ran while
+// the first half was being decoded.  One routine per code format, so that what a decoder computes is stored from
+// the registers it was computed in (behind a common merge point every value was copied once more).
+// UB: bitwidth, with kPlanesFlag for a tile of a bit-plane block.
+template <uint32_t UB, uint32_t LIM>
+__device__ __forceinline__ bool dq_item(const char* item, int r, int lane, uint32_t lane_addr, uint32_t a_empty_s,
+                                        uint32_t a_empty_par, unsigned long long* slot_empty, Ctrl* c, int32_t* status) {
+  __half2 s2, z2;
+  if constexpr ((UB & kPlanesFlag) != 0) {       // table state of the committed bitwidth at a fixed place
+    s2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut)[r]);
+    z2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut + 256)[r]);
+  } else {
+    s2 = __half2half2(reinterpret_cast<const __half*>(item + UB * 2048)[r]);
+    z2 = __half2half2(reinterpret_cast<const __half*>(item + UB * 2048 + 256)[r]);
+  }
+#pragma unroll 1
+  for (int h = 0; h < 2; ++h) {
+    __half2 w[32];
+    if constexpr ((UB & kPlanesFlag) != 0) decode_half_planes<(int)(UB & ~kPlanesFlag)>(item, r, h, s2, z2, w);
+    else decode_half<(int)UB>(reinterpret_cast<const uint4*>(item) + r, h, s2, z2, w);
+    if (h == 0) {
+      if (!mbar_wait_s<LIM>(a_empty_s, a_empty_par, c, status)) return false;
+      tc_fence_after();
+    } else {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(slot_empty);    // this warp has read its rows of the tile
+    }
+    tmem_st32(lane_addr + h * 32, w);
+  }
+  return true;
+}
+
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
 // PLANES: the instantiation that also reads blocks of overlaid bit-planes; launched only for a layer that holds one
@@ -953,35 +986,23 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             if (!ok) break;
           }
           const char* item = wring + rp.s * kSlotBytes;
-#pragma unroll 1
-          for (int h = 0; h < 2; ++h) {
-            __half2 w[32];
-            switch (bits) {
-              case 8: decode_item_half<8>(item, r, h, w); break;
-              case 4: decode_item_half<4>(item, r, h, w); break;
-              case 3: decode_item_half<3>(item, r, h, w); break;
-              case 2: decode_item_half<2>(item, r, h, w); break;
-              default:
-                if constexpr (PLANES) {          // a bit-plane tile: table state of the committed bitwidth at a fixed place
-                  const __half2 s2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut)[r]);
-                  const __half2 z2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut + 256)[r]);
-                  if (bits == (kPlanesFlag | 4)) decode_half_planes<4>(item, r, h, s2, z2, w);
-                  else if (bits == (kPlanesFlag | 3)) decode_half_planes<3>(item, r, h, s2, z2, w);
-                  else decode_half_planes<2>(item, r, h, s2, z2, w);
-                }
-                break;
-            }
-            if (h == 0) {
-              // The slot is free once the MMAs of the group's previous tile have read it; they ran while the
-              // half above was being decoded.
-              ok = mbar_wait_s<LIM>(smem_u32(&c->a_empty[grp]), use_par ^ 1, c, status);
-              if (!ok) break;
-              tc_fence_after();
-            } else {
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&c->empty[rp.s]);   // this warp has read its rows of the tile
-            }
-            tmem_st32(lane_addr + h * 32, w);
+          const uint32_t ae_s = smem_u32(&c->a_empty[grp]);
+          unsigned long long* slot_empty = &c->empty[rp.s];
+          switch (bits) {
+            case 8: ok = dq_item<8, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
+            case 4: ok = dq_item<4, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
+            case 3: ok = dq_item<3, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
+            case 2: ok = dq_item<2, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
+            default:
+              if constexpr (PLANES) {
+                if (bits == (kPlanesFlag | 4))
+                  ok = dq_item<kPlanesFlag | 4, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
+                else if (bits == (kPlanesFlag | 3))
+                  ok = dq_item<kPlanesFlag | 3, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
+                else
+                  ok = dq_item<kPlanesFlag | 2, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
+              }
+              break;
           }
           if (!ok) break;
           // hand the tile over: both stores have landed, then one arrival per warp

@@ -145,6 +145,40 @@ __device__ inline __half2 dq_pair_k(uint32_t biased, uint32_t bias, __half2 s2, 
   return __hfma2(__hsub2(u32_as_h2(biased), u32_as_h2(bias)), s2, z2);
 }
 
+// (a & b) | c as ONE instruction.  Written out because the compiler, given two immediates, emits an AND and an
+// OR; with the constants in registers the three-input logic unit does both.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+// fp16 constant whose mantissa reads a field that starts at bit POS as an integer: 2^(10 - POS) has its unit in
+// the last place at bit POS, so (field << POS) | bits(2^(10 - POS)) = 2^(10 - POS) + field, exactly.
+template <int POS>
+__device__ __forceinline__ constexpr uint32_t field_magic() {
+  return (uint32_t)((25 - POS) << 10) * 0x00010001u;
+}
+// The pair of W-bit fields at bit POS of the two half-words of `word` -> (field * scale + zero-point) as half2.
+template <int POS, int W>
+__device__ __forceinline__ __half2 dq_field(uint32_t word, __half2 s2, __half2 z2) {
+  constexpr uint32_t mask = (((1u << W) - 1u) << POS) * 0x00010001u;
+  constexpr uint32_t magic = field_magic<POS>();
+  return dq_pair_k(and_or(word, mask, magic), magic, s2, z2);
+}
+// The same for a 2-bit field, with (BITS == 3) the code's third bit from bit p / 16 + p of `hw` put just above it.
+template <int POS, int BITS>
+__device__ __forceinline__ __half2 dq_field23(uint32_t word, uint32_t hw, int p, __half2 s2, __half2 z2) {
+  constexpr uint32_t mask = (3u << POS) * 0x00010001u;
+  constexpr uint32_t magic = field_magic<POS>();
+  uint32_t v = and_or(word, mask, magic);
+  if constexpr (BITS == 3) {
+    const int t = POS + 2;                       // where the third bit goes
+    const uint32_t hi = p >= t ? (hw >> (p - t)) : (hw << (t - p));
+    v = and_or(hi, (1u << t) * 0x00010001u, v);
+  }
+  return dq_pair_k(v, magic, s2, z2);
+}
+
 // Quarter t (0 .. 3) of a row-group: out[p] = weights (32t + 2p, 32t + 2p + 1), p = 0 .. 15.
 // `row_units` points at unit 0 of the row inside a tile image (shared or global memory); unit j
 // of the same row is kUnitStride uint4 further on.
@@ -180,30 +214,36 @@ __device__ __forceinline__ void decode_quarter(const uint4* row_units, int t, __
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint32_t w8 = w[i] >> 8;
-      out[4 * i + 0] = dq_pair_k((w[i] & 0x000f000fu) | 0x64006400u, 0x64006400u, s2, z2);
-      out[4 * i + 1] = dq_pair_k((w[i] & 0x00f000f0u) | 0x54005400u, 0x54005400u, s2, z2);
-      out[4 * i + 2] = dq_pair_k((w8 & 0x000f000fu) | 0x64006400u, 0x64006400u, s2, z2);
-      out[4 * i + 3] = dq_pair_k((w8 & 0x00f000f0u) | 0x54005400u, 0x54005400u, s2, z2);
+      out[4 * i + 0] = dq_field<0, 4>(w[i], s2, z2);
+      out[4 * i + 1] = dq_field<4, 4>(w[i], s2, z2);
+      out[4 * i + 2] = dq_field<0, 4>(w8, s2, z2);
+      out[4 * i + 3] = dq_field<4, 4>(w8, s2, z2);
     }
   } else {
     // 2 bits: words 2(t%2), 2(t%2)+1 of unit t/2.  3 bits: the same low-plane words plus word t of unit 2.
+    // A half-word holds eight 2-bit fields; fields 0 .. 3 are read where they lie (see dq_field), one shift by 8
+    // per word brings fields 4 .. 7 to the same places.  The third bit of a 3-bit code is moved to the place
+    // just above its field, where it reads 4.
     const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + (t >> 1) * kUnitStride) +
                                                      2 * (t & 1));
     const uint32_t w[2] = {u.x, u.y};
     uint32_t hw = 0;
     if constexpr (BITS == 3) hw = reinterpret_cast<const uint32_t*>(row_units + 2 * kUnitStride)[t];
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
+    for (int i = 0; i < 2; ++i) {
+      const uint32_t w8 = w[i] >> 8;
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
         const int p = 8 * i + m;                   // pair index inside the quarter = inside the high-plane word
-        uint32_t v = ((w[i] >> (2 * m)) & 0x00030003u) | 0x64006400u;
-        if constexpr (BITS == 3) {
-          const uint32_t hi = p >= 2 ? (hw >> (p - 2)) : (hw << (2 - p));
-          v |= hi & 0x00040004u;
+        const uint32_t src = m < 4 ? w[i] : w8;
+        switch (m & 3) {
+          case 0: out[p] = dq_field23<0, BITS>(src, hw, p, s2, z2); break;
+          case 1: out[p] = dq_field23<2, BITS>(src, hw, p, s2, z2); break;
+          case 2: out[p] = dq_field23<4, BITS>(src, hw, p, s2, z2); break;
+          default: out[p] = dq_field23<6, BITS>(src, hw, p, s2, z2); break;
         }
-        out[p] = dq_pair(v, s2, z2);
       }
+    }
   }
 }
 
