@@ -414,35 +414,81 @@ __device__ __forceinline__ void decode_item_half(const char* item, int r, int h,
   decode_half<BITS>(row_units, h, s2, z2, w);
 }
 
-// One slot item, dequantized by one warp of its group: row r of the tile, both K-halves, into the group's operand
-// slot in tensor memory.  The slot is free once the MMAs of the group's previous tile have read it; they ran while
-// the first half was being decoded.  One routine per code format, so that what a decoder computes is stored from
-// the registers it was computed in (behind a common merge point every value was copied once more).
+// predicated arrival (no branch around it)
+__device__ __forceinline__ void mbar_arrive_if_s(uint32_t bar_s, bool pred) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(bar_s),
+               "r"((uint32_t)pred)
+               : "memory");
+}
+
+// What a dequantizer warp carries from tile to tile.
+struct DqState {
+  uint32_t sq;                                   // number of my next slot item
+  uint32_t s, par;                               // its ring slot and the parity of its full-barrier phase
+  uint32_t a_par;                                // parity of the next "operand slot free" phase of my group
+  uint32_t known;                                // the producer of my items has armed every one below this number
+};
+
+// The tiles of one unit that fall to this warp's group (`count` of them, `step` slot items apart), all in one code
+// format: row r of each tile, both K-halves, into the group's operand slot in tensor memory.  The slot is free once
+// the MMAs of the group's previous tile have read it; they ran while the first half was being decoded.  One routine
+// per code format, with the tile loop inside: what a decoder computes is stored from the registers it was computed
+// in, and nothing about the format is decided per tile.  The per-tile control path is a chain of dependent
+// instructions that the decoders of the other groups do not hide, so it is kept as short as it gets.
 // UB: bitwidth, with kPlanesFlag for a tile of a bit-plane block.
 template <uint32_t UB, uint32_t LIM>
-__device__ __forceinline__ bool dq_item(const char* item, int r, int lane, uint32_t lane_addr, uint32_t a_empty_s,
-                                        uint32_t a_empty_par, unsigned long long* slot_empty, Ctrl* c, int32_t* status) {
-  __half2 s2, z2;
-  if constexpr ((UB & kPlanesFlag) != 0) {       // table state of the committed bitwidth at a fixed place
-    s2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut)[r]);
-    z2 = __half2half2(reinterpret_cast<const __half*>(item + kPlaneSlotLut + 256)[r]);
-  } else {
-    s2 = __half2half2(reinterpret_cast<const __half*>(item + UB * 2048)[r]);
-    z2 = __half2half2(reinterpret_cast<const __half*>(item + UB * 2048 + 256)[r]);
-  }
+__device__ __forceinline__ bool dq_run(DqState& st, uint32_t count, uint32_t step, uint32_t n_slots, uint32_t wring_s,
+                                       int r, bool lane0, uint32_t lane_addr, uint32_t full_s, uint32_t empty_s,
+                                       uint32_t a_full_s, uint32_t a_empty_s, Ctrl* c, int32_t* status) {
 #pragma unroll 1
-  for (int h = 0; h < 2; ++h) {
-    __half2 w[32];
-    if constexpr ((UB & kPlanesFlag) != 0) decode_half_planes<(int)(UB & ~kPlanesFlag)>(item, r, h, s2, z2, w);
-    else decode_half<(int)UB>(reinterpret_cast<const uint4*>(item) + r, h, s2, z2, w);
-    if (h == 0) {
-      if (!mbar_wait_s<LIM>(a_empty_s, a_empty_par, c, status)) return false;
-      tc_fence_after();
-    } else {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(slot_empty);    // this warp has read its rows of the tile
+  for (; count; --count) {
+    // A slot's full barrier is looked at only once the item is known to have been armed (the phase before it has
+    // then completed, so the parity cannot be mistaken); the producer is usually several items ahead, and one
+    // look at its counter covers them.
+    if (st.known <= st.sq) {
+      st.known = c->issued[st.sq & 1];
+      if (st.known <= st.sq) {
+        if (!flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->issued[st.sq & 1])), st.sq, c, status)) return false;
+        st.known = st.sq + 1;
+      }
     }
-    tmem_st32(lane_addr + h * 32, w);
+    if (!mbar_wait_s<LIM>(full_s + 8 * st.s, st.par, c, status)) return false;
+    const uint32_t item_s = wring_s + st.s * kSlotBytes;
+    __half2 s2, z2;
+    {
+      constexpr uint32_t lut = (UB & kPlanesFlag) != 0 ? (uint32_t)kPlaneSlotLut : (UB & 63u) * 2048u;
+      uint16_t sv, zv;
+      asm volatile("ld.shared.u16 %0, [%1];" : "=h"(sv) : "r"(item_s + lut + 2 * r));
+      asm volatile("ld.shared.u16 %0, [%1];" : "=h"(zv) : "r"(item_s + lut + 256 + 2 * r));
+      s2 = __half2half2(__ushort_as_half(sv));
+      z2 = __half2half2(__ushort_as_half(zv));
+    }
+    const char* item = reinterpret_cast<const char*>(c) + kCtrlBytes + st.s * kSlotBytes;
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
+      __half2 w[32];
+      if constexpr ((UB & kPlanesFlag) != 0) decode_half_planes<(int)(UB & ~kPlanesFlag)>(item, r, h, s2, z2, w);
+      else decode_half<(int)UB>(reinterpret_cast<const uint4*>(item) + r, h, s2, z2, w);
+      if (h == 0) {
+        if (!mbar_wait_s<LIM>(a_empty_s, st.a_par ^ 1, c, status)) return false;
+        tc_fence_after();
+      } else {
+        __syncwarp();
+        mbar_arrive_if_s(empty_s + 8 * st.s, lane0);   // this warp has read its rows of the tile
+      }
+      tmem_st32(lane_addr + h * 32, w);
+    }
+    // hand the tile over: both stores have landed, then one arrival per warp
+    tmem_wait_st();
+    tc_fence_before();
+    mbar_arrive_if_s(a_full_s, lane0);
+    st.a_par ^= 1u;
+    st.sq += step;
+    st.s += step;
+    if (st.s >= n_slots) {                       // step never exceeds the number of slots
+      st.s -= n_slots;
+      st.par ^= 1u;
+    }
   }
   return true;
 }
@@ -958,7 +1004,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     constexpr uint32_t kStride = NMAT == 2 ? 2 : 4;  // groups per matrix = distance between my tiles
     uint32_t seq_unit = 0;                           // slot items before the current unit
     uint32_t base = 0;                               // tiles of one matrix before the current unit
-    uint32_t uses = 0;                               // tiles I have taken so far (parity of my slot's use)
+    DqState st;
+    st.sq = st.s = st.par = st.a_par = st.known = 0;
+    const uint32_t wring_s = smem_u32(wring);
+    const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
+    const uint32_t a_full_s = smem_u32(&c->a_full[grp]), a_empty_s = smem_u32(&c->a_empty[grp]);
+    const bool lane0 = lane == 0;
     bool ok = true;
     for (int i = 0; ok; ++i) {
       const int u = next_unit<LIM>((uint32_t)i, c, status);
@@ -970,49 +1021,33 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       const uint32_t bits = qm ? ubits[NMAT - 1] : ubits[0];
       const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
-      if (bits != 16) {                              // the MMA reads 16-bit tiles straight from shared memory
-        // Tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my first one
-        // in this unit is group j0, then every kStride-th.
-        const uint32_t j0 = (gsub - base) & (kStride - 1);
+      // Tile k of a matrix (counted over all units) goes to that matrix's group k mod kStride: my first one
+      // in this unit is group j0, then every kStride-th.
+      const uint32_t j0 = (gsub - base) & (kStride - 1);
+      if (bits != 16 && j0 < ng) {                   // the MMA reads 16-bit tiles straight from shared memory
+        const uint32_t count = (ng - j0 + kStride - 1) / kStride;
         const uint32_t step = kStride * W;
-        uint32_t sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
-        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
-#pragma unroll 1
-        for (uint32_t j = j0; ok && j < ng; j += kStride) {
-          const uint32_t use_par = uses & 1u;
-          ++uses;
-          if (c->issued[sq & 1] <= sq || !mbar_try(&c->full[rp.s], rp.par)) {
-            ok = wait_issued<LIM>(sq, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[rp.s]), rp.par, c, status);
-            if (!ok) break;
-          }
-          const char* item = wring + rp.s * kSlotBytes;
-          const uint32_t ae_s = smem_u32(&c->a_empty[grp]);
-          unsigned long long* slot_empty = &c->empty[rp.s];
-          switch (bits) {
-            case 8: ok = dq_item<8, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
-            case 4: ok = dq_item<4, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
-            case 3: ok = dq_item<3, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
-            case 2: ok = dq_item<2, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status); break;
-            default:
-              if constexpr (PLANES) {
-                if (bits == (kPlanesFlag | 4))
-                  ok = dq_item<kPlanesFlag | 4, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
-                else if (bits == (kPlanesFlag | 3))
-                  ok = dq_item<kPlanesFlag | 3, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
-                else
-                  ok = dq_item<kPlanesFlag | 2, LIM>(item, r, lane, lane_addr, ae_s, use_par ^ 1, slot_empty, c, status);
-              }
-              break;
-          }
-          if (!ok) break;
-          // hand the tile over: both stores have landed, then one arrival per warp
-          tmem_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&c->a_full[grp]);
-          sq += step;
-          ring_advance(rp, step, (uint32_t)n_slots);
+        st.sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
+        const RingPos rp = ring_pos(st.sq, (uint32_t)n_slots);
+        st.s = rp.s;
+        st.par = rp.par;
+        st.known = 0;                                // my items of this unit may be another producer's than before
+#define PW_DQ_RUN(UB) \
+  dq_run<UB, LIM>(st, count, step, (uint32_t)n_slots, wring_s, r, lane0, lane_addr, full_s, empty_s, a_full_s, a_empty_s, c, status)
+        switch (bits) {
+          case 8: ok = PW_DQ_RUN(8); break;
+          case 4: ok = PW_DQ_RUN(4); break;
+          case 3: ok = PW_DQ_RUN(3); break;
+          case 2: ok = PW_DQ_RUN(2); break;
+          default:
+            if constexpr (PLANES) {
+              if (bits == (kPlanesFlag | 4)) ok = PW_DQ_RUN(kPlanesFlag | 4);
+              else if (bits == (kPlanesFlag | 3)) ok = PW_DQ_RUN(kPlanesFlag | 3);
+              else ok = PW_DQ_RUN(kPlanesFlag | 2);
+            }
+            break;
         }
+#undef PW_DQ_RUN
       }
       base += ng;
       seq_unit += ng * W;
@@ -1207,7 +1242,7 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
     int ns = (kMaxDynSmem - kCtrlBytes - n_bslots[phase] * bslot_bytes) / kSlotBytes;
     if (ns > kMaxSlots) ns = kMaxSlots;
     ns &= ~1;                                    // an even number of slots: one set per producer
-    if (ns < 4) return PW_ERR_NOMEM;
+    if (ns < 6) return PW_ERR_NOMEM;             // the dequantizers advance up to six slot items at a time
     n_slots[phase] = ns;
     smem[phase] = kCtrlBytes + ns * kSlotBytes + n_bslots[phase] * bslot_bytes;
   }
