@@ -286,19 +286,25 @@ __device__ __forceinline__ void decode_quarter_planes(const char* image, int r, 
   const uint32_t h1 = reinterpret_cast<const uint32_t*>(image + kPlaneSlotBit1 + r * 16)[t];
   uint32_t h0 = 0;
   if constexpr (Q == 4) h0 = reinterpret_cast<const uint32_t*>(image + kPlaneSlotBit0 + r * 16)[t];
+  // The top two bits of pair m of a word sit at bit 2m of both half-words.  Shifted up by Q - 2 places they stand
+  // where the leading bits of a Q-bit code belong when the unit of the fp16 constant is at bit 2(m mod 4) (see
+  // dq_field); the plane bits below them are moved to their places and merged, one instruction each.
+  constexpr int up = Q - 2;
 #pragma unroll
-  for (int i = 0; i < 2; ++i)
+  for (int i = 0; i < 2; ++i) {
+    const uint32_t lo4 = w[i] << up, hi4 = w[i] >> (8 - up);   // pairs 0 .. 3 / 4 .. 7 of the word at bits up + 2(m mod 4)
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
-      const int p = 8 * i + m;
-      constexpr int up = Q - 2;                    // the top two bits sit `up` places above bit 0 of the code
-      const uint32_t top = 2 * m >= up ? (w[i] >> (2 * m - up)) : (w[i] << (up - 2 * m));
-      uint32_t v = (top & (0x00030003u << up)) | 0x64006400u;
-      const uint32_t b1 = p >= up - 1 ? (h1 >> (p - (up - 1))) : (h1 << ((up - 1) - p));
-      v |= b1 & (0x00010001u << (up - 1));
-      if constexpr (Q == 4) v |= (h0 >> p) & 0x00010001u;
-      out[p] = dq_pair(v, s2, z2);
+      const int p = 8 * i + m;                     // pair index inside the quarter = bit of the plane words
+      const int U = 2 * (m & 3);                   // where the code's last bit goes
+      const uint32_t magic = (uint32_t)((25 - U) << 10) * 0x00010001u;
+      uint32_t v = and_or(m < 4 ? lo4 : hi4, (3u << (U + up)) * 0x00010001u, magic);
+      const int t1 = U + up - 1;
+      v = and_or(p >= t1 ? (h1 >> (p - t1)) : (h1 << (t1 - p)), (1u << t1) * 0x00010001u, v);
+      if constexpr (Q == 4) v = and_or(p >= U ? (h0 >> (p - U)) : (h0 << (U - p)), (1u << U) * 0x00010001u, v);
+      out[p] = dq_pair_k(v, magic, s2, z2);
     }
+  }
 }
 template <int Q>
 __device__ __forceinline__ void decode_half_planes(const char* image, int r, int h, __half2 s2, __half2 z2, __half2* out) {
