@@ -446,6 +446,10 @@ def run_gpu(args):
         pwbuild.build()
     replicas.barrier(device)
     peaks = measured_peaks()
+    if args.only == "prefill":
+        print(json.dumps({"metric": "prefill TFLOP/s", "data": "synthetic",
+                          "prefill": run_prefill(device, peaks, steps=min(args.steps, 20), warmup=3)}))
+        return
     cfg = synth.CONFIGS[args.config]
     if args.uniform_bits:
         import dataclasses
@@ -465,6 +469,11 @@ def run_gpu(args):
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize(device)
+    if args.only == "demote":
+        ms_alone = time_region(step, 30, device) / 30
+        print(json.dumps({"metric": "demote GB/s", "data": "synthetic",
+                          "demote": run_demote(ctx, cfg, layers, device, peaks, step, ms_alone)}))
+        return
     sampler = ClockSampler(device.index or 0)
     n0 = ctx.pw_launch_count()
     sampler.start()
@@ -915,6 +924,8 @@ def main():
                     help="diagnostic: give every routed block this bitwidth instead of the configured mix")
     ap.add_argument("--steady-seconds", type=float, default=0.6,
                     help="least duration of the steady-state region (0: just --steps steps, for profiler captures)")
+    ap.add_argument("--only", default="", choices=["", "prefill", "demote"],
+                    help="run one of the extra regions alone and print it (small commands for profiler captures)")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-extra", action="store_true")
     ap.add_argument("--skip-graph", action="store_true", help="leave out the CUDA-graph replay of the step")

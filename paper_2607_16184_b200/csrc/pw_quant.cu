@@ -121,6 +121,110 @@ __global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restri
   }
 }
 
+// 4 bits -> 2 bits without touching a weight.  A group has at most 16 distinct values, one per source code, and
+// the demote Q(D(.)) is a function of the code alone: minimum and maximum are the values of the smallest and the
+// largest code present, and new_code(c) = clamp(rint((D(c) - lo) / scale')) is non-decreasing in c.  So the four
+// lanes of a row-group evaluate it on the 16 codes (four each, the arithmetic of the general kernel, bit for
+// bit), turn the table into three thresholds t_k = number of source codes whose new code is below k, and every
+// code becomes [c >= t_1] + [c >= t_2] + [c >= t_3]: nibbles spread to bytes, one add of (128 - t_k) per
+// threshold puts the comparison into bit 7 of each byte, three logic operations make the two result bits.
+// About 7 instructions per weight instead of 17, and two conversions per weight fewer.
+__global__ void __launch_bounds__(512, 3) requant_4to2_kernel(const void* __restrict__ src_codes, uint32_t cols,
+                                                              void* __restrict__ dst_codes) {
+  const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
+  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
+  const size_t tile = (size_t)rt * ng + g;
+  const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_bytes(4);
+  const uint4 u = __ldg(reinterpret_cast<const uint4*>(tb + slice_word_offset<4>(r, q, 0)));
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+  const float s = __half2float(*reinterpret_cast<const __half*>(tb + tile_scale_offset(4, r)));
+  const float z = __half2float(*reinterpret_cast<const __half*>(tb + tile_zp_offset(4, r)));
+
+  // smallest and largest code of the group: a page written by the quantizer always uses 0 and 15 (the extremes
+  // of the group map to them), which two zero-nibble tests see; any other page takes the exact scan
+  uint32_t has0 = 0, has15 = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    has0 |= (w[i] - 0x11111111u) & ~w[i] & 0x88888888u;
+    has15 |= (~w[i] - 0x11111111u) & w[i] & 0x88888888u;
+  }
+  uint32_t flags = (has0 != 0 ? 1u : 0u) | (has15 != 0 ? 2u : 0u);
+  flags |= __shfl_xor_sync(0xffffffffu, flags, 1);
+  flags |= __shfl_xor_sync(0xffffffffu, flags, 2);
+  int cmin = 0, cmax = 15;
+  if (__any_sync(0xffffffffu, flags != 3u)) {
+    int code[32];
+    unpack_slice<4>(w, code);
+    int mn = code[0], mx = code[0];
+#pragma unroll
+    for (int i = 1; i < 32; ++i) {
+      mn = min(mn, code[i]);
+      mx = max(mx, code[i]);
+    }
+#pragma unroll
+    for (int d = 1; d <= 2; d <<= 1) {
+      mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    }
+    cmin = mn;
+    cmax = mx;
+  }
+
+  // scale and zero-point of the new page: the general quantizer's arithmetic on the two extreme values
+  constexpr int L = 3;
+  float lo = dequant_exact(cmin, s, z);
+  const float hi = dequant_exact(cmax, s, z);
+  if (lo == 0.0f) lo = 0.0f;  // store -0 as +0
+  const float rng = __fsub_rn(hi, lo);
+  __half sh;
+  if (rng == 0.0f) {
+    sh = __ushort_as_half((unsigned short)0x3c00);
+  } else {
+    sh = __float2half_rn(__fdiv_rn(rng, (float)L));
+    if ((__half_as_ushort(sh) & 0x7fff) == 0) sh = __ushort_as_half((unsigned short)0x0001);
+  }
+  const float rinv = __fdiv_rn(1.0f, __half2float(sh));
+
+  // my four entries of the code table -> per k, how many of them reach k (5 bits each)
+  uint32_t reach = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float v = dequant_exact(4 * q + j, s, z);
+    const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v, lo), rinv));
+    const uint32_t nc = c < (uint32_t)L ? c : (uint32_t)L;
+    reach += (nc >= 1u ? 1u : 0u) | (nc >= 2u ? 1u << 5 : 0u) | (nc >= 3u ? 1u << 10 : 0u);
+  }
+  reach += __shfl_xor_sync(0xffffffffu, reach, 1);
+  reach += __shfl_xor_sync(0xffffffffu, reach, 2);
+  // byte-wise x + (128 - t) has bit 7 set exactly when x >= t (x <= 15, 0 <= t <= 16: no carry between bytes)
+  const uint32_t k1 = (112u + (reach & 31u)) * 0x01010101u;            // 128 - t_1, t_1 = 16 - reach_1
+  const uint32_t k2 = (112u + ((reach >> 5) & 31u)) * 0x01010101u;
+  const uint32_t k3 = (112u + ((reach >> 10) & 31u)) * 0x01010101u;
+
+  uint32_t half_bytes[4];                          // per source word: 8 new codes, a byte in each half-word
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t zc[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {                  // nibbles 0, 2 of each half-word, then nibbles 1, 3
+      const uint32_t x = (e ? w[i] >> 4 : w[i]) & 0x0f0f0f0fu;
+      const uint32_t y1 = x + k1, y2 = x + k2, y3 = x + k3;
+      uint32_t b0;                                 // bit 7: (c >= t1 and not c >= t2) or c >= t3 = bit 0 of the count
+      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(y1), "r"(y2), "r"(y3));
+      zc[e] = and_or(b0 >> 7, 0x01010101u, (y2 >> 6) & 0x02020202u);   // new code in bits 0-1 of every byte
+    }
+    const uint32_t m = zc[0] | (zc[1] << 2);       // byte 0: pairs 0, 1; byte 1: pairs 2, 3 (4 bits used of each)
+    half_bytes[i] = (m | (m >> 4)) & 0x00ff00ffu;  // the four codes of a half-word in its low byte
+  }
+  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(2);
+  *reinterpret_cast<uint2*>(db + slice_word_offset<2>(r, q, 0)) =
+      make_uint2(half_bytes[0] | (half_bytes[1] << 8), half_bytes[2] | (half_bytes[3] << 8));
+  if (q == 0) {
+    *reinterpret_cast<__half*>(db + tile_scale_offset(2, r)) = sh;
+    *reinterpret_cast<__half*>(db + tile_zp_offset(2, r)) = __float2half_rn(lo);
+  }
+}
+
 // TILED -> CANONICAL (EXPORT = true) or CANONICAL -> TILED, same bitwidth.
 template <int BITS, bool EXPORT>
 __global__ void __launch_bounds__(512) relayout_kernel(const void* __restrict__ src_codes, uint32_t cols,
@@ -230,7 +334,8 @@ static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void
       if (SB > 3) quant_tile_kernel<SK, SB, (SB > 3 ? 3 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
     case 2:
-      quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SK == SRC_TILED && SB == 4) requant_4to2_kernel<<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      else quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       break;
   }
 }

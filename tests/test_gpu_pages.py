@@ -83,6 +83,32 @@ def test_demote_chain_16_4_2(ctx, orc):
     assert pages_equal(export_to_oracle(ctx, p2, orc), ref)
 
 
+def test_demote_4_to_2_of_pages_that_do_not_use_their_code_range(ctx, orc):
+    """A 4-bit page from elsewhere (imported) need not contain code 0 and code 15 in every group: the demote then
+    takes minimum and maximum from the codes that are present.  Groups of every kind side by side."""
+    rows, cols = 128, 1024
+    rng = np.random.default_rng(11)
+    codes = rng.integers(0, 16, (rows, cols), dtype=np.uint8)
+    codes[0:32, :] = rng.integers(3, 12, (32, cols))                 # neither extreme
+    codes[32:64, :] = rng.integers(0, 9, (32, cols))                 # no 15 (almost surely a 0)
+    codes[64:96, :] = rng.integers(5, 16, (32, cols))                # no 0
+    codes[96, :128] = 7                                              # a single level
+    codes[97, :128] = np.where(np.arange(128) % 2 == 0, 2, 13)       # two levels
+    scales = rng.uniform(1e-3, 2e-2, (rows, cols // 128)).astype(np.float16)
+    zps = rng.uniform(-0.2, 0.05, (rows, cols // 128)).astype(np.float16)
+    zps[98, 0] = np.float16(-0.0)
+    codes[98, :128] = rng.integers(0, 16, 128)
+    codes[98, 5] = 0
+    stream = np.packbits(np.unpackbits(codes.reshape(-1, 1), axis=1, bitorder="little")[:, :4].reshape(-1),
+                         bitorder="little")
+    ref4 = orc.Page(stream, scales.view(np.uint16).copy(), zps.view(np.uint16).copy(), rows, cols, 4)
+    assert np.array_equal(orc.unpack_codes(ref4), codes)
+    dev4 = import_from_oracle(ctx, ref4)
+    dev2 = ctx.pw_demote_block(dev4, 2)
+    torch.cuda.synchronize()
+    assert pages_equal(export_to_oracle(ctx, dev2, orc), orc.demote_block(ref4, 2))
+
+
 @pytest.mark.parametrize("bits", [16, 8, 4, 3, 2])
 def test_import_export_round_trip(ctx, orc, bits):
     cfg = synth.CONFIGS["tiny"]
