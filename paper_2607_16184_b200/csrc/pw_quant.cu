@@ -37,53 +37,63 @@ __device__ __forceinline__ void load_slice_words(const char* tb, int r, int q, u
   }
 }
 
-template <int SRC_KIND, int SRC_BITS, int DST_BITS>
-__global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restrict__ src_codes, uint32_t cols,
-                                                         void* __restrict__ dst_codes) {
-  const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
-  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
-  const size_t tile = (size_t)rt * ng + g;
-
-  float v[32];
-  __half2 h16[SRC_BITS == 16 ? 16 : 1];             // the packed halves of a 16-bit source
+// Words of my slice of tile (rt, g) of the source, as they lie in memory (an fp16 matrix or a tile image).
+template <int SRC_KIND, int SRC_BITS>
+__device__ __forceinline__ void load_source_slice(const void* __restrict__ src_codes, uint32_t cols, int rt, int g, int ng,
+                                                  int r, int q, uint32_t* raw) {
   if constexpr (SRC_KIND == SRC_RAW) {
     const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(src_codes) +
                                                     ((size_t)rt * kTileRows + r) * cols + (size_t)g * kGroup + 32 * q);
-    uint4 u[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) u[i] = __ldg(p + i);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const __half2* h = reinterpret_cast<const __half2*>(&u[i]);
+      const uint4 u = __ldg(p + i);
+      raw[4 * i] = u.x;
+      raw[4 * i + 1] = u.y;
+      raw[4 * i + 2] = u.z;
+      raw[4 * i + 3] = u.w;
+    }
+  } else {
+    const char* tb = reinterpret_cast<const char*>(src_codes) + ((size_t)rt * ng + g) * tile_bytes(SRC_BITS);
+    load_slice_words<SRC_BITS>(tb, r, q, raw);
+  }
+}
+
+// NT: tiles per CTA (group g and, NT == 2, group g + n_groups / 2 of the same row tile).  The loads of all of
+// them are issued before the first is worked on: twice the bytes in flight per thread, and the second tile's
+// latency is covered by the first one's arithmetic.
+template <int SRC_KIND, int SRC_BITS, int DST_BITS, int NT>
+__global__ void __launch_bounds__(512, NT == 2 ? 2 : 3) quant_tile_kernel(const void* __restrict__ src_codes, uint32_t cols,
+                                                                          void* __restrict__ dst_codes) {
+  const int rt = blockIdx.y, ng = gridDim.x * NT;
+  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
+  constexpr int NWS = SliceWords<SRC_BITS>::kWords;
+  uint32_t raw[NT][NWS];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float2 f = __half22float2(h[j]);
-        h16[4 * i + j] = h[j];
-        v[8 * i + 2 * j] = f.x;
-        v[8 * i + 2 * j + 1] = f.y;
-      }
+  for (int k = 0; k < NT; ++k)
+    load_source_slice<SRC_KIND, SRC_BITS>(src_codes, cols, rt, blockIdx.x + k * gridDim.x, ng, r, q, raw[k]);
+
+#pragma unroll
+  for (int k = 0; k < NT; ++k) {
+  const int g = blockIdx.x + k * gridDim.x;
+  const size_t tile = (size_t)rt * ng + g;
+  float v[32];
+  __half2 h16[SRC_BITS == 16 ? 16 : 1];             // the packed halves of a 16-bit source
+  if constexpr (SRC_BITS == 16) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      h16[i] = u32_as_h2(raw[k][i]);
+      const float2 f = __half22float2(h16[i]);
+      v[2 * i] = f.x;
+      v[2 * i + 1] = f.y;
     }
   } else {
     const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_bytes(SRC_BITS);
-    constexpr int NW = SliceWords<SRC_BITS>::kWords;
-    uint32_t w[NW];
-    load_slice_words<SRC_BITS>(tb, r, q, w);
-    if constexpr (SRC_BITS == 16) {
+    int code[32];
+    unpack_slice<SRC_BITS>(raw[k], code);
+    const float s = __half2float(*reinterpret_cast<const __half*>(tb + tile_scale_offset(SRC_BITS, r)));
+    const float z = __half2float(*reinterpret_cast<const __half*>(tb + tile_zp_offset(SRC_BITS, r)));
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        h16[i] = u32_as_h2(w[i]);
-        float2 f = __half22float2(h16[i]);
-        v[2 * i] = f.x;
-        v[2 * i + 1] = f.y;
-      }
-    } else {
-      int code[32];
-      unpack_slice<SRC_BITS>(w, code);
-      const float s = __half2float(*reinterpret_cast<const __half*>(tb + tile_scale_offset(SRC_BITS, r)));
-      const float z = __half2float(*reinterpret_cast<const __half*>(tb + tile_zp_offset(SRC_BITS, r)));
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = dequant_exact(code[i], s, z);
-    }
+    for (int i = 0; i < 32; ++i) v[i] = dequant_exact(code[i], s, z);
   }
 
   char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(DST_BITS);
@@ -96,9 +106,7 @@ __global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restri
       for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
       *reinterpret_cast<uint4*>(db + slice_word_offset<16>(r, q, 4 * i)) = o;
     }
-    return;
-  }
-
+  } else {
   int code[32];
   __half sh;
   float lo;
@@ -118,6 +126,8 @@ __global__ void __launch_bounds__(512, 3) quant_tile_kernel(const void* __restri
   if (q == 0) {
     *reinterpret_cast<__half*>(db + tile_scale_offset(DST_BITS, r)) = sh;
     *reinterpret_cast<__half*>(db + tile_zp_offset(DST_BITS, r)) = __float2half_rn(lo);
+  }
+  }
   }
 }
 
@@ -318,24 +328,33 @@ static pw_status check_page_buffers(const pw_page* p, int bits, int layout) {
   return PW_OK;
 }
 
+// 16-bit sources take two tiles per CTA when the block has an even number of groups.
+template <int SK, int SB, int DB>
+static void launch_quant(dim3 grid, cudaStream_t s, const void* sc, uint32_t cols, pw_page* d) {
+  if (SB == 16 && DB < 16 && grid.x % 2 == 0)
+    quant_tile_kernel<SK, SB, DB, (SB == 16 && DB < 16 ? 2 : 1)><<<dim3(grid.x / 2, grid.y), 512, 0, s>>>(sc, cols, d->codes);
+  else
+    quant_tile_kernel<SK, SB, DB, 1><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+}
+
 template <int SK, int SB>
 static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void* sc, uint32_t cols, pw_page* d) {
   switch (dst_bits) {
     case 16:
-      if (SK == SRC_RAW) quant_tile_kernel<SK, SB, 16><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SK == SRC_RAW) launch_quant<SK, SB, 16>(grid, s, sc, cols, d);
       break;
     case 8:
-      if (SB > 8) quant_tile_kernel<SK, SB, (SB > 8 ? 8 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SB > 8) launch_quant<SK, SB, (SB > 8 ? 8 : 2)>(grid, s, sc, cols, d);
       break;
     case 4:
-      if (SB > 4) quant_tile_kernel<SK, SB, (SB > 4 ? 4 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SB > 4) launch_quant<SK, SB, (SB > 4 ? 4 : 2)>(grid, s, sc, cols, d);
       break;
     case 3:
-      if (SB > 3) quant_tile_kernel<SK, SB, (SB > 3 ? 3 : 2)><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SB > 3) launch_quant<SK, SB, (SB > 3 ? 3 : 2)>(grid, s, sc, cols, d);
       break;
     case 2:
       if (SK == SRC_TILED && SB == 4) requant_4to2_kernel<<<grid, 512, 0, s>>>(sc, cols, d->codes);
-      else quant_tile_kernel<SK, SB, 2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      else launch_quant<SK, SB, 2>(grid, s, sc, cols, d);
       break;
   }
 }
