@@ -48,8 +48,11 @@ typedef enum {
 
 typedef enum { PW_GATE = 0, PW_UP = 1, PW_DOWN = 2 } pw_kind;
 
-/* Which expert-FFN kernel family pw_moe_forward uses.  AUTO is TENSOR: the tensor-core kernels are the
- * faster ones at every batch size, one token included. */
+/* Which expert-FFN kernel family pw_moe_forward uses.  The paper's runtime has one kernel and no such switch
+ * (Sec. 3.3); a caller leaves this at AUTO, which is TENSOR: the tensor-core kernels are the faster ones at
+ * every batch size, one token included, and they pick the decode or the prefill instantiation (token tiles of
+ * up to 64 or of 128) from the batch themselves.  SIMT is an independent second implementation kept for
+ * cross-checks; it does not read PW_LAYOUT_PLANES pages. */
 typedef enum {
   PW_MODE_AUTO = 0,
   PW_MODE_SIMT = 1,  /* CUDA-core kernel, thread per weight row: an independent second implementation */
@@ -122,8 +125,10 @@ typedef struct {
 /* Bytes of device workspace a context with this configuration needs (0 if cfg is invalid). */
 size_t pw_workspace_bytes(const pw_config* cfg);
 
-/* Creates a context on the current device.  cfg->workspace is zero-initialised
- * and the call returns after that has completed.
+/* Creates a context on the current device: the host object that holds the weight page table of Sec. 3.1 (one
+ * row per (layer, expert, kind), at first empty) and the offsets of the routing and operand buffers of
+ * Sec. 3.3 inside the caller's workspace.  cfg->workspace is zero-initialised and the call returns after that
+ * has completed.
  * Errors: INVALID_ARG, SHAPE, ALIGN, NOMEM (workspace too small), CUDA. */
 pw_status pw_create(pw_ctx** ctx, const pw_config* cfg);
 
@@ -159,9 +164,15 @@ pw_status pw_quantize_block(pw_ctx* ctx, const void* w_fp16, uint32_t rows, uint
  * pw_moe_forward runs on another.  Errors: INVALID_ARG, BITS, ALIGN, STATE (src not TILED). */
 pw_status pw_demote_block(pw_ctx* ctx, const pw_page* src, int dst_bits, pw_page* dst, pw_stream stream);
 
-/* Layout conversion, same bitwidth: TILED -> CANONICAL (export) and CANONICAL -> TILED (import).
- * dst buffers are caller-allocated, same sizes as src; the call fills dst's header fields.
- * Export is how pages are compared bit for bit and saved; import restores them. */
+/* Layout conversion, same bitwidth: TILED -> CANONICAL (export) and CANONICAL -> TILED (import).  What a page
+ * row holds is Sec. 3.1's: the codes of the block at its committed bitwidth and the state needed to decode them
+ * (here a scale and a zero-point per group); CANONICAL is that content in an order that does not depend on the
+ * kernels.  dst buffers are caller-allocated, same sizes as src; the call fills dst's header fields.
+ * Export is how pages are compared bit for bit and saved; import restores them.
+ * Shapes (every page-building call): cols must be a multiple of the group size, 128, as the format asks, and
+ * rows a multiple of 128 as well -- a TILED page is made of whole 128-row tiles (the MMA's M); the expert
+ * matrices of the model families of Table 1 all satisfy both.  Anything else: PW_ERR_SHAPE.
+ * Errors: INVALID_ARG, BITS, SHAPE, ALIGN, STATE (wrong source layout). */
 pw_status pw_export_page(pw_ctx* ctx, const pw_page* src_tiled, pw_page* dst_canonical, pw_stream stream);
 pw_status pw_import_page(pw_ctx* ctx, const pw_page* src_canonical, pw_page* dst_tiled, pw_stream stream);
 
@@ -280,7 +291,8 @@ pw_status pw_moe_forward(pw_ctx* ctx, int layer, const void* hidden_fp16, const 
 pw_status pw_moe_forward_host(pw_ctx* ctx, int layer, const void* hidden_host, const float* logits_host, int T,
                               int top_k, float* out_host, pw_mode mode, pw_stream stream);
 
-/* Copies the routing of the last forward call out of the workspace (device pointers, any may
+/* The routing decision of the last forward call (Sec. 2.1: top-k experts per token and their gates; Sec. 3.3:
+ * the grouping of the routed pairs by expert), copied out of the workspace (device pointers, any may
  * be NULL): topk_ids int32 [T, k], gates fp32 [T, k], counts int32 [E], offsets int32 [E+1],
  * perm int32 [T*k] (pair ids p = t*k + j sorted by expert, then by p). */
 pw_status pw_get_routing(pw_ctx* ctx, int32_t* topk_ids, float* gates, int32_t* counts, int32_t* offsets,
@@ -424,6 +436,8 @@ pw_status pw_plan_queue_peek(const pw_plan_queue* queue, int32_t stage, uint64_t
 
 /* Eq. 7: bytes to release = max(0, free_block_threshold + 1 - free_blocks) * kv_block_bytes. */
 uint64_t pw_kv_pressure_bytes(int64_t free_block_threshold, int64_t free_blocks, uint64_t kv_block_bytes);
+
+/* ---- measurement and test aids (no counterpart in the paper) ----------------------------- */
 
 /* Synchronises the device and returns the device status word (PW_OK, PW_ERR_TIMEOUT, ...),
  * then clears it. */

@@ -701,58 +701,22 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // all eight k-steps of it into its own partial accumulator; a quantized tile k is dequantized by the
     // matrix's group k mod IPM, so with npart == IPM every dequantizer group has an issuer of its own.
     // The epilogue adds the partials.
-    if constexpr (!HELP) {
     const int iss = warp - kWarpMma;
     const int my_m = iss / IPM, my_j = iss % IPM;
-    if (lane == 0 && my_j < npart) {
-      uint32_t seq_unit = 0;                        // slot items before the current unit
-      uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
-      uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
-      uint32_t ucount = 0;
-      // Accumulators: partial (m, j) of a unit sits at buffer base + (m * npart + j) * nb_rows.  A unit whose
-      // accumulators fit half of the accumulator columns takes one of two buffers in turn, so that its MMAs
-      // overlap the epilogue of the unit before it; a wider unit takes both.
-      uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
-      const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
-      const uint32_t b_lo_base = smem_u32(bslots) >> 4;
-      const uint32_t w_lo_base = smem_u32(wring) >> 4;
-      const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
-      const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
-      const uint32_t a_base = tmem + acol;
-      bool ok = true;
-      for (int i = 0; ok; ++i, ++ucount) {
-        const int u = next_unit<LIM>((uint32_t)i, c, status);
-        if (u < 0) break;
-        const Unit un = load_unit(units, u);
-        uint32_t ubits[NMAT];
-#pragma unroll
-        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
-        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
-        // slot items per group of the unit (W) and the offset of my matrix's inside a group
-        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
-        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
-        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
-        const int nb_rows = (un.ntok + 15) & ~15;
-        const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
-        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
-        const uint32_t b_step = (uint32_t)(2 * nb_rows);
-        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
-        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
-        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
-        uint32_t bt = base + j0;                     // token-tile number
-        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
-        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
-        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
-        const bool wide = NMAT * npart * nb_rows > acol / 2;
-        const uint32_t dbuf = wide ? 0u : dtoggle;
-        if (!wide) dtoggle ^= 1u;
-        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
-        // the epilogue has drained the buffer(s) this unit accumulates into
-        if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
-        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
-        if (!ok) break;
-        tc_fence_after();
+    const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
+    const uint32_t b_lo_base = smem_u32(bslots) >> 4;
+    const uint32_t w_lo_base = smem_u32(wring) >> 4;
+    const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
+    const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
+    const uint32_t a_base = tmem + acol;
+    const uint32_t a_lo_lbo = (2048u >> 4) << 16;                   // A descriptor (16-bit tiles): LBO 2048 B
+    // My tiles of one unit (every npart-th group from j0 on): token tile, operand (a 16-bit tile's two halves from
+    // the ring, or the operand slot of the group that dequantized the tile), eight MMAs, hand-backs.  One body for
+    // both instantiations of the issuer role below.
+    auto issue_tiles = [&](uint32_t j0, uint32_t ng, uint32_t base, uint32_t W, uint32_t my_bits, uint32_t d_t,
+                           uint32_t b_lo_unit, uint32_t b_step, uint32_t idesc, uint32_t& bt, RingPos& bp, uint32_t& sq,
+                           RingPos& rp, uint32_t& upar) -> bool {
+        bool ok = true;
         uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
 #pragma unroll 1
         for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
@@ -802,43 +766,18 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           bt += (uint32_t)npart;
           ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
         }
-        if (ok) {
-          if (wide || dbuf == 0) {
-            tc_commit(&c->d_full[0]);
-            ++duse0;
-          }
-          if (wide || dbuf == 1) {
-            tc_commit(&c->d_full[1]);
-            ++duse1;
-          }
-        }
-        base += ng;
-        seq_unit += ng * W;
-      }
-    }
-    } else {
-    const int iss = warp - kWarpMma;
-    const int my_m = iss / IPM, my_j = iss % IPM;
-    // Wide token tiles leave no room for a second accumulator buffer, so the epilogue of a unit is not
-    // overlapped: here the four issuer warps share it with the four epilogue warps (they take the upper
-    // half of the token columns of their lane quarter), lane 0 of the warps with an accumulator of their own
-    // issuing the unit's MMAs first.  Every lane tracks the per-unit state; only lane 0 uses the issuing part.
-    const bool issuing = my_j < npart;
-    const int hq = warp & 3;
-    const int hr = hq * 32 + lane;
-    const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
-    {
+        return ok;
+    };
+    if constexpr (!HELP) {
+    if (lane == 0 && my_j < npart) {
       uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
       uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
       uint32_t ucount = 0;
+      // Accumulators: partial (m, j) of a unit sits at buffer base + (m * npart + j) * nb_rows.  A unit whose
+      // accumulators fit half of the accumulator columns takes one of two buffers in turn, so that its MMAs
+      // overlap the epilogue of the unit before it; a wider unit takes both.
       uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
-      const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
-      const uint32_t b_lo_base = smem_u32(bslots) >> 4;
-      const uint32_t w_lo_base = smem_u32(wring) >> 4;
-      const uint32_t af_s = smem_u32(&c->a_full[0]), ae_s = smem_u32(&c->a_empty[0]);
-      const uint32_t bf_s = smem_u32(&c->b_full[0]), be_s = smem_u32(&c->b_empty[0]);
-      const uint32_t a_base = tmem + acol;
       bool ok = true;
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = next_unit<LIM>((uint32_t)i, c, status);
@@ -857,7 +796,69 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
         const uint32_t b_step = (uint32_t)(2 * nb_rows);
-        const uint32_t a_lo_lbo = (2048u >> 4) << 16;                 // A descriptor (16-bit tiles): LBO 2048 B
+        // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        uint32_t bt = base + j0;                     // token-tile number
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const uint32_t dbuf = wide ? 0u : dtoggle;
+        if (!wide) dtoggle ^= 1u;
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        // the epilogue has drained the buffer(s) this unit accumulates into
+        if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
+        if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
+        if (!ok) break;
+        tc_fence_after();
+        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
+        if (ok) {
+          if (wide || dbuf == 0) {
+            tc_commit(&c->d_full[0]);
+            ++duse0;
+          }
+          if (wide || dbuf == 1) {
+            tc_commit(&c->d_full[1]);
+            ++duse1;
+          }
+        }
+        base += ng;
+        seq_unit += ng * W;
+      }
+    }
+    } else {
+    // Wide token tiles leave no room for a second accumulator buffer, so the epilogue of a unit is not
+    // overlapped: here the four issuer warps share it with the four epilogue warps (they take the upper
+    // half of the token columns of their lane quarter), lane 0 of the warps with an accumulator of their own
+    // issuing the unit's MMAs first.  Every lane tracks the per-unit state; only lane 0 uses the issuing part.
+    const bool issuing = my_j < npart;
+    const int hq = warp & 3;
+    const int hr = hq * 32 + lane;
+    const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
+    {
+      uint32_t seq_unit = 0;                        // slot items before the current unit
+      uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
+      uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
+      uint32_t ucount = 0;
+      uint32_t dtoggle = 0, duse0 = 0, duse1 = 0;
+      bool ok = true;
+      for (int i = 0; ok; ++i, ++ucount) {
+        const int u = next_unit<LIM>((uint32_t)i, c, status);
+        if (u < 0) break;
+        const Unit un = load_unit(units, u);
+        uint32_t ubits[NMAT];
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+        const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
+        // slot items per group of the unit (W) and the offset of my matrix's inside a group
+        const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
+        const uint32_t my_off = my_m ? slot_items(ubits[0]) : 0u;
+        const uint32_t ng = (uint32_t)(un.g1 - un.g0);
+        const int nb_rows = (un.ntok + 15) & ~15;
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(nb_rows >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // B descriptor: leading byte offset = nb_rows * 16 (field at bit 16), advance 2 * nb_rows k-chunk units per k-step
+        const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
+        const uint32_t b_step = (uint32_t)(2 * nb_rows);
         // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
         const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
         uint32_t bt = base + j0;                     // token-tile number
@@ -875,55 +876,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         tc_fence_after();
-        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
-#pragma unroll 1
-        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
-          // the token tile of this group (a tile is looked at only once it is known to have been armed)
-          if (c->b_issued <= bt) {
-            ok = flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, c, status);
-            if (!ok) break;
-          }
-          ok = mbar_wait_s<LIM>(bf_s + 8 * bp.s, bp.par, c, status);
-          if (!ok) break;
-          const uint32_t b_lo = b_lo_unit + bp.s * (uint32_t)(bslot_bytes >> 4);
-          if (my_bits == 16) {
-            // each K-half lies in its own slot as a K-major core-matrix image (k-steps 0 .. 3, 4 KB apart)
-            RingPos hp = rp;
-#pragma unroll 1
-            for (uint32_t hh = 0; hh < 2; ++hh) {
-              ok = wait_issued<LIM>(sq + hh, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[hp.s]), hp.par, c, status);
-              if (!ok) break;
-              tc_fence_after();
-              const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
-              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
-              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
-              tc_commit(&c->empty[hp.s]);
-              ring_advance(hp, 1, (uint32_t)n_slots);
-            }
-            if (!ok) break;
-            sq += (uint32_t)npart * W;
-            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
-          } else {
-            // the group that dequantizes this tile, and the parity of this use of its operand slot
-            const uint32_t k = base + j;
-            const uint32_t grp = NMAT == 2 ? 2u * (uint32_t)my_m + (k & 1u) : (k & 3u);
-            const uint32_t use_par = (upar >> grp) & 1u;
-            upar ^= 1u << grp;
-            const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
-            const uint32_t a_t = a_base + grp * 64;
-            ok = mbar_wait_s<LIM>(f0, use_par, c, status);
-            if (!ok) break;
-            tc_fence_after();
-            // all eight k-steps of the tile, then one commit hands the group's operand slot back
-            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
-            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
-            tc_commit_s(e0);
-          }
-          tc_commit_s(be_s + 8 * bp.s);
-          later = 1;
-          bt += (uint32_t)npart;
-          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
-        }
+        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
             if (ok) {
               if (wide || dbuf == 0) tc_commit(&c->d_full[0]);
               if (wide || dbuf == 1) tc_commit(&c->d_full[1]);
