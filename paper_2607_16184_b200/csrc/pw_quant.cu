@@ -131,16 +131,18 @@ __global__ void __launch_bounds__(512, NT == 2 ? 2 : 3) quant_tile_kernel(const 
   }
 }
 
-// 4 bits -> 2 bits without touching a weight.  A group has at most 16 distinct values, one per source code, and
-// the demote Q(D(.)) is a function of the code alone: minimum and maximum are the values of the smallest and the
-// largest code present, and new_code(c) = clamp(rint((D(c) - lo) / scale')) is non-decreasing in c.  So the four
-// lanes of a row-group evaluate it on the 16 codes (four each, the arithmetic of the general kernel, bit for
-// bit), turn the table into three thresholds t_k = number of source codes whose new code is below k, and every
-// code becomes [c >= t_1] + [c >= t_2] + [c >= t_3]: nibbles spread to bytes, one add of (128 - t_k) per
-// threshold puts the comparison into bit 7 of each byte, three logic operations make the two result bits.
-// About 7 instructions per weight instead of 17, and two conversions per weight fewer.
-__global__ void __launch_bounds__(512, 3) requant_4to2_kernel(const void* __restrict__ src_codes, uint32_t cols,
-                                                              void* __restrict__ dst_codes) {
+// 4 bits -> 3 or 2 bits without touching a weight.  A group has at most 16 distinct values, one per source code,
+// and the demote Q(D(.)) is a function of the code alone: minimum and maximum are the values of the smallest and
+// the largest code present, and new_code(c) = clamp(rint((D(c) - lo) / scale')) is non-decreasing in c.  So the
+// four lanes of a row-group evaluate it on the 16 codes (four each, the arithmetic of the general kernel, bit for
+// bit), turn the table into L thresholds t_k = number of source codes whose new code is below k, and every code
+// becomes [c >= t_1] + .. + [c >= t_L]: nibbles spread to bytes, one add of (128 - t_k) per threshold puts the
+// comparison into bit 7 of each byte, and because the comparisons are nested a few three-input logic operations
+// give the bits of their count.  To 2 bits: about 10 instructions per weight instead of 17, and two conversions
+// per weight fewer.
+template <int DB>
+__global__ void __launch_bounds__(512, 3) requant_from4_kernel(const void* __restrict__ src_codes, uint32_t cols,
+                                                               void* __restrict__ dst_codes) {
   const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
   const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
   const size_t tile = (size_t)rt * ng + g;
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(512, 3) requant_4to2_kernel(const void* __rest
   }
 
   // scale and zero-point of the new page: the general quantizer's arithmetic on the two extreme values
-  constexpr int L = 3;
+  constexpr int L = (1 << DB) - 1;
   float lo = dequant_exact(cmin, s, z);
   const float hi = dequant_exact(cmax, s, z);
   if (lo == 0.0f) lo = 0.0f;  // store -0 as +0
@@ -195,43 +197,61 @@ __global__ void __launch_bounds__(512, 3) requant_4to2_kernel(const void* __rest
   }
   const float rinv = __fdiv_rn(1.0f, __half2float(sh));
 
-  // my four entries of the code table -> per k, how many of them reach k (5 bits each)
-  uint32_t reach = 0;
+  // my four entries of the code table -> per k, how many of them reach k (5 bits each: the sums stay <= 16)
+  unsigned long long reach = 0;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const float v = dequant_exact(4 * q + j, s, z);
     const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v, lo), rinv));
     const uint32_t nc = c < (uint32_t)L ? c : (uint32_t)L;
-    reach += (nc >= 1u ? 1u : 0u) | (nc >= 2u ? 1u << 5 : 0u) | (nc >= 3u ? 1u << 10 : 0u);
+#pragma unroll
+    for (int k = 1; k <= L; ++k) reach += (unsigned long long)(nc >= (uint32_t)k ? 1u : 0u) << (5 * (k - 1));
   }
   reach += __shfl_xor_sync(0xffffffffu, reach, 1);
   reach += __shfl_xor_sync(0xffffffffu, reach, 2);
   // byte-wise x + (128 - t) has bit 7 set exactly when x >= t (x <= 15, 0 <= t <= 16: no carry between bytes)
-  const uint32_t k1 = (112u + (reach & 31u)) * 0x01010101u;            // 128 - t_1, t_1 = 16 - reach_1
-  const uint32_t k2 = (112u + ((reach >> 5) & 31u)) * 0x01010101u;
-  const uint32_t k3 = (112u + ((reach >> 10) & 31u)) * 0x01010101u;
+  uint32_t kk[L];                                  // 128 - t_k in every byte, t_k = 16 - reach_k
+#pragma unroll
+  for (int k = 0; k < L; ++k) kk[k] = (112u + (uint32_t)((reach >> (5 * k)) & 31u)) * 0x01010101u;
 
-  uint32_t half_bytes[4];                          // per source word: 8 new codes, a byte in each half-word
+  uint32_t half_bytes[4];                          // per source word: the low two bits of 8 new codes, a byte in each half-word
+  uint32_t third = 0;                              // DB == 3: the plane of the third bits, bit P / 16 + P for pair P
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    uint32_t zc[2];
+    uint32_t zc[2], hv[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {                  // nibbles 0, 2 of each half-word, then nibbles 1, 3
       const uint32_t x = (e ? w[i] >> 4 : w[i]) & 0x0f0f0f0fu;
-      const uint32_t y1 = x + k1, y2 = x + k2, y3 = x + k3;
-      uint32_t b0;                                 // bit 7: (c >= t1 and not c >= t2) or c >= t3 = bit 0 of the count
-      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(y1), "r"(y2), "r"(y3));
-      zc[e] = and_or(b0 >> 7, 0x01010101u, (y2 >> 6) & 0x02020202u);   // new code in bits 0-1 of every byte
+      uint32_t y[L];
+#pragma unroll
+      for (int k = 0; k < L; ++k) y[k] = x + kk[k];
+      // the comparisons are nested (t_1 <= t_2 <= ..), so bit 0 of their count is ((y1 & ~y2) | y3) & ~y4 | .. and
+      // bit 1 is (y2 & ~y4) | y6, bit 2 is y4 -- all in bit 7 of every byte
+      uint32_t b0, b1;
+      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(y[0]), "r"(y[1]), "r"(y[2]));
+      if constexpr (DB == 3) {
+        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(y[3]), "r"(y[4]));
+        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(y[5]), "r"(y[6]));
+        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b1) : "r"(y[1]), "r"(y[3]), "r"(y[5]));
+        const uint32_t t = (y[3] >> 7) & 0x01010101u;
+        hv[e] = (t | (t >> 6)) & 0x00050005u;      // bits 0, 2 (16, 18): the pairs 0, 2 (e = 0) or 1, 3 of this word
+      } else {
+        b1 = y[1];
+        hv[e] = 0;
+      }
+      zc[e] = and_or(b0 >> 7, 0x01010101u, (b1 >> 6) & 0x02020202u);   // low two bits of the new code in every byte
     }
     const uint32_t m = zc[0] | (zc[1] << 2);       // byte 0: pairs 0, 1; byte 1: pairs 2, 3 (4 bits used of each)
     half_bytes[i] = (m | (m >> 4)) & 0x00ff00ffu;  // the four codes of a half-word in its low byte
+    if constexpr (DB == 3) third |= (hv[0] | (hv[1] << 1)) << (4 * i);
   }
-  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(2);
-  *reinterpret_cast<uint2*>(db + slice_word_offset<2>(r, q, 0)) =
+  char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(DB);
+  *reinterpret_cast<uint2*>(db + slice_word_offset<DB>(r, q, 0)) =
       make_uint2(half_bytes[0] | (half_bytes[1] << 8), half_bytes[2] | (half_bytes[3] << 8));
+  if constexpr (DB == 3) *reinterpret_cast<uint32_t*>(db + slice_word_offset<3>(r, q, 2)) = third;
   if (q == 0) {
-    *reinterpret_cast<__half*>(db + tile_scale_offset(2, r)) = sh;
-    *reinterpret_cast<__half*>(db + tile_zp_offset(2, r)) = __float2half_rn(lo);
+    *reinterpret_cast<__half*>(db + tile_scale_offset(DB, r)) = sh;
+    *reinterpret_cast<__half*>(db + tile_zp_offset(DB, r)) = __float2half_rn(lo);
   }
 }
 
@@ -350,10 +370,11 @@ static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void
       if (SB > 4) launch_quant<SK, SB, (SB > 4 ? 4 : 2)>(grid, s, sc, cols, d);
       break;
     case 3:
-      if (SB > 3) launch_quant<SK, SB, (SB > 3 ? 3 : 2)>(grid, s, sc, cols, d);
+      if (SK == SRC_TILED && SB == 4) requant_from4_kernel<3><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      else if (SB > 3) launch_quant<SK, SB, (SB > 3 ? 3 : 2)>(grid, s, sc, cols, d);
       break;
     case 2:
-      if (SK == SRC_TILED && SB == 4) requant_4to2_kernel<<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SK == SRC_TILED && SB == 4) requant_from4_kernel<2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
       else launch_quant<SK, SB, 2>(grid, s, sc, cols, d);
       break;
   }

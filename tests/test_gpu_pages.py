@@ -83,7 +83,8 @@ def test_demote_chain_16_4_2(ctx, orc):
     assert pages_equal(export_to_oracle(ctx, p2, orc), ref)
 
 
-def test_demote_4_to_2_of_pages_that_do_not_use_their_code_range(ctx, orc):
+@pytest.mark.parametrize("dst", [3, 2])
+def test_demote_from_4_bits_of_pages_that_do_not_use_their_code_range(ctx, orc, dst):
     """A 4-bit page from elsewhere (imported) need not contain code 0 and code 15 in every group: the demote then
     takes minimum and maximum from the codes that are present.  Groups of every kind side by side."""
     rows, cols = 128, 1024
@@ -104,9 +105,9 @@ def test_demote_4_to_2_of_pages_that_do_not_use_their_code_range(ctx, orc):
     ref4 = orc.Page(stream, scales.view(np.uint16).copy(), zps.view(np.uint16).copy(), rows, cols, 4)
     assert np.array_equal(orc.unpack_codes(ref4), codes)
     dev4 = import_from_oracle(ctx, ref4)
-    dev2 = ctx.pw_demote_block(dev4, 2)
+    low = ctx.pw_demote_block(dev4, dst)
     torch.cuda.synchronize()
-    assert pages_equal(export_to_oracle(ctx, dev2, orc), orc.demote_block(ref4, 2))
+    assert pages_equal(export_to_oracle(ctx, low, orc), orc.demote_block(ref4, dst))
 
 
 @pytest.mark.parametrize("bits", [16, 8, 4, 3, 2])
