@@ -77,3 +77,47 @@ def test_two_step_descent_releases_the_sum_of_the_steps(res):
         row.transfer_done(upper)
     assert start - row.gpu_bytes() == (M[16] - M[4]) + (M[4] - M[2]) == M[16] - M[2]
     assert sorted(b for b, s in row.state.items() if s == res.CPU) == [4, 16]
+
+
+def test_planes_leave_above_the_committed_precision_and_return_before_it_is_raised(res):
+    # a 14336 x 4096 block: a plane is one bit of every weight = 7,340,032 bytes; the leading planes with the
+    # table states of the three bitwidths are 3584 tiles x 5632 bytes
+    plane, top = 14336 * 4096 // 8, (14336 // 128) * (4096 // 128) * 5632
+    assert (plane, top) == (7340032, 20185088)
+    M = size_table()
+    row = res.PlaneRow(top, plane)
+    row.commit(4)
+    for p in (3, 4):
+        with pytest.raises(res.IllegalTransition):
+            row.offload(p)                            # q_i = 4 reads both planes
+    row.commit(3)                                     # lower q_i first ...
+    with pytest.raises(res.IllegalTransition):
+        row.offload(3)
+    row.offload(4)                                    # ... then the plane it no longer reads moves out
+    with pytest.raises(res.IllegalTransition):
+        row.commit(4)                                 # on its way out
+    assert row.gpu_bytes() == top + 2 * plane         # its buffer still exists
+    row.transfer_done(4)
+    assert row.gpu_bytes() == top + plane
+    row.commit(2)
+    row.offload(3)
+    row.transfer_done(3)
+    # Eq. 3 on the size table: 4 -> 2 bits releases M^4 - M^2 = two planes (the table state is the same size)
+    assert 2 * plane == M[4] - M[2] == 31195136 - 16515072
+    with pytest.raises(res.IllegalTransition):
+        row.commit(3)                                 # CPU-resident
+    with pytest.raises(res.IllegalTransition):
+        row.transfer_done(3)                          # no transfer in flight
+    row.reload(3)
+    with pytest.raises(res.IllegalTransition):
+        row.commit(3)                                 # still in transfer
+    row.transfer_done(3)
+    row.commit(3)
+    with pytest.raises(res.IllegalTransition):
+        row.commit(4)                                 # plane 4 is still away
+    row.reload(4)
+    row.transfer_done(4)
+    row.commit(4)
+    assert row.committed == 4 and row.gpu_bytes() == top + 2 * plane
+    with pytest.raises(res.IllegalTransition):
+        row.commit(5)
