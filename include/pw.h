@@ -267,6 +267,30 @@ pw_status pw_reload_page(pw_ctx* ctx, int layer, int expert, int kind, int bits,
 pw_status pw_page_state(pw_ctx* ctx, int layer, int expert, int kind, int bits, int* state_out);
 pw_status pw_drop_page(pw_ctx* ctx, int layer, int expert, int kind, int bits);
 
+/* The same for a row that holds a block of overlaid bit-planes (PW_LAYOUT_PLANES), the paper's own case
+ * (Sec. 2.2, Sec. 3.1): the unit of movement is a plane.  Plane 3 (the BIT1 buffer, at `scales` of the block's
+ * header) is what reading at 3 bits adds to reading at 2 bits, plane 4 (BIT0, at `zps`) what 4 bits add to 3;
+ * the leading planes (TOP) hold the table state of every bitwidth and never leave.  The two ordering rules,
+ * checked on the host before anything is enqueued:
+ *   - offload: a plane that the committed bitwidth of the row reads cannot leave (STATE) -- publish the block
+ *     at a lower bitwidth first;
+ *   - reload: pw_set_page_table refuses (STATE) a bitwidth that reads a plane which is CPU_RESIDENT or
+ *     IN_TRANSFER, and accepts it once pw_plane_state reports GPU_RESIDENT (give the header the address the
+ *     plane was reloaded to).
+ * A plane is one buffer of `bit_bytes` (pw_plane_bytes), so each direction is one asynchronous copy on `stream`.
+ * pw_offload_plane: block = the block's header (layout PLANES; only rows, cols and the plane's pointer are
+ * used), plane = 3 or 4, host_dst = bit_bytes of (pinned) host memory.  The device buffer may be released once
+ * pw_plane_state reports CPU_RESIDENT and every forward call enqueued before the commit that lowered the
+ * bitwidth has finished.  Lowering the precision by q -> q' bits thus releases (q - q') * rows * cols / 8 bytes
+ * of GPU memory (Eq. 3).
+ * pw_reload_plane: host_src = the buffer the plane was offloaded to, dev_dst = bit_bytes of device memory.
+ * Errors: INVALID_ARG (also: not the buffer of the offload), BITS (plane not 3 or 4), SHAPE, ALIGN, STATE, CUDA. */
+pw_status pw_offload_plane(pw_ctx* ctx, int layer, int expert, int kind, const pw_page* block, int plane,
+                           void* host_dst, pw_stream stream);
+pw_status pw_reload_plane(pw_ctx* ctx, int layer, int expert, int kind, int plane, const void* host_src, void* dev_dst,
+                          pw_stream stream);
+pw_status pw_plane_state(pw_ctx* ctx, int layer, int expert, int kind, int plane, int* state_out);
+
 /* ---- forward ------------------------------------------------------------------------ */
 
 /* One MoE layer (Sec. 2.1, Sec. 3.3): top_k routing of T tokens over the E routed experts

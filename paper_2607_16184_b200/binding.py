@@ -28,6 +28,7 @@ GROUP = 128
 EXPORTS = ("pw_workspace_bytes", "pw_create", "pw_destroy", "pw_page_bytes", "pw_quantize_block", "pw_demote_block",
            "pw_export_page", "pw_import_page", "pw_plane_bytes", "pw_quantize_planes", "pw_export_planes", "pw_set_page_table", "pw_get_page_table", "pw_query_row",
            "pw_offload_page", "pw_reload_page", "pw_page_state", "pw_drop_page",
+           "pw_offload_plane", "pw_reload_plane", "pw_plane_state",
            "pw_moe_forward", "pw_moe_forward_host", "pw_get_routing", "pw_route_tokens_static", "pw_observe", "pw_observation_summary", "pw_plan_step", "pw_plan_queue_create", "pw_plan_queue_destroy", "pw_plan_queue_step", "pw_plan_queue_peek", "pw_kv_pressure_bytes",
            "pw_last_device_status",
            "pw_kernel_timing", "pw_get_kernel_times", "pw_launch_count", "pw_debug_set_wait", "pw_status_str")
@@ -114,6 +115,12 @@ def load():
     L.pw_page_state.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_int)]
     L.pw_drop_page.restype = i32
     L.pw_drop_page.argtypes = [vp, i32, i32, i32, i32]
+    L.pw_offload_plane.restype = i32
+    L.pw_offload_plane.argtypes = [vp, i32, i32, i32, C.POINTER(pw_page), i32, vp, vp]
+    L.pw_reload_plane.restype = i32
+    L.pw_reload_plane.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp]
+    L.pw_plane_state.restype = i32
+    L.pw_plane_state.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_int)]
     L.pw_moe_forward.restype = i32
     L.pw_moe_forward.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp]
     L.pw_moe_forward_host.restype = i32
@@ -486,6 +493,28 @@ class Context:
 
     def pw_drop_page(self, layer: int, expert: int, kind: int, bits: int):
         _check(self.L.pw_drop_page(self.handle, layer, expert, kind, bits), "pw_drop_page")
+
+    def pw_offload_plane(self, layer: int, expert: int, kind: int, block: "PlanePage", plane: int,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Starts the copy of plane 3 (BIT1) or 4 (BIT0) of a bit-plane block to pinned host memory; returns it."""
+        _, _, bb = pw_plane_bytes(block.rows, block.cols)
+        host = torch.empty(bb, dtype=torch.uint8).pin_memory()
+        _check(self.L.pw_offload_plane(self.handle, layer, expert, kind, C.byref(block.c), plane, host.data_ptr(),
+                                       _stream_ptr(stream)), "pw_offload_plane")
+        return host
+
+    def pw_reload_plane(self, layer: int, expert: int, kind: int, plane: int, host: torch.Tensor,
+                        stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """Starts the copy of an offloaded plane back into a fresh device buffer; returns the buffer."""
+        dst = torch.empty(host.numel(), dtype=torch.uint8, device=self.device)
+        _check(self.L.pw_reload_plane(self.handle, layer, expert, kind, plane, host.data_ptr(), dst.data_ptr(),
+                                      _stream_ptr(stream)), "pw_reload_plane")
+        return dst
+
+    def pw_plane_state(self, layer: int, expert: int, kind: int, plane: int) -> int:
+        st = C.c_int()
+        _check(self.L.pw_plane_state(self.handle, layer, expert, kind, plane, C.byref(st)), "pw_plane_state")
+        return int(st.value)
 
     # ---- forward ----
     def pw_moe_forward(self, layer: int, hidden: torch.Tensor, router_logits: torch.Tensor, top_k: int,

@@ -192,10 +192,9 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
     if (e.expert >= c.n_experts && (p.bits != 16 || planes)) return PW_ERR_STATE;
     if (e.desired_bits != 0 && !bits_ok(e.desired_bits)) return PW_ERR_BITS;
     // q_i is only set to a bitwidth whose page is GPU-resident (Sec. 3.1): not while it is away or on its way
-    if (!planes) {
-      const pw_status rs = residency_check_commit(ctx, row_index(ctx, e.layer, e.expert, e.kind), p);
-      if (rs != PW_OK) return rs;
-    }
+    const size_t ridx = row_index(ctx, e.layer, e.expert, e.kind);
+    const pw_status rs = planes ? residency_check_commit_planes(ctx, ridx, p) : residency_check_commit(ctx, ridx, p);
+    if (rs != PW_OK) return rs;
   }
   // The rows travel in the parameter space of a small kernel, 64 at a time: the update is ordered on the
   // stream like any kernel and never queues behind a large copy on a DMA engine (a page being reloaded on a
@@ -224,6 +223,7 @@ extern "C" pw_status pw_set_page_table(pw_ctx* ctx, const pw_table_entry* entrie
       ctx->host_rows[idx] = e;
       ctx->host_valid[idx] = 1;
       if (e.page.layout != PW_LAYOUT_PLANES) residency_note_commit(ctx, idx, e.page);
+      else residency_note_commit_planes(ctx, idx, e.page);
     }
     commit_rows_kernel<<<1, kCommitBatch, 0, stream>>>(batch, dtab);
     ctx->launches++;

@@ -86,7 +86,7 @@ namespace pw {
 // Residency record of the page of one page-table row at one bitwidth (Sec. 3.1: GPU-resident, CPU-resident
 // or in transfer).  A transfer is a copy enqueued on a stream plus an event behind it; the record moves on
 // to `heading` when a later call finds the event complete.
-constexpr int kBitLevels = 5;                      // 16, 8, 4, 3, 2
+constexpr int kBitLevels = 7;                      // pages at 16, 8, 4, 3, 2 bits; planes 3 and 4 of a bit-plane block
 struct PageRecord {
   uint8_t state;        // PW_STATE_*
   uint8_t heading;      // state the page reaches when its transfer has finished
@@ -95,6 +95,8 @@ struct PageRecord {
   cudaEvent_t ev;       // created on first use
 };
 inline int bit_level(int bits) { return bits == 16 ? 0 : bits == 8 ? 1 : bits == 4 ? 2 : bits == 3 ? 3 : bits == 2 ? 4 : -1; }
+// record of the plane that reading at `plane` bits adds to reading at plane - 1 bits (3: BIT1, 4: BIT0)
+inline int plane_level(int plane) { return plane == 3 ? 5 : plane == 4 ? 6 : -1; }
 }  // namespace pw
 
 struct pw_ctx {
@@ -149,6 +151,9 @@ int residency_poll(pw_ctx* ctx, size_t row, int bits);
 pw_status residency_check_commit(pw_ctx* ctx, size_t row, const pw_page& page);
 void residency_note_commit(pw_ctx* ctx, size_t row, const pw_page& page);
 void residency_teardown(pw_ctx* ctx);
+// the same for a row that is committed to a block of bit-planes read at page.bits: the planes 3 .. bits
+pw_status residency_check_commit_planes(pw_ctx* ctx, size_t row, const pw_page& page);
+void residency_note_commit_planes(pw_ctx* ctx, size_t row, const pw_page& page);
 pw_status launch_ffn_simt(pw_ctx* ctx, int layer, int T, int k, cudaStream_t s);
 pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, int ksplit, cudaStream_t s);
 int tensor_token_tile(const pw_ctx* ctx, int T, int k);

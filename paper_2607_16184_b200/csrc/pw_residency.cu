@@ -36,6 +36,32 @@ void residency_note_commit(pw_ctx* ctx, size_t row, const pw_page& page) {
   r->dev = page.codes;
 }
 
+static int poll_record(PageRecord* r) {
+  if (r->state == PW_STATE_IN_TRANSFER && r->ev && cudaEventQuery(r->ev) == cudaSuccess) {
+    r->state = r->heading;
+    if (r->state == PW_STATE_CPU_RESIDENT) r->dev = nullptr;
+  }
+  return r->state;
+}
+
+// A block of bit-planes read at q bits needs the planes 3 .. q on the GPU (Sec. 3.1: the bitwidth is raised only
+// once the planes it reads are back).
+pw_status residency_check_commit_planes(pw_ctx* ctx, size_t row, const pw_page& page) {
+  for (int p = 3; p <= page.bits; ++p) {
+    const int st = poll_record(&ctx->records[row * kBitLevels + plane_level(p)]);
+    if (st == PW_STATE_IN_TRANSFER || st == PW_STATE_CPU_RESIDENT) return PW_ERR_STATE;
+  }
+  return PW_OK;
+}
+
+void residency_note_commit_planes(pw_ctx* ctx, size_t row, const pw_page& page) {
+  for (int p = 3; p <= page.bits; ++p) {
+    PageRecord* r = &ctx->records[row * kBitLevels + plane_level(p)];
+    r->state = PW_STATE_GPU_RESIDENT;
+    r->dev = p == 3 ? page.scales : page.zps;
+  }
+}
+
 void residency_teardown(pw_ctx* ctx) {
   if (!ctx->records) return;
   for (size_t i = 0; i < ctx->n_rows * kBitLevels; ++i)
@@ -136,5 +162,73 @@ extern "C" pw_status pw_page_state(pw_ctx* ctx, int layer, int expert, int kind,
     return PW_ERR_INVALID_ARG;
   if (bit_level(bits) < 0) return PW_ERR_BITS;
   *state_out = residency_poll(ctx, row_index(ctx, layer, expert, kind), bits);
+  return PW_OK;
+}
+
+// ---- planes of a bit-plane block ---------------------------------------------------------------
+
+static pw_status check_plane_args(const pw_ctx* ctx, int layer, int expert, int kind, int plane) {
+  if (layer < 0 || layer >= ctx->cfg.n_layers || expert < 0 || expert >= ctx->ws.S || kind < 0 || kind > 2)
+    return PW_ERR_INVALID_ARG;
+  return plane_level(plane) < 0 ? PW_ERR_BITS : PW_OK;
+}
+
+extern "C" pw_status pw_offload_plane(pw_ctx* ctx, int layer, int expert, int kind, const pw_page* block, int plane,
+                                      void* host_dst, pw_stream stream) {
+  if (!ctx || !block || !host_dst) return PW_ERR_INVALID_ARG;
+  pw_status st = check_plane_args(ctx, layer, expert, kind, plane);
+  if (st != PW_OK) return st;
+  if (block->layout != PW_LAYOUT_PLANES || block->group != kGroup) return PW_ERR_STATE;
+  const pw_config& c = ctx->cfg;
+  const uint32_t er = kind == PW_DOWN ? c.hidden : c.ffn, ec = kind == PW_DOWN ? c.ffn : c.hidden;
+  if (block->rows != er || block->cols != ec) return PW_ERR_SHAPE;
+  void* dev = plane == 3 ? block->scales : block->zps;
+  if (!dev) return PW_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dev) & 15) return PW_ERR_ALIGN;
+  const size_t row = row_index(ctx, layer, expert, kind);
+  // the committed bitwidth is lowered first, then the plane it no longer reads moves out
+  const pw_page& cur = ctx->host_rows[row].page;
+  if (ctx->host_valid[row] && cur.layout == PW_LAYOUT_PLANES && cur.bits >= plane) return PW_ERR_STATE;
+  PageRecord* r = &ctx->records[row * kBitLevels + plane_level(plane)];
+  const int now = poll_record(r);
+  if (now == PW_STATE_IN_TRANSFER || now == PW_STATE_CPU_RESIDENT) return PW_ERR_STATE;
+  size_t bit_bytes = 0;
+  pw_plane_bytes(block->rows, block->cols, nullptr, &bit_bytes);
+  st = start_transfer(r, host_dst, dev, bit_bytes, cudaMemcpyDeviceToHost, stream);
+  if (st != PW_OK) return st;
+  r->state = PW_STATE_IN_TRANSFER;
+  r->heading = PW_STATE_CPU_RESIDENT;
+  r->dev = dev;
+  r->host = host_dst;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_reload_plane(pw_ctx* ctx, int layer, int expert, int kind, int plane, const void* host_src,
+                                     void* dev_dst, pw_stream stream) {
+  if (!ctx || !host_src || !dev_dst) return PW_ERR_INVALID_ARG;
+  pw_status st = check_plane_args(ctx, layer, expert, kind, plane);
+  if (st != PW_OK) return st;
+  if (reinterpret_cast<uintptr_t>(dev_dst) & 15) return PW_ERR_ALIGN;
+  const size_t row = row_index(ctx, layer, expert, kind);
+  PageRecord* r = &ctx->records[row * kBitLevels + plane_level(plane)];
+  if (poll_record(r) != PW_STATE_CPU_RESIDENT) return PW_ERR_STATE;
+  if (r->host != host_src) return PW_ERR_INVALID_ARG;     // not the buffer this plane was offloaded to
+  const pw_config& c = ctx->cfg;
+  size_t bit_bytes = 0;
+  pw_plane_bytes(kind == PW_DOWN ? c.hidden : c.ffn, kind == PW_DOWN ? c.ffn : c.hidden, nullptr, &bit_bytes);
+  st = start_transfer(r, dev_dst, host_src, bit_bytes, cudaMemcpyHostToDevice, stream);
+  if (st != PW_OK) return st;
+  r->state = PW_STATE_IN_TRANSFER;
+  r->heading = PW_STATE_GPU_RESIDENT;
+  r->dev = dev_dst;
+  return PW_OK;
+}
+
+extern "C" pw_status pw_plane_state(pw_ctx* ctx, int layer, int expert, int kind, int plane, int* state_out) {
+  if (!ctx || !state_out) return PW_ERR_INVALID_ARG;
+  const pw_status st = check_plane_args(ctx, layer, expert, kind, plane);
+  if (st != PW_OK) return st;
+  PageRecord* r = &ctx->records[row_index(ctx, layer, expert, kind) * kBitLevels + plane_level(plane)];
+  *state_out = poll_record(r);
   return PW_OK;
 }

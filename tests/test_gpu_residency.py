@@ -125,3 +125,103 @@ def test_argument_errors_enqueue_nothing():
         assert ctx.pw_launch_count() == n0
     finally:
         ctx.close()
+
+
+def test_planes_leave_and_return_following_the_oracle():
+    """A row that holds overlaid bit-planes: the precision is lowered by publishing the same buffers at fewer
+    bits, the planes above it move to host memory, and come back before the precision is raised again."""
+    from oracle import oracle as orc
+    from oracle import planes as PL
+    from oracle import residency as R
+    cfg = synth.LayerConfig("planes_res", 4, 2, 256, 512, 24, routing="normal")
+    ctx = make_ctx(cfg, n_layers=1)
+    try:
+        blocks, refs, entries = [], [], []
+        for e in range(cfg.n_experts):
+            for u in range(3):
+                w = synth.block_weights(cfg, 0, e, u, device="cuda")
+                blk = ctx.pw_quantize_planes(w)
+                blocks.append(blk)
+                refs.append(PL.quantize_planes(w.cpu().numpy()))
+                entries.append((0, e, u, blk.at(4)))
+        ctx.pw_set_page_table(entries)
+        e, u = 1, B.PW_UP
+        row, blk = (0, e, u), blocks[e * 3 + u]
+        _, top_bytes, bit_bytes = B.pw_plane_bytes(blk.rows, blk.cols)
+        orow = R.PlaneRow(top_bytes, bit_bytes)
+        orow.commit(4)
+        x = synth.activations(cfg, device="cuda")
+        lg = synth.router_logits(cfg, device="cuda")
+
+        def forward_matches(q):
+            views = [PL.view(r, q if i == e * 3 + u else 4) for i, r in enumerate(refs)]
+            out = ctx.pw_moe_forward(0, x, lg, cfg.top_k)
+            ref = orc.moe_forward(x.cpu().numpy(), lg.cpu().numpy(), cfg.top_k, views)
+            d = out.cpu().numpy().astype(np.float64) - ref
+            assert np.abs(d).max() <= 2e-2 and np.linalg.norm(d) / np.linalg.norm(ref) <= 5e-3
+            return out.clone()
+
+        def same_states():
+            for p in (3, 4):
+                assert ctx.pw_plane_state(*row, p) == orow.state[p]
+
+        out4 = forward_matches(4)
+        same_states()
+        for p in (3, 4):                                            # q_i = 4 reads both planes
+            expect(STATE_ERR, ctx.pw_offload_plane, *row, blk, p)
+            with pytest.raises(R.IllegalTransition):
+                orow.offload(p)
+        # lower to 2 bits (a new header, no kernel), then both planes move out on a side stream
+        ctx.pw_set_page_table([(0, e, u, blk.at(2))])
+        orow.commit(2)
+        forward_matches(2)
+        image1, image0 = blk.bit1.clone(), blk.bit0.clone()
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            torch.cuda._sleep(200_000_000)                          # ~0.1 s: the copies behind it cannot have finished
+            host1 = ctx.pw_offload_plane(*row, blk, 3, stream=side)
+            host0 = ctx.pw_offload_plane(*row, blk, 4, stream=side)
+        orow.offload(3)
+        orow.offload(4)
+        same_states()                                               # in transfer
+        expect(STATE_ERR, ctx.pw_set_page_table, [(0, e, u, blk.at(3))])
+        with pytest.raises(R.IllegalTransition):
+            orow.commit(3)
+        side.synchronize()
+        orow.transfer_done(3)
+        orow.transfer_done(4)
+        same_states()                                               # CPU-resident
+        assert orow.gpu_bytes() == top_bytes
+        assert torch.equal(host1, image1.cpu()) and torch.equal(host0, image0.cpu())
+        blk.bit1.fill_(0xEE)                                        # the device buffers are released (here: trashed)
+        blk.bit0.fill_(0xEE)
+        forward_matches(2)                                          # the 2-bit view does not touch them
+        expect(STATE_ERR, ctx.pw_set_page_table, [(0, e, u, blk.at(3))])
+        expect(STATE_ERR, ctx.pw_offload_plane, *row, blk, 3)       # already away
+        expect(ARG_ERR, ctx.pw_reload_plane, *row, 3, host0)        # not the buffer plane 3 went to
+        # raise to 3 bits: plane 3 comes back first
+        new1 = ctx.pw_reload_plane(*row, 3, host1, stream=side)
+        orow.reload(3)
+        side.synchronize()
+        orow.transfer_done(3)
+        same_states()
+        back = B.PlanePage(blk.rows, blk.cols, _buffers=(blk.top, new1, blk.bit0), bits=3)
+        ctx.pw_set_page_table([(0, e, u, back)])
+        orow.commit(3)
+        forward_matches(3)
+        expect(STATE_ERR, ctx.pw_set_page_table, [(0, e, u, back.at(4))])   # plane 4 is still on the host
+        new0 = ctx.pw_reload_plane(*row, 4, host0, stream=side)
+        orow.reload(4)
+        side.synchronize()
+        orow.transfer_done(4)
+        full = B.PlanePage(blk.rows, blk.cols, _buffers=(blk.top, new1, new0), bits=4)
+        ctx.pw_set_page_table([(0, e, u, full)])
+        orow.commit(4)
+        same_states()
+        assert torch.equal(new1, image1) and torch.equal(new0, image0)
+        assert torch.equal(forward_matches(4), out4)                # the bits of the first call
+        assert orow.gpu_bytes() == top_bytes + 2 * bit_bytes
+        assert ctx.pw_last_device_status() == 0
+    finally:
+        ctx.close()
