@@ -20,7 +20,8 @@
 //                it to its issuer once per tile, while it decodes the first half of its next tile in registers;
 //   warps 16,18  weight producers: producer P arms the slot items with number = P mod 2 (which sit in the
 //                slots = P mod 2) and issues their copies, as far ahead as the ring allows; producer 0 also
-//                claims the CTA's units from a global counter and posts them on the CTA's work list;
+//                claims the CTA's units from a global counter and posts them (the unit and the bitwidths of its
+//                pages) on the CTA's work list in shared memory, the only place the other roles learn of them;
 //   warp 17      token-tile producer (its own few slots, never holds back the weight stream);
 //   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  A tcgen05.mma holds its issuing
 //                thread for ~100 cycles whatever its size, so the issuers work in parallel: issuer j of a
@@ -40,6 +41,8 @@
 // that the ordinary one keeps its decode switch and its registers.
 #include <cuda.h>
 
+#include <cstddef>
+
 #include <new>
 
 #include "pw_common.cuh"
@@ -51,7 +54,7 @@ constexpr int kSlotBytes = 17408;               // one ring slot: an 8-bit item 
 constexpr int kMaxSlots = 16;
 constexpr int kMaxASlots = 4;                  // operand slots in tensor memory, one per group (64 columns = a 128 x 128 tile)
 constexpr int kMaxBSlots = 5;
-constexpr int kCtrlBytes = 1024;
+constexpr int kCtrlBytes = 1536;
 constexpr int kMaxDynSmem = 232448;            // 227 KB
 constexpr int kDqWarps = 16;
 constexpr int kWarpCodes = 16, kWarpTokens = 17, kWarpCodes2 = 18, kWarpMma = 19, kIssuers = 4, kWarpEpi = 23;
@@ -81,7 +84,11 @@ struct Ctrl {                                  // lives at the start of dynamic 
   // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
   volatile int32_t sched_unit[32];
+  // the posted units themselves (entry i & 15), with the bitwidths of their pages packed into the spare word: what
+  // every role needs to know about a unit, so that only the producers read the unit list and the page table
+  alignas(16) Unit desc[16];                   // read and written 16 bytes at a time
 };
+static_assert(offsetof(Ctrl, desc) % 16 == 0, "descriptor alignment");
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
 
@@ -359,9 +366,10 @@ __device__ __forceinline__ int next_unit(uint32_t i, Ctrl* c, int32_t* status) {
   return -2;
 }
 // A unit of the list.  The gate/up list is written by the kernel directly ahead of this one in the stream, possibly
-// while this grid is already resident; no role reads it before producer 0 has waited for that kernel and posted the
-// unit, so an ordinary cached load sees final data -- what it must not be is a load through the non-coherent path,
-// which the compiler may choose for a `const __restrict__` pointer: hence the explicit cache operator.
+// while this grid is already resident.  Only the two weight producers read it, after they have waited for that
+// kernel (grid_dep_sync), so an ordinary cached load sees final data -- what it must not be is a load through the
+// non-coherent path, which the compiler may choose for a `const __restrict__` pointer: hence the explicit cache
+// operator.  Every other role gets the unit from producer 0 through shared memory (load_desc).
 __device__ __forceinline__ Unit load_unit(const Unit* units, int u) {
   const int4* p = reinterpret_cast<const int4*>(units + u);
   const int4 a = __ldca(p), b = __ldca(p + 1);
@@ -374,6 +382,23 @@ __device__ __forceinline__ Unit load_unit(const Unit* units, int u) {
   un.g1 = b.y;
   un.split = b.z;
   un.pad_ = b.w;
+  return un;
+}
+// Unit i of this CTA's work list as producer 0 posted it (after next_unit has returned its index).
+__device__ __forceinline__ Unit load_desc(const Ctrl* c, uint32_t i) {
+  const uint32_t a_s = smem_u32(&c->desc[i & 15]);
+  int4 a, b;
+  asm volatile("ld.volatile.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "r"(a_s));
+  asm volatile("ld.volatile.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "r"(a_s + 16));
+  Unit un;
+  un.seg = a.x;
+  un.row_tile = a.y;
+  un.tok0 = a.z;
+  un.ntok = a.w;
+  un.g0 = b.x;
+  un.g1 = b.y;
+  un.split = b.z;
+  un.pad_ = b.w;                                 // bitwidths: matrix 0 in bits 0-7, matrix 1 in bits 8-15
   return un;
 }
 // Bitwidth of a page-table row as the kernel's roles pass it around: the bitwidth, with kPlanesFlag for a block of
@@ -586,20 +611,36 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       if (PHASE == 0) grid_dep_sync();
       // the work list: unit blockIdx.x first, then whatever the global counter hands out
       int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
-      if (P == 0) {
-        c->sched_unit[0] = u;
+      Unit un;
+      DevRow rw[NMAT];
+      auto fetch_info = [&](int uu) {
+        un = load_unit(units, uu);
+#pragma unroll
+        for (int m = 0; m < NMAT; ++m) rw[m] = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+      };
+      // producer 0 posts a unit: its index, and the unit with the bitwidths of its pages for the other roles
+      auto post = [&](uint32_t idx, int uu) {
+        if (uu >= 0) {
+          Unit d = un;
+          d.pad_ = (int32_t)(row_ubits<PLANES>(rw[0]) | (row_ubits<PLANES>(rw[NMAT - 1]) << 8));
+          int4* dp = reinterpret_cast<int4*>(&c->desc[idx & 15]);
+          dp[0] = make_int4(d.seg, d.row_tile, d.tok0, d.ntok);
+          dp[1] = make_int4(d.g0, d.g1, d.split, d.pad_);
+        }
+        c->sched_unit[idx & 31] = uu;
         __threadfence_block();
-        c->sched_n = 1;
-      }
+        c->sched_n = idx + 1;
+      };
+      if (u >= 0) fetch_info(u);
+      if (P == 0) post(0u, u);
       for (int i = 0; ok && u >= 0; ++i) {
-        const Unit un = load_unit(units, u);
         int claimed = 0;
         // per matrix of the unit: bitwidth, bytes of a tile image, address of the unit's first tile;
         // consecutive groups of a row tile are consecutive tiles of the page
         MatSrc ms[NMAT];
 #pragma unroll
         for (int m = 0; m < NMAT; ++m) {
-          const DevRow row = rows[un.seg * 3 + (PHASE == 0 ? m : 2)];
+          const DevRow& row = rw[m];
           const bool planes = PLANES && row.valid == 2;
           ms[m].bits = row.bits;
           ms[m].q = planes ? row.bits : 0u;
@@ -657,11 +698,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         }
         if (P == 0) {
           u = claimed < n_units ? claimed : -1;
-          c->sched_unit[(i + 1) & 31] = u;
-          __threadfence_block();
-          c->sched_n = (uint32_t)i + 2;
+          if (u >= 0) fetch_info(u);
+          post((uint32_t)i + 1, u);
         } else {
           u = next_unit<LIM>((uint32_t)i + 1, c, status);
+          if (u >= 0) fetch_info(u);
         }
       }
     }
@@ -675,7 +716,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       for (int i = 0; ok; ++i) {
         const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
-        const Unit un = load_unit(units, u);
+        const Unit un = load_desc(c, (uint32_t)i);
         const int nb_rows = (un.ntok + 15) & ~15;
         const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
         for (int g = un.g0; ok && g < un.g1; ++g) {
@@ -782,10 +823,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
-        const Unit un = load_unit(units, u);
+        const Unit un = load_desc(c, (uint32_t)i);
         uint32_t ubits[NMAT];
 #pragma unroll
-        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+        for (int m = 0; m < NMAT; ++m) ubits[m] = ((uint32_t)un.pad_ >> (8 * m)) & 0xffu;
         const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
         // slot items per group of the unit (W) and the offset of my matrix's inside a group
         const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
@@ -845,10 +886,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       for (int i = 0; ok; ++i, ++ucount) {
         const int u = next_unit<LIM>((uint32_t)i, c, status);
         if (u < 0) break;
-        const Unit un = load_unit(units, u);
+        const Unit un = load_desc(c, (uint32_t)i);
         uint32_t ubits[NMAT];
 #pragma unroll
-        for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+        for (int m = 0; m < NMAT; ++m) ubits[m] = ((uint32_t)un.pad_ >> (8 * m)) & 0xffu;
         const uint32_t my_bits = my_m ? ubits[NMAT - 1] : ubits[0];
         // slot items per group of the unit (W) and the offset of my matrix's inside a group
         const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
@@ -967,10 +1008,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     for (int i = 0; ok; ++i) {
       const int u = next_unit<LIM>((uint32_t)i, c, status);
       if (u < 0) break;
-      const Unit un = load_unit(units, u);
+      const Unit un = load_desc(c, (uint32_t)i);
       uint32_t ubits[NMAT];
 #pragma unroll
-      for (int m = 0; m < NMAT; ++m) ubits[m] = row_ubits<PLANES>(rows[un.seg * 3 + (PHASE == 0 ? m : 2)]);
+      for (int m = 0; m < NMAT; ++m) ubits[m] = ((uint32_t)un.pad_ >> (8 * m)) & 0xffu;
       const uint32_t bits = qm ? ubits[NMAT - 1] : ubits[0];
       const uint32_t W = slot_items(ubits[0]) + (NMAT == 2 ? slot_items(ubits[NMAT - 1]) : 0u);
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
@@ -1016,7 +1057,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     for (int i = 0; ok; ++i, ++ucount) {
       const int u = next_unit<LIM>((uint32_t)i, c, status);
       if (u < 0) break;
-      const Unit un = load_unit(units, u);
+      const Unit un = load_desc(c, (uint32_t)i);
       const int nb_rows = (un.ntok + 15) & ~15;
       const bool wide = NMAT * npart * nb_rows > acol / 2;
       const uint32_t dbuf = wide ? 0u : dtoggle;
