@@ -754,6 +754,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // My tiles of one unit (every npart-th group from j0 on): token tile, operand (a 16-bit tile's two halves from
     // the ring, or the operand slot of the group that dequantized the tile), eight MMAs, hand-backs.  One body for
     // both instantiations of the issuer role below.
+    uint32_t b_known = 0;                          // token tiles known to have been armed
     auto issue_tiles = [&](uint32_t j0, uint32_t ng, uint32_t base, uint32_t W, uint32_t my_bits, uint32_t d_t,
                            uint32_t b_lo_unit, uint32_t b_step, uint32_t idesc, uint32_t& bt, RingPos& bp, uint32_t& sq,
                            RingPos& rp, uint32_t& upar) -> bool {
@@ -761,10 +762,15 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
 #pragma unroll 1
         for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
-          // the token tile of this group (a tile is looked at only once it is known to have been armed)
-          if (c->b_issued <= bt) {
-            ok = flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, c, status);
-            if (!ok) break;
+          // the token tile of this group (a tile is looked at only once it is known to have been armed; the
+          // producer is usually ahead, and one look at its counter covers the tiles up to it)
+          if (b_known <= bt) {
+            b_known = c->b_issued;
+            if (b_known <= bt) {
+              ok = flag_wait<LIM>(smem_u32(const_cast<uint32_t*>(&c->b_issued)), bt, c, status);
+              if (!ok) break;
+              b_known = bt + 1;
+            }
           }
           ok = mbar_wait_s<LIM>(bf_s + 8 * bp.s, bp.par, c, status);
           if (!ok) break;
@@ -805,7 +811,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           tc_commit_s(be_s + 8 * bp.s);
           later = 1;
           bt += (uint32_t)npart;
-          ring_advance(bp, (uint32_t)npart, (uint32_t)n_bslots);
+          bp.s += (uint32_t)npart;                   // npart < n_bslots: one wrap at most
+          if (bp.s >= (uint32_t)n_bslots) {
+            bp.s -= (uint32_t)n_bslots;
+            bp.par ^= 1u;
+          }
         }
         return ok;
     };
