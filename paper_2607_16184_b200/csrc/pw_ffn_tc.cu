@@ -33,6 +33,10 @@
 //                between two accumulator buffers, so the next unit's MMAs overlap the epilogue.
 //                Token tiles wider than 64 leave no second buffer: the HELP instantiation, launched for
 //                those, has the four issuer warps share the epilogue of every wide unit.
+//                Wide token tiles also leave the gate/up kernel one accumulator per matrix: there the two issuers
+//                of a matrix take turns on it, tile by tile (a turn word in shared memory between tcgen05 fences
+//                keeps the MMAs of an accumulator in tile order), so that one issuer's waits and hand-backs run
+//                while the other issues.
 // Every wait is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing
 // work, frees its tensor memory and returns.
 // A block in the overlaid bit-plane format (Sec. 2.2, Sec. 3.1) is a slot item like any quantized tile: its
@@ -80,6 +84,10 @@ struct Ctrl {                                  // lives at the start of dynamic 
   // its slot items below this number.
   volatile uint32_t issued[2];
   volatile uint32_t b_issued;                  // token tiles armed so far (same purpose, for the token-tile slots)
+  // Accumulators that two issuers share (wide token tiles leave room for fewer accumulators than issuers): tiles
+  // issued on accumulator a so far.  The issuer of the next tile waits for its turn, so the MMAs of an accumulator
+  // enter the tensor pipe in tile order whoever issues them.
+  volatile uint32_t turn[4];
   // Work list of this CTA: the weight producer claims units from a global counter and posts them here;
   // entry i & 31 is valid once sched_n > i (the producer is never more than a ring of slots ahead of the others), -1 ends the list.
   volatile uint32_t sched_n;
@@ -545,7 +553,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
   constexpr int IPM = kIssuers / NMAT;           // issuers per matrix = dequantizer groups per matrix
   int npart = IPM;
   while (npart > 1 && NMAT * npart * nt_tile + kMaxASlots * 64 > kTmemCols) npart >>= 1;
-  const int n_issuers = NMAT * npart;            // active issuers
+  // Active issuers per matrix: one per accumulator, except in the gate/up kernel for wide token tiles, where the
+  // two issuers of a matrix take turns on its one accumulator (the down kernel's token tiles then leave too few
+  // token-tile slots for four issuers: it lost 10 %).
+  constexpr bool kSharedAcc = HELP && PHASE == 0;
+  const int ipa = kSharedAcc ? IPM : npart;
+  const int n_issuers = NMAT * ipa;
   const int acol = NMAT * npart * nt_tile;       // the operand slot of group g sits at acol + 64 * g
   const int G = gridDim.x;
 
@@ -569,6 +582,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     c->abort_flag = 0;
     c->issued[0] = c->issued[1] = 0;
     c->b_issued = 0;
+    c->turn[0] = c->turn[1] = c->turn[2] = c->turn[3] = 0;
     c->sched_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -755,13 +769,28 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // the ring, or the operand slot of the group that dequantized the tile), eight MMAs, hand-backs.  One body for
     // both instantiations of the issuer role below.
     uint32_t b_known = 0;                          // token tiles known to have been armed
+    // accumulator of this issuer (several issuers per accumulator when npart < IPM) and its turn word
+    const uint32_t my_p = (uint32_t)my_j & (uint32_t)(npart - 1);
+    constexpr bool shared_acc = kSharedAcc;
+    const uint32_t npart_log = npart == 4 ? 2u : npart == 2 ? 1u : 0u;
+    const uint32_t turn_s = smem_u32(const_cast<uint32_t*>(&c->turn[my_m * npart + (int)my_p]));
     auto issue_tiles = [&](uint32_t j0, uint32_t ng, uint32_t base, uint32_t W, uint32_t my_bits, uint32_t d_t,
                            uint32_t b_lo_unit, uint32_t b_step, uint32_t idesc, uint32_t& bt, RingPos& bp, uint32_t& sq,
                            RingPos& rp, uint32_t& upar) -> bool {
         bool ok = true;
-        uint32_t later = 0;                          // becomes 1 after my first tile: accumulate onto earlier ones
+        // accumulate onto earlier tiles: after my first tile, and from the start when the accumulator's first tile
+        // of this unit is another issuer's
+        uint32_t later = j0 >= (uint32_t)npart ? 1u : 0u;
+        // my MMAs are in the pipe: the accumulator's next tile may follow
+        auto release_turn = [&](uint32_t tord) {
+          if (shared_acc) {
+            tc_fence_before();
+            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_s), "r"(tord + 1) : "memory");
+          }
+        };
 #pragma unroll 1
-        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)npart) {
+        for (uint32_t j = j0; ok && j < ng; j += (uint32_t)ipa) {
+          const uint32_t tord = (base + j) >> npart_log;   // number of this tile among the tiles of its accumulator
           // the token tile of this group (a tile is looked at only once it is known to have been armed; the
           // producer is usually ahead, and one look at its counter covers the tiles up to it)
           if (b_known <= bt) {
@@ -781,17 +810,19 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
               ok = wait_issued<LIM>(sq + hh, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[hp.s]), hp.par, c, status);
+              if (ok && shared_acc && hh == 0 && tord > 0) ok = flag_wait<LIM>(turn_s, tord - 1, c, status);
               if (!ok) break;
               tc_fence_after();
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
               tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
+              if (hh == 1) release_turn(tord);
               mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
               tc_commit(&c->empty[hp.s]);
               ring_advance(hp, 1, (uint32_t)n_slots);
             }
             if (!ok) break;
-            sq += (uint32_t)npart * W;
-            ring_advance(rp, (uint32_t)npart * W, (uint32_t)n_slots);
+            sq += (uint32_t)ipa * W;
+            ring_advance(rp, (uint32_t)ipa * W, (uint32_t)n_slots);
           } else {
             // the group that dequantizes this tile, and the parity of this use of its operand slot
             const uint32_t k = base + j;
@@ -801,26 +832,24 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
             ok = mbar_wait_s<LIM>(f0, use_par, c, status);
+            if (ok && shared_acc && tord > 0) ok = flag_wait<LIM>(turn_s, tord - 1, c, status);
             if (!ok) break;
             tc_fence_after();
             // all eight k-steps of the tile, then one commit hands the group's operand slot back
             tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
             tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            release_turn(tord);
             tc_commit_s(e0);
           }
           tc_commit_s(be_s + 8 * bp.s);
           later = 1;
-          bt += (uint32_t)npart;
-          bp.s += (uint32_t)npart;                   // npart < n_bslots: one wrap at most
-          if (bp.s >= (uint32_t)n_bslots) {
-            bp.s -= (uint32_t)n_bslots;
-            bp.par ^= 1u;
-          }
+          bt += (uint32_t)ipa;
+          ring_advance(bp, (uint32_t)ipa, (uint32_t)n_bslots);
         }
         return ok;
     };
     if constexpr (!HELP) {
-    if (lane == 0 && my_j < npart) {
+    if (lane == 0 && my_j < ipa) {
       uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
       uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
@@ -848,7 +877,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
         const uint32_t b_step = (uint32_t)(2 * nb_rows);
         // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
-        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(ipa - 1);
         uint32_t bt = base + j0;                     // token-tile number
         RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
@@ -856,7 +885,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const bool wide = NMAT * npart * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
-        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + (int)my_p) * nb_rows);
         // the epilogue has drained the buffer(s) this unit accumulates into
         if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
         if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
@@ -882,7 +911,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // overlapped: here the four issuer warps share it with the four epilogue warps (they take the upper
     // half of the token columns of their lane quarter), lane 0 of the warps with an accumulator of their own
     // issuing the unit's MMAs first.  Every lane tracks the per-unit state; only lane 0 uses the issuing part.
-    const bool issuing = my_j < npart;
+    const bool issuing = my_j < ipa;
     const int hq = warp & 3;
     const int hr = hq * 32 + lane;
     const uint32_t hlane_addr = tmem + ((uint32_t)(hq * 32) << 16);
@@ -911,7 +940,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const uint32_t b_lo_unit = b_lo_base | ((uint32_t)nb_rows << 16);
         const uint32_t b_step = (uint32_t)(2 * nb_rows);
         // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
-        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(npart - 1);
+        const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(ipa - 1);
         uint32_t bt = base + j0;                     // token-tile number
         RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
@@ -919,7 +948,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const bool wide = NMAT * npart * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
-        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + my_j) * nb_rows);
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + (int)my_p) * nb_rows);
         if (lane == 0 && issuing) {
           do {
         // the epilogue has drained the buffer(s) this unit accumulates into
@@ -1242,10 +1271,18 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
     const int nmat = phase == 0 ? 2 : 1;
     int npart = kIssuers / nmat;
     while (npart > 1 && nmat * npart * nt_tile + kMaxASlots * 64 > kTmemCols) npart >>= 1;
-    n_bslots[phase] = npart + 1 > kMaxBSlots ? kMaxBSlots : npart + 1;
-    int ns = (kMaxDynSmem - kCtrlBytes - n_bslots[phase] * bslot_bytes) / kSlotBytes;
-    if (ns > kMaxSlots) ns = kMaxSlots;
-    ns &= ~1;                                    // an even number of slots: one set per producer
+    // every issuer of a matrix works on a token tile of its own, one more is on its way -- fewer when the tiles are
+    // so wide that the weight ring would fall below six slots
+    const int ipa = phase == 0 && nt_tile > 64 ? kIssuers / nmat : npart;   // active issuers per matrix (the kernel's rule)
+    int nb = ipa + 1 > kMaxBSlots ? kMaxBSlots : ipa + 1;
+    int ns = 0;
+    for (;; --nb) {
+      ns = (kMaxDynSmem - kCtrlBytes - nb * bslot_bytes) / kSlotBytes;
+      if (ns > kMaxSlots) ns = kMaxSlots;
+      ns &= ~1;                                  // an even number of slots: one set per producer
+      if (ns >= 6 || nb <= npart + 1) break;
+    }
+    n_bslots[phase] = nb;
     if (ns < 6) return PW_ERR_NOMEM;             // the dequantizers advance up to six slot items at a time
     n_slots[phase] = ns;
     smem[phase] = kCtrlBytes + ns * kSlotBytes + n_bslots[phase] * bslot_bytes;
