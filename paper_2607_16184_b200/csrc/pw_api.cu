@@ -50,6 +50,7 @@ WsMap make_wsmap(const pw_config& c) {
   m.units_gu = take(sizeof(Unit) * (size_t)m.max_units);
   m.units_dn = take(sizeof(Unit) * (size_t)m.max_units);
   m.n_units = take(16);
+  m.done = take(4 * 8 * (size_t)m.Rmax);
   m.xt = take((size_t)c.hidden * 2 * m.Rpad);
   m.ht = take((size_t)c.ffn * 2 * m.Rpad);
   m.y = take(m.y_slots * c.hidden * 4);

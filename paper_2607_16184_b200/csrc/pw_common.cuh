@@ -55,6 +55,7 @@ struct WsMap {
   size_t units_gu;    // Unit[max_units]
   size_t units_dn;    // Unit[max_units]
   size_t n_units;     // int32[4]
+  size_t done;        // int32[Rmax * 8]: gate/up units finished, per (first operand row of a token tile, K range of the down projection)
   size_t xt;          // fp16 operand rows, k-chunk major: [H/8][Rpad][8]
   size_t ht;          // fp16 SwiGLU output,  k-chunk major: [F/8][Rpad][8]
   size_t y;           // float [y_slots][H]  split-K partial outputs of the down projection
@@ -169,9 +170,12 @@ void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 // are visible; a thread calls it before it reads anything that kernel wrote.  grid_dep_trigger() lets the
 // kernel after this one be placed as soon as SMs free up; a kernel calls it only after its own
 // grid_dep_sync(), so "my CTA has been placed" implies that every kernel two or more steps back in the chain
-// has completed.  That is what allows the down kernel to start streaming weight pages at once (its unit list
-// and the page-table rows are written two steps back or earlier) and to wait only before its first token
-// tile; the gate/up kernel's unit list is written one step back, so its weight producers wait as well.
+// has completed.  That is what allows the down kernel to start streaming weight pages at once (its unit list,
+// the zeroed completion counters and the page-table rows are written two steps back or earlier); the gate/up
+// kernel's unit list is written one step back, so its weight producers wait as well.  The down kernel is the
+// one exception to "sync, then trigger": it never waits for the gate/up kernel as a whole but, unit by unit,
+// for the completion counters that kernel's epilogue raises (WsMap::done), and the kernel after it reads
+// nothing of the gate/up kernel's and waits for the down kernel before it reads anything at all.
 // With the timing events between the kernels the attribute has no effect.
 __device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -37,6 +37,11 @@
 //                of a matrix take turns on it, tile by tile (a turn word in shared memory between tcgen05 fences
 //                keeps the MMAs of an accumulator in tile order), so that one issuer's waits and hand-backs run
 //                while the other issues.
+// The two kernels of a call overlap: the down kernel's CTAs are placed on the SMs the gate/up kernel's CTAs leave,
+// stream their weight pages at once, and start a unit when the gate/up units that write the SwiGLU rows of its K
+// range have been counted in (a counter per token tile and K range, raised by the gate/up epilogue behind a
+// fence, read with an acquire load by the down kernel's token-tile producer); the down list goes K range
+// outermost so that the ranges finished first are multiplied first.
 // Every wait is bounded; when one runs out the CTA records PW_ERR_TIMEOUT in the status word, stops issuing
 // work, frees its tensor memory and returns.
 // A block in the overlaid bit-plane format (Sec. 2.2, Sec. 3.1) is a slot item like any quantized tile: its
@@ -526,6 +531,20 @@ __device__ __forceinline__ bool dq_run(DqState& st, uint32_t count, uint32_t ste
   return true;
 }
 
+// A warp has stored its share of the SwiGLU rows of a gate/up unit: count it in for the K range of the down
+// projection that the unit's FFN rows belong to.  The down kernel, which may already be running on SMs this kernel
+// has left, starts a unit when every warp of every gate/up unit it reads has been counted (see the token-tile
+// producer); the fence before the count makes the rows visible to it.
+__device__ __forceinline__ void signal_rows_done(int32_t* done, int tok0, int row_tile, int n_row_tiles, int dn_splits, int lane) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) {
+    int sp = 0;                                    // K range sp of the down projection covers [sp * n / splits, (sp + 1) * n / splits)
+    while (sp + 1 < dn_splits && ((sp + 1) * n_row_tiles) / dn_splits <= row_tile) ++sp;
+    atomicAdd(done + (size_t)tok0 * dn_splits + sp, 1);
+  }
+}
+
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
 // PLANES: the instantiation that also reads blocks of overlaid bit-planes; launched only for a layer that holds one
@@ -538,7 +557,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t* __restrict__ n_units_ptr,
               const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
               __half* __restrict__ ht, float* __restrict__ y, int H, size_t y_split_stride,
-              int32_t* __restrict__ work_counter, int32_t* __restrict__ status, uint32_t hook) {
+              int32_t* __restrict__ work_counter, int32_t* __restrict__ status, int32_t* done, int dn_splits,
+              int ffn_tiles, uint32_t hook) {
   constexpr uint32_t LIM = SHORT ? kTestWaitPolls : kDefaultWaitPolls;
   extern __shared__ __align__(1024) char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
@@ -599,8 +619,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
   const uint32_t tmem = c->tmem_base;
   // This CTA may have been placed while the kernel before this one is still finishing on other SMs.  Work
   // counters, page-table rows and the unit counts were written two or more kernels back and are final (see
-  // grid_dep_sync).  What the kernel directly ahead writes is not: the token rows (both kernels; the
-  // token-tile producer waits for them) and the gate/up unit list (PHASE 0; the weight producers wait).
+  // grid_dep_sync).  What the kernel directly ahead writes is not: the token rows (the gate/up kernel's
+  // token-tile producer waits for the kernel that gathers them, the down kernel's for the completion counters of
+  // the gate/up units, one unit at a time) and the gate/up unit list (PHASE 0; the weight producers wait).
 
   // Units are claimed dynamically: CTA b starts with unit b, every further one comes from the global counter
   // (the weight producer claims, the other roles follow its list).
@@ -723,7 +744,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
   } else if (warp == kWarpTokens) {
     // ---------------- token-tile producer ----------------
     if (lane == 0) {
-      grid_dep_sync();
+      // The gate/up kernel waits for the kernel ahead of it (which gathers its token rows).  The down kernel does
+      // not wait for the gate/up kernel as a whole: its CTAs take the SMs that kernel's CTAs leave one by one, and
+      // a unit starts as soon as the gate/up units that write the rows it multiplies have been counted in.
+      if (PHASE == 0) grid_dep_sync();
       grid_dep_trigger();
       uint32_t bcount = 0;
       bool ok = true;
@@ -733,6 +757,28 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const Unit un = load_desc(c, (uint32_t)i);
         const int nb_rows = (un.ntok + 15) & ~15;
         const CUtensorMap* map = &tmaps.m[(nb_rows >> 4) - 1];
+        if (PHASE == 1) {
+          // every warp that stores rows of a gate/up unit counts itself in: the four epilogue warps, and the four
+          // issuer warps as well where they share the epilogue (that kernel's rule for a wide unit)
+          const bool helped = HELP && 2 * nb_rows > nt_tile;
+          const int need = (helped ? 8 : 4) * (un.g1 - un.g0);
+          const int32_t* flag = done + (size_t)un.tok0 * dn_splits + un.split;
+          int seen = 0;
+          for (uint32_t n = 0;; ++n) {
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+            if (seen >= need) break;
+            // the gate/up kernel gave up (a wait of its own ran out), or this wait has lasted 2 s
+            if (n >= LIM * 64u || *reinterpret_cast<volatile int32_t*>(status) == (int)PW_ERR_TIMEOUT) {
+              c->abort_flag = 1;
+              atomicMax(status, (int)PW_ERR_TIMEOUT);
+              ok = false;
+              break;
+            }
+            __nanosleep(300);
+          }
+          if (!ok) break;
+          asm volatile("fence.proxy.async.global;" ::: "memory");   // the rows were written with ordinary stores; the copies below read them through the async proxy
+        }
         for (int g = un.g0; ok && g < un.g1; ++g) {
           if ((hook & 1u) && bcount == 1) {        // test hook: leave the tile unarmed, so that the waits on it run out
             ok = false;
@@ -975,17 +1021,15 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (!ok) break;
         if (wide) {
           tc_fence_after();
-          uint32_t written = 0;
-          for (int p = 0; p < npart; ++p)
-            if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
+          const uint32_t p0 = base & (uint32_t)(npart - 1), nq = ng < (uint32_t)npart ? ng : (uint32_t)npart;
           const int row = un.row_tile * kTileRows + hr;
           const int half = ((nb_rows / 16 + 1) / 2) * 16;         // the epilogue warps take [0, half)
           for (int c0 = half; c0 < nb_rows; c0 += 16) {
             float a[16], b[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
-            for (int p = 0; p < npart; ++p) {
-              if (!((written >> p) & 1u)) continue;
+            for (uint32_t q = 0; q < nq; ++q) {
+              const int p = (int)((p0 + q) & (uint32_t)(npart - 1));
               float t[16];
               tmem_ld16(hlane_addr + p * nb_rows + c0, t);
               tmem_wait_ld();
@@ -1017,6 +1061,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             mbar_arrive(&c->d_empty[0]);
             mbar_arrive(&c->d_empty[1]);
           }
+          if (PHASE == 0) signal_rows_done(done, un.tok0, un.row_tile, ffn_tiles, dn_splits, lane);
         }
         base += ng;
         seq_unit += ng * W;
@@ -1107,12 +1152,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       tc_fence_after();
       const int row = un.row_tile * kTileRows + r;
       const uint32_t dbase = lane_addr + dbuf * (uint32_t)(acol / 2);
-      // partial accumulator p holds the tiles base + j with (base + j) mod npart == p: it has been written in
-      // this unit only if there is such a j below the unit's group count
+      // Partial accumulator p holds the tiles base + j with (base + j) mod npart == p.  They are added starting
+      // with the one that holds the unit's first tile, so that the order of the sum depends on the unit alone
+      // and not on how many tiles this CTA has seen before it (units are claimed in a different order from run
+      // to run): a forward call repeats bit for bit.
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
-      uint32_t written = 0;
-      for (int p = 0; p < npart; ++p)
-        if ((((uint32_t)p - base) & (uint32_t)(npart - 1)) < ng) written |= 1u << p;
+      const uint32_t p0 = base & (uint32_t)(npart - 1), nq = ng < (uint32_t)npart ? ng : (uint32_t)npart;
       base += ng;
       // with helpers, the issuer warps take the upper half of the token columns of a wide unit
       const int c_end = HELP && wide ? ((nb_rows / 16 + 1) / 2) * 16 : nb_rows;
@@ -1120,8 +1165,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         float a[16], b[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
-        for (int p = 0; p < npart; ++p) {              // add the issuers' partial sums, in order
-          if (!((written >> p) & 1u)) continue;
+        for (uint32_t q = 0; q < nq; ++q) {            // add the issuers' partial sums, in the unit's tile order
+          const int p = (int)((p0 + q) & (uint32_t)(npart - 1));
           float t[16];
           tmem_ld16(dbase + p * nb_rows + c0, t);
           tmem_wait_ld();
@@ -1157,6 +1202,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (wide || dbuf == 0) mbar_arrive_n(&c->d_empty[0], n_arr);
         if (wide || dbuf == 1) mbar_arrive_n(&c->d_empty[1], n_arr);
       }
+      // (after the accumulators have been handed back: the fence in there waits for the stores above)
+      if (PHASE == 0) signal_rows_done(done, un.tok0, un.row_tile, ffn_tiles, dn_splits, lane);
       if (wide || dbuf == 0) ++duse0;
       if (wide || dbuf == 1) ++duse1;
     }
@@ -1197,7 +1244,7 @@ static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, Tma
 }
 
 typedef void (*FfnKernel)(const DevRow*, const Unit*, const int32_t*, const TmapSet, int, int, int, int, __half*, float*, int, size_t,
-                          int32_t*, int32_t*, uint32_t);
+                          int32_t*, int32_t*, int32_t*, int, int, uint32_t);
 static FfnKernel ffn_kernel_of(int phase, int help, int planes) {
   static const FfnKernel tab[8] = {
       ffn_tc_kernel<0, false, false, false>, ffn_tc_kernel<1, false, false, false>, ffn_tc_kernel<0, true, false, false>,
@@ -1302,15 +1349,14 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
                               dim3(kThreads), (size_t)smem[0], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
                               n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
-                              work_counter, status, ctx->test_hook));
+                              work_counter, status, reinterpret_cast<int32_t*>(b + w.done), ksplit, c.ffn / kTileRows, ctx->test_hook));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
   PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
                               n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
-                              (size_t)R * c.hidden, work_counter + 1, status, 0u));
+                              (size_t)R * c.hidden, work_counter + 1, status, reinterpret_cast<int32_t*>(b + w.done), ksplit, c.ffn / kTileRows, 0u));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
-  (void)ksplit;
   return PW_OK;
 }
 

@@ -228,12 +228,16 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
                                                      const int2* __restrict__ tile_tab, int max_tiles,
                                                      const int32_t* __restrict__ n_units, int nt_tile, int ksplit,
                                                      int ng_gu, int ng_dn, int dn_token_tile_outer,
-                                                     Unit* __restrict__ units_gu, Unit* __restrict__ units_dn) {
+                                                     Unit* __restrict__ units_gu, Unit* __restrict__ units_dn,
+                                                     int32_t* __restrict__ done) {
   grid_dep_sync();
   grid_dep_trigger();
   if (nt_tile > 0) {
     const int gt = (blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
     const int n_threads = gridDim.x * gridDim.y * blockDim.x;
+    // completion counters of the gate/up units, one per (first operand row of a token tile, K range of the down
+    // projection): the down kernel starts a unit as soon as the rows it multiplies are there
+    for (int i = gt; i < offsets[S] * ksplit; i += n_threads) done[i] = 0;
     for (int phase = 0; phase < 2; ++phase) {
       const int total = n_units[phase], TT = n_units[2 + phase];
       const int splits = phase == 0 ? 1 : ksplit;
@@ -256,7 +260,11 @@ __global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ h
           rs = u / TT;
           j = u - rs * TT;
         }
-        const int rt = rs / splits, sp = rs - rt * splits;
+        // down projection: K range outermost, so that the units whose SwiGLU rows are finished first (the gate/up
+        // list goes through the FFN rows in order) come first
+        const int RT = RS / splits;
+        const int sp = phase == 1 && !tt_outer ? rs / RT : rs % splits;
+        const int rt = phase == 1 && !tt_outer ? rs - sp * RT : rs / splits;
         const int2 t = tab[j];
         const int n = counts[t.x];
         Unit un;
@@ -461,7 +469,7 @@ pw_status launch_route(pw_ctx* ctx, int layer, const void* hidden, const float* 
                               reinterpret_cast<const int2*>(b + w.tile_tab), w.max_tiles,
                               reinterpret_cast<const int32_t*>(b + w.n_units), nt_tile, ksplit, c.hidden / kGroup,
                               c.ffn / kGroup, dn_tt_outer, reinterpret_cast<Unit*>(b + w.units_gu),
-                              reinterpret_cast<Unit*>(b + w.units_dn)));
+                              reinterpret_cast<Unit*>(b + w.units_dn), reinterpret_cast<int32_t*>(b + w.done)));
   ctx->launches += 2;
   PW_CUDA_OK(cudaGetLastError());
   return PW_OK;

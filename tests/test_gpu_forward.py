@@ -211,6 +211,31 @@ def test_forward_is_bitwise_reproducible(mode):
         ctx.close()
 
 
+def test_forward_repeats_bit_for_bit_when_the_tile_counts_are_odd():
+    """More units than CTAs, so the later units are claimed in an order that changes from run to run, and odd
+    numbers of K tiles per unit (3 for gate/up, 5 for down), so a unit's first tile falls on a different
+    partial accumulator depending on what its CTA ran before: the partials are added starting from the one
+    that holds the unit's first tile, and the result does not depend on that history."""
+    cfg = synth.LayerConfig("odd_tiles", 96, 6, 384, 640, 64, n_shared=1, routing="normal", bit_rule="iid5")
+    ctx = make_ctx(cfg, max_tokens=cfg.tokens, n_layers=1)
+    try:
+        build_layer(ctx, cfg, 0, None)
+        x = synth.activations(cfg, device="cuda")
+        logits = synth.router_logits(cfg, device="cuda")
+        first = ctx.pw_moe_forward(0, x, logits, cfg.top_k).clone()
+        side = torch.cuda.Stream()
+        for i in range(60):
+            if i % 5 == 0:
+                with torch.cuda.stream(side):        # other work on the device shifts which CTA finishes first
+                    torch.cuda._sleep(100000)
+            again = ctx.pw_moe_forward(0, x, logits, cfg.top_k)
+            assert torch.equal(first.view(torch.int32), again.view(torch.int32)), i
+        torch.cuda.synchronize()
+        assert ctx.pw_last_device_status() == 0
+    finally:
+        ctx.close()
+
+
 def test_back_to_back_calls_with_different_routing(orc):
     """Consecutive calls reuse the workspace (unit lists, counters, operand buffers) while the kernels of the
     call before may still be draining: alternate two token sets and check every result against the oracle."""
