@@ -133,50 +133,52 @@ __global__ void __launch_bounds__(512, NT == 2 ? 2 : 3) quant_tile_kernel(const 
 
 // 4 bits -> 3 or 2 bits without touching a weight.  A group has at most 16 distinct values, one per source code,
 // and the demote Q(D(.)) is a function of the code alone: minimum and maximum are the values of the smallest and
-// the largest code present, and new_code(c) = clamp(rint((D(c) - lo) / scale')) is non-decreasing in c.  So the
-// four lanes of a row-group evaluate it on the 16 codes (four each, the arithmetic of the general kernel, bit for
-// bit), turn the table into L thresholds t_k = number of source codes whose new code is below k, and every code
-// becomes [c >= t_1] + .. + [c >= t_L]: nibbles spread to bytes, one add of (128 - t_k) per threshold puts the
-// comparison into bit 7 of each byte, and because the comparisons are nested a few three-input logic operations
-// give the bits of their count.  To 2 bits: about 10 instructions per weight instead of 17, and two conversions
-// per weight fewer.
+// the largest code present, and new_code(c) = clamp(rint((D(c) - lo) / scale')) is non-decreasing in c.  One thread
+// owns a whole group (a row of a tile: 16 words), so the group's work is done once and not by each of four lanes:
+// it evaluates the general kernel's arithmetic, bit for bit, on the 16 codes, turns the table into L thresholds
+// t_k = number of source codes whose new code is below k, and every code becomes [c >= t_1] + .. + [c >= t_L]:
+// nibbles spread to bytes, one add of (128 - t_k) per threshold puts the comparison into bit 7 of each byte, and
+// because the comparisons are nested a few three-input logic operations give the bits of their count.
+constexpr int kRequantThreads = 256;              // two tiles per CTA
 template <int DB>
-__global__ void __launch_bounds__(512, 3) requant_from4_kernel(const void* __restrict__ src_codes, uint32_t cols,
-                                                               void* __restrict__ dst_codes) {
-  const int g = blockIdx.x, rt = blockIdx.y, ng = gridDim.x;
-  const int r = threadIdx.x >> 2, q = threadIdx.x & 3;
-  const size_t tile = (size_t)rt * ng + g;
+__global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const void* __restrict__ src_codes, uint32_t n_tiles,
+                                                                        void* __restrict__ dst_codes) {
+  const int r = threadIdx.x & (kTileRows - 1);
+  const size_t tile = (size_t)blockIdx.x * (kRequantThreads / kTileRows) + (threadIdx.x >> 7);
+  if (tile >= n_tiles) return;
   const char* tb = reinterpret_cast<const char*>(src_codes) + tile * tile_bytes(4);
-  const uint4 u = __ldg(reinterpret_cast<const uint4*>(tb + slice_word_offset<4>(r, q, 0)));
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+  uint32_t w[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(tb + slice_word_offset<4>(r, q, 0)));
+    w[4 * q] = u.x;
+    w[4 * q + 1] = u.y;
+    w[4 * q + 2] = u.z;
+    w[4 * q + 3] = u.w;
+  }
   const float s = __half2float(*reinterpret_cast<const __half*>(tb + tile_scale_offset(4, r)));
   const float z = __half2float(*reinterpret_cast<const __half*>(tb + tile_zp_offset(4, r)));
 
   // smallest and largest code of the group: a page written by the quantizer always uses 0 and 15 (the extremes
-  // of the group map to them), which two zero-nibble tests see; any other page takes the exact scan
+  // of the group map to them), which two zero-nibble tests see (bit 3 of a nibble of x - 0x1111.. & ~x is set for
+  // the lowest zero nibble of x; ~x - k = ~(x + k)); any other page takes the exact scan
   uint32_t has0 = 0, has15 = 0;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    has0 |= (w[i] - 0x11111111u) & ~w[i] & 0x88888888u;
-    has15 |= (~w[i] - 0x11111111u) & w[i] & 0x88888888u;
+  for (int i = 0; i < 16; ++i) {
+    has0 |= (w[i] - 0x11111111u) & ~w[i];
+    has15 |= ~(w[i] + 0x11111111u) & w[i];
   }
-  uint32_t flags = (has0 != 0 ? 1u : 0u) | (has15 != 0 ? 2u : 0u);
-  flags |= __shfl_xor_sync(0xffffffffu, flags, 1);
-  flags |= __shfl_xor_sync(0xffffffffu, flags, 2);
   int cmin = 0, cmax = 15;
-  if (__any_sync(0xffffffffu, flags != 3u)) {
-    int code[32];
-    unpack_slice<4>(w, code);
-    int mn = code[0], mx = code[0];
+  if (((has0 & 0x88888888u) == 0) | ((has15 & 0x88888888u) == 0)) {
+    int mn = 15, mx = 0;
 #pragma unroll
-    for (int i = 1; i < 32; ++i) {
-      mn = min(mn, code[i]);
-      mx = max(mx, code[i]);
-    }
+    for (int i = 0; i < 16; ++i) {
 #pragma unroll
-    for (int d = 1; d <= 2; d <<= 1) {
-      mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
-      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+      for (int j = 0; j < 8; ++j) {
+        const int c = (int)((w[i] >> (4 * j)) & 15u);
+        mn = min(mn, c);
+        mx = max(mx, c);
+      }
     }
     cmin = mn;
     cmax = mx;
@@ -197,27 +199,32 @@ __global__ void __launch_bounds__(512, 3) requant_from4_kernel(const void* __res
   }
   const float rinv = __fdiv_rn(1.0f, __half2float(sh));
 
-  // my four entries of the code table -> per k, how many of them reach k (5 bits each: the sums stay <= 16)
-  unsigned long long reach = 0;
+  // t_k = how many of the 16 source codes get a new code below k.  The new code is min(rint(x), L) with
+  // x = (D(c) - lo) * rinv (negative for a code below the smallest one present: new code 0), and with ties to even
+  // rint(x) >= k  <=>  x >= k - 0.5 (k even), x > k - 0.5 (k odd): no conversion to an integer is needed.
+  uint32_t below[L];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float v = dequant_exact(4 * q + j, s, z);
-    const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v, lo), rinv));
-    const uint32_t nc = c < (uint32_t)L ? c : (uint32_t)L;
+  for (int k = 0; k < L; ++k) below[k] = 0;
 #pragma unroll
-    for (int k = 1; k <= L; ++k) reach += (unsigned long long)(nc >= (uint32_t)k ? 1u : 0u) << (5 * (k - 1));
+  for (int c = 0; c < 16; ++c) {
+    const float x = __fmul_rn(__fsub_rn(dequant_exact(c, s, z), lo), rinv);
+#pragma unroll
+    for (int k = 1; k <= L; ++k) {
+      const float edge = (float)k - 0.5f;
+      const bool reached = (k & 1) ? x > edge : x >= edge;
+      below[k - 1] += reached ? 0u : 1u;
+    }
   }
-  reach += __shfl_xor_sync(0xffffffffu, reach, 1);
-  reach += __shfl_xor_sync(0xffffffffu, reach, 2);
   // byte-wise x + (128 - t) has bit 7 set exactly when x >= t (x <= 15, 0 <= t <= 16: no carry between bytes)
-  uint32_t kk[L];                                  // 128 - t_k in every byte, t_k = 16 - reach_k
+  uint32_t kk[L];
 #pragma unroll
-  for (int k = 0; k < L; ++k) kk[k] = (112u + (uint32_t)((reach >> (5 * k)) & 31u)) * 0x01010101u;
+  for (int k = 0; k < L; ++k) kk[k] = (128u - below[k]) * 0x01010101u;
 
-  uint32_t half_bytes[4];                          // per source word: the low two bits of 8 new codes, a byte in each half-word
-  uint32_t third = 0;                              // DB == 3: the plane of the third bits, bit P / 16 + P for pair P
+  uint32_t half_bytes[16];                         // per source word: the low two bits of 8 new codes, a byte in each half-word
+  uint32_t third[4];                               // DB == 3, per slice: the plane of the third bits, bit P / 16 + P for pair P
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 16; ++i) {
+    if ((i & 3) == 0) third[i >> 2] = 0;
     uint32_t zc[2], hv[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {                  // nibbles 0, 2 of each half-word, then nibbles 1, 3
@@ -243,16 +250,20 @@ __global__ void __launch_bounds__(512, 3) requant_from4_kernel(const void* __res
     }
     const uint32_t m = zc[0] | (zc[1] << 2);       // byte 0: pairs 0, 1; byte 1: pairs 2, 3 (4 bits used of each)
     half_bytes[i] = (m | (m >> 4)) & 0x00ff00ffu;  // the four codes of a half-word in its low byte
-    if constexpr (DB == 3) third |= (hv[0] | (hv[1] << 1)) << (4 * i);
+    if constexpr (DB == 3) third[i >> 2] |= (hv[0] | (hv[1] << 1)) << (4 * (i & 3));
   }
+  // slices 2h and 2h + 1 of a row share a 16-byte chunk of the destination tile
   char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(DB);
-  *reinterpret_cast<uint2*>(db + slice_word_offset<DB>(r, q, 0)) =
-      make_uint2(half_bytes[0] | (half_bytes[1] << 8), half_bytes[2] | (half_bytes[3] << 8));
-  if constexpr (DB == 3) *reinterpret_cast<uint32_t*>(db + slice_word_offset<3>(r, q, 2)) = third;
-  if (q == 0) {
-    *reinterpret_cast<__half*>(db + tile_scale_offset(DB, r)) = sh;
-    *reinterpret_cast<__half*>(db + tile_zp_offset(DB, r)) = __float2half_rn(lo);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const uint32_t* hb = half_bytes + 8 * h;
+    *reinterpret_cast<uint4*>(db + slice_word_offset<DB>(r, 2 * h, 0)) =
+        make_uint4(hb[0] | (hb[1] << 8), hb[2] | (hb[3] << 8), hb[4] | (hb[5] << 8), hb[6] | (hb[7] << 8));
   }
+  if constexpr (DB == 3)
+    *reinterpret_cast<uint4*>(db + slice_word_offset<3>(r, 0, 2)) = make_uint4(third[0], third[1], third[2], third[3]);
+  *reinterpret_cast<__half*>(db + tile_scale_offset(DB, r)) = sh;
+  *reinterpret_cast<__half*>(db + tile_zp_offset(DB, r)) = __float2half_rn(lo);
 }
 
 // TILED -> CANONICAL (EXPORT = true) or CANONICAL -> TILED, same bitwidth.
@@ -357,6 +368,12 @@ static void launch_quant(dim3 grid, cudaStream_t s, const void* sc, uint32_t col
     quant_tile_kernel<SK, SB, DB, 1><<<grid, 512, 0, s>>>(sc, cols, d->codes);
 }
 
+template <int DB>
+static void launch_requant_from4(dim3 grid, cudaStream_t s, const void* sc, pw_page* d) {
+  const uint32_t n_tiles = grid.x * grid.y, per_cta = kRequantThreads / kTileRows;
+  requant_from4_kernel<DB><<<(n_tiles + per_cta - 1) / per_cta, kRequantThreads, 0, s>>>(sc, n_tiles, d->codes);
+}
+
 template <int SK, int SB>
 static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void* sc, uint32_t cols, pw_page* d) {
   switch (dst_bits) {
@@ -370,11 +387,11 @@ static void launch_quant_dst(int dst_bits, dim3 grid, cudaStream_t s, const void
       if (SB > 4) launch_quant<SK, SB, (SB > 4 ? 4 : 2)>(grid, s, sc, cols, d);
       break;
     case 3:
-      if (SK == SRC_TILED && SB == 4) requant_from4_kernel<3><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SK == SRC_TILED && SB == 4) launch_requant_from4<3>(grid, s, sc, d);
       else if (SB > 3) launch_quant<SK, SB, (SB > 3 ? 3 : 2)>(grid, s, sc, cols, d);
       break;
     case 2:
-      if (SK == SRC_TILED && SB == 4) requant_from4_kernel<2><<<grid, 512, 0, s>>>(sc, cols, d->codes);
+      if (SK == SRC_TILED && SB == 4) launch_requant_from4<2>(grid, s, sc, d);
       else launch_quant<SK, SB, 2>(grid, s, sc, cols, d);
       break;
   }
