@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(512, NT == 2 ? 2 : 3) quant_tile_kernel(const 
 // owns a whole group (a row of a tile: 16 words), so the group's work is done once and not by each of four lanes:
 // it evaluates the general kernel's arithmetic, bit for bit, on the 16 codes, turns the table into L thresholds
 // t_k = number of source codes whose new code is below k, and every code becomes [c >= t_1] + .. + [c >= t_L]:
-// nibbles spread to bytes, one add of (128 - t_k) per threshold puts the comparison into bit 7 of each byte, and
-// because the comparisons are nested a few three-input logic operations give the bits of their count.
+// one add and one three-input logic operation per threshold compare all eight nibbles of a code word at once, and
+// because the comparisons are nested a few more logic operations give the bits of their count.
 constexpr int kRequantThreads = 256;              // two tiles per CTA
 template <int DB>
 __global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const void* __restrict__ src_codes, uint32_t n_tiles,
@@ -199,58 +199,71 @@ __global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const vo
   }
   const float rinv = __fdiv_rn(1.0f, __half2float(sh));
 
-  // t_k = how many of the 16 source codes get a new code below k.  The new code is min(rint(x), L) with
-  // x = (D(c) - lo) * rinv (negative for a code below the smallest one present: new code 0), and with ties to even
-  // rint(x) >= k  <=>  x >= k - 0.5 (k even), x > k - 0.5 (k odd): no conversion to an integer is needed.
-  uint32_t below[L];
+  // t_k = how many of the 16 source codes get a new code below k = 16 - (codes that reach k).  The new code is
+  // min(rint(x), L) with x = (D(c) - lo) * rinv (negative for a code below the smallest one present: new code 0;
+  // NaN when the source's largest value overflowed fp16: new code 0 as well, as the conversion to an integer of
+  // the general kernel gives), and with ties to even rint(x) >= k  <=>  x > k - 0.5 (k odd), x >= k - 0.5 (k even),
+  // the latter being x > the float just below k - 0.5.  Each comparison x > e is one saturating multiply-add --
+  // sat((x - e) * 2^40) is 1 for x > e and 0 otherwise (also for NaN); the rounding of the sum keeps sign and
+  // zero-ness -- and one add, both on the multiply-add pipe that the logic operations below leave idle.
+  float reach[L];
 #pragma unroll
-  for (int k = 0; k < L; ++k) below[k] = 0;
+  for (int k = 0; k < L; ++k) reach[k] = 0.0f;
 #pragma unroll
   for (int c = 0; c < 16; ++c) {
     const float x = __fmul_rn(__fsub_rn(dequant_exact(c, s, z), lo), rinv);
 #pragma unroll
     for (int k = 1; k <= L; ++k) {
+      constexpr float kBig = 1099511627776.0f;     // 2^40
       const float edge = (float)k - 0.5f;
-      const bool reached = (k & 1) ? x > edge : x >= edge;
-      below[k - 1] += reached ? 0u : 1u;
+      const float ulp = edge >= 4.0f ? 4.76837158203125e-7f : edge >= 2.0f ? 2.384185791015625e-7f : 1.1920928955078125e-7f;
+      const float e = (k & 1) ? edge : edge - ulp;
+      reach[k - 1] += __saturatef(fmaf(x, kBig, -e * kBig));
     }
   }
-  // byte-wise x + (128 - t) has bit 7 set exactly when x >= t (x <= 15, 0 <= t <= 16: no carry between bytes)
-  uint32_t kk[L];
+  // The comparison c >= t_k on all eight nibbles of a word at once.  With c = 8 h + l: for t <= 8 it is
+  // h | (l >= t), for t > 8 it is h & (l >= t - 8), and l >= t' (0 <= t' <= 8) is bit 3 of l + (8 - t'), which never
+  // carries out of the nibble.  So per threshold one add on the word with the h bits masked out, and one majority
+  // function of (sum, word, m_k) -- m_k all ones for t_k <= 8 (or), zero above (and) -- leave the flag in bit 3 of
+  // every nibble.  With n = 16 - t codes reaching k: 8 - t' = n - 8 for n >= 8, n below.
+  uint32_t kk[L], mk[L];
 #pragma unroll
-  for (int k = 0; k < L; ++k) kk[k] = (128u - below[k]) * 0x01010101u;
+  for (int k = 0; k < L; ++k) {
+    const uint32_t n = __float2uint_rn(reach[k]);
+    kk[k] = (n >= 8u ? n - 8u : n) * 0x11111111u;
+    mk[k] = n >= 8u ? 0xffffffffu : 0u;
+  }
 
-  uint32_t half_bytes[16];                         // per source word: the low two bits of 8 new codes, a byte in each half-word
+  uint32_t half_bytes[16];                         // per source word: the 2-bit codes of 8 weights, a byte in each half-word
   uint32_t third[4];                               // DB == 3, per slice: the plane of the third bits, bit P / 16 + P for pair P
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     if ((i & 3) == 0) third[i >> 2] = 0;
-    uint32_t zc[2], hv[2];
+    const uint32_t low = w[i] & 0x77777777u;
+    uint32_t f[L];
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {                  // nibbles 0, 2 of each half-word, then nibbles 1, 3
-      const uint32_t x = (e ? w[i] >> 4 : w[i]) & 0x0f0f0f0fu;
-      uint32_t y[L];
-#pragma unroll
-      for (int k = 0; k < L; ++k) y[k] = x + kk[k];
-      // the comparisons are nested (t_1 <= t_2 <= ..), so bit 0 of their count is ((y1 & ~y2) | y3) & ~y4 | .. and
-      // bit 1 is (y2 & ~y4) | y6, bit 2 is y4 -- all in bit 7 of every byte
-      uint32_t b0, b1;
-      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(y[0]), "r"(y[1]), "r"(y[2]));
-      if constexpr (DB == 3) {
-        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(y[3]), "r"(y[4]));
-        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(y[5]), "r"(y[6]));
-        asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b1) : "r"(y[1]), "r"(y[3]), "r"(y[5]));
-        const uint32_t t = (y[3] >> 7) & 0x01010101u;
-        hv[e] = (t | (t >> 6)) & 0x00050005u;      // bits 0, 2 (16, 18): the pairs 0, 2 (e = 0) or 1, 3 of this word
-      } else {
-        b1 = y[1];
-        hv[e] = 0;
-      }
-      zc[e] = and_or(b0 >> 7, 0x01010101u, (b1 >> 6) & 0x02020202u);   // low two bits of the new code in every byte
+    for (int k = 0; k < L; ++k) asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(f[k]) : "r"(low + kk[k]), "r"(w[i]), "r"(mk[k]));
+    // the comparisons are nested (t_1 <= t_2 <= ..), so bit 0 of their count is ((f1 & ~f2) | f3) & ~f4 | .. and
+    // bit 1 is (f2 & ~f4) | f6, bit 2 is f4 -- all in bit 3 of every nibble
+    uint32_t b0, b1;
+    asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(f[0]), "r"(f[1]), "r"(f[2]));
+    if constexpr (DB == 3) {
+      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(f[3]), "r"(f[4]));
+      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b0) : "r"(b0), "r"(f[5]), "r"(f[6]));
+      asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b1) : "r"(f[1]), "r"(f[3]), "r"(f[5]));
+      // third bits: nibble a of the word (flag in bit 4 a + 3) -> bit a of its half-word.  Moved to bit 4 a + 1, the
+      // shifts by 1, 4, 7, 10 bring a = 0 .. 3 to bits 0 .. 3 and no two copies share a bit (4 a - 3 j is different
+      // for every a and j): one high product.
+      const uint32_t g = __umulhi((f[3] >> 2) & 0x22222222u, (1u << 31) + (1u << 28) + (1u << 25) + (1u << 22));
+      third[i >> 2] |= (g & 0x000f000fu) << (4 * (i & 3));
+    } else {
+      b1 = f[1];
     }
-    const uint32_t m = zc[0] | (zc[1] << 2);       // byte 0: pairs 0, 1; byte 1: pairs 2, 3 (4 bits used of each)
-    half_bytes[i] = (m | (m >> 4)) & 0x00ff00ffu;  // the four codes of a half-word in its low byte
-    if constexpr (DB == 3) third[i >> 2] |= (hv[0] | (hv[1] << 1)) << (4 * (i & 3));
+    // low two bits of every new code into the low bits of its nibble, then the four codes of a half-word into its
+    // low byte (what lands in the upper byte is dropped by the byte permute below)
+    const uint32_t t = and_or(b0 >> 3, 0x11111111u, (b1 >> 2) & 0x22222222u);
+    const uint32_t u = (t | (t >> 2)) & 0x0f0f0f0fu;
+    half_bytes[i] = u | (u >> 4);
   }
   // slices 2h and 2h + 1 of a row share a 16-byte chunk of the destination tile
   char* db = reinterpret_cast<char*>(dst_codes) + tile * tile_bytes(DB);
@@ -258,7 +271,8 @@ __global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const vo
   for (int h = 0; h < 2; ++h) {
     const uint32_t* hb = half_bytes + 8 * h;
     *reinterpret_cast<uint4*>(db + slice_word_offset<DB>(r, 2 * h, 0)) =
-        make_uint4(hb[0] | (hb[1] << 8), hb[2] | (hb[3] << 8), hb[4] | (hb[5] << 8), hb[6] | (hb[7] << 8));
+        make_uint4(__byte_perm(hb[0], hb[1], 0x6240), __byte_perm(hb[2], hb[3], 0x6240), __byte_perm(hb[4], hb[5], 0x6240),
+                   __byte_perm(hb[6], hb[7], 0x6240));
   }
   if constexpr (DB == 3)
     *reinterpret_cast<uint4*>(db + slice_word_offset<3>(r, 0, 2)) = make_uint4(third[0], third[1], third[2], third[3]);
