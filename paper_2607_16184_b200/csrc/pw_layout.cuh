@@ -86,6 +86,49 @@ __device__ inline void unpack_slice(const uint32_t* w, int (&code)[32]) {
   }
 }
 
+// Two signed integers saturated to BITS-bit unsigned codes and packed, a above b, under the low bits of c moved
+// up by 2 * BITS: one instruction clamps and packs two codes.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack2_sat(int a, int b, uint32_t c) {
+  uint32_t d;
+  if constexpr (BITS == 8) asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  else if constexpr (BITS == 4) asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  else asm("cvt.pack.sat.u2.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// pack_slice for codes that have not been clamped from above yet (8, 4 or 2 bits): the same words, built from the
+// top of each word down with the saturating pack.
+template <int BITS>
+__device__ inline void pack_slice_sat(const int (&code)[32], uint32_t* w) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      w[i] = pack2_sat<8>(code[4 * i + 1], code[4 * i], pack2_sat<8>(code[4 * i + 3], code[4 * i + 2], 0u));
+  } else if constexpr (BITS == 4) {
+    // low half-word: the even codes of the word's eight, four bits each; high half-word: the odd ones
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int* c = code + 8 * i;
+      uint32_t v = pack2_sat<4>(c[7], c[5], 0u);
+      v = pack2_sat<4>(c[3], c[1], v);
+      v = pack2_sat<4>(c[6], c[4], v);
+      w[i] = pack2_sat<4>(c[2], c[0], v);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int* c = code + 16 * i;
+      uint32_t v = 0;
+#pragma unroll
+      for (int m = 3; m >= 0; --m) v = pack2_sat<2>(c[4 * m + 3], c[4 * m + 1], v);   // odd codes, from the top
+#pragma unroll
+      for (int m = 3; m >= 0; --m) v = pack2_sat<2>(c[4 * m + 2], c[4 * m], v);       // even codes below them
+      w[i] = v;
+    }
+  }
+}
+
 template <int BITS>
 __device__ inline void pack_slice(const int (&code)[32], uint32_t* w) {
   if constexpr (BITS == 8) {

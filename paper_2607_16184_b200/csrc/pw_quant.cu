@@ -110,10 +110,15 @@ __global__ void __launch_bounds__(512, NT == 2 ? 2 : 3) quant_tile_kernel(const 
   int code[32];
   __half sh;
   float lo;
-  group_quantize<SRC_BITS == 16>(v, h16, (1 << DST_BITS) - 1, code, sh, lo);
   constexpr int NW = SliceWords<DST_BITS>::kWords;
   uint32_t w[NW];
-  pack_slice<DST_BITS>(code, w);
+  if constexpr (DST_BITS == 3) {
+    group_quantize<SRC_BITS == 16>(v, h16, (1 << DST_BITS) - 1, code, sh, lo);
+    pack_slice<DST_BITS>(code, w);
+  } else {                                           // the upper clamp of the codes is the pack's saturation
+    group_quantize<SRC_BITS == 16, false>(v, h16, (1 << DST_BITS) - 1, code, sh, lo);
+    pack_slice_sat<DST_BITS>(code, w);
+  }
   if constexpr (DST_BITS == 8) {
     *reinterpret_cast<uint4*>(db + slice_word_offset<8>(r, q, 0)) = make_uint4(w[0], w[1], w[2], w[3]);
     *reinterpret_cast<uint4*>(db + slice_word_offset<8>(r, q, 4)) = make_uint4(w[4], w[5], w[6], w[7]);

@@ -11,7 +11,9 @@ namespace pw {
 
 // v: my 32 values; h16: the same as packed halves when the source was 16-bit (FROM_HALVES).  Returns my 32
 // codes, the group's scale and its minimum (the zero-point), identical on the four lanes of the row-group.
-template <bool FROM_HALVES>
+// CLAMP = false leaves the codes as rint((w - lo) / scale) without the upper clamp (never negative; a huge
+// quotient saturates at INT_MAX, NaN gives 0): for a caller whose packing saturates (pack_slice_sat).
+template <bool FROM_HALVES, bool CLAMP = true>
 __device__ __forceinline__ void group_quantize(const float (&v)[32], const __half2* h16, int L, int (&code)[32],
                                                __half& sh, float& lo_out) {
   // minimum and maximum of my 32 values (of fp16 sources taken on the packed halves: half as many operations,
@@ -54,8 +56,12 @@ __device__ __forceinline__ void group_quantize(const float (&v)[32], const __hal
   for (int i = 0; i < 32; ++i) {
     // round half to even and convert in one step (the product is never negative; a huge one saturates), then
     // clamp: the same code as clamp(rint(x), 0, L)
-    const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v[i], lo), rinv));
-    code[i] = (int)(c < (uint32_t)L ? c : (uint32_t)L);
+    if constexpr (CLAMP) {
+      const uint32_t c = __float2uint_rn(__fmul_rn(__fsub_rn(v[i], lo), rinv));
+      code[i] = (int)(c < (uint32_t)L ? c : (uint32_t)L);
+    } else {
+      code[i] = __float2int_rn(__fmul_rn(__fsub_rn(v[i], lo), rinv));
+    }
   }
   lo_out = lo;
 }
