@@ -177,6 +177,9 @@ void timing_mark(pw_ctx* ctx, int i, cudaStream_t s);
 // for the completion counters that kernel's epilogue raises (WsMap::done), and the kernel after it reads
 // nothing of the gate/up kernel's and waits for the down kernel before it reads anything at all.
 // With the timing events between the kernels the attribute has no effect.
+// Pointer qualifiers follow from this: `const __restrict__` (which allows non-coherent loads) only on data that
+// is final when the kernel is placed -- pages, page-table rows, anything written two or more kernels back; a
+// buffer that the kernel directly ahead writes is passed as a plain pointer and read after grid_dep_sync().
 __device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -222,11 +222,13 @@ __global__ void __launch_bounds__(1024) permute_kernel(const float* __restrict__
 // The same grid first writes the two unit lists from the tables of the permute kernel: unit u of a list is
 // (row tile, K split) pair u / TT and token tile u mod TT.
 constexpr int kGatherChunks = 4;
-__global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ row_token,
-                                                     const int32_t* __restrict__ offsets, int S, int H8, int Rpad,
-                                                     uint4* __restrict__ xt, const int32_t* __restrict__ counts,
-                                                     const int2* __restrict__ tile_tab, int max_tiles,
-                                                     const int32_t* __restrict__ n_units, int nt_tile, int ksplit,
+// row_token, offsets, counts, tile_tab and n_units are written by the kernel directly ahead, during this kernel's
+// lifetime: no __restrict__ on them, so that their loads cannot become non-coherent ones.
+__global__ void __launch_bounds__(256) gather_kernel(const uint4* __restrict__ hidden, const int32_t* row_token,
+                                                     const int32_t* offsets, int S, int H8, int Rpad,
+                                                     uint4* __restrict__ xt, const int32_t* counts,
+                                                     const int2* tile_tab, int max_tiles,
+                                                     const int32_t* n_units, int nt_tile, int ksplit,
                                                      int ng_gu, int ng_dn, int dn_token_tile_outer,
                                                      Unit* __restrict__ units_gu, Unit* __restrict__ units_dn,
                                                      int32_t* __restrict__ done) {
@@ -307,7 +309,7 @@ constexpr int kCombineCols = 64, kCombineRows = 4, kMaxSplit = 8;
 // prompt (thousands of tokens: fewer, fatter CTAs), one for a decode batch (more CTAs for the few tokens).
 template <int kCombineChunks>
 __global__ void __launch_bounds__(kCombineCols * kCombineRows)
-    combine_kernel(const float4* __restrict__ y, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
+    combine_kernel(const float4* y /* written by the kernel directly ahead */, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
                    int T, int k, int n_shared, int H4, int ksplit, size_t split_stride4, float4* __restrict__ out) {
   grid_dep_sync();
   grid_dep_trigger();
@@ -379,7 +381,7 @@ __global__ void __launch_bounds__(kCombineCols * kCombineRows)
 // are those of combine_kernel (splits added in split order, times the gate, terms added in choice order).
 template <int U>
 __global__ void __launch_bounds__(128)
-    combine_stream_kernel(const float4* __restrict__ y, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
+    combine_stream_kernel(const float4* y /* written by the kernel directly ahead */, const float* __restrict__ gates, const int32_t* __restrict__ inv_perm,
                           int T, int k, int n_shared, int H4, int ksplit, size_t split_stride4, float4* __restrict__ out) {
   grid_dep_sync();
   grid_dep_trigger();
