@@ -228,6 +228,19 @@ __device__ __forceinline__ void tc_commit(unsigned long long* b) {
 __device__ __forceinline__ void tc_commit_s(uint32_t bar_s) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_s) : "memory");
 }
+// predicated forms for code that the whole warp runs and one lane acts on
+__device__ __forceinline__ void tc_commit_if_s(uint32_t bar_s, uint32_t on) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar_s),
+      "r"(on)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n_if_s(uint32_t bar_s, uint32_t n, uint32_t on) {
+  asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q mbarrier.arrive.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar_s),
+               "r"(n), "r"(on)
+               : "memory");
+}
 // A operand in tensor memory
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
@@ -251,30 +264,34 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint
 // NK consecutive k-steps of one item issued from one asm block (the issuing thread gets few issue slots,
 // so every instruction around an MMA counts).  Descriptors are passed as (lo, hi) words; only lo moves.
 // TS: A in tensor memory at a_tmem (+a_step per k-step).  `acc0`: accumulate flag of the first k-step.
+// `on`: the whole warp runs the issuer's code with the same values (so that the operands can live in uniform
+// registers), and the lane with on != 0 issues.
 template <int NK>
 __device__ __forceinline__ void tc_mma_ts_burst(uint32_t d_tmem, uint32_t a_tmem, uint32_t a_step, uint32_t b_lo,
-                                                uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t acc0) {
+                                                uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t acc0, uint32_t on) {
   asm volatile(
-      "{\n\t.reg .pred p, t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
+      "{\n\t.reg .pred p, t, q;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
       "setp.ne.b32 p, %7, 0;\n\t"
+      "setp.ne.b32 q, %8, 0;\n\t"
       "setp.eq.b32 t, 0, 0;\n\t"
       "mov.b64 bd, {%3, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %6, p;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %6, p;\n\t"
       "add.u32 lo, %3, %5;\n\tadd.u32 a, %1, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
       "}" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
+      "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0), "r"(on)
       : "memory");
   if (NK == 4) {
     asm volatile(
-        "{\n\t.reg .pred t;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
+        "{\n\t.reg .pred t, q;\n\t.reg .b64 bd;\n\t.reg .b32 lo, a;\n\t"
         "setp.eq.b32 t, 0, 0;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
         "mad.lo.u32 lo, %5, 2, %3;\n\tmad.lo.u32 a, %2, 2, %1;\n\tmov.b64 bd, {lo, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
         "add.u32 lo, lo, %5;\n\tadd.u32 a, a, %2;\n\tmov.b64 bd, {lo, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %6, t;\n\t"
         "}" ::"r"(d_tmem),
-        "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        "r"(a_tmem), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(on)
         : "memory");
   }
 }
@@ -282,28 +299,30 @@ __device__ __forceinline__ void tc_mma_ts_burst(uint32_t d_tmem, uint32_t a_tmem
 template <int NK>
 __device__ __forceinline__ void tc_mma_ss_burst(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step,
                                                 uint32_t b_lo, uint32_t b_hi, uint32_t b_step, uint32_t idesc,
-                                                uint32_t acc0) {
+                                                uint32_t acc0, uint32_t on) {
   asm volatile(
-      "{\n\t.reg .pred p, t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
+      "{\n\t.reg .pred p, t, q;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
       "setp.ne.b32 p, %8, 0;\n\t"
+      "setp.ne.b32 q, %9, 0;\n\t"
       "setp.eq.b32 t, 0, 0;\n\t"
       "mov.b64 ad, {%1, %2};\n\tmov.b64 bd, {%4, %5};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, p;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, p;\n\t"
       "add.u32 la, %1, %3;\n\tadd.u32 lb, %4, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
       "}" ::"r"(d_tmem),
-      "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0)
+      "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(acc0), "r"(on)
       : "memory");
   if (NK == 4) {
     asm volatile(
-        "{\n\t.reg .pred t;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
+        "{\n\t.reg .pred t, q;\n\t.reg .b64 ad, bd;\n\t.reg .b32 la, lb;\n\t"
         "setp.eq.b32 t, 0, 0;\n\t"
+        "setp.ne.b32 q, %8, 0;\n\t"
         "mad.lo.u32 la, %3, 2, %1;\n\tmad.lo.u32 lb, %6, 2, %4;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
         "add.u32 la, la, %3;\n\tadd.u32 lb, lb, %6;\n\tmov.b64 ad, {la, %2};\n\tmov.b64 bd, {lb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %7, t;\n\t"
         "}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc)
+        "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(on)
         : "memory");
   }
 }
@@ -566,7 +585,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
   char* bslots = wring + n_slots * kSlotBytes;
   const int bslot_bytes = nt_tile * 256;
   constexpr int NMAT = PHASE == 0 ? 2 : 1;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the warp number, broadcast: what follows from it (role, group, slot and barrier addresses) is then known to the
+  // compiler as the same in all lanes and can be computed and kept in uniform registers
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int n_units = n_units_ptr[PHASE];
   // tensor-memory columns: partial accumulators first ([matrix][partial][nt_tile]), dequantized-operand
   // slots after them.  Partials per matrix: as many as issuers per matrix, while two operand slots still fit.
@@ -802,7 +823,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // all eight k-steps of it into its own partial accumulator; a quantized tile k is dequantized by the
     // matrix's group k mod IPM, so with npart == IPM every dequantizer group has an issuer of its own.
     // The epilogue adds the partials.
+    // The whole warp runs the issuer's code on the same values -- the warp number is broadcast so that the compiler
+    // knows it -- and lane 0 issues, commits and arrives: descriptors and addresses computed by a converged warp
+    // can stay in uniform registers, which is where the MMA takes its operands from.
     const int iss = warp - kWarpMma;
+    const uint32_t on = lane == 0 ? 1u : 0u;
     const int my_m = iss / IPM, my_j = iss % IPM;
     const uint32_t desc_hi = (uint32_t)(make_kmajor_desc(0, 0) >> 32);
     const uint32_t b_lo_base = smem_u32(bslots) >> 4;
@@ -831,7 +856,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         auto release_turn = [&](uint32_t tord) {
           if (shared_acc) {
             tc_fence_before();
-            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_s), "r"(tord + 1) : "memory");
+            if (on) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_s), "r"(tord + 1) : "memory");
           }
         };
 #pragma unroll 1
@@ -860,10 +885,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
               if (!ok) break;
               tc_fence_after();
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
-              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh);
+              tc_mma_ss_burst<4>(d_t, a_lo, desc_hi, 256, b_lo + 4 * hh * b_step, desc_hi, b_step, idesc, later | hh, on);
               if (hh == 1) release_turn(tord);
-              mbar_arrive_n(&c->empty[hp.s], 3);       // with the commit: the four arrivals of the slot's phase
-              tc_commit(&c->empty[hp.s]);
+              mbar_arrive_n_if_s(smem_u32(&c->empty[hp.s]), 3, on);   // with the commit: the four arrivals of the slot's phase
+              tc_commit_if_s(smem_u32(&c->empty[hp.s]), on);
               ring_advance(hp, 1, (uint32_t)n_slots);
             }
             if (!ok) break;
@@ -882,12 +907,12 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             if (!ok) break;
             tc_fence_after();
             // all eight k-steps of the tile, then one commit hands the group's operand slot back
-            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later);
-            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u);
+            tc_mma_ts_burst<4>(d_t, a_t, 8, b_lo, desc_hi, b_step, idesc, later, on);
+            tc_mma_ts_burst<4>(d_t, a_t + 32, 8, b_lo + 4 * b_step, desc_hi, b_step, idesc, 1u, on);
             release_turn(tord);
-            tc_commit_s(e0);
+            tc_commit_if_s(e0, on);
           }
-          tc_commit_s(be_s + 8 * bp.s);
+          tc_commit_if_s(be_s + 8 * bp.s, on);
           later = 1;
           bt += (uint32_t)ipa;
           ring_advance(bp, (uint32_t)ipa, (uint32_t)n_bslots);
@@ -895,7 +920,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         return ok;
     };
     if constexpr (!HELP) {
-    if (lane == 0 && my_j < ipa) {
+    if (my_j < ipa) {
       uint32_t seq_unit = 0;                        // slot items before the current unit
       uint32_t base = 0;                            // tiles of one matrix (= token tiles) before the current unit
       uint32_t upar = 0;                            // per group: parity of the next use of its operand slot
@@ -940,11 +965,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
         if (ok) {
           if (wide || dbuf == 0) {
-            tc_commit(&c->d_full[0]);
+            tc_commit_if_s(smem_u32(&c->d_full[0]), on);
             ++duse0;
           }
           if (wide || dbuf == 1) {
-            tc_commit(&c->d_full[1]);
+            tc_commit_if_s(smem_u32(&c->d_full[1]), on);
             ++duse1;
           }
         }
@@ -995,7 +1020,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
         const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + (int)my_p) * nb_rows);
-        if (lane == 0 && issuing) {
+        if (issuing) {
           do {
         // the epilogue has drained the buffer(s) this unit accumulates into
         if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
@@ -1004,8 +1029,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         tc_fence_after();
         ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
             if (ok) {
-              if (wide || dbuf == 0) tc_commit(&c->d_full[0]);
-              if (wide || dbuf == 1) tc_commit(&c->d_full[1]);
+              if (wide || dbuf == 0) tc_commit_if_s(smem_u32(&c->d_full[0]), on);
+              if (wide || dbuf == 1) tc_commit_if_s(smem_u32(&c->d_full[1]), on);
             }
           } while (false);
         }
