@@ -212,6 +212,27 @@ __device__ __forceinline__ void bulk_g2s_s(uint32_t dst_s, const void* src, uint
                "l"(src), "r"(bytes), "r"(bar_s)
                : "memory");
 }
+// predicated forms (the whole warp runs the producer's code, one lane acts)
+__device__ __forceinline__ void mbar_expect_tx_if_s(uint32_t bar_s, uint32_t bytes, uint32_t on) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar_s),
+      "r"(bytes), "r"(on)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_if_s(uint32_t dst_s, const void* src, uint32_t bytes, uint32_t bar_s, uint32_t on) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %4, 0;\n\t"
+      "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}" ::"r"(dst_s),
+      "l"(src), "r"(bytes), "r"(bar_s), "r"(on)
+      : "memory");
+}
+__device__ __forceinline__ void tma_2d_g2s_if_s(uint32_t dst_s, const CUtensorMap* map, int x, int y, uint32_t bar_s, uint32_t on) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n\t}" ::"r"(dst_s),
+      "l"(map), "r"(x), "r"(y), "r"(bar_s), "r"(on)
+      : "memory");
+}
 __device__ __forceinline__ void tma_2d_g2s(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
@@ -651,8 +672,10 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // ---------------- weight producers ----------------
     // Two single-thread producers share the stream: producer P arms the slot items with number = P mod 2,
     // which (even slot count) always land in the slots = P mod 2, so each keeps the state of its own slots.
-    // Producer 0 also claims the units.
-    if (lane == 0) {
+    // Producer 0 also claims the units.  The whole warp runs the loop on the same values; lane 0 arms, copies,
+    // claims and posts.
+    {
+      const uint32_t on = lane == 0 ? 1u : 0u;
       const uint32_t P = warp == kWarpCodes ? 0u : 1u;
       uint32_t seq = 0, s = 0;                     // number and slot of the next slot item of the stream
       // A slot is free for slot item seq once the phase seq / n_slots - 1 of its empty barrier has completed
@@ -676,16 +699,18 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       };
       // producer 0 posts a unit: its index, and the unit with the bitwidths of its pages for the other roles
       auto post = [&](uint32_t idx, int uu) {
-        if (uu >= 0) {
-          Unit d = un;
-          d.pad_ = (int32_t)(row_ubits<PLANES>(rw[0]) | (row_ubits<PLANES>(rw[NMAT - 1]) << 8));
-          int4* dp = reinterpret_cast<int4*>(&c->desc[idx & 15]);
-          dp[0] = make_int4(d.seg, d.row_tile, d.tok0, d.ntok);
-          dp[1] = make_int4(d.g0, d.g1, d.split, d.pad_);
+        if (on) {
+          if (uu >= 0) {
+            Unit d = un;
+            d.pad_ = (int32_t)(row_ubits<PLANES>(rw[0]) | (row_ubits<PLANES>(rw[NMAT - 1]) << 8));
+            int4* dp = reinterpret_cast<int4*>(&c->desc[idx & 15]);
+            dp[0] = make_int4(d.seg, d.row_tile, d.tok0, d.ntok);
+            dp[1] = make_int4(d.g0, d.g1, d.split, d.pad_);
+          }
+          c->sched_unit[idx & 31] = uu;
+          __threadfence_block();
+          c->sched_n = idx + 1;
         }
-        c->sched_unit[idx & 31] = uu;
-        __threadfence_block();
-        c->sched_n = idx + 1;
       };
       if (u >= 0) fetch_info(u);
       if (P == 0) post(0u, u);
@@ -711,7 +736,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 #pragma unroll 1
         for (int g = 0; ok && g < ng; ++g) {
           // claim the next unit half-way through this one: the answer is back long before it is needed
-          if (P == 0 && g == claim_at) claimed = atomicAdd(work_counter, 1) + G;
+          if (P == 0 && g == claim_at) {
+            int got = 0;
+            if (on) got = atomicAdd(work_counter, 1);
+            claimed = __shfl_sync(0xffffffffu, got, 0) + G;
+          }
 #pragma unroll
           for (int m = 0; m < NMAT; ++m) {
             const bool f16 = ms[m].bits == 16;
@@ -731,17 +760,17 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
                 if (pass) ok = mbar_wait_s<LIM>(smem_u32(&c->empty[s]), (pass - 1) & 1, c, status);
                 if (!ok) break;
                 const uint32_t bar_s = full_s + 8 * s;
-                mbar_expect_tx_s(bar_s, bytes);
+                mbar_expect_tx_if_s(bar_s, bytes, on);
                 const uint32_t slot_s = wring_s + s * kSlotBytes;
                 if (q) {
-                  bulk_g2s_s(slot_s, src, kPlaneTopCodes, bar_s);
-                  bulk_g2s_s(slot_s + kPlaneSlotLut, src + plane_lut_offset((int)q), 512, bar_s);
-                  if (q >= 3) bulk_g2s_s(slot_s + kPlaneSlotBit1, b1, kPlaneBitTile, bar_s);
-                  if (q == 4) bulk_g2s_s(slot_s + kPlaneSlotBit0, b0, kPlaneBitTile, bar_s);
+                  bulk_g2s_if_s(slot_s, src, kPlaneTopCodes, bar_s, on);
+                  bulk_g2s_if_s(slot_s + kPlaneSlotLut, src + plane_lut_offset((int)q), 512, bar_s, on);
+                  if (q >= 3) bulk_g2s_if_s(slot_s + kPlaneSlotBit1, b1, kPlaneBitTile, bar_s, on);
+                  if (q == 4) bulk_g2s_if_s(slot_s + kPlaneSlotBit0, b0, kPlaneBitTile, bar_s, on);
                 } else {
-                  bulk_g2s_s(slot_s, src, bytes, bar_s);
+                  bulk_g2s_if_s(slot_s, src, bytes, bar_s, on);
                 }
-                c->issued[P] = seq + 2;                // my next slot item is seq + 2
+                if (on) c->issued[P] = seq + 2;        // my next slot item is seq + 2
               }
               ++seq;
               if (++s == (uint32_t)n_slots) {
@@ -764,7 +793,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     }
   } else if (warp == kWarpTokens) {
     // ---------------- token-tile producer ----------------
-    if (lane == 0) {
+    // (the whole warp runs the loop on the same values; lane 0 arms and copies)
+    {
+      const uint32_t on = lane == 0 ? 1u : 0u;
       // The gate/up kernel waits for the kernel ahead of it (which gathers its token rows).  The down kernel does
       // not wait for the gate/up kernel as a whole: its CTAs take the SMs that kernel's CTAs leave one by one, and
       // a unit starts as soon as the gate/up units that write the rows it multiplies have been counted in.
@@ -787,6 +818,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           int seen = 0;
           for (uint32_t n = 0;; ++n) {
             asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+            seen = __shfl_sync(0xffffffffu, seen, 0);    // one answer for the warp
             if (seen >= need) break;
             // the gate/up kernel gave up (a wait of its own ran out), or this wait has lasted 2 s
             if (n >= LIM * 64u || *reinterpret_cast<volatile int32_t*>(status) == (int)PW_ERR_TIMEOUT) {
@@ -809,10 +841,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
           const int bs = bcount % n_bslots;
           ok = mbar_wait_s<LIM>(smem_u32(&c->b_empty[bs]), ((bcount / n_bslots) & 1) ^ 1, c, status);
           if (!ok) break;
-          mbar_expect_tx(&c->b_full[bs], nb_rows * 256);
-          tma_2d_g2s(bslots + (size_t)bs * bslot_bytes, map, un.tok0 * 2, g * 16, &c->b_full[bs]);
+          const uint32_t bf_bar = smem_u32(&c->b_full[bs]);
+          mbar_expect_tx_if_s(bf_bar, (uint32_t)(nb_rows * 256), on);
+          tma_2d_g2s_if_s(smem_u32(bslots) + (uint32_t)(bs * bslot_bytes), map, un.tok0 * 2, g * 16, bf_bar, on);
           ++bcount;
-          c->b_issued = bcount;
+          if (on) c->b_issued = bcount;
         }
       }
     }
