@@ -179,6 +179,25 @@ def time_region(fn, steps, device):
     return e0.elapsed_time(e1)
 
 
+def time_region_chunks(fn, steps, device, chunk=50):
+    """time_region with an event every `chunk` steps as well (one event per 50 calls does not disturb the chain):
+    returns the total and the per-step times of the chunks, for a median and a best figure."""
+    torch.cuda.synchronize(device)
+    replicas.barrier(device)
+    marks = [torch.cuda.Event(enable_timing=True)]
+    marks[0].record()
+    for i in range(steps):
+        fn(i)
+        if (i + 1) % chunk == 0 or i + 1 == steps:
+            marks.append(torch.cuda.Event(enable_timing=True))
+            marks[-1].record()
+    torch.cuda.synchronize(device)
+    replicas.barrier(device)
+    bounds = [min((j + 1) * chunk, steps) - j * chunk for j in range(len(marks) - 1)]
+    per_step = [marks[j].elapsed_time(marks[j + 1]) / n for j, n in enumerate(bounds) if n == chunk]
+    return marks[0].elapsed_time(marks[-1]), per_step
+
+
 def cpu_oracle_sample(cfg, layer_pages_host, x, logits, n_tokens):
     """Times the CPU oracle, as it stands, on the first n_tokens tokens of the batch."""
     from oracle import oracle
@@ -511,10 +530,13 @@ def run_gpu(args):
     n_steady = max(args.steps, int(np.ceil(args.steady_seconds / (ms_step * 1e-3))))
     sampler2 = ClockSampler(device.index or 0)
     sampler2.start()
-    ms_steady = time_region(step, n_steady, device) / n_steady
+    ms_steady_total, chunk_ms = time_region_chunks(step, n_steady, device)
+    ms_steady = ms_steady_total / n_steady
     clocks2 = sampler2.stop()
     kavg2, _ = kernel_pass(ctx, step, n_steady, device)
     steady = {"steps": n_steady, "ms_per_step": ms_steady, "tokens_per_s": T / (ms_steady * 1e-3),
+              "median_ms_per_step": float(np.median(chunk_ms)) if chunk_ms else None,      # over chunks of 50 steps
+              "best_ms_per_step": float(np.min(chunk_ms)) if chunk_ms else None,
               "sm_mhz": clocks2["sm_mhz"], "reasons": clocks2["reasons"],
               "roofline_frac": gbs(gu_kernel_bytes, kavg2["ffn_gate_up"]) / peaks["hbm_gbs"],
               "gate_up_ms": kavg2["ffn_gate_up"], "down_ms": kavg2["ffn_down"],
