@@ -513,6 +513,22 @@ __device__ __forceinline__ void signal_rows_done(int32_t* done, int tok0, int ro
   }
 }
 
+// Accumulators per matrix of a unit with nb_rows token columns.  The decode kernels give a unit as many partial
+// accumulators per matrix as there are issuers per matrix.  For token tiles wider than 32 that fills more than half
+// of the accumulator columns: the unit takes both accumulator buffers, and its epilogue cannot overlap the next
+// unit's MMAs.  The SHARE instantiations, launched where the epilogue is a large part of a unit (units of at most
+// kShortUnitTiles weight tiles), give such a unit fewer accumulators instead, the issuers of a matrix taking turns
+// on them tile by tile (the turn word below), and it keeps to one buffer: fine-grained decode, down kernel -12 %,
+// gate/up -4 %.  On long units the turns buy nothing, and the code for them costs the gate/up kernel 1 %.
+constexpr int kShortUnitTiles = 32;
+template <bool SHARE, int NMAT>
+__device__ __forceinline__ int unit_accumulators(int npart, int nb_rows, int acol) {
+  int npe = npart;
+  if (SHARE)
+    while (npe > 1 && NMAT * npe * nb_rows > acol / 2) npe >>= 1;
+  return npe;
+}
+
 // PHASE 0: units of (expert, 128 FFN rows, token tile): gate and up pages -> Ht.
 // PHASE 1: units of (expert, 128 hidden rows, token tile, K range): down page -> Y[split].
 // PLANES: the instantiation that also reads blocks of overlaid bit-planes; launched only for a layer that holds one
@@ -520,7 +536,7 @@ __device__ __forceinline__ void signal_rows_done(int32_t* done, int tok0, int ro
 // SHORT: the instantiation with the short wait limit (kTestWaitPolls instead of kDefaultWaitPolls), for the test of
 // the failure path.  hook: test hook, bit 0 = the token-tile producer stops before its second tile (so that the
 // waits on it run out).
-template <int PHASE, bool HELP, bool PLANES, bool SHORT>
+template <int PHASE, bool HELP, bool PLANES, bool SHORT, bool SHARE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t* __restrict__ n_units_ptr,
               const __grid_constant__ TmapSet tmaps, int Rpad, int nt_tile, int n_bslots, int n_slots,
@@ -801,28 +817,35 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
     // the ring, or the operand slot of the group that dequantized the tile), eight MMAs, hand-backs.  One body for
     // both instantiations of the issuer role below.
     uint32_t b_known = 0;                          // token tiles known to have been armed
-    // accumulator of this issuer (several issuers per accumulator when npart < IPM) and its turn word
-    const uint32_t my_p = (uint32_t)my_j & (uint32_t)(npart - 1);
-    constexpr bool shared_acc = kSharedAcc;
-    const uint32_t npart_log = npart == 4 ? 2u : npart == 2 ? 1u : 0u;
-    const uint32_t turn_s = smem_u32(const_cast<uint32_t*>(&c->turn[my_m * npart + (int)my_p]));
+    // npe: accumulators per matrix of the unit (unit_accumulators); tile k of the matrix goes to accumulator
+    // k mod npe.  When that is fewer than the issuers of the matrix, the tiles of an accumulator are issued in
+    // order by different issuers: its turn word holds 1 + the number of the last tile whose MMAs are in the pipe.
+    // Never more than two issuers share an accumulator (half of the accumulator columns always holds two token
+    // tiles of the down kernel, one per matrix of the gate/up kernel), so the only other writer of the word a tile
+    // waits on is the issuer of the tile before it -- which writes a later number only after that tile.  The first
+    // tile of a unit on an accumulator waits for nobody: the buffer was handed back by the epilogue.
     auto issue_tiles = [&](uint32_t j0, uint32_t ng, uint32_t base, uint32_t W, uint32_t my_bits, uint32_t d_t,
                            uint32_t b_lo_unit, uint32_t b_step, uint32_t idesc, uint32_t& bt, RingPos& bp, uint32_t& sq,
-                           RingPos& rp, uint32_t& upar) -> bool {
+                           RingPos& rp, uint32_t& upar, uint32_t npe) -> bool {
         bool ok = true;
+        const bool shared_acc = SHARE ? npe < (uint32_t)ipa : kSharedAcc;
+        const uint32_t turn_s = smem_u32(const_cast<uint32_t*>(&c->turn[my_m * npart + (my_j & ((int)npe - 1))]));
         // accumulate onto earlier tiles: after my first tile, and from the start when the accumulator's first tile
         // of this unit is another issuer's
-        uint32_t later = j0 >= (uint32_t)npart ? 1u : 0u;
+        uint32_t later = j0 >= npe ? 1u : 0u;
         // my MMAs are in the pipe: the accumulator's next tile may follow
-        auto release_turn = [&](uint32_t tord) {
+        auto release_turn = [&](uint32_t k) {
           if (shared_acc) {
             tc_fence_before();
-            if (on) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_s), "r"(tord + 1) : "memory");
+            // (a maximum, not a store: the issuer that goes first in the next unit may already have written a later
+            // number when the one that closes this unit gets here)
+            if (on) asm volatile("red.shared.max.u32 [%0], %1;" ::"r"(turn_s), "r"(k + 1) : "memory");
           }
         };
 #pragma unroll 1
         for (uint32_t j = j0; ok && j < ng; j += (uint32_t)ipa) {
-          const uint32_t tord = (base + j) >> npart_log;   // number of this tile among the tiles of its accumulator
+          const uint32_t tord = base + j;              // number of this tile among the tiles of its matrix
+          const bool after = shared_acc && j >= npe;   // another issuer's tile of this unit precedes it on the accumulator
           // the token tile of this group (a tile is looked at only once it is known to have been armed; the
           // producer is usually ahead, and one look at its counter covers the tiles up to it)
           if (b_known <= bt) {
@@ -842,7 +865,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 #pragma unroll 1
             for (uint32_t hh = 0; hh < 2; ++hh) {
               ok = wait_issued<LIM>(sq + hh, c, status) && mbar_wait_s<LIM>(smem_u32(&c->full[hp.s]), hp.par, c, status);
-              if (ok && shared_acc && hh == 0 && tord > 0) ok = flag_wait<LIM>(turn_s, tord - 1, c, status);
+              if (ok && after && hh == 0) ok = flag_wait<LIM>(turn_s, tord - npe, c, status);
               if (!ok) break;
               tc_fence_after();
               const uint32_t a_lo = (w_lo_base + hp.s * (kSlotBytes >> 4)) | a_lo_lbo;
@@ -864,7 +887,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
             const uint32_t f0 = af_s + 8 * grp, e0 = ae_s + 8 * grp;       // barriers of the group's operand slot
             const uint32_t a_t = a_base + grp * 64;
             ok = mbar_wait_s<LIM>(f0, use_par, c, status);
-            if (ok && shared_acc && tord > 0) ok = flag_wait<LIM>(turn_s, tord - 1, c, status);
+            if (ok && after) ok = flag_wait<LIM>(turn_s, tord - npe, c, status);
             if (!ok) break;
             tc_fence_after();
             // all eight k-steps of the tile, then one commit hands the group's operand slot back
@@ -914,16 +937,17 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
         RingPos rp = ring_pos(sq, (uint32_t)n_slots);
-        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const int npe = unit_accumulators<SHARE, NMAT>(npart, nb_rows, acol);
+        const bool wide = NMAT * npe * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
-        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + (int)my_p) * nb_rows);
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npe + (my_j & (npe - 1))) * nb_rows);
         // the epilogue has drained the buffer(s) this unit accumulates into
         if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[0]), (duse0 & 1) ^ 1, c, status);
         if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         tc_fence_after();
-        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
+        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar, (uint32_t)npe);
         if (ok) {
           if (wide || dbuf == 0) {
             tc_commit_if_s(smem_u32(&c->d_full[0]), on);
@@ -977,10 +1001,11 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
         RingPos rp = ring_pos(sq, (uint32_t)n_slots);
-        const bool wide = NMAT * npart * nb_rows > acol / 2;
+        const int npe = unit_accumulators<SHARE, NMAT>(npart, nb_rows, acol);
+        const bool wide = NMAT * npe * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
         if (!wide) dtoggle ^= 1u;
-        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npart + (int)my_p) * nb_rows);
+        const uint32_t d_t = tmem + dbuf * (uint32_t)(acol / 2) + (uint32_t)((my_m * npe + (my_j & (npe - 1))) * nb_rows);
         if (issuing) {
           do {
         // the epilogue has drained the buffer(s) this unit accumulates into
@@ -988,7 +1013,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (ok && (wide || dbuf == 1)) ok = mbar_wait_s<LIM>(smem_u32(&c->d_empty[1]), (duse1 & 1) ^ 1, c, status);
         if (!ok) break;
         tc_fence_after();
-        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar);
+        ok = issue_tiles(j0, ng, base, W, my_bits, d_t, b_lo_unit, b_step, idesc, bt, bp, sq, rp, upar, (uint32_t)npe);
             if (ok) {
               if (wide || dbuf == 0) tc_commit_if_s(smem_u32(&c->d_full[0]), on);
               if (wide || dbuf == 1) tc_commit_if_s(smem_u32(&c->d_full[1]), on);
@@ -1007,7 +1032,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         if (!ok) break;
         if (wide) {
           tc_fence_after();
-          const uint32_t p0 = base & (uint32_t)(npart - 1), nq = ng < (uint32_t)npart ? ng : (uint32_t)npart;
+          const uint32_t p0 = base & (uint32_t)(npe - 1), nq = ng < (uint32_t)npe ? ng : (uint32_t)npe;
           const int row = un.row_tile * kTileRows + hr;
           const int half = ((nb_rows / 16 + 1) / 2) * 16;         // the epilogue warps take [0, half)
           for (int c0 = half; c0 < nb_rows; c0 += 16) {
@@ -1015,14 +1040,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 #pragma unroll
             for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
             for (uint32_t q = 0; q < nq; ++q) {
-              const int p = (int)((p0 + q) & (uint32_t)(npart - 1));
+              const int p = (int)((p0 + q) & (uint32_t)(npe - 1));
               float t[16];
               tmem_ld16(hlane_addr + p * nb_rows + c0, t);
               tmem_wait_ld();
 #pragma unroll
               for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
               if (PHASE == 0) {
-                tmem_ld16(hlane_addr + (npart + p) * nb_rows + c0, t);
+                tmem_ld16(hlane_addr + (npe + p) * nb_rows + c0, t);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
@@ -1129,7 +1154,8 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       if (u < 0) break;
       const Unit un = load_desc(c, (uint32_t)i);
       const int nb_rows = (un.ntok + 15) & ~15;
-      const bool wide = NMAT * npart * nb_rows > acol / 2;
+      const int npe = unit_accumulators<SHARE, NMAT>(npart, nb_rows, acol);    // the issuers' rule
+      const bool wide = NMAT * npe * nb_rows > acol / 2;
       const uint32_t dbuf = wide ? 0u : dtoggle;
       if (!wide) dtoggle ^= 1u;
       if (wide || dbuf == 0) ok = mbar_wait_s<LIM>(smem_u32(&c->d_full[0]), duse0 & 1, c, status);
@@ -1143,7 +1169,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
       // and not on how many tiles this CTA has seen before it (units are claimed in a different order from run
       // to run): a forward call repeats bit for bit.
       const uint32_t ng = (uint32_t)(un.g1 - un.g0);
-      const uint32_t p0 = base & (uint32_t)(npart - 1), nq = ng < (uint32_t)npart ? ng : (uint32_t)npart;
+      const uint32_t p0 = base & (uint32_t)(npe - 1), nq = ng < (uint32_t)npe ? ng : (uint32_t)npe;
       base += ng;
       // with helpers, the issuer warps take the upper half of the token columns of a wide unit
       const int c_end = HELP && wide ? ((nb_rows / 16 + 1) / 2) * 16 : nb_rows;
@@ -1152,14 +1178,14 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 #pragma unroll
         for (int j = 0; j < 16; ++j) a[j] = b[j] = 0.0f;
         for (uint32_t q = 0; q < nq; ++q) {            // add the issuers' partial sums, in the unit's tile order
-          const int p = (int)((p0 + q) & (uint32_t)(npart - 1));
+          const int p = (int)((p0 + q) & (uint32_t)(npe - 1));
           float t[16];
           tmem_ld16(dbase + p * nb_rows + c0, t);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; ++j) a[j] = __fadd_rn(a[j], t[j]);
           if (PHASE == 0) {
-            tmem_ld16(dbase + (npart + p) * nb_rows + c0, t);
+            tmem_ld16(dbase + (npe + p) * nb_rows + c0, t);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 16; ++j) b[j] = __fadd_rn(b[j], t[j]);
@@ -1231,7 +1257,11 @@ static bool make_maps(EncodeTiledFn enc, void* base, int n_chunks, int Rpad, Tma
 
 typedef void (*FfnKernel)(const DevRow*, const Unit*, const int32_t*, const TmapSet, int, int, int, int, __half*, float*, int, size_t,
                           int32_t*, int32_t*, int32_t*, int, int, uint32_t);
-static FfnKernel ffn_kernel_of(int phase, int help, int planes) {
+// share: the instantiation whose wide units take fewer accumulators (decode kernels only)
+static FfnKernel ffn_kernel_of(int phase, int help, int planes, int share = 0) {
+  static const FfnKernel shared[4] = {ffn_tc_kernel<0, false, false, false, true>, ffn_tc_kernel<1, false, false, false, true>,
+                                      ffn_tc_kernel<0, false, true, false, true>, ffn_tc_kernel<1, false, true, false, true>};
+  if (share && !help) return shared[phase + 2 * planes];
   static const FfnKernel tab[8] = {
       ffn_tc_kernel<0, false, false, false>, ffn_tc_kernel<1, false, false, false>, ffn_tc_kernel<0, true, false, false>,
       ffn_tc_kernel<1, true, false, false>,  ffn_tc_kernel<0, false, true, false>,  ffn_tc_kernel<1, false, true, false>,
@@ -1258,6 +1288,9 @@ static pw_status tc_setup(pw_ctx* ctx) {
   }
   for (int i = 0; i < 8; ++i)
     PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_of(i & 1, (i >> 1) & 1, (i >> 2) & 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxDynSmem));
+  for (int i = 0; i < 4; ++i)
+    PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_of(i & 1, 0, (i >> 1) & 1, 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     kMaxDynSmem));
   PW_CUDA_OK(cudaFuncSetAttribute(ffn_kernel_short(), cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
   ctx->tc_state = st;
@@ -1331,13 +1364,16 @@ pw_status launch_ffn_tensor(pw_ctx* ctx, int layer, int T, int k, int nt_tile, i
   const bool planes = planes_layer(ctx, layer);
   // a context with a lowered wait limit (pw_debug_set_wait) runs the gate/up kernel's short-limit instantiation
   const bool short_wait = ctx->wait_polls != 0 && !help && !planes;
-  PW_CUDA_OK(launch_dependent(short_wait ? ffn_kernel_short() : ffn_kernel_of(0, help, planes), dim3(ctx->num_sms),
+  // short units (few weight tiles between two epilogues): the instantiations that keep wide units to one buffer
+  const int share_gu = 2 * (c.hidden / kGroup) <= kShortUnitTiles;
+  const int share_dn = (c.ffn / kGroup + ksplit - 1) / ksplit <= kShortUnitTiles;
+  PW_CUDA_OK(launch_dependent(short_wait ? ffn_kernel_short() : ffn_kernel_of(0, help, planes, share_gu), dim3(ctx->num_sms),
                               dim3(kThreads), (size_t)smem[0], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_gu), n_units, st->xt, w.Rpad, nt_tile, n_bslots[0],
                               n_slots[0], reinterpret_cast<__half*>(b + w.ht), (float*)nullptr, c.hidden, (size_t)0,
                               work_counter, status, reinterpret_cast<int32_t*>(b + w.done), ksplit, c.ffn / kTileRows, ctx->test_hook));
   timing_mark(ctx, PW_K_FFN_DOWN, s);
-  PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
+  PW_CUDA_OK(launch_dependent(ffn_kernel_of(1, help, planes, share_dn), dim3(ctx->num_sms), dim3(kThreads), (size_t)smem[1], s, rows,
                               reinterpret_cast<const Unit*>(b + w.units_dn), n_units, st->ht, w.Rpad, nt_tile, n_bslots[1],
                               n_slots[1], (__half*)nullptr, reinterpret_cast<float*>(b + w.y), c.hidden,
                               (size_t)R * c.hidden, work_counter + 1, status, reinterpret_cast<int32_t*>(b + w.done), ksplit, c.ffn / kTileRows, 0u));
