@@ -316,10 +316,17 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 struct RingPos {
   uint32_t s, par;                               // slot, parity of the full-barrier phase
 };
-__device__ __forceinline__ RingPos ring_pos(uint32_t seq, uint32_t n_slots) {
-  const uint32_t q = seq / n_slots;
+// `recip` = floor(2^32 / n_slots), computed once per kernel: the high product is the quotient or one less, which
+// one comparison corrects -- a division by a run-time number is some twenty instructions, and every role does
+// one or two at every unit boundary.
+__device__ __forceinline__ RingPos ring_pos(uint32_t seq, uint32_t n_slots, uint32_t recip) {
+  uint32_t q = __umulhi(seq, recip);
   RingPos p;
   p.s = seq - q * n_slots;
+  if (p.s >= n_slots) {
+    p.s -= n_slots;
+    ++q;
+  }
   p.par = q & 1u;
   return p;
 }
@@ -567,6 +574,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
   const int n_issuers = NMAT * ipa;
   const int acol = NMAT * npart * nt_tile;       // the operand slot of group g sits at acol + 64 * g
   const int G = gridDim.x;
+  const uint32_t recip_w = 0xffffffffu / (uint32_t)n_slots, recip_b = 0xffffffffu / (uint32_t)n_bslots;   // see ring_pos
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxSlots; ++i) {
@@ -934,9 +942,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
         const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(ipa - 1);
         uint32_t bt = base + j0;                     // token-tile number
-        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots, recip_b);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
-        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots, recip_w);
         const int npe = unit_accumulators<SHARE, NMAT>(npart, nb_rows, acol);
         const bool wide = NMAT * npe * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
@@ -998,9 +1006,9 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         // my first tile of the unit and what follows from its number: token-tile slot, ring slot, group
         const uint32_t j0 = ((uint32_t)my_j - base) & (uint32_t)(ipa - 1);
         uint32_t bt = base + j0;                     // token-tile number
-        RingPos bp = ring_pos(bt, (uint32_t)n_bslots);
+        RingPos bp = ring_pos(bt, (uint32_t)n_bslots, recip_b);
         uint32_t sq = seq_unit + j0 * W + my_off;    // first slot item of my tile (16-bit tiles only)
-        RingPos rp = ring_pos(sq, (uint32_t)n_slots);
+        RingPos rp = ring_pos(sq, (uint32_t)n_slots, recip_w);
         const int npe = unit_accumulators<SHARE, NMAT>(npart, nb_rows, acol);
         const bool wide = NMAT * npe * nb_rows > acol / 2;
         const uint32_t dbuf = wide ? 0u : dtoggle;
@@ -1117,7 +1125,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
         const uint32_t count = (ng - j0 + kStride - 1) / kStride;
         const uint32_t step = kStride * W;
         st.sq = seq_unit + j0 * W + (qm ? slot_items(ubits[0]) : 0u);
-        const RingPos rp = ring_pos(st.sq, (uint32_t)n_slots);
+        const RingPos rp = ring_pos(st.sq, (uint32_t)n_slots, recip_w);
         st.s = rp.s;
         st.par = rp.par;
         st.known = 0;                                // my items of this unit may be another producer's than before
