@@ -236,6 +236,38 @@ def test_forward_repeats_bit_for_bit_when_the_tile_counts_are_odd():
         ctx.close()
 
 
+def test_many_calls_with_wide_token_tiles_on_short_units(orc):
+    """Short contractions (4 K-tiles per gate/up unit, 16 per down unit), several units per CTA, token tiles wider than 32: the kernels
+    whose wide units share accumulators, two issuers taking turns on each.  One issuer is regularly a unit ahead
+    of the other at a unit boundary; the turn word must survive that (an earlier version lost a turn there and
+    ran into its bounded waits once in a few hundred units).  Several hundred calls over three layers of mixed
+    pages, every call checked against the first of its layer bit for bit, one of them against the oracle."""
+    cfg = synth.LayerConfig("wide_short", 16, 2, 512, 2048, 512, routing="normal", bit_rule="iid5", n_layers=3)
+    ctx = make_ctx(cfg, max_tokens=cfg.tokens, n_layers=3)
+    try:
+        pages = [build_layer(ctx, cfg, l, None)[0] for l in range(3)]
+        x = synth.activations(cfg, device="cuda")
+        logits = synth.router_logits(cfg, device="cuda")
+        first = [ctx.pw_moe_forward(l, x, logits, cfg.top_k).clone() for l in range(3)]
+        counts = ctx.pw_get_routing(cfg.tokens, cfg.top_k)["counts"].cpu().numpy()
+        assert counts.min() > 32                              # every expert takes wide token tiles
+        for i in range(450):
+            l = i % 3
+            again = ctx.pw_moe_forward(l, x, logits, cfg.top_k)
+            if i % 50 == 0:
+                assert ctx.pw_last_device_status() == 0, i
+            assert torch.equal(first[l].view(torch.int32), again.view(torch.int32)), i
+        torch.cuda.synchronize()
+        assert ctx.pw_last_device_status() == 0
+        opages = [export_to_oracle(ctx, p, orc) for p in pages[1]]
+        sample = list(range(0, cfg.tokens, 16))
+        ref = orc.moe_forward(x.cpu().numpy(), logits.cpu().numpy(), cfg.top_k, opages, tokens=sample)
+        max_abs, rel_f = error_metrics(first[1].cpu().numpy()[sample], ref[sample])
+        assert max_abs <= MAX_ABS and rel_f <= REL_F, (max_abs, rel_f)
+    finally:
+        ctx.close()
+
+
 def test_back_to_back_calls_with_different_routing(orc):
     """Consecutive calls reuse the workspace (unit lists, counters, operand buffers) while the kernels of the
     call before may still be draining: alternate two token sets and check every result against the oracle."""
