@@ -477,7 +477,7 @@ __device__ __forceinline__ bool dq_run(DqState& st, uint32_t count, uint32_t ste
       z2 = __half2half2(__ushort_as_half(zv));
     }
     const char* item = reinterpret_cast<const char*>(c) + kCtrlBytes + st.s * kSlotBytes;
-#pragma unroll 1
+#pragma unroll
     for (int h = 0; h < 2; ++h) {
       __half2 w[32];
       if constexpr ((UB & kPlanesFlag) != 0) decode_half_planes<(int)(UB & ~kPlanesFlag)>(item, r, h, s2, z2, w);
