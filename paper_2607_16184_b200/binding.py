@@ -366,16 +366,23 @@ class PlanePage:
 class Context:
     """Owns the workspace tensor and the ``pw_ctx``; methods carry the names of the C calls."""
 
+    GUARD_BYTE = 0xA5
+
     def __init__(self, n_layers: int, n_experts: int, n_shared: int, hidden: int, ffn: int, max_tokens: int,
-                 max_top_k: int, device="cuda"):
+                 max_top_k: int, device="cuda", guard_bytes: int = 0):
+        """``guard_bytes`` > 0 puts that many bytes of a known pattern in front of and behind the workspace
+        (``workspace_guards_intact`` looks at them): a check that no kernel writes outside it."""
         self.L = load()
         self.device = torch.device(device)
         cfg = pw_config(n_layers, n_experts, n_shared, hidden, ffn, GROUP, max_tokens, max_top_k, None, 0)
         nbytes = self.L.pw_workspace_bytes(C.byref(cfg))
         if nbytes == 0:
             raise PwError(1, "pw_workspace_bytes")
-        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
-        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        guard = (guard_bytes + 255) // 256 * 256
+        self.workspace = torch.full((nbytes + 256 + 2 * guard,), self.GUARD_BYTE, dtype=torch.uint8, device=self.device) \
+            if guard else torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + guard + 255) // 256 * 256
+        self._ws_span = (base - self.workspace.data_ptr(), nbytes)
         cfg.workspace, cfg.workspace_bytes = base, nbytes
         self.cfg = cfg
         self.handle = C.c_void_p()
@@ -384,6 +391,13 @@ class Context:
         self.n_segments = n_experts + n_shared
         self._committed = {}          # (layer, expert, kind) -> the page the row points to
         self.obs = None               # accumulators of the observation taps while they are on
+
+    def workspace_guards_intact(self) -> bool:
+        """True when the bytes in front of and behind the workspace still hold the guard pattern."""
+        off, nbytes = self._ws_span
+        torch.cuda.synchronize(self.device)
+        front, back = self.workspace[:off], self.workspace[off + nbytes:]
+        return bool((front == self.GUARD_BYTE).all().item()) and bool((back == self.GUARD_BYTE).all().item())
 
     def close(self):
         if self.handle:
