@@ -304,11 +304,16 @@ __device__ __forceinline__ void decode_half(const uint4* row_units, int h, __hal
 //   TOP   5632 B per tile: the two leading bits of every code in the 2-bit arrangement above (4096 B), then the
 //         lookup-table state of each bitwidth the planes can be read at: 128 scales + 128 zero-points (fp16) for
 //         2 bits, the same for 3 bits, the same for 4 bits.  The table is affine, entry c = zero-point + c * scale.
-//   BIT1  2048 B per tile: the third bit.  Row r owns 16 bytes at r * 16; word w of them covers k = 32w .. 32w+31:
-//         bit m (m < 16) belongs to k = 32w + 2m, bit 16 + m to k = 32w + 2m + 1.
+//   BIT1  2048 B per tile: the third bit.  Row r owns 16 bytes at r * 16; word w of them covers k = 32w .. 32w+31,
+//         the even k in its low half-word, the odd k in its high half-word, pair P = (k = 32w + 2P, 32w + 2P + 1)
+//         at bit plane_bit_pos(P) of each: the eight pairs that share a word of top codes take eight consecutive
+//         bits, first the four whose top codes are read in place (at every other bit), then, in the bits between,
+//         the four whose top codes are read after a shift by 8 -- so that one shift of the plane word puts the
+//         bits of four pairs where the decoder wants them (see decode_quarter_planes).
 //   BIT0  the fourth bit, same arrangement.
 // Read at q bits the code of a weight is its first q bits, c4 >> (4 - q): q = 2 needs TOP alone, q = 3 TOP and
 // BIT1, q = 4 all three.  Lowering the precision moves and computes nothing.
+__host__ __device__ constexpr int plane_bit_pos(int P) { return 8 * (P >> 3) + 2 * (P & 3) + ((P >> 2) & 1); }
 constexpr int kPlaneTopCodes = 4096;
 constexpr int kPlaneTopTile = kPlaneTopCodes + 3 * 512;
 constexpr int kPlaneBitTile = 2048;
@@ -331,20 +336,25 @@ __device__ __forceinline__ void decode_quarter_planes(const char* image, int r, 
   if constexpr (Q == 4) h0 = reinterpret_cast<const uint32_t*>(image + kPlaneSlotBit0 + r * 16)[t];
   // The top two bits of pair m of a word sit at bit 2m of both half-words.  Shifted up by Q - 2 places they stand
   // where the leading bits of a Q-bit code belong when the unit of the fp16 constant is at bit 2(m mod 4) (see
-  // dq_field); the plane bits below them are moved to their places and merged, one instruction each.
+  // dq_field).  The plane bits below them: pairs 0 .. 3 of word i have theirs at bits 8i, 8i + 2, 8i + 4, 8i + 6 of
+  // the plane word, pairs 4 .. 7 at the odd bits between, so one shift per word, plane and group of four pairs
+  // moves four of them to their places at once, and one logic instruction each merges them.
   constexpr int up = Q - 2;
+  auto moved = [](uint32_t x, int s) { return s >= 0 ? x >> s : x << -s; };   // s is a constant after unrolling
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     const uint32_t lo4 = w[i] << up, hi4 = w[i] >> (8 - up);   // pairs 0 .. 3 / 4 .. 7 of the word at bits up + 2(m mod 4)
+    // plane bits of pairs 0 .. 3 / 4 .. 7 at bits 2(m mod 4) + up - 1 (third bit) and 2(m mod 4) (fourth bit)
+    const uint32_t a1 = moved(h1, 8 * i - (up - 1)), b1 = moved(h1, 8 * i + 1 - (up - 1));
+    const uint32_t a0 = h0 >> (8 * i), b0 = h0 >> (8 * i + 1);
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
-      const int p = 8 * i + m;                     // pair index inside the quarter = bit of the plane words
+      const int p = 8 * i + m;                     // pair index inside the quarter
       const int U = 2 * (m & 3);                   // where the code's last bit goes
       const uint32_t magic = (uint32_t)((25 - U) << 10) * 0x00010001u;
       uint32_t v = and_or(m < 4 ? lo4 : hi4, (3u << (U + up)) * 0x00010001u, magic);
-      const int t1 = U + up - 1;
-      v = and_or(p >= t1 ? (h1 >> (p - t1)) : (h1 << (t1 - p)), (1u << t1) * 0x00010001u, v);
-      if constexpr (Q == 4) v = and_or(p >= U ? (h0 >> (p - U)) : (h0 << (U - p)), (1u << U) * 0x00010001u, v);
+      v = and_or(m < 4 ? a1 : b1, (1u << (U + up - 1)) * 0x00010001u, v);
+      if constexpr (Q == 4) v = and_or(m < 4 ? a0 : b0, (1u << U) * 0x00010001u, v);
       out[p] = dq_pair_k(v, magic, s2, z2);
     }
   }

@@ -8,13 +8,14 @@
 
 namespace pw {
 
-// word of plane bits of one 32-weight slice: bit m (m < 16) = weight 2m, bit 16 + m = weight 2m + 1
+// word of plane bits of one 32-weight slice: pair P = weights (2P, 2P + 1) at bit plane_bit_pos(P) of the low and
+// of the high half-word
 __device__ __forceinline__ uint32_t plane_word(const int (&code)[32], int bit) {
   uint32_t v = 0;
 #pragma unroll
   for (int m = 0; m < 16; ++m) {
-    v |= (uint32_t)((code[2 * m] >> bit) & 1) << m;
-    v |= (uint32_t)((code[2 * m + 1] >> bit) & 1) << (16 + m);
+    v |= (uint32_t)((code[2 * m] >> bit) & 1) << plane_bit_pos(m);
+    v |= (uint32_t)((code[2 * m + 1] >> bit) & 1) << (16 + plane_bit_pos(m));
   }
   return v;
 }
@@ -93,16 +94,16 @@ __global__ void __launch_bounds__(512) export_planes_kernel(const char* __restri
     const uint32_t b = reinterpret_cast<const uint32_t*>(bit1 + tile * kPlaneBitTile + r * 16)[q];
 #pragma unroll
     for (int m = 0; m < 16; ++m) {
-      code[2 * m] = (code[2 * m] << 1) | ((b >> m) & 1);
-      code[2 * m + 1] = (code[2 * m + 1] << 1) | ((b >> (16 + m)) & 1);
+      code[2 * m] = (code[2 * m] << 1) | ((b >> plane_bit_pos(m)) & 1);
+      code[2 * m + 1] = (code[2 * m + 1] << 1) | ((b >> (16 + plane_bit_pos(m))) & 1);
     }
   }
   if constexpr (Q == 4) {
     const uint32_t b = reinterpret_cast<const uint32_t*>(bit0 + tile * kPlaneBitTile + r * 16)[q];
 #pragma unroll
     for (int m = 0; m < 16; ++m) {
-      code[2 * m] = (code[2 * m] << 1) | ((b >> m) & 1);
-      code[2 * m + 1] = (code[2 * m + 1] << 1) | ((b >> (16 + m)) & 1);
+      code[2 * m] = (code[2 * m] << 1) | ((b >> plane_bit_pos(m)) & 1);
+      code[2 * m + 1] = (code[2 * m + 1] << 1) | ((b >> (16 + plane_bit_pos(m))) & 1);
     }
   }
   const size_t elem = row * cols + (size_t)g * kGroup + 32 * q;
