@@ -53,6 +53,13 @@ __host__ __device__ inline int slice_word_offset(int r, int q, int i) {
   return (2 * 128 + r) * 16 + q * 4;
 }
 
+// Where the single-bit plane of a 32-weight slice (the third bit of a 3-bit page, the planes of a bit-plane block)
+// keeps the bit of pair P = weights (2P, 2P + 1), in the low half-word for the even and in the high half-word for
+// the odd weight.  The eight pairs that share a word of 2-bit fields take eight consecutive bits: the four whose
+// fields are read in place at the even bits, the four read after the shift by 8 at the odd bits between -- one
+// shift of the plane word then moves the bits of four pairs to where the decoder merges them.
+__host__ __device__ constexpr int plane_bit_pos(int P) { return 8 * (P >> 3) + 2 * (P & 3) + ((P >> 2) & 1); }
+
 template <int BITS>
 __device__ inline void unpack_slice(const uint32_t* w, int (&code)[32]) {
   if constexpr (BITS == 8) {
@@ -79,8 +86,8 @@ __device__ inline void unpack_slice(const uint32_t* w, int (&code)[32]) {
     if constexpr (BITS == 3) {
 #pragma unroll
       for (int m = 0; m < 16; ++m) {
-        code[2 * m] |= ((w[2] >> m) & 1) << 2;
-        code[2 * m + 1] |= ((w[2] >> (16 + m)) & 1) << 2;
+        code[2 * m] |= ((w[2] >> plane_bit_pos(m)) & 1) << 2;
+        code[2 * m + 1] |= ((w[2] >> (16 + plane_bit_pos(m))) & 1) << 2;
       }
     }
   }
@@ -165,8 +172,8 @@ __device__ inline void pack_slice(const int (&code)[32], uint32_t* w) {
       uint32_t v = 0;
 #pragma unroll
       for (int m = 0; m < 16; ++m) {
-        v |= (uint32_t)((code[2 * m] >> 2) & 1) << m;
-        v |= (uint32_t)((code[2 * m + 1] >> 2) & 1) << (16 + m);
+        v |= (uint32_t)((code[2 * m] >> 2) & 1) << plane_bit_pos(m);
+        v |= (uint32_t)((code[2 * m + 1] >> 2) & 1) << (16 + plane_bit_pos(m));
       }
       w[2] = v;
     }
@@ -208,17 +215,14 @@ __device__ __forceinline__ __half2 dq_field(uint32_t word, __half2 s2, __half2 z
   constexpr uint32_t magic = field_magic<POS>();
   return dq_pair_k(and_or(word, mask, magic), magic, s2, z2);
 }
-// The same for a 2-bit field, with (BITS == 3) the code's third bit from bit p / 16 + p of `hw` put just above it.
+// The same for a 2-bit field, with (BITS == 3) the code's third bit, already moved to bit POS + 2 of `hi`, put just
+// above it.
 template <int POS, int BITS>
-__device__ __forceinline__ __half2 dq_field23(uint32_t word, uint32_t hw, int p, __half2 s2, __half2 z2) {
+__device__ __forceinline__ __half2 dq_field23(uint32_t word, uint32_t hi, __half2 s2, __half2 z2) {
   constexpr uint32_t mask = (3u << POS) * 0x00010001u;
   constexpr uint32_t magic = field_magic<POS>();
   uint32_t v = and_or(word, mask, magic);
-  if constexpr (BITS == 3) {
-    const int t = POS + 2;                       // where the third bit goes
-    const uint32_t hi = p >= t ? (hw >> (p - t)) : (hw << (t - p));
-    v = and_or(hi, (1u << t) * 0x00010001u, v);
-  }
+  if constexpr (BITS == 3) v = and_or(hi, (1u << (POS + 2)) * 0x00010001u, v);
   return dq_pair_k(v, magic, s2, z2);
 }
 
@@ -266,7 +270,8 @@ __device__ __forceinline__ void decode_quarter(const uint4* row_units, int t, __
     // 2 bits: words 2(t%2), 2(t%2)+1 of unit t/2.  3 bits: the same low-plane words plus word t of unit 2.
     // A half-word holds eight 2-bit fields; fields 0 .. 3 are read where they lie (see dq_field), one shift by 8
     // per word brings fields 4 .. 7 to the same places.  The third bit of a 3-bit code is moved to the place
-    // just above its field, where it reads 4.
+    // just above its field, where it reads 4: the plane word keeps the bits of fields 0 .. 3 of word i at bits
+    // 8i, 8i + 2, .. and those of fields 4 .. 7 at the odd bits between (plane_bit_pos), so two shifts per word do.
     const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint32_t*>(row_units + (t >> 1) * kUnitStride) +
                                                      2 * (t & 1));
     const uint32_t w[2] = {u.x, u.y};
@@ -275,15 +280,17 @@ __device__ __forceinline__ void decode_quarter(const uint4* row_units, int t, __
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       const uint32_t w8 = w[i] >> 8;
+      // third bits of fields 0 .. 3 / 4 .. 7 at bits 2(m mod 4) + 2
+      const uint32_t ha = i == 0 ? hw << 2 : hw >> 6, hb = i == 0 ? hw << 1 : hw >> 7;
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
-        const int p = 8 * i + m;                   // pair index inside the quarter = inside the high-plane word
-        const uint32_t src = m < 4 ? w[i] : w8;
+        const int p = 8 * i + m;                   // pair index inside the quarter
+        const uint32_t src = m < 4 ? w[i] : w8, hi = m < 4 ? ha : hb;
         switch (m & 3) {
-          case 0: out[p] = dq_field23<0, BITS>(src, hw, p, s2, z2); break;
-          case 1: out[p] = dq_field23<2, BITS>(src, hw, p, s2, z2); break;
-          case 2: out[p] = dq_field23<4, BITS>(src, hw, p, s2, z2); break;
-          default: out[p] = dq_field23<6, BITS>(src, hw, p, s2, z2); break;
+          case 0: out[p] = dq_field23<0, BITS>(src, hi, s2, z2); break;
+          case 1: out[p] = dq_field23<2, BITS>(src, hi, s2, z2); break;
+          case 2: out[p] = dq_field23<4, BITS>(src, hi, s2, z2); break;
+          default: out[p] = dq_field23<6, BITS>(src, hi, s2, z2); break;
         }
       }
     }
@@ -313,7 +320,6 @@ __device__ __forceinline__ void decode_half(const uint4* row_units, int h, __hal
 //   BIT0  the fourth bit, same arrangement.
 // Read at q bits the code of a weight is its first q bits, c4 >> (4 - q): q = 2 needs TOP alone, q = 3 TOP and
 // BIT1, q = 4 all three.  Lowering the precision moves and computes nothing.
-__host__ __device__ constexpr int plane_bit_pos(int P) { return 8 * (P >> 3) + 2 * (P & 3) + ((P >> 2) & 1); }
 constexpr int kPlaneTopCodes = 4096;
 constexpr int kPlaneTopTile = kPlaneTopCodes + 3 * 512;
 constexpr int kPlaneBitTile = 2048;

@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const vo
   }
 
   uint32_t half_bytes[16];                         // per source word: the 2-bit codes of 8 weights, a byte in each half-word
-  uint32_t third[4];                               // DB == 3, per slice: the plane of the third bits, bit P / 16 + P for pair P
+  uint32_t third[4];                               // DB == 3, per slice: the plane of the third bits (plane_bit_pos)
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     if ((i & 3) == 0) third[i >> 2] = 0;
@@ -258,9 +258,13 @@ __global__ void __launch_bounds__(kRequantThreads) requant_from4_kernel(const vo
       asm("lop3.b32 %0, %1, %2, %3, 0xBA;" : "=r"(b1) : "r"(f[1]), "r"(f[3]), "r"(f[5]));
       // third bits: nibble a of the word (flag in bit 4 a + 3) -> bit a of its half-word.  Moved to bit 4 a + 1, the
       // shifts by 1, 4, 7, 10 bring a = 0 .. 3 to bits 0 .. 3 and no two copies share a bit (4 a - 3 j is different
-      // for every a and j): one high product.
+      // for every a and j): one high product.  The plane keeps the four pairs of source word i at every other
+      // bit from plane_bit_pos(4 (i mod 4)) on, so the four bits are spread to every other place first.
       const uint32_t g = __umulhi((f[3] >> 2) & 0x22222222u, (1u << 31) + (1u << 28) + (1u << 25) + (1u << 22));
-      third[i >> 2] |= (g & 0x000f000fu) << (4 * (i & 3));
+      uint32_t sp = g & 0x000f000fu;
+      sp = (sp | (sp << 2)) & 0x00330033u;
+      sp = (sp | (sp << 1)) & 0x00550055u;
+      third[i >> 2] |= sp << plane_bit_pos(4 * (i & 3));
     } else {
       b1 = f[1];
     }
