@@ -351,16 +351,20 @@ __device__ __forceinline__ void decode_quarter_planes(const char* image, int r, 
   for (int i = 0; i < 2; ++i) {
     const uint32_t lo4 = w[i] << up, hi4 = w[i] >> (8 - up);   // pairs 0 .. 3 / 4 .. 7 of the word at bits up + 2(m mod 4)
     // plane bits of pairs 0 .. 3 / 4 .. 7 at bits 2(m mod 4) + up - 1 (third bit) and 2(m mod 4) (fourth bit)
-    const uint32_t a1 = moved(h1, 8 * i - (up - 1)), b1 = moved(h1, 8 * i + 1 - (up - 1));
-    const uint32_t a0 = h0 >> (8 * i), b0 = h0 >> (8 * i + 1);
+    uint32_t a1 = moved(h1, 8 * i - (up - 1)), b1 = moved(h1, 8 * i + 1 - (up - 1));
+    if constexpr (Q == 4) {
+      // third and fourth bits of four pairs side by side (bits 2(m mod 4) + 1 and 2(m mod 4)): merged once per four
+      // pairs, so that a pair takes its two low bits with one instruction
+      a1 = and_or(a1, 0x00aa00aau, (h0 >> (8 * i)) & 0x00550055u);
+      b1 = and_or(b1, 0x00aa00aau, (h0 >> (8 * i + 1)) & 0x00550055u);
+    }
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
       const int p = 8 * i + m;                     // pair index inside the quarter
       const int U = 2 * (m & 3);                   // where the code's last bit goes
       const uint32_t magic = (uint32_t)((25 - U) << 10) * 0x00010001u;
       uint32_t v = and_or(m < 4 ? lo4 : hi4, (3u << (U + up)) * 0x00010001u, magic);
-      v = and_or(m < 4 ? a1 : b1, (1u << (U + up - 1)) * 0x00010001u, v);
-      if constexpr (Q == 4) v = and_or(m < 4 ? a0 : b0, (1u << U) * 0x00010001u, v);
+      v = and_or(m < 4 ? a1 : b1, (Q == 4 ? 3u << U : 1u << U) * 0x00010001u, v);
       out[p] = dq_pair_k(v, magic, s2, z2);
     }
   }
