@@ -11,9 +11,12 @@
 // written to tensor memory, which the MMA then reads as its A operand.  The token tile (B operand) comes
 // from the k-chunk-major operand buffers with one 2-D TMA copy per group.
 //
-// One persistent CTA per SM, 27 warps.  The control roles are single threads with short dependent
-// instruction chains: they share the schedulers with the arithmetic-heavy dequantizers, and every
-// instruction of theirs waits its turn, so each of them does as little per item as possible.
+// One persistent CTA per SM, 27 warps.  The control roles have short dependent instruction chains: they share
+// the schedulers with the arithmetic-heavy dequantizers, and every instruction of theirs waits its turn, so each
+// of them does as little per item as possible.  Each runs as a whole, converged warp on the same values, lane 0
+// being a predicate on the instructions with an effect (copies, MMAs, commits, arrivals): the MMA, the bulk copy
+// and the barrier operations take their operands from uniform registers, which a single lane inside a divergent
+// branch can only fill by moving every operand over for every instruction.
 //   warps 0-15   dequantize: four groups of four warps; tile k of a matrix goes to that matrix's group
 //                k mod (groups per matrix); warp w owns TMEM lanes 32*(w%4).., one weight row per thread;
 //                a group has one operand slot of 64 columns in tensor memory (a whole tile, K 0..127) and hands
@@ -23,11 +26,13 @@
 //                claims the CTA's units from a global counter and posts them (the unit and the bitwidths of its
 //                pages) on the CTA's work list in shared memory, the only place the other roles learn of them;
 //   warp 17      token-tile producer (its own few slots, never holds back the weight stream);
-//   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  A tcgen05.mma holds its issuing
-//                thread for ~100 cycles whatever its size, so the issuers work in parallel: issuer j of a
+//   warps 19-22  MMA issuers (warp 19 also allocates tensor memory).  Issuing a tcgen05.mma costs its warp tens of
+//                cycles whatever its size, so the issuers work in parallel: issuer j of a
 //                matrix issues all eight k-steps of the tiles k = j mod (issuers per matrix) into its own
 //                partial accumulator -- with as many issuers as groups, each dequantizer group has an
-//                issuer of its own -- and no two threads ever accumulate into the same columns;
+//                issuer of its own -- and no two threads ever accumulate into the same columns at the same time
+//                (the SHARE instantiations let the two issuers of an accumulator take turns on it where a
+//                unit's token tile is wide, see unit_accumulators);
 //   warps 23-26  epilogue: adds the partials; SwiGLU -> fp16 operand of the down projection (PHASE 0), or the
 //                fp32 split-K partial of the down projection (PHASE 1).  Narrow token tiles alternate
 //                between two accumulator buffers, so the next unit's MMAs overlap the epilogue.
@@ -622,7 +627,7 @@ ffn_tc_kernel(const DevRow* __restrict__ rows, const Unit* units, const int32_t*
 
   if (warp == kWarpCodes || warp == kWarpCodes2) {
     // ---------------- weight producers ----------------
-    // Two single-thread producers share the stream: producer P arms the slot items with number = P mod 2,
+    // Two producer warps share the stream: producer P arms the slot items with number = P mod 2,
     // which (even slot count) always land in the slots = P mod 2, so each keeps the state of its own slots.
     // Producer 0 also claims the units.  The whole warp runs the loop on the same values; lane 0 arms, copies,
     // claims and posts.
